@@ -1,0 +1,203 @@
+"""CPU oracle for the gradient-dropping hot path (Aji & Heafield 2017, Section 4, Algorithm 1).
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain definition that the CUDA library is
+checked against.  It shares no code with the CUDA path, imports nothing from the product
+package, and may be imported only by tests, by the smoke check and by the benchmark's
+cpu-baseline leg.  Every function is pinned by tests that do not go through this module's own
+formulas (brute-force rank counts, closed forms, library selection routines, the payload ratios
+the paper prints); no function here is "parity unpinned".
+
+What the path computes (Algorithm 1, in its order):
+
+  1. grad += residuals                      (fp32 add, round to nearest even)
+  2. select threshold: R% of |grad| smaller  (single threshold on |value|, Section 4 par. 1)
+  3. kept[i] = grad[i] where |grad[i]| is above the threshold, else 0
+  4. residuals = grad - kept                 (the dropped mass stays local)
+  5. return sparse(kept)                     (index + value pairs, 8 bytes per survivor;
+                                              the "50x less data at 99%" of Section 5.1)
+
+Readings taken where the paper is silent:
+  * exactly k = n - floor(n * drop_ppm / 1e6) entries are kept per threshold scope; the
+    order used is (|v| bit pattern descending, index ascending), so ties at the cut go to
+    the lower index; the reported threshold tau is the smallest kept |v| bit pattern
+    (0xFFFFFFFF when nothing is kept);
+  * a scope is either the whole gradient ("global") or each parameter tensor on its own
+    ("locally to each matrix", Section 4 last paragraph);
+  * two-value quantisation (Section 5.4, "averages of values being quantized"): one pair
+    (mean of kept entries with sign bit 0, mean of kept entries with sign bit 1) per layer,
+    survivors packed as index | signbit << 31; the residual still holds only the dropped mass;
+  * the server applies a push as p[idx - shard_start] += alpha * value (Section 3: a server
+    owns 1/N of the parameters); this oracle evaluates that sum in fp64.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+SCOPE_GLOBAL = 0
+SCOPE_PER_LAYER = 1
+VALUES_FP32 = 0
+VALUES_TWO_MEANS = 1
+
+_ABS_MASK = np.uint32(0x7FFFFFFF)
+TAU_NONE = 0xFFFFFFFF
+
+
+def kept_count(n: int, drop_ppm: int) -> int:
+    """Entries kept out of n when drop_ppm parts per million are dropped (Algorithm 1, step 2).
+
+    dropped = floor(n * drop_ppm / 1e6), kept = the rest; Python integers, so no rounding.
+    """
+    if n < 0 or not (0 <= drop_ppm <= 1_000_000):
+        raise ValueError("bad n or drop_ppm")
+    return n - (n * drop_ppm) // 1_000_000
+
+
+def scopes_of(layer_off, scope_mode: int):
+    """Index ranges over which one threshold is selected (Section 4, last paragraph)."""
+    layer_off = [int(x) for x in layer_off]
+    if scope_mode == SCOPE_GLOBAL:
+        return [(layer_off[0], layer_off[-1])]
+    if scope_mode == SCOPE_PER_LAYER:
+        return [(layer_off[i], layer_off[i + 1]) for i in range(len(layer_off) - 1)]
+    raise ValueError("bad scope_mode")
+
+
+def magnitude_keys(v: np.ndarray) -> np.ndarray:
+    """|v| as the unsigned integer whose order equals the order of |v| for finite floats."""
+    assert v.dtype == np.float32
+    return v.view(np.uint32) & _ABS_MASK
+
+
+def _kept_in_scope(keys: np.ndarray, k: int, method: str):
+    """Indices (local, ascending) of the k largest keys, ties to the lower index, and tau.
+
+    The order is made strict by the composite  key << 32 | (0xFFFFFFFF - index): a larger
+    composite means larger |v|, or equal |v| and a lower index.  "sort" sorts all composites;
+    "select" uses a partial selection of the same composites (the k-th element of a strict
+    total order is unique, so both give the same set).
+    """
+    n = keys.shape[0]
+    if k == 0:
+        return np.empty(0, dtype=np.int64), TAU_NONE
+    comp = (keys.astype(np.uint64) << np.uint64(32)) | (
+        np.uint64(0xFFFFFFFF) - np.arange(n, dtype=np.uint64))
+    if method == "sort":
+        top = np.sort(comp)[n - k:]
+    elif method == "select":
+        top = np.partition(comp, n - k)[n - k:]
+    else:
+        raise ValueError("bad method")
+    tau = int(top.min() >> np.uint64(32))
+    local = (np.uint64(0xFFFFFFFF) - (top & np.uint64(0xFFFFFFFF))).astype(np.int64)
+    local.sort()
+    return local, tau
+
+
+def compress(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GLOBAL,
+             value_mode=VALUES_FP32, method="sort"):
+    """One GradDrop call (Algorithm 1) for one worker's flat fp32 gradient.
+
+    grad, residual : float32 arrays of n elements (not modified).
+    layer_off      : n_layers + 1 ascending offsets, first 0, last n.
+    shard_off      : n_shards + 1 ascending offsets, first 0, last n (Section 3's 1/N pieces).
+    Returns a dict with
+      idx       uint32[k_total]  survivor positions, ascending (two-means: idx | sign << 31)
+      val       float32[k_total] survivor values, bit-for-bit v[idx]  (fp32 mode)
+      residual  float32[n]       v where dropped, +0.0 where kept
+      tau       uint32[n_scopes] smallest kept |v| bit pattern per scope (0xFFFFFFFF: none kept)
+      shard_cnt_off uint32[n_shards+1] survivors with index below each shard boundary
+      means     float32[n_layers, 2], counts int64[n_layers, 2], sums float64[n_layers, 2]
+                (two-means mode; column 0 = sign bit clear, column 1 = sign bit set)
+    """
+    g = np.ascontiguousarray(grad, dtype=np.float32)
+    r = np.ascontiguousarray(residual, dtype=np.float32)
+    n = g.shape[0]
+    assert r.shape[0] == n
+    layer_off = [int(x) for x in layer_off]
+    shard_off = [int(x) for x in shard_off]
+    assert layer_off[0] == 0 and layer_off[-1] == n
+    assert shard_off[0] == 0 and shard_off[-1] == n
+
+    v = g + r                                   # step 1: one IEEE binary32 add per element
+    keys = magnitude_keys(v)
+
+    kept_parts, taus = [], []
+    for lo, hi in scopes_of(layer_off, scope_mode):
+        k = kept_count(hi - lo, drop_ppm)       # step 2
+        local, tau = _kept_in_scope(keys[lo:hi], k, method)
+        kept_parts.append(local + lo)
+        taus.append(tau)
+    kept = np.concatenate(kept_parts) if kept_parts else np.empty(0, dtype=np.int64)
+
+    new_residual = v.copy()                     # step 4: residuals = grad - kept
+    new_residual[kept] = np.float32(0.0)
+    val = v[kept]                               # step 3/5: the values that travel
+
+    shard_cnt_off = np.searchsorted(kept, np.asarray(shard_off, dtype=np.int64),
+                                    side="left").astype(np.uint32)
+    out = {
+        "idx": kept.astype(np.uint32),
+        "val": val,
+        "residual": new_residual,
+        "tau": np.asarray(taus, dtype=np.uint32),
+        "shard_cnt_off": shard_cnt_off,
+        "v": v,
+    }
+    if value_mode == VALUES_TWO_MEANS:
+        if n > (1 << 31):
+            raise ValueError("two-means packing needs n <= 2^31")
+        n_layers = len(layer_off) - 1
+        sums = np.zeros((n_layers, 2), dtype=np.float64)
+        cnts = np.zeros((n_layers, 2), dtype=np.int64)
+        sign = (val.view(np.uint32) >> np.uint32(31)).astype(np.int64)
+        layer = np.searchsorted(np.asarray(layer_off, dtype=np.int64), kept, side="right") - 1
+        # unbuffered accumulation: one fp64 add per survivor, in ascending index order
+        np.add.at(sums, (layer, sign), val.astype(np.float64))
+        np.add.at(cnts, (layer, sign), 1)
+        with np.errstate(invalid="ignore", divide="ignore"):
+            means = np.where(cnts > 0, sums / np.maximum(cnts, 1), 0.0).astype(np.float32)
+        out["idx"] = (kept.astype(np.uint32) | (sign.astype(np.uint32) << np.uint32(31)))
+        out["means"], out["counts"], out["sums"] = means, cnts, sums
+    elif value_mode != VALUES_FP32:
+        raise ValueError("bad value_mode")
+    return out
+
+
+def decode_push(push_idx, push_val, value_mode=VALUES_FP32, means=None, layer_off=None):
+    """Positions and fp32 values a push stands for (the server-side decompress)."""
+    idx = np.asarray(push_idx, dtype=np.uint32)
+    if value_mode == VALUES_FP32:
+        return idx.astype(np.int64), np.asarray(push_val, dtype=np.float32)
+    pos = (idx & _ABS_MASK).astype(np.int64)
+    sign = (idx >> np.uint32(31)).astype(np.int64)
+    layer = np.searchsorted(np.asarray(layer_off, dtype=np.int64), pos, side="right") - 1
+    return pos, np.asarray(means, dtype=np.float32)[layer, sign]
+
+
+def apply_pushes(params, shard_start, pushes, alpha=1.0, value_mode=VALUES_FP32, layer_off=None):
+    """fp64 reference of the server-side scatter-add into one parameter shard (Section 3).
+
+    params  : float32[shard_len], the shard's parameters before the pushes.
+    pushes  : list of dicts with "idx" (+ "val", or "means" in two-means mode); only entries
+              whose position falls in [shard_start, shard_start + shard_len) are applied.
+    Returns (ref, bound): ref = p0 + sum alpha * value in fp64, and bound = |p0| + sum
+    |alpha * value| (the magnitude the 1e-6 relative tolerance is taken against).
+    """
+    p0 = np.asarray(params, dtype=np.float32)
+    ref = p0.astype(np.float64)
+    bound = np.abs(ref)
+    a = float(np.float32(alpha))
+    lo, hi = int(shard_start), int(shard_start) + p0.shape[0]
+    for push in pushes:
+        pos, val = decode_push(push["idx"], push.get("val"), value_mode, push.get("means"),
+                               layer_off)
+        m = (pos >= lo) & (pos < hi)
+        contrib = a * val[m].astype(np.float64)
+        np.add.at(ref, pos[m] - lo, contrib)
+        np.add.at(bound, pos[m] - lo, np.abs(contrib))
+    return ref, bound
+
+
+def residual_reset(n: int) -> np.ndarray:
+    """The state before the first call: nothing has been dropped yet (Section 4, par. 2)."""
+    return np.zeros(n, dtype=np.float32)

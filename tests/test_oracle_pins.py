@@ -1,0 +1,370 @@
+"""Pins for the CPU oracle: every check here is independent of the oracle's own formulas.
+
+Brute-force rank counts in pure Python, closed forms, library selection routines, exact
+rational arithmetic, and the payload ratios the paper prints (tests/golden/payload_ratios.txt).
+"""
+import itertools
+import math
+import os
+import struct
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import graddrop_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def f32_bits(x) -> int:
+    return struct.unpack("<I", struct.pack("<f", float(x)))[0]
+
+
+def brute_force_kept(v, k):
+    """O(n^2): entry i is kept iff fewer than k entries precede it in (|v| desc, index asc)."""
+    keys = [f32_bits(x) & 0x7FFFFFFF for x in v]
+    kept = []
+    for i, ki in enumerate(keys):
+        ahead = 0
+        for j, kj in enumerate(keys):
+            if kj > ki or (kj == ki and j < i):
+                ahead += 1
+        if ahead < k:
+            kept.append(i)
+    return kept
+
+
+def run_flat(v, drop_ppm, **kw):
+    """GradDrop of v itself: the residual is -0.0 everywhere, the one value with x + r == x bit for bit."""
+    g = np.asarray(v, dtype=np.float32)
+    r = np.full_like(g, -0.0)
+    n = g.shape[0]
+    return orc.compress(g, r, [0, n], [0, n], drop_ppm, **kw)
+
+
+# ---------------------------------------------------------------- kept-count formula
+def test_kept_count_values():
+    assert orc.kept_count(1 << 20, 990_000) == 10_486
+    assert orc.kept_count(1 << 30, 999_000) == 1_073_742
+    assert orc.kept_count(10, 990_000) == 1
+    assert orc.kept_count(0, 990_000) == 0
+    assert orc.kept_count(7, 0) == 7
+    assert orc.kept_count(7, 1_000_000) == 0
+    # the six tensors of the MNIST-shaped workload at 99 %
+    sizes = [784 * 4096, 4096, 4096 * 4096, 4096, 40960, 10]
+    assert [orc.kept_count(s, 990_000) for s in sizes] == [32113, 41, 167773, 41, 410, 1]
+    assert orc.kept_count(sum(sizes), 990_000) == 200_377
+    # equals ceil((1 - R) n) evaluated exactly
+    for n in (1, 3, 99, 100, 101, 12345, 1 << 20):
+        for ppm in (0, 1, 900_000, 990_000, 999_000, 999_999, 1_000_000):
+            assert orc.kept_count(n, ppm) == math.ceil(Fraction(n) * (1 - Fraction(ppm, 1_000_000)))
+
+
+def test_paper_payload_ratios():
+    rec = {}
+    with open(os.path.join(GOLDEN, "payload_ratios.txt")) as fh:
+        for line in fh:
+            if line.strip() and not line.startswith("#"):
+                parts = line.split()
+                rec[parts[0]] = parts[1]
+    ratio99 = float(rec["ratio_dense_over_sparse_at_99pct"])
+    min_ratio = float(rec["min_ratio_984_to_99"])
+    for n in (100, 1000, 1 << 20, 137_585_000):
+        out = run_flat(np.arange(1, n + 1, dtype=np.float32) if n <= 1000 else
+                       np.random.default_rng(0).standard_normal(n).astype(np.float32), 990_000,
+                       method="select")
+        sparse_bytes = out["idx"].nbytes + out["val"].nbytes
+        assert out["idx"].dtype == np.uint32 and out["val"].dtype == np.float32
+        got = 4 * n / sparse_bytes
+        if n % 100 == 0:
+            assert got == ratio99
+        else:
+            assert abs(got - ratio99) / ratio99 < 1e-4
+    k984 = orc.kept_count(10**6, 984_000)
+    k99 = orc.kept_count(10**6, 990_000)
+    assert k984 / k99 > min_ratio and k984 / k99 == pytest.approx(1.6)
+
+
+# ---------------------------------------------------------------- brute force on tiny vectors
+ALPHABET = [0.0, -0.0, 1.0, -1.0, 2.0, -2.0, 1e-45, -3.5]
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4])
+def test_exhaustive_tiny_vectors_all_k(n):
+    ppms = sorted({(d * 1_000_000) // n for d in range(n + 1)} | {1_000_000, 0, 999_999, 1})
+    for v in itertools.product(ALPHABET, repeat=n):
+        for ppm in ppms:
+            k = n - (n * ppm) // 1_000_000
+            want = brute_force_kept(v, k)
+            out = run_flat(v, ppm)
+            assert out["idx"].tolist() == want, (v, ppm)
+            if k:
+                assert int(out["tau"][0]) == min(f32_bits(v[i]) & 0x7FFFFFFF for i in want)
+            else:
+                assert int(out["tau"][0]) == 0xFFFFFFFF
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_brute_force_random_with_ties(seed):
+    rng = np.random.default_rng(seed)
+    n = int(rng.integers(5, 400))
+    # few distinct magnitudes => many ties at the cut
+    v = rng.choice(np.array([0.0, -0.0, 0.5, -0.5, 0.75, 3.0, -3.0, 1e-40], dtype=np.float32), size=n)
+    for ppm in (0, 500_000, 900_000, 990_000, 1_000_000):
+        for method in ("sort", "select"):
+            out = run_flat(v, ppm, method=method)
+            assert out["idx"].tolist() == brute_force_kept(v.tolist(), orc.kept_count(n, ppm))
+
+
+def test_brute_force_per_layer_and_shards():
+    rng = np.random.default_rng(11)
+    sizes = [10, 0, 37, 1, 128, 5]
+    layer_off = np.concatenate([[0], np.cumsum(sizes)]).tolist()
+    n = layer_off[-1]
+    g = rng.standard_normal(n).astype(np.float32)
+    g[rng.integers(0, n, 40)] = 0.25           # ties
+    r = (rng.standard_normal(n) * 0.1).astype(np.float32)
+    shard_off = [0, 7, 7, 100, n]
+    out = orc.compress(g, r, layer_off, shard_off, 900_000, scope_mode=orc.SCOPE_PER_LAYER)
+    v = [float(np.float32(a) + np.float32(b)) for a, b in zip(g, r)]
+    want = []
+    for li, s in enumerate(sizes):
+        lo = layer_off[li]
+        k = s - (s * 900_000) // 1_000_000
+        want += [lo + i for i in brute_force_kept(v[lo:lo + s], k)]
+    assert out["idx"].tolist() == want
+    assert out["shard_cnt_off"].tolist() == [sum(1 for i in want if i < b) for b in shard_off]
+    assert [int(t) for t in out["tau"]][1] == 0xFFFFFFFF        # empty layer keeps nothing
+
+
+# ---------------------------------------------------------------- invariants
+def check_invariants(g, r, layer_off, shard_off, ppm, scope_mode, out):
+    v = (g + r).astype(np.float32)
+    keys = v.view(np.uint32) & np.uint32(0x7FFFFFFF)
+    idx = out["idx"].astype(np.int64) & 0x7FFFFFFF if out["idx"].dtype == np.uint32 and "means" in out \
+        else out["idx"].astype(np.int64)
+    kept_mask = np.zeros(v.shape[0], dtype=bool)
+    kept_mask[idx] = True
+    assert np.all(np.diff(idx) > 0)                                   # strictly ascending
+    # kept + residual reassemble v bit for bit
+    res_bits = out["residual"].view(np.uint32)
+    assert np.all(res_bits[kept_mask] == 0)
+    assert np.array_equal(res_bits[~kept_mask], v.view(np.uint32)[~kept_mask])
+    if "means" not in out:
+        assert np.array_equal(out["val"].view(np.uint32), v.view(np.uint32)[idx])
+    for si, (lo, hi) in enumerate(orc.scopes_of(layer_off, scope_mode)):
+        k = (hi - lo) - ((hi - lo) * ppm) // 1_000_000
+        m = kept_mask[lo:hi]
+        assert int(m.sum()) == k
+        if 0 < k < hi - lo:
+            kk, dk = keys[lo:hi][m], keys[lo:hi][~m]
+            tau = int(out["tau"][si])
+            assert int(kk.min()) == tau and int(dk.max()) <= tau
+            ties = np.flatnonzero(keys[lo:hi] == tau)
+            kept_ties, dropped_ties = ties[m[ties]], ties[~m[ties]]
+            if len(kept_ties) and len(dropped_ties):
+                assert kept_ties.max() < dropped_ties.min()
+    sc = out["shard_cnt_off"].astype(np.int64)
+    assert np.all(np.diff(sc) >= 0) and sc[0] == 0 and sc[-1] == idx.shape[0]
+
+
+@pytest.mark.parametrize("seed", range(4))
+@pytest.mark.parametrize("scope_mode", [orc.SCOPE_GLOBAL, orc.SCOPE_PER_LAYER])
+def test_invariants_random(seed, scope_mode):
+    rng = np.random.default_rng(100 + seed)
+    sizes = rng.integers(0, 5000, size=7).tolist()
+    layer_off = np.concatenate([[0], np.cumsum(sizes)]).tolist()
+    n = layer_off[-1]
+    g = rng.laplace(0, 1e-3, n).astype(np.float32)
+    g[rng.random(n) < 0.3] = 0.0
+    r = np.where(rng.random(n) < 0.5, rng.laplace(0, 1e-3, n), 0).astype(np.float32)
+    shard_off = [0, n // 3, n // 2, n]
+    for ppm in (0, 900_000, 990_000, 999_000, 1_000_000):
+        out = orc.compress(g, r, layer_off, shard_off, ppm, scope_mode=scope_mode)
+        check_invariants(g, r, layer_off, shard_off, ppm, scope_mode, out)
+
+
+# ---------------------------------------------------------------- closed forms
+def test_closed_form_distinct_magnitudes():
+    n = 1000
+    rng = np.random.default_rng(5)
+    m = rng.permutation(n) + 1                               # magnitudes m / 1024, all distinct
+    sign = rng.choice([-1.0, 1.0], n)
+    v = (sign * m / 1024.0).astype(np.float32)
+    for ppm in (500_000, 900_000, 990_000, 999_000):
+        k = orc.kept_count(n, ppm)
+        out = run_flat(v, ppm)
+        assert sorted(m[out["idx"]].tolist()) == list(range(n - k + 1, n + 1))
+        assert int(out["tau"][0]) == f32_bits((n - k + 1) / 1024.0)
+
+
+def test_closed_form_degenerate_inputs():
+    n = 257
+    for c in (0.0, -0.0, 3.25, -3.25):
+        for ppm in (900_000, 990_000):
+            k = orc.kept_count(n, ppm)
+            out = run_flat(np.full(n, c, dtype=np.float32), ppm)
+            assert out["idx"].tolist() == list(range(k))         # ties go to the lowest indices
+            assert int(out["tau"][0]) == f32_bits(c) & 0x7FFFFFFF
+            assert np.array_equal(out["val"].view(np.uint32), np.full(k, f32_bits(c), dtype=np.uint32))
+    v = np.random.default_rng(1).standard_normal(n).astype(np.float32)
+    out = run_flat(v, 0)                                         # R = 0: everything travels
+    assert out["idx"].tolist() == list(range(n)) and not out["residual"].any()
+    assert np.all(out["residual"].view(np.uint32) == 0)
+    out = run_flat(v, 1_000_000)                                 # R = 100 %: nothing travels
+    assert out["idx"].size == 0 and np.array_equal(out["residual"], v)
+    # k = 1 is the lowest-index arg-max of |v|
+    v[[17, 200]] = [-9.0, 9.0]
+    out = run_flat(v, orc_ppm_for_k1(n))
+    assert out["idx"].tolist() == [17] and out["val"].tolist() == [-9.0]
+
+
+def orc_ppm_for_k1(n):
+    ppm = ((n - 1) * 1_000_000 + n - 1) // n
+    assert orc.kept_count(n, ppm) == 1
+    return ppm
+
+
+def test_signed_zero_and_subnormals_are_preserved():
+    v = np.array([-0.0, 1e-45, -1e-45, 0.0, 5.0, -1e-39], dtype=np.float32)
+    out = run_flat(v, 500_000)                                   # keeps 3: 5.0, -1e-39, then 1e-45 (idx 1)
+    assert out["idx"].tolist() == [1, 4, 5]
+    assert [f32_bits(x) for x in out["val"]] == [f32_bits(1e-45), f32_bits(5.0), f32_bits(-1e-39)]
+    assert [f32_bits(x) for x in out["residual"]] == [0x80000000, 0, f32_bits(-1e-45), 0, 0, 0]
+
+
+# ---------------------------------------------------------------- library selection routines
+@pytest.mark.parametrize("seed", range(3))
+def test_threshold_equals_library_selection(seed):
+    rng = np.random.default_rng(200 + seed)
+    n = 50_000 + seed * 777
+    g = rng.laplace(0, 1e-3, n).astype(np.float32)
+    r = rng.laplace(0, 1e-4, n).astype(np.float32)
+    for ppm in (900_000, 990_000, 999_000):
+        k = orc.kept_count(n, ppm)
+        out = orc.compress(g, r, [0, n], [0, n], ppm)
+        a = np.abs(g + r)
+        tau_f = np.partition(a, n - k)[n - k]
+        assert np.uint32(out["tau"][0]).view(np.float32) == tau_f
+        tv = torch.kthvalue(torch.from_numpy(a), n - k + 1).values.item()
+        assert np.uint32(out["tau"][0]).view(np.float32) == np.float32(tv)
+        if np.unique(a).size == n:                                # tie-free: top-k set is unique
+            top = torch.topk(torch.from_numpy(a), k).indices.numpy()
+            assert np.array_equal(np.sort(top), out["idx"].astype(np.int64))
+        mask = np.zeros(n, dtype=bool)
+        mask[out["idx"]] = True
+        assert np.array_equal(np.flatnonzero(mask), out["idx"].astype(np.int64))
+
+
+def test_select_method_equals_sort_method():
+    rng = np.random.default_rng(9)
+    n = 1 << 20
+    g = rng.laplace(0, 1e-3, n).astype(np.float32)
+    g[rng.random(n) < 0.6] = 0.0
+    r = np.zeros(n, dtype=np.float32)
+    layer_off = [0, 1000, 1000, 300_000, n]
+    for scope_mode in (orc.SCOPE_GLOBAL, orc.SCOPE_PER_LAYER):
+        for ppm in (300_000, 990_000):                            # 30 % drop cuts inside the zero ties
+            a = orc.compress(g, r, layer_off, [0, n], ppm, scope_mode=scope_mode, method="sort")
+            b = orc.compress(g, r, layer_off, [0, n], ppm, scope_mode=scope_mode, method="select")
+            for key in ("idx", "val", "residual", "tau", "shard_cnt_off"):
+                assert np.array_equal(a[key].view(np.uint32), b[key].view(np.uint32))
+
+
+# ---------------------------------------------------------------- error feedback over steps
+def test_nothing_is_lost_over_steps():
+    """Integer-valued gradients make every fp32 add exact: sent mass + residual == sum of gradients."""
+    rng = np.random.default_rng(3)
+    n, steps = 4096, 12
+    layer_off, shard_off = [0, 100, n], [0, n // 2, n]
+    r = orc.residual_reset(n)
+    sent = np.zeros(n, dtype=np.int64)
+    total = np.zeros(n, dtype=np.int64)
+    for _ in range(steps):
+        g = rng.integers(-1024, 1025, n).astype(np.float32)
+        total += g.astype(np.int64)
+        out = orc.compress(g, r, layer_off, shard_off, 990_000, scope_mode=orc.SCOPE_PER_LAYER)
+        sent[out["idx"]] += out["val"].astype(np.int64)
+        r = out["residual"]
+    assert np.array_equal(sent + r.astype(np.int64), total)
+    assert np.abs(r).max() > 1024                                 # residuals really accumulated
+
+
+# ---------------------------------------------------------------- two-value quantisation
+def test_two_means_closed_form_and_independent_sum():
+    rng = np.random.default_rng(21)
+    layer_off = [0, 300, 300, 1000]
+    n = layer_off[-1]
+    g = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    big = rng.choice(n, 64, replace=False)
+    g[big] = np.where(rng.random(64) < 0.5, 2.5, -1.5).astype(np.float32)   # kept values are exactly +2.5 / -1.5
+    r = np.zeros(n, dtype=np.float32)
+    out = orc.compress(g, r, layer_off, [0, 500, n], 950_000, scope_mode=orc.SCOPE_GLOBAL,
+                       value_mode=orc.VALUES_TWO_MEANS)
+    k = orc.kept_count(n, 950_000)
+    assert k == 50
+    pos = (out["idx"] & np.uint32(0x7FFFFFFF)).astype(np.int64)
+    sign = out["idx"] >> np.uint32(31)
+    assert set(pos.tolist()) <= set(big.tolist())
+    assert np.array_equal(sign, (g[pos] < 0).astype(np.uint32))
+    for li in (0, 2):
+        in_l = (pos >= layer_off[li]) & (pos < layer_off[li + 1])
+        for sg, c in ((0, 2.5), (1, -1.5)):
+            cnt = int(np.sum(in_l & (sign == sg)))
+            assert out["counts"][li, sg] == cnt
+            assert out["means"][li, sg] == (np.float32(c) if cnt else np.float32(0.0))
+    assert out["counts"][1].tolist() == [0, 0] and out["means"][1].tolist() == [0.0, 0.0]
+    assert out["counts"].sum() == k
+    # residual holds the dropped mass only (the quantisation error is not fed back)
+    plain = orc.compress(g, r, layer_off, [0, 500, n], 950_000)
+    assert np.array_equal(plain["residual"].view(np.uint32), out["residual"].view(np.uint32))
+    assert np.array_equal(plain["idx"], pos.astype(np.uint32))
+
+    # general values: means against exactly rounded sums (math.fsum), independent of numpy's add
+    g2 = rng.laplace(0, 1e-3, n).astype(np.float32)
+    out2 = orc.compress(g2, r, layer_off, [0, n], 900_000, scope_mode=orc.SCOPE_PER_LAYER,
+                        value_mode=orc.VALUES_TWO_MEANS)
+    pos2 = (out2["idx"] & np.uint32(0x7FFFFFFF)).astype(np.int64)
+    for li in range(3):
+        for sg in (0, 1):
+            sel = [float(g2[p]) for p in pos2 if layer_off[li] <= p < layer_off[li + 1]
+                   and (f32_bits(g2[p]) >> 31) == sg]
+            want = np.float32(math.fsum(sel) / len(sel)) if sel else np.float32(0)
+            assert abs(float(out2["means"][li, sg]) - float(want)) <= 1e-6 * abs(float(want))
+
+
+# ---------------------------------------------------------------- server-side apply
+def test_apply_against_exact_rationals():
+    rng = np.random.default_rng(8)
+    n, shard_start, shard_len = 600, 150, 300
+    p0 = (rng.standard_normal(shard_len) * 0.01).astype(np.float32)
+    pushes = []
+    for w in range(3):
+        g = rng.laplace(0, 1e-3, n).astype(np.float32)
+        out = orc.compress(g, np.zeros(n, np.float32), [0, n], [0, n], 900_000)
+        pushes.append({"idx": out["idx"], "val": out["val"]})
+    alpha = 0.5
+    ref, bound = orc.apply_pushes(p0, shard_start, pushes, alpha=alpha)
+    exact = [Fraction(float(x)) for x in p0]
+    mag = [abs(Fraction(float(x))) for x in p0]
+    for push in pushes:
+        for i, x in zip(push["idx"].tolist(), push["val"].tolist()):
+            if shard_start <= i < shard_start + shard_len:
+                exact[i - shard_start] += Fraction(alpha) * Fraction(x)
+                mag[i - shard_start] += abs(Fraction(alpha) * Fraction(x))
+    for j in range(shard_len):
+        assert abs(Fraction(float(ref[j])) - exact[j]) <= Fraction(1, 10**14) * max(mag[j], Fraction(1, 10**30))
+        assert abs(Fraction(float(bound[j])) - mag[j]) <= Fraction(1, 10**14) * max(mag[j], Fraction(1, 10**30))
+
+
+def test_apply_two_means_decode():
+    layer_off = [0, 4, 10]
+    means = np.array([[0.5, -0.25], [2.0, -3.0]], dtype=np.float32)
+    idx = np.array([1, 3 | (1 << 31), 4 | (1 << 31), 9], dtype=np.uint32)
+    pos, val = orc.decode_push(idx, None, orc.VALUES_TWO_MEANS, means, layer_off)
+    assert pos.tolist() == [1, 3, 4, 9] and val.tolist() == [0.5, -0.25, -3.0, 2.0]
+    ref, _ = orc.apply_pushes(np.ones(6, np.float32), 4, [{"idx": idx, "means": means}],
+                              value_mode=orc.VALUES_TWO_MEANS, layer_off=layer_off)
+    assert ref.tolist() == [-2.0, 1.0, 1.0, 1.0, 1.0, 3.0]
