@@ -1,0 +1,203 @@
+/*
+ * gd.h - C ABI of the gradient-dropping library (libgd.so, CUDA, sm_100a).
+ *
+ * The library implements the hot path of "Sparse Communication for Distributed Gradient
+ * Descent" (Aji & Heafield, EMNLP 2017): Algorithm 1 (GradDrop) on the worker side and the
+ * decompress + scatter-add of sparse pushes on the server side (Section 3).
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory of the current device; "HOST" pointers are
+ *     ordinary host memory that is read before the call returns.
+ *   - A stream argument is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - Unless stated otherwise a call only enqueues work on the stream and returns; it never
+ *     synchronises and never allocates or frees device memory.  All device buffers, the
+ *     residual and the workspace included, are owned by the caller.
+ *   - Every function returns a gd_status_t.  Argument errors are detected on the host before
+ *     anything is enqueued.  Conditions detected on the device (a bounded wait that ran out,
+ *     an inconsistent count) are written to a status word in the workspace and are returned
+ *     by gd_status(); device code never traps, asserts or spins without a limit.
+ *   - No CUDA headers are needed to include this file.
+ */
+#ifndef GD_H
+#define GD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GD_OK = 0,
+  GD_ERR_INVALID_ARG = -1,    /* NULL / misaligned pointer, offsets not ascending, bad enum value */
+  GD_ERR_TOO_LARGE = -2,      /* n beyond what uint32 indices (or 31-bit packed indices) can address */
+  GD_ERR_WORKSPACE = -3,      /* workspace missing or smaller than gd_workspace_bytes() */
+  GD_ERR_CUDA = -4,           /* a CUDA runtime call failed (launch, memset, copy) */
+  GD_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait gave up; outputs of that call are invalid */
+  GD_ERR_INTERNAL = -6        /* device-side consistency check failed; outputs of that call are invalid */
+} gd_status_t;
+
+enum { GD_SCOPE_GLOBAL = 0, GD_SCOPE_PER_LAYER = 1 };
+enum { GD_VALUES_FP32 = 0, GD_VALUES_TWO_MEANS = 1 };
+
+/* gd_compress_args.flags */
+enum {
+  GD_FLAG_NO_PREDICTION = 1u  /* do not predict the threshold from a sample: always select over the
+                                 whole dense vector (same results, more memory traffic) */
+};
+
+const char* gd_status_string(int status);
+
+/*
+ * Entries kept in one threshold scope of n_scope elements when drop_ppm parts per million are
+ * dropped: k = n_scope - floor(n_scope * drop_ppm / 1e6), in 64-bit integers.
+ * Algorithm 1, "Select threshold: R% of |grad| is smaller"; R is passed as an integer so that
+ * every party computes the same count.  drop_ppm must be <= 1000000.
+ */
+int gd_kept_count(uint64_t n_scope, uint32_t drop_ppm, uint64_t* k_out);
+
+/*
+ * Total survivors of one gd_compress call, so that outputs can be sized before the launch.
+ * layer_off: HOST, n_layers + 1 ascending offsets (first 0, last n).  Section 4, last paragraph:
+ * the threshold is chosen "locally to each matrix" (GD_SCOPE_PER_LAYER: one scope per layer) or
+ * globally (GD_SCOPE_GLOBAL: one scope [0, n)).
+ */
+int gd_total_kept(const uint64_t* layer_off, uint32_t n_layers, int scope_mode, uint32_t drop_ppm,
+                  uint64_t* k_total_out);
+
+/* Bytes of device workspace gd_compress needs for these arguments (same meaning as in gd_compress_args). */
+int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, int scope_mode,
+                       uint32_t drop_ppm, size_t* bytes_out);
+
+/* Bytes of device workspace gd_decompress_apply needs. */
+int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes_out);
+
+/*
+ * gd_compress - Algorithm 1 (GradDrop) for one worker's flat fp32 gradient.
+ *
+ *   v[i]      = grad[i] + residual[i]                  (one fp32 add, round to nearest, no flush to zero)
+ *   per scope: keep exactly k entries, the largest by |v| (order: bit pattern of |v| descending,
+ *              then index ascending); tau = smallest kept |v| bit pattern (0xFFFFFFFF if k = 0)
+ *   out       = survivors of all scopes in ascending index: out_idx[t], out_val[t] = v[out_idx[t]]
+ *   residual  = v where dropped, +0.0f where kept      (Algorithm 1: residuals <- grad - dropped)
+ *   out_shard_cnt_off[j] = number of survivors with index < shard_off[j]   (Section 3: the
+ *              gradient is split into N pieces, one per server)
+ *   two-means mode (Section 5.4, quantisation by "the averages of values being quantized"): per
+ *              layer, mu+ = mean of kept v with sign bit 0 and mu- = mean of kept v with sign bit 1
+ *              (fp64 accumulation, rounded to fp32, +0.0f for an empty group); out_idx[t] carries
+ *              index | signbit << 31 and out_val is not written.  The residual is unchanged by the
+ *              value mode: it holds the dropped mass only.
+ *
+ * Results are bit-exact functions of (grad, residual, offsets, drop_ppm) except the two means,
+ * whose fp64 partial sums are combined in an unspecified order.  Non-finite inputs are ordered by
+ * their bit pattern (NaN above Inf above finite); NaN payloads follow the device's fp32 add.
+ * grad, residual, the outputs and the workspace must not overlap.  Calls that share a workspace
+ * must be ordered (same stream, or otherwise serialised).
+ */
+typedef struct gd_compress_args {
+  const float* grad;          /* device, n fp32, 16-byte aligned, read-only */
+  float* residual;            /* device, n fp32, 16-byte aligned, in/out */
+  uint64_t n;                 /* <= 2^32 (GD_VALUES_FP32) or <= 2^31 (GD_VALUES_TWO_MEANS) */
+  const uint64_t* layer_off;  /* HOST, n_layers + 1 ascending offsets, [0] = 0, last = n */
+  uint32_t n_layers;          /* >= 1 */
+  uint32_t n_shards;          /* >= 1 */
+  const uint64_t* shard_off;  /* HOST, n_shards + 1 ascending offsets, [0] = 0, last = n */
+  uint32_t drop_ppm;          /* 990000 = 99 %, 999000 = 99.9 % */
+  int32_t scope_mode;         /* GD_SCOPE_* */
+  int32_t value_mode;         /* GD_VALUES_* */
+  uint32_t flags;             /* GD_FLAG_* */
+  uint32_t* out_idx;          /* device, gd_total_kept() words */
+  float* out_val;             /* device, gd_total_kept() fp32; may be NULL in two-means mode */
+  uint32_t* out_shard_cnt_off;/* device, n_shards + 1 words */
+  uint32_t* out_tau;          /* device, one word per scope (1, or n_layers); may be NULL */
+  float* out_means;           /* device, n_layers x 2 fp32 (mu+, mu-); two-means mode only */
+  void* workspace;            /* device, 256-byte aligned, >= gd_workspace_bytes() */
+  size_t workspace_bytes;
+} gd_compress_args;
+
+int gd_compress(const gd_compress_args* args, void* stream);
+
+/*
+ * One sparse push as produced by gd_compress (all pointers device memory).  The entries that
+ * are applied are [shard_cnt_off[0], shard_cnt_off[n_shards]) of idx / val, n_shards being the
+ * shard count of the gd_apply_args the push is used with.  A server that owns one shard j passes
+ * the worker's out_shard_cnt_off + j.
+ */
+typedef struct gd_push {
+  const uint32_t* idx;
+  const float* val;              /* NULL in two-means mode */
+  const uint32_t* shard_cnt_off;
+  const float* means;            /* n_layers x 2, two-means mode only */
+} gd_push;
+
+/*
+ * gd_decompress_apply - the server side of Section 3: each server owns 1/N of the parameters
+ * and adds the pushed pieces into it.  For every push in array order and every entry of it
+ * whose index lies in a shard [shard_off[j], shard_off[j+1]):
+ *     params[j][index - shard_off[j]] += alpha * value
+ * with value = val[t] (fp32 mode) or the mean of the entry's layer and sign (two-means mode).
+ * One fused multiply-add in fp32 per entry; with alpha = 1 the result is fl32(p + value).
+ * Pushes are applied one after another in stream order; indices inside one push are unique.
+ * Entries whose index lies outside every shard are skipped.  The optimiser is not part of
+ * this library.
+ */
+typedef struct gd_apply_args {
+  float* const* params;        /* HOST array of n_shards device pointers */
+  const uint64_t* shard_off;   /* HOST, n_shards + 1 ascending global offsets */
+  uint32_t n_shards;
+  uint32_t n_pushes;
+  const gd_push* pushes;       /* HOST array of n_pushes */
+  int32_t value_mode;          /* GD_VALUES_* */
+  float alpha;
+  const uint64_t* layer_off;   /* HOST, n_layers + 1; two-means mode only */
+  uint32_t n_layers;
+  uint32_t reserved;
+  void* workspace;             /* device, 256-byte aligned, >= gd_apply_workspace_bytes() */
+  size_t workspace_bytes;
+} gd_apply_args;
+
+int gd_decompress_apply(const gd_apply_args* args, void* stream);
+
+/* residual <- +0.0f: the state before the first step, when nothing has been dropped yet (Section 4). */
+int gd_residual_reset(float* residual, uint64_t n, void* stream);
+
+/*
+ * Synchronises the stream and returns the device status word the last gd_compress left in this
+ * workspace (GD_OK, GD_ERR_DEVICE_TIMEOUT or GD_ERR_INTERNAL), or GD_ERR_CUDA.
+ */
+int gd_status(const void* workspace, void* stream);
+
+/* Diagnostics of the last gd_compress on this workspace (synchronises the stream). */
+typedef struct gd_stats {
+  int32_t status;
+  uint32_t n_scopes;
+  uint32_t n_scopes_predicted;  /* scopes whose threshold was found from the predicted candidate list */
+  uint32_t n_scopes_dense;      /* scopes that needed selection over the whole dense range */
+  uint64_t n_candidates;        /* candidates emitted by the fused pass, over all scopes */
+  uint64_t n_kept;              /* survivors written */
+} gd_stats;
+
+int gd_get_stats(const void* workspace, void* stream, gd_stats* out);
+
+/*
+ * gd_step_host - one whole step for a caller whose gradient lives in host memory: copies grad_host
+ * to the device buffer args->grad, runs gd_compress and then gd_decompress_apply (apply may be
+ * NULL), and copies the push (indices, values or means, shard offsets) back to the host buffers.
+ * Synchronises the stream before returning.  Host buffers should be page-locked for full copy
+ * bandwidth.  k_total = gd_total_kept() entries are copied to idx_host / val_host.
+ */
+typedef struct gd_host_io {
+  const float* grad_host;        /* HOST, n fp32 */
+  uint32_t* idx_host;            /* HOST, k_total words, or NULL */
+  float* val_host;               /* HOST, k_total fp32, or NULL */
+  uint32_t* shard_cnt_off_host;  /* HOST, n_shards + 1 words, or NULL */
+  float* means_host;             /* HOST, n_layers x 2 fp32, or NULL */
+} gd_host_io;
+
+int gd_step_host(const gd_compress_args* args, const gd_apply_args* apply, const gd_host_io* io, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GD_H */

@@ -1,0 +1,358 @@
+// Host side of libgd.so: argument checks, the per-call plan (scopes, tile tables, workspace
+// layout) and the C entry points declared in include/gd.h.
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "gd_internal.cuh"
+
+namespace gd {
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+inline uint64_t kept_count(uint64_t n, uint32_t drop_ppm) {
+  return n - (n * (uint64_t)drop_ppm) / 1000000ull;   // n <= 2^32, drop_ppm <= 1e6: no overflow
+}
+
+// How one scope is sampled for the prediction and how many candidate slots it gets.  A scope of
+// ns elements keeping k: m stratified samples are read and the predicted lower bound is the rank-th
+// largest sample key.  rank is chosen so that, for independent samples, the number of entries at or
+// above the prediction is at least k with a margin of six standard deviations plus 12.5 %.  Small
+// scopes are sampled completely, which makes the prediction the exact threshold.  None of this
+// affects results: a scope whose prediction fails is selected densely.
+void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint64_t* cap) {
+  if (k == 0 || ns == 0) { *m = 0; *rank = 0; *cap = 0; return; }
+  double target = 1024.0 * (double)ns / (double)k;
+  if (target < 32768.0) target = 32768.0;
+  if (target > 1048576.0) target = 1048576.0;
+  const uint64_t mt = (uint64_t)target;
+  if (mt * 2 >= ns) {
+    *m = ns;
+    *rank = k;
+    uint64_t c = 2 * k + 1024;
+    *cap = c < ns ? c : ns;
+    return;
+  }
+  *m = mt;
+  const double x = (double)k * (double)mt / (double)ns;
+  const double y = 3.0 + std::sqrt(9.0 + 1.125 * x + 1.0);
+  uint64_t r = (uint64_t)std::ceil(y * y);
+  if (r > mt) r = mt;
+  if (r < 1) r = 1;
+  *rank = r;
+  uint64_t c = 2 * k + 128 * (ns / mt) + 1024;
+  *cap = c < ns ? c : ns;
+}
+
+struct Plan {
+  std::vector<ScopeDesc> scopes;
+  std::vector<uint32_t> tile0[L_COUNT];
+  std::vector<uint64_t> samp_off;
+  uint32_t tiles[L_COUNT] = {0, 0, 0, 0, 0};
+  uint64_t samp_total = 0, cand_total = 0, k_total = 0;
+  uint32_t n_scopes = 0;
+  // workspace layout (byte offsets)
+  size_t off_ctl = 0, off_state = 0, off_hist = 0, off_sums = 0, off_cnts = 0, off_desc_emit = 0,
+         off_desc_cand = 0, off_desc_dcomp = 0, zero_bytes = 0;
+  size_t off_tables = 0, tables_bytes = 0;
+  size_t t_scopes = 0, t_tile0[L_COUNT] = {0, 0, 0, 0, 0}, t_samp_off = 0, t_layer_off = 0, t_shard_off = 0;
+  size_t off_samp = 0, off_cand_idx = 0, off_cand_val = 0, total_bytes = 0;
+};
+
+int check_offsets(const uint64_t* off, uint32_t count, uint64_t* n_out) {
+  if (!off || count == 0) return GD_ERR_INVALID_ARG;
+  if (off[0] != 0) return GD_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < count; ++i)
+    if (off[i + 1] < off[i]) return GD_ERR_INVALID_ARG;
+  *n_out = off[count];
+  return GD_OK;
+}
+
+int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, int scope_mode, uint32_t drop_ppm,
+              uint32_t flags, Plan* P) {
+  uint64_t n = 0;
+  int rc = check_offsets(layer_off, n_layers, &n);
+  if (rc != GD_OK) return rc;
+  if (n_shards == 0 || drop_ppm > 1000000u) return GD_ERR_INVALID_ARG;
+  if (scope_mode != GD_SCOPE_GLOBAL && scope_mode != GD_SCOPE_PER_LAYER) return GD_ERR_INVALID_ARG;
+  if (n > (1ull << 32)) return GD_ERR_TOO_LARGE;
+  const bool predict = !(flags & GD_FLAG_NO_PREDICTION);
+  const uint32_t ns_count = scope_mode == GD_SCOPE_GLOBAL ? 1u : n_layers;
+  P->n_scopes = ns_count;
+  P->scopes.resize(ns_count);
+  for (int l = 0; l < L_COUNT; ++l) P->tile0[l].assign(ns_count + 1, 0);
+  P->samp_off.assign(ns_count + 1, 0);
+  uint64_t tiles[L_COUNT] = {0, 0, 0, 0, 0};
+  uint64_t out_base = 0, cand_base = 0, samp_base = 0;
+  for (uint32_t s = 0; s < ns_count; ++s) {
+    ScopeDesc& d = P->scopes[s];
+    d.lo = scope_mode == GD_SCOPE_GLOBAL ? 0 : layer_off[s];
+    d.hi = scope_mode == GD_SCOPE_GLOBAL ? n : layer_off[s + 1];
+    const uint64_t ns = d.hi - d.lo;
+    d.k = kept_count(ns, drop_ppm);
+    d.out_base = out_base;
+    out_base += d.k;
+    uint64_t m = 0, rank = 0, cap = 0;
+    if (predict) plan_prediction(ns, d.k, &m, &rank, &cap);
+    d.cand_base = cand_base;
+    d.cand_cap = cap;
+    cand_base += (cap + 3) / 4 * 4;
+    d.samp_base = samp_base;
+    d.samp_m = m;
+    d.samp_rank = rank;
+    samp_base += m;
+    for (int l = 0; l < L_COUNT; ++l) P->tile0[l][s] = (uint32_t)tiles[l];
+    P->samp_off[s] = d.samp_base;
+    if (ns) {
+      tiles[L_EMIT] += (d.hi + kTile - 1) / kTile - d.lo / kTile;
+      tiles[L_DSEL] += (ns + kDenseSelTile - 1) / kDenseSelTile;
+      tiles[L_DCOMP] += (ns + kTile - 1) / kTile;
+    }
+    tiles[L_SAMP] += (m + kTile - 1) / kTile;
+    tiles[L_CAND] += (cap + kTile - 1) / kTile;
+  }
+  for (int l = 0; l < L_COUNT; ++l) {
+    if (tiles[l] > 0x7FFFFFFFull) return GD_ERR_TOO_LARGE;
+    P->tile0[l][ns_count] = (uint32_t)tiles[l];
+    P->tiles[l] = (uint32_t)tiles[l];
+  }
+  P->samp_off[ns_count] = samp_base;
+  P->samp_total = samp_base;
+  P->cand_total = cand_base;
+  P->k_total = out_base;
+
+  size_t off = 0;
+  P->off_ctl = off;          off = align_up(off + sizeof(Ctl));
+  P->off_state = off;        off = align_up(off + sizeof(ScopeState) * ns_count);
+  P->off_hist = off;         off = align_up(off + sizeof(unsigned long long) * kRadixBins0 * (size_t)ns_count);
+  P->off_sums = off;         off = align_up(off + sizeof(double) * 2 * (size_t)n_layers);
+  P->off_cnts = off;         off = align_up(off + sizeof(unsigned long long) * 2 * (size_t)n_layers);
+  P->off_desc_emit = off;    off = align_up(off + 16 * (size_t)P->tiles[L_EMIT]);
+  P->off_desc_cand = off;    off = align_up(off + 16 * (size_t)P->tiles[L_CAND]);
+  P->off_desc_dcomp = off;   off = align_up(off + 16 * (size_t)P->tiles[L_DCOMP]);
+  P->zero_bytes = off;
+  P->off_tables = off;
+  size_t t = 0;
+  P->t_scopes = t;           t = align_up(t + sizeof(ScopeDesc) * ns_count);
+  for (int l = 0; l < L_COUNT; ++l) { P->t_tile0[l] = t; t = align_up(t + sizeof(uint32_t) * (ns_count + 1)); }
+  P->t_samp_off = t;         t = align_up(t + sizeof(uint64_t) * (ns_count + 1));
+  P->t_layer_off = t;        t = align_up(t + sizeof(uint64_t) * ((size_t)n_layers + 1));
+  P->t_shard_off = t;        t = align_up(t + sizeof(uint64_t) * ((size_t)n_shards + 1));
+  P->tables_bytes = t;
+  off += t;
+  P->off_samp = off;         off = align_up(off + sizeof(float) * P->samp_total);
+  P->off_cand_idx = off;     off = align_up(off + sizeof(uint32_t) * P->cand_total);
+  P->off_cand_val = off;     off = align_up(off + sizeof(float) * P->cand_total);
+  P->total_bytes = off;
+  return GD_OK;
+}
+
+}  // namespace
+
+}  // namespace gd
+
+using namespace gd;
+
+extern "C" {
+
+const char* gd_status_string(int status) {
+  switch (status) {
+    case GD_OK: return "ok";
+    case GD_ERR_INVALID_ARG: return "invalid argument";
+    case GD_ERR_TOO_LARGE: return "gradient too large for 32-bit indices";
+    case GD_ERR_WORKSPACE: return "workspace missing or too small";
+    case GD_ERR_CUDA: return "CUDA runtime error";
+    case GD_ERR_DEVICE_TIMEOUT: return "bounded device-side wait timed out";
+    case GD_ERR_INTERNAL: return "device-side consistency check failed";
+    default: return "unknown status";
+  }
+}
+
+int gd_kept_count(uint64_t n_scope, uint32_t drop_ppm, uint64_t* k_out) {
+  if (!k_out || drop_ppm > 1000000u) return GD_ERR_INVALID_ARG;
+  if (n_scope > (1ull << 32)) return GD_ERR_TOO_LARGE;
+  *k_out = kept_count(n_scope, drop_ppm);
+  return GD_OK;
+}
+
+int gd_total_kept(const uint64_t* layer_off, uint32_t n_layers, int scope_mode, uint32_t drop_ppm,
+                  uint64_t* k_total_out) {
+  if (!k_total_out || drop_ppm > 1000000u) return GD_ERR_INVALID_ARG;
+  if (scope_mode != GD_SCOPE_GLOBAL && scope_mode != GD_SCOPE_PER_LAYER) return GD_ERR_INVALID_ARG;
+  uint64_t n = 0;
+  int rc = check_offsets(layer_off, n_layers, &n);
+  if (rc != GD_OK) return rc;
+  if (n > (1ull << 32)) return GD_ERR_TOO_LARGE;
+  uint64_t total = 0;
+  if (scope_mode == GD_SCOPE_GLOBAL) {
+    total = kept_count(n, drop_ppm);
+  } else {
+    for (uint32_t l = 0; l < n_layers; ++l) total += kept_count(layer_off[l + 1] - layer_off[l], drop_ppm);
+  }
+  *k_total_out = total;
+  return GD_OK;
+}
+
+int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, int scope_mode,
+                       uint32_t drop_ppm, size_t* bytes_out) {
+  if (!bytes_out) return GD_ERR_INVALID_ARG;
+  try {
+    Plan P;
+    int rc = make_plan(layer_off, n_layers, n_shards, scope_mode, drop_ppm, 0u, &P);
+    if (rc != GD_OK) return rc;
+    *bytes_out = P.total_bytes;
+    return GD_OK;
+  } catch (const std::bad_alloc&) {
+    return GD_ERR_INVALID_ARG;
+  }
+}
+
+int gd_compress(const gd_compress_args* a, void* stream_v) {
+  if (!a) return GD_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  try {
+    Plan P;
+    int rc = make_plan(a->layer_off, a->n_layers, a->n_shards, a->scope_mode, a->drop_ppm, a->flags, &P);
+    if (rc != GD_OK) return rc;
+    uint64_t n_sh = 0;
+    rc = check_offsets(a->shard_off, a->n_shards, &n_sh);
+    if (rc != GD_OK) return rc;
+    const uint64_t n = a->layer_off[a->n_layers];
+    if (n_sh != n || a->n != n) return GD_ERR_INVALID_ARG;
+    if (a->value_mode != GD_VALUES_FP32 && a->value_mode != GD_VALUES_TWO_MEANS) return GD_ERR_INVALID_ARG;
+    if (a->value_mode == GD_VALUES_TWO_MEANS && n > (1ull << 31)) return GD_ERR_TOO_LARGE;
+    if (a->flags & ~(uint32_t)GD_FLAG_NO_PREDICTION) return GD_ERR_INVALID_ARG;
+    if (n && (!a->grad || !a->residual)) return GD_ERR_INVALID_ARG;
+    if (((uintptr_t)a->grad | (uintptr_t)a->residual) & 15u) return GD_ERR_INVALID_ARG;
+    if (!a->out_shard_cnt_off) return GD_ERR_INVALID_ARG;
+    if (P.k_total && !a->out_idx) return GD_ERR_INVALID_ARG;
+    if (P.k_total && a->value_mode == GD_VALUES_FP32 && !a->out_val) return GD_ERR_INVALID_ARG;
+    if (a->value_mode == GD_VALUES_TWO_MEANS && !a->out_means) return GD_ERR_INVALID_ARG;
+    if (!a->workspace || ((uintptr_t)a->workspace & (kAlign - 1))) return GD_ERR_WORKSPACE;
+    if (a->workspace_bytes < P.total_bytes) return GD_ERR_WORKSPACE;
+
+    // host image of the tables
+    std::vector<unsigned char> blob(P.tables_bytes, 0);
+    std::memcpy(blob.data() + P.t_scopes, P.scopes.data(), sizeof(ScopeDesc) * P.n_scopes);
+    for (int l = 0; l < L_COUNT; ++l)
+      std::memcpy(blob.data() + P.t_tile0[l], P.tile0[l].data(), sizeof(uint32_t) * (P.n_scopes + 1));
+    std::memcpy(blob.data() + P.t_samp_off, P.samp_off.data(), sizeof(uint64_t) * (P.n_scopes + 1));
+    std::memcpy(blob.data() + P.t_layer_off, a->layer_off, sizeof(uint64_t) * ((size_t)a->n_layers + 1));
+    std::memcpy(blob.data() + P.t_shard_off, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
+
+    unsigned char* ws = (unsigned char*)a->workspace;
+    if (cudaMemsetAsync(ws, 0, P.zero_bytes, stream) != cudaSuccess) return GD_ERR_CUDA;
+    if (cudaMemcpyAsync(ws + P.off_tables, blob.data(), P.tables_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      return GD_ERR_CUDA;
+
+    DevTables T;
+    std::memset(&T, 0, sizeof(T));
+    T.grad = a->grad;
+    T.residual = a->residual;
+    T.n = n;
+    T.n_scopes = P.n_scopes;
+    T.n_layers = a->n_layers;
+    T.n_shards = a->n_shards;
+    T.flags = a->flags;
+    T.value_mode = a->value_mode;
+    T.k_total = P.k_total;
+    T.ctl = (Ctl*)(ws + P.off_ctl);
+    T.state = (ScopeState*)(ws + P.off_state);
+    T.hist = (unsigned long long*)(ws + P.off_hist);
+    T.sums = (double*)(ws + P.off_sums);
+    T.cnts = (unsigned long long*)(ws + P.off_cnts);
+    T.desc_emit = (uint64_t*)(ws + P.off_desc_emit);
+    T.desc_cand = (uint64_t*)(ws + P.off_desc_cand);
+    T.desc_dcomp = (uint64_t*)(ws + P.off_desc_dcomp);
+    const unsigned char* tb = ws + P.off_tables;
+    T.scopes = (const ScopeDesc*)(tb + P.t_scopes);
+    for (int l = 0; l < L_COUNT; ++l) T.tile0[l] = (const uint32_t*)(tb + P.t_tile0[l]);
+    T.samp_off = (const uint64_t*)(tb + P.t_samp_off);
+    T.layer_off = (const uint64_t*)(tb + P.t_layer_off);
+    T.shard_off = (const uint64_t*)(tb + P.t_shard_off);
+    T.samp_val = (float*)(ws + P.off_samp);
+    T.cand_idx = (uint32_t*)(ws + P.off_cand_idx);
+    T.cand_val = (float*)(ws + P.off_cand_val);
+    T.out_idx = a->out_idx;
+    T.out_val = a->out_val;
+    T.out_shard_cnt_off = a->out_shard_cnt_off;
+    T.out_tau = a->out_tau;
+    T.out_means = a->out_means;
+
+    uint32_t tiles[L_COUNT];
+    for (int l = 0; l < L_COUNT; ++l) tiles[l] = P.tiles[l];
+    if (!(a->flags & GD_FLAG_NO_PREDICTION)) {
+      // dense kernels are still enqueued: they return at once unless a prediction failed
+    } else {
+      tiles[L_SAMP] = 0;
+      tiles[L_CAND] = 0;
+    }
+    if (launch_compress(T, tiles, P.samp_total, stream) != cudaSuccess) return GD_ERR_CUDA;
+    return GD_OK;
+  } catch (const std::bad_alloc&) {
+    return GD_ERR_INVALID_ARG;
+  }
+}
+
+int gd_residual_reset(float* residual, uint64_t n, void* stream) {
+  if (n == 0) return GD_OK;
+  if (!residual) return GD_ERR_INVALID_ARG;
+  if (cudaMemsetAsync(residual, 0, sizeof(float) * n, (cudaStream_t)stream) != cudaSuccess) return GD_ERR_CUDA;
+  return GD_OK;
+}
+
+int gd_get_stats(const void* workspace, void* stream, gd_stats* out) {
+  if (!workspace || !out) return GD_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return GD_ERR_CUDA;
+  Ctl c;
+  if (cudaMemcpy(&c, workspace, sizeof(Ctl), cudaMemcpyDeviceToHost) != cudaSuccess) return GD_ERR_CUDA;
+  out->status = c.status;
+  out->n_scopes = c.n_scopes;
+  out->n_scopes_predicted = c.n_scopes_predicted;
+  out->n_scopes_dense = c.n_scopes_dense;
+  out->n_candidates = c.n_candidates;
+  out->n_kept = c.n_kept;
+  return GD_OK;
+}
+
+int gd_status(const void* workspace, void* stream) {
+  gd_stats s;
+  int rc = gd_get_stats(workspace, stream, &s);
+  return rc != GD_OK ? rc : s.status;
+}
+
+int gd_step_host(const gd_compress_args* a, const gd_apply_args* apply, const gd_host_io* io, void* stream_v) {
+  if (!a || !io || !io->grad_host) return GD_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  uint64_t k_total = 0;
+  int rc = gd_total_kept(a->layer_off, a->n_layers, a->scope_mode, a->drop_ppm, &k_total);
+  if (rc != GD_OK) return rc;
+  if (a->n && cudaMemcpyAsync((void*)a->grad, io->grad_host, sizeof(float) * a->n, cudaMemcpyHostToDevice, stream) !=
+                  cudaSuccess)
+    return GD_ERR_CUDA;
+  rc = gd_compress(a, stream_v);
+  if (rc != GD_OK) return rc;
+  if (apply) {
+    rc = gd_decompress_apply(apply, stream_v);
+    if (rc != GD_OK) return rc;
+  }
+  cudaError_t e = cudaSuccess;
+  if (io->idx_host && k_total)
+    e = cudaMemcpyAsync(io->idx_host, a->out_idx, sizeof(uint32_t) * k_total, cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess && io->val_host && k_total && a->value_mode == GD_VALUES_FP32)
+    e = cudaMemcpyAsync(io->val_host, a->out_val, sizeof(float) * k_total, cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess && io->shard_cnt_off_host)
+    e = cudaMemcpyAsync(io->shard_cnt_off_host, a->out_shard_cnt_off, sizeof(uint32_t) * ((size_t)a->n_shards + 1),
+                        cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess && io->means_host && a->value_mode == GD_VALUES_TWO_MEANS)
+    e = cudaMemcpyAsync(io->means_host, a->out_means, sizeof(float) * 2 * (size_t)a->n_layers, cudaMemcpyDeviceToHost,
+                        stream);
+  if (e != cudaSuccess) return GD_ERR_CUDA;
+  return gd_status(a->workspace, stream_v);
+}
+
+}  // extern "C"

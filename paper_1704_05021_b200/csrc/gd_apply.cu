@@ -1,0 +1,141 @@
+// gd_decompress_apply: the server side of the parameter-sharded exchange (Section 3 of Aji &
+// Heafield 2017).  Each push is a list of (index, value) survivors; every entry is routed to the
+// shard that owns its index and added to that shard's parameters.
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "gd_internal.cuh"
+
+namespace gd {
+
+namespace {
+
+constexpr size_t kAlignA = 256;
+inline size_t align_up_a(size_t x) { return (x + kAlignA - 1) / kAlignA * kAlignA; }
+
+struct ApplyDev {
+  float* const* params;        // [n_shards] device pointers
+  const uint64_t* shard_off;   // [n_shards + 1]
+  const uint64_t* layer_off;   // [n_layers + 1] (two-means mode)
+  uint32_t n_shards, n_layers;
+  int32_t value_mode;
+  float alpha;
+  const uint32_t* idx;
+  const float* val;
+  const uint32_t* cnt_off;
+  const float* means;
+};
+
+// Segmented scatter-add: the entries [cnt_off[0], cnt_off[n_shards]) of one push, one thread per
+// entry in a grid-stride loop.  Indices inside one push are unique, so a plain read-modify-write is
+// enough; pushes are separate launches in stream order.
+__global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__ ApplyDev A) {
+  const uint64_t begin = A.cnt_off[0], end = A.cnt_off[A.n_shards];
+  const uint64_t lo_all = A.shard_off[0], hi_all = A.shard_off[A.n_shards];
+  const uint64_t stride = (uint64_t)gridDim.x * kThreads;
+  for (uint64_t p = begin + (uint64_t)blockIdx.x * kThreads + threadIdx.x; p < end; p += stride) {
+    const uint32_t w = __ldcs(A.idx + p);
+    uint64_t pos = w;
+    float x;
+    if (A.value_mode == GD_VALUES_TWO_MEANS) {
+      pos = w & kAbsMask;
+      const uint32_t l = range_of(A.layer_off, A.n_layers, pos);
+      x = __ldg(A.means + 2 * (size_t)l + (w >> 31));
+    } else {
+      x = __ldcs(A.val + p);
+    }
+    if (pos < lo_all || pos >= hi_all) continue;
+    const uint32_t j = range_of(A.shard_off, A.n_shards, pos);
+    float* dst = A.params[j] + (pos - A.shard_off[j]);
+    *dst = __fmaf_rn(A.alpha, x, *dst);
+  }
+}
+
+int g_sm_count = 0;
+
+}  // namespace
+
+}  // namespace gd
+
+using namespace gd;
+
+extern "C" {
+
+int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes_out) {
+  if (!bytes_out || n_shards == 0) return GD_ERR_INVALID_ARG;
+  size_t b = align_up_a(sizeof(float*) * (size_t)n_shards);
+  b += align_up_a(sizeof(uint64_t) * ((size_t)n_shards + 1));
+  b += align_up_a(sizeof(uint64_t) * ((size_t)n_layers + 1));
+  *bytes_out = b;
+  return GD_OK;
+}
+
+int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
+  if (!a || !a->params || !a->shard_off || a->n_shards == 0) return GD_ERR_INVALID_ARG;
+  if (a->n_pushes && !a->pushes) return GD_ERR_INVALID_ARG;
+  if (a->value_mode != GD_VALUES_FP32 && a->value_mode != GD_VALUES_TWO_MEANS) return GD_ERR_INVALID_ARG;
+  const bool two_means = a->value_mode == GD_VALUES_TWO_MEANS;
+  if (two_means && (!a->layer_off || a->n_layers == 0)) return GD_ERR_INVALID_ARG;
+  for (uint32_t j = 0; j < a->n_shards; ++j) {
+    if (a->shard_off[j + 1] < a->shard_off[j]) return GD_ERR_INVALID_ARG;
+    if (a->shard_off[j + 1] > a->shard_off[j] && !a->params[j]) return GD_ERR_INVALID_ARG;
+  }
+  if (a->shard_off[a->n_shards] > (1ull << 32)) return GD_ERR_TOO_LARGE;
+  if (two_means)
+    for (uint32_t l = 0; l < a->n_layers; ++l)
+      if (a->layer_off[l + 1] < a->layer_off[l]) return GD_ERR_INVALID_ARG;
+  for (uint32_t w = 0; w < a->n_pushes; ++w) {
+    const gd_push& p = a->pushes[w];
+    if (!p.idx || !p.shard_cnt_off) return GD_ERR_INVALID_ARG;
+    if (two_means ? !p.means : !p.val) return GD_ERR_INVALID_ARG;
+  }
+  const uint32_t n_layers = two_means ? a->n_layers : 0;
+  size_t need = 0;
+  gd_apply_workspace_bytes(a->n_shards, n_layers, &need);
+  if (!a->workspace || ((uintptr_t)a->workspace & (kAlignA - 1)) || a->workspace_bytes < need) return GD_ERR_WORKSPACE;
+  if (a->n_pushes == 0) return GD_OK;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  try {
+    const size_t o_params = 0;
+    const size_t o_shard = align_up_a(sizeof(float*) * (size_t)a->n_shards);
+    const size_t o_layer = o_shard + align_up_a(sizeof(uint64_t) * ((size_t)a->n_shards + 1));
+    std::vector<unsigned char> blob(need, 0);
+    std::memcpy(blob.data() + o_params, a->params, sizeof(float*) * (size_t)a->n_shards);
+    std::memcpy(blob.data() + o_shard, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
+    if (two_means) std::memcpy(blob.data() + o_layer, a->layer_off, sizeof(uint64_t) * ((size_t)n_layers + 1));
+    unsigned char* ws = (unsigned char*)a->workspace;
+    if (cudaMemcpyAsync(ws, blob.data(), need, cudaMemcpyHostToDevice, stream) != cudaSuccess) return GD_ERR_CUDA;
+
+    if (g_sm_count == 0) {
+      int dev = 0, sms = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return GD_ERR_CUDA;
+      g_sm_count = sms;
+    }
+    ApplyDev A;
+    std::memset(&A, 0, sizeof(A));
+    A.params = (float* const*)(ws + o_params);
+    A.shard_off = (const uint64_t*)(ws + o_shard);
+    A.layer_off = (const uint64_t*)(ws + o_layer);
+    A.n_shards = a->n_shards;
+    A.n_layers = n_layers;
+    A.value_mode = a->value_mode;
+    A.alpha = a->alpha;
+    for (uint32_t w = 0; w < a->n_pushes; ++w) {
+      const gd_push& p = a->pushes[w];
+      A.idx = p.idx;
+      A.val = p.val;
+      A.cnt_off = p.shard_cnt_off;
+      A.means = p.means;
+      apply_kernel<<<(unsigned)g_sm_count * 8u, kThreads, 0, stream>>>(A);
+      if (cudaPeekAtLastError() != cudaSuccess) return GD_ERR_CUDA;
+    }
+    return GD_OK;
+  } catch (const std::bad_alloc&) {
+    return GD_ERR_INVALID_ARG;
+  }
+}
+
+}  // extern "C"

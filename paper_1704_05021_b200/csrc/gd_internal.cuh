@@ -1,0 +1,156 @@
+// Shared declarations of the gradient-dropping kernels (device tables, workspace layout,
+// small PTX helpers).  Internal to libgd.so; the public interface is include/gd.h.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gd.h"
+
+namespace gd {
+
+constexpr int kThreads = 256;           // threads per CTA in every tiled kernel
+constexpr int kWarps = kThreads / 32;
+constexpr uint32_t kTile = 4096;        // elements per tile of the streaming kernels
+constexpr uint32_t kDenseSelTile = 32768;  // elements per CTA in the dense histogram passes
+constexpr int kRadixBits0 = 11;         // 31-bit magnitude key = 11 + 10 + 10 bits
+constexpr int kRadixBins0 = 1 << kRadixBits0;
+constexpr int kShift0 = 20, kShift1 = 10, kShift2 = 0;
+constexpr uint32_t kAbsMask = 0x7FFFFFFFu;
+constexpr uint32_t kLookbackSpinLimit = 1u << 21;  // polls before a look-back wait gives up
+
+// Kinds of tiled launches; each has its own tile -> scope table.
+enum Launch : int { L_EMIT = 0, L_SAMP = 1, L_CAND = 2, L_DSEL = 3, L_DCOMP = 4, L_COUNT = 5 };
+// Views a selection can run over.
+enum View : int { V_SAMPLE = 0, V_CAND = 1, V_DENSE = 2 };
+
+// Look-back descriptor flags (low two bits of a 64-bit word; the count sits above them).
+enum : uint64_t { F_INVALID = 0, F_AGG = 1, F_PREFIX = 2, F_ABORT = 3 };
+
+struct ScopeDesc {       // built on the host for every call, read-only on the device
+  uint64_t lo, hi;       // element range [lo, hi) of the scope in the flat gradient
+  uint64_t k;            // entries kept
+  uint64_t out_base;     // first slot of the scope in out_idx / out_val
+  uint64_t cand_base;    // first slot of the scope in the candidate buffers
+  uint64_t cand_cap;     // slots reserved for the scope's candidates
+  uint64_t samp_base;    // first slot of the scope in the sample buffer
+  uint64_t samp_m;       // samples drawn from the scope
+  uint64_t samp_rank;    // the prediction is the samp_rank-th largest sample key
+};
+
+struct SelState {        // running state of one radix selection
+  uint32_t prefix;       // digits fixed so far
+  uint32_t pad;
+  uint64_t rank;         // rank still to find inside the prefix bucket
+  uint64_t gt;           // elements strictly above the prefix bucket so far
+};
+
+struct ScopeState {      // zeroed at the start of every call
+  uint64_t cand_count;   // candidates the fused pass counted (may exceed cand_cap)
+  uint32_t tau_lo;       // predicted lower bound of the threshold key
+  uint32_t tau;          // threshold key: smallest kept |v| bit pattern
+  uint64_t q;            // ties at tau that are kept (the lowest indices)
+  uint64_t gt;           // entries with key > tau
+  SelState sel[3];       // one per view
+  uint32_t done[3][3];   // finished tiles per view and pass
+  uint32_t used_dense;   // 1 if the dense path produced this scope's result
+};
+
+struct Ctl {             // zeroed at the start of every call
+  int32_t status;
+  uint32_t ticket[L_COUNT];
+  uint32_t n_scopes;
+  uint32_t n_scopes_predicted;
+  uint32_t n_scopes_dense;
+  uint32_t pad;
+  uint64_t n_candidates;
+  uint64_t n_kept;
+};
+
+struct DevTables {       // passed by value to every kernel
+  const float* grad;
+  float* residual;
+  uint64_t n;
+  uint32_t n_scopes, n_layers, n_shards;
+  uint32_t flags;
+  int32_t value_mode;
+  uint32_t pad;
+  uint64_t k_total;
+  // zeroed region
+  Ctl* ctl;
+  ScopeState* state;
+  unsigned long long* hist;          // [n_scopes][kRadixBins0]
+  double* sums;                      // [n_layers][2]
+  unsigned long long* cnts;          // [n_layers][2]
+  uint64_t* desc_emit;               // [tiles(L_EMIT)]
+  uint64_t* desc_cand;               // [tiles(L_CAND)][2]
+  uint64_t* desc_dcomp;              // [tiles(L_DCOMP)][2]
+  // uploaded tables
+  const ScopeDesc* scopes;           // [n_scopes]
+  const uint32_t* tile0[L_COUNT];    // [n_scopes + 1] first tile of each scope per launch kind
+  const uint64_t* samp_off;          // [n_scopes + 1]
+  const uint64_t* layer_off;         // [n_layers + 1]
+  const uint64_t* shard_off;         // [n_shards + 1]
+  // buffers
+  float* samp_val;
+  uint32_t* cand_idx;
+  float* cand_val;
+  // outputs
+  uint32_t* out_idx;
+  float* out_val;
+  uint32_t* out_shard_cnt_off;
+  uint32_t* out_tau;
+  float* out_means;
+};
+
+// ---------------------------------------------------------------- device helpers
+__device__ __forceinline__ uint64_t ld_relaxed_u64(const uint64_t* p) {
+  uint64_t v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(uint64_t* p, uint64_t v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31u; }
+__device__ __forceinline__ uint32_t lanemask_lt() {
+  uint32_t m;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+__device__ __forceinline__ uint64_t pack_desc(uint64_t flag, uint64_t value) { return (value << 2) | flag; }
+
+// Largest s in [0, n_scopes) with tile0[s] <= t (tile0 has n_scopes + 1 entries, ascending; scopes
+// without tiles repeat their successor's value, so the scope found is the one that owns tile t).
+__device__ __forceinline__ uint32_t scope_of_tile(const uint32_t* __restrict__ tile0, uint32_t n_scopes, uint32_t t) {
+  uint32_t lo = 0, hi = n_scopes;  // invariant: tile0[lo] <= t < tile0[hi]
+  while (hi - lo > 1) {
+    uint32_t mid = (lo + hi) >> 1;
+    if (__ldg(tile0 + mid) <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// Largest l in [0, count) with off[l] <= x, for ascending off[0..count] with off[0] <= x < off[count];
+// entries that repeat (empty ranges) resolve to the last one, i.e. the non-empty range holding x.
+__device__ __forceinline__ uint32_t range_of(const uint64_t* __restrict__ off, uint32_t count, uint64_t x) {
+  uint32_t lo = 0, hi = count;
+  while (hi - lo > 1) {
+    uint32_t mid = (lo + hi) >> 1;
+    if (__ldg(off + mid) <= x) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// True when the scope's result comes from the candidate list the fused pass emitted: the
+// prediction was a valid lower bound (at least k candidates) and the list did not overflow.
+__device__ __forceinline__ bool predicted_ok(const DevTables& T, const ScopeDesc& d, const ScopeState& st) {
+  if (T.flags & GD_FLAG_NO_PREDICTION) return false;
+  uint64_t m = st.cand_count;
+  return m >= d.k && m <= d.cand_cap;
+}
+
+// Host-side entry points of the kernel groups (defined in the .cu files).
+cudaError_t launch_compress(const DevTables& T, const uint32_t* tiles_per_launch, uint64_t samp_total, cudaStream_t stream);
+
+}  // namespace gd
