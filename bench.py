@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the gradient-dropping hot path: dense-gradient GB/s through compress + apply.
+
+One step = gd_compress (residual add, threshold select, compaction, residual rewrite) followed by
+gd_decompress_apply of the push into all parameter shards, on one flat fp32 gradient that is
+already resident in device memory.  value = 4 * n bytes * steps / time, summed over the ranks
+(each rank is an independent replica: the path has no exchange between GPUs).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+Prints one JSON line.  --impl reference times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "dense-gradient GB/s through compress+apply"
+UNIT = "GB/s"
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def workload_config(w, extra=None):
+    cfg = {
+        "workload": f"config {w.config}: {w.name}, n={w.n}, drop_ppm={w.drop_ppm}, "
+                    f"scope={'global' if w.scope_mode == 0 else 'per-layer'}, "
+                    f"values={'fp32' if w.value_mode == 0 else 'two-means'}, shards={w.n_shards}",
+        "n": w.n, "drop_ppm": w.drop_ppm, "n_layers": len(w.layer_off) - 1, "n_shards": w.n_shards,
+        "parallelism": "replicas only (no exchange between GPUs)",
+    }
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+# ---------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1]))
+                    smax.append(float(p[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     p[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ---------------------------------------------------------------- CPU oracle legs
+ORACLE_SAMPLE_LIMIT = 1 << 26
+
+
+def oracle_sample(w):
+    """A bounded sample of the workload for the CPU oracle (about 2^26 elements at most).
+
+    Returns (sample workload, function step -> numpy gradient, description).
+    """
+    from paper_1704_05021_b200 import workloads as W
+    if w.n <= ORACLE_SAMPLE_LIMIT:
+        return w, (lambda step: W.make_gradient(w, step, "cpu").numpy()), "the whole workload"
+    if len(w.layer_off) == 2:
+        sw = W.workload(w.config, scale_log2=26)
+        text = f"2^26 of {w.n} elements drawn from the same distribution, same drop ratio and shard count"
+        return sw, (lambda step: W.make_gradient(sw, step, "cpu").numpy()), text
+    sizes = [(w.layer_off[i + 1] - w.layer_off[i]) * ORACLE_SAMPLE_LIMIT // w.n for i in range(len(w.layer_off) - 1)]
+    sw = W.small_layered(len(sizes), sizes, w.drop_ppm, w.scope_mode, w.value_mode, w.n_shards)
+
+    def grad(step):
+        import numpy as np
+        full = W.make_gradient(w, step, "cpu").numpy()
+        return np.concatenate([full[w.layer_off[i]:w.layer_off[i] + sizes[i]] for i in range(len(sizes))])
+
+    return sw, grad, f"the leading {ORACLE_SAMPLE_LIMIT / w.n:.0%} of every layer ({sw.n} of {w.n} elements)"
+
+
+def time_oracle_step(w_full, steps: int, warmup: int):
+    """Oracle compress + apply on the bounded sample; returns (GB/s, ms per step, sample text)."""
+    import numpy as np
+    import torch
+    from oracle import graddrop_oracle as orc
+    torch.set_num_threads(1)
+    sw, grad_of, sample = oracle_sample(w_full)
+    grads = [grad_of(s) for s in range(min(steps + warmup, 2))]
+    r = orc.residual_reset(sw.n)
+    params = np.zeros(sw.n, dtype=np.float32)
+    times = []
+    for it in range(warmup + steps):
+        g = grads[it % len(grads)]
+        t0 = time.perf_counter()
+        out = orc.compress(g, r, sw.layer_off, sw.shard_off, sw.drop_ppm, sw.scope_mode, sw.value_mode)
+        for j in range(sw.n_shards):
+            lo, hi = sw.shard_off[j], sw.shard_off[j + 1]
+            ref, _ = orc.apply_pushes(params[lo:hi], lo, [out], value_mode=sw.value_mode, layer_off=sw.layer_off)
+            params[lo:hi] = ref.astype(np.float32)
+        dt = time.perf_counter() - t0
+        r = out["residual"]
+        if it >= warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    return 4.0 * sw.n / (ms * 1e-3) / 1e9, ms, sample
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_1704_05021_b200 import workloads as W
+    w = W.workload(args.config)
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    gbs, ms, sample = time_oracle_step(w, steps, warmup)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(w, {"timed_steps": steps, "timed_warmup": warmup}),
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------- the CUDA arm
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1704_05021_b200 import binding as B
+    from paper_1704_05021_b200 import workloads as W
+    from paper_1704_05021_b200.session import GradDropSession
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.load_library()
+
+    w = W.workload(args.config)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
+                           B.GD_FLAG_NO_PREDICTION if args.no_prediction else 0, dev)
+    params = W.make_params(w, dev)
+    views = sess.shard_views(params)
+    pool = max(1, min(args.steps + args.warmup, args.pool))
+    grads = [W.make_gradient(w, s, dev) for s in range(pool)]
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for it in range(args.warmup):
+        sess.compress(grads[it % pool])
+        sess.apply(views)
+    barrier()
+    if sess.status() != B.GD_OK:
+        raise RuntimeError(f"device status {sess.status()} after warm-up")
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    B.gd_profile_enable(True)
+    B.gd_profile_collect()
+    launches0 = B.gd_launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    ev[0].record()
+    for it in range(args.steps):
+        sess.compress(grads[(args.warmup + it) % pool])
+        sess.apply(views)
+        ev[it + 1].record()
+    barrier()
+    launches = B.gd_launch_count() - launches0
+    fused_ms = B.gd_profile_collect()
+    B.gd_profile_enable(False)
+    clocks = sampler.stop() if rank == 0 else None
+    stats = sess.stats()
+    if stats["status"] != B.GD_OK:
+        raise RuntimeError(f"device status {stats['status']} in the timed region")
+    total_ms = ev[0].elapsed_time(ev[-1])
+    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * 4.0 * w.n * args.steps / (total_ms * 1e-3) / 1e9
+
+    # end to end through the host entry point: gradient in page-locked host memory, push read back
+    e2e = None
+    if not args.no_e2e:
+        k = sess.k_total
+        g_host = torch.empty(w.n, dtype=torch.float32, pin_memory=True)
+        g_host.copy_(grads[0])
+        idx_host = torch.empty(max(k, 1), dtype=torch.int32, pin_memory=True)
+        val_host = torch.empty(max(k, 1), dtype=torch.float32, pin_memory=True)
+        off_host = torch.empty(w.n_shards + 1, dtype=torch.int32, pin_memory=True)
+        means_host = torch.empty(len(w.layer_off) - 1, 2, dtype=torch.float32, pin_memory=True)
+        g_dev = torch.empty(w.n, dtype=torch.float32, device=dev)
+        call = sess.compress_call(g_dev)
+        acall = sess.apply_call(views)
+        e2e_steps = max(1, min(args.steps, 5))
+        two = w.value_mode == B.GD_VALUES_TWO_MEANS
+        for _ in range(2):
+            B.gd_step_host(call, acall, g_host, idx_host, None if two else val_host, off_host,
+                           means_host if two else None)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            B.gd_step_host(call, acall, g_host, idx_host, None if two else val_host, off_host,
+                           means_host if two else None)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        d2h = 4 * (w.n_shards + 1) + 4 * k + (8 * (len(w.layer_off) - 1) if two else 4 * k)
+        e2e = {"value": world * 4.0 * w.n * e2e_steps / dt / 1e9, "unit": UNIT, "h2d_bytes_per_step": 4 * w.n,
+               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": 1e3 * dt / e2e_steps}
+        del g_host, g_dev
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = read_peaks()
+    fused_avg_ms = sum(fused_ms) / len(fused_ms) if fused_ms else None
+    cand_per_call = stats["n_candidates"]
+    fused_bytes = 12.0 * w.n + 8.0 * cand_per_call         # read g, read r, write r; candidates written
+    roofline = {"bound": "hbm", "kernel": "add_emit_kernel", "achieved": None, "peak": peak, "unit": "GB/s",
+                "frac": None, "traffic": None, "peak_kind": f"of {peak_kind}",
+                "algorithmic_bytes_per_launch": fused_bytes, "launches_timed": len(fused_ms)}
+    if fused_avg_ms:
+        roofline["achieved"] = fused_bytes / (fused_avg_ms * 1e-3) / 1e9
+        roofline["frac"] = roofline["achieved"] / peak
+        roofline["avg_launch_ms"] = fused_avg_ms
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(traffic_path) as fh:
+            tr = json.load(fh)
+        per_elt = tr.get(f"config{w.config}", tr.get("default"))
+        if per_elt is not None:
+            roofline["traffic"] = float(per_elt["add_emit_dram_bytes_per_element"]) * w.n
+            roofline["traffic_source"] = per_elt.get("source")
+    except Exception:
+        pass
+    k_frac = sess.k_total / max(w.n, 1)
+    per_surv = 16.0 if w.value_mode == B.GD_VALUES_TWO_MEANS else 24.0
+    alg_step_bytes = (12.0 + per_surv * k_frac) * w.n
+    step_frac = (alg_step_bytes / (ms_per_step * 1e-3) / 1e9) / peak
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        gbs, cms, sample = time_oracle_step(w, 1, 0)
+        cpu = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample, "ms_per_step": cms}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": workload_config(w, {
+            "l2": "inputs larger than L2" if 4 * w.n > 126e6 * 2 else "inputs fit in L2; not flushed between steps",
+            "gradient_pool": pool, "prediction": not args.no_prediction}),
+        "step_ms": {"min": min(step_ms), "median": statistics.median(step_ms), "max": max(step_ms)},
+        "step_roofline": {"algorithmic_bytes_per_step": alg_step_bytes, "frac_of_peak": step_frac,
+                          "frac_of_8000": (alg_step_bytes / (ms_per_step * 1e-3) / 1e9) / 8000.0},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+        "clocks": clocks, "stats": stats,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=5, help="workload 1..5 (default 5: 2^30 elements, 8 shards)")
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--pool", type=int, default=10, help="distinct gradients kept on the device and cycled")
+    ap.add_argument("--no-prediction", action="store_true", help="force the dense selection path")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "cuda":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -197,6 +197,19 @@ typedef struct gd_host_io {
 
 int gd_step_host(const gd_compress_args* args, const gd_apply_args* apply, const gd_host_io* io, void* stream);
 
+/*
+ * Measurement hooks (no counterpart in the paper).  While enabled, every gd_compress call records
+ * a pair of CUDA events on its stream around the fused full pass (the kernel that streams the
+ * dense gradient and residual once); gd_profile_collect waits for the recorded pairs, writes their
+ * durations in milliseconds (oldest first, at most `capacity`) and forgets them.  At most 4096
+ * pairs are held between two collects; later launches are not recorded.  Not thread-safe.
+ */
+int gd_profile_enable(int enable);
+int gd_profile_collect(float* ms_out, uint32_t capacity, uint32_t* count_out);
+
+/* Number of kernels this library has launched in this process (memsets and copies not counted). */
+int gd_launch_count(uint64_t* count_out);
+
 #ifdef __cplusplus
 }
 #endif

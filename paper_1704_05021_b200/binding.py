@@ -31,6 +31,7 @@ GD_FLAG_NO_PREDICTION = 1
 EXPORTS = [
     "gd_status_string", "gd_kept_count", "gd_total_kept", "gd_workspace_bytes", "gd_apply_workspace_bytes",
     "gd_compress", "gd_decompress_apply", "gd_residual_reset", "gd_status", "gd_get_stats", "gd_step_host",
+    "gd_profile_enable", "gd_profile_collect", "gd_launch_count",
 ]
 
 
@@ -105,6 +106,9 @@ def load_library():
     lib.gd_status.argtypes = [C.c_void_p, C.c_void_p]
     lib.gd_get_stats.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(_Stats)]
     lib.gd_step_host.argtypes = [C.POINTER(_CompressArgs), C.POINTER(_ApplyArgs), C.POINTER(_HostIo), C.c_void_p]
+    lib.gd_profile_enable.argtypes = [C.c_int]
+    lib.gd_profile_collect.argtypes = [C.POINTER(C.c_float), C.c_uint32, C.POINTER(C.c_uint32)]
+    lib.gd_launch_count.argtypes = [C.POINTER(C.c_uint64)]
     for name in EXPORTS:
         if name != "gd_status_string":
             getattr(lib, name).restype = C.c_int
@@ -243,3 +247,20 @@ def gd_step_host(call: CompressCall, apply: Optional[ApplyCall], grad_host: torc
     io = _HostIo(_ptr(grad_host), _ptr(idx_host), _ptr(val_host), _ptr(shard_cnt_off_host), _ptr(means_host))
     ap = C.byref(apply.args) if apply is not None else None
     _check(load_library().gd_step_host(C.byref(call.args), ap, C.byref(io), _stream_handle(stream)), "gd_step_host")
+
+
+def gd_profile_enable(enable: bool) -> None:
+    _check(load_library().gd_profile_enable(1 if enable else 0), "gd_profile_enable")
+
+
+def gd_profile_collect(capacity: int = 4096) -> list:
+    buf = (C.c_float * capacity)()
+    cnt = C.c_uint32(0)
+    _check(load_library().gd_profile_collect(buf, capacity, C.byref(cnt)), "gd_profile_collect")
+    return [buf[i] for i in range(cnt.value)]
+
+
+def gd_launch_count() -> int:
+    out = C.c_uint64(0)
+    _check(load_library().gd_launch_count(C.byref(out)), "gd_launch_count")
+    return out.value

@@ -151,7 +151,35 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, i
   return GD_OK;
 }
 
+// measurement hooks
+constexpr uint32_t kProfilePairs = 4096;
+bool g_profile_on = false;
+cudaEvent_t g_ev_begin[kProfilePairs], g_ev_end[kProfilePairs];
+uint32_t g_ev_created = 0, g_ev_used = 0;
+bool g_pair_open = false;
+uint64_t g_launches = 0;
+
 }  // namespace
+
+void note_launches(uint32_t count) { g_launches += count; }
+
+void profile_mark(cudaStream_t stream, bool begin) {
+  if (!g_profile_on) return;
+  if (begin) {
+    g_pair_open = false;
+    if (g_ev_used >= kProfilePairs) return;
+    if (g_ev_used >= g_ev_created) {
+      if (cudaEventCreate(&g_ev_begin[g_ev_created]) != cudaSuccess) return;
+      if (cudaEventCreate(&g_ev_end[g_ev_created]) != cudaSuccess) { cudaEventDestroy(g_ev_begin[g_ev_created]); return; }
+      ++g_ev_created;
+    }
+    if (cudaEventRecord(g_ev_begin[g_ev_used], stream) == cudaSuccess) g_pair_open = true;
+  } else if (g_pair_open) {
+    cudaEventRecord(g_ev_end[g_ev_used], stream);
+    ++g_ev_used;
+    g_pair_open = false;
+  }
+}
 
 }  // namespace gd
 
@@ -285,12 +313,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
 
     uint32_t tiles[L_COUNT];
     for (int l = 0; l < L_COUNT; ++l) tiles[l] = P.tiles[l];
-    if (!(a->flags & GD_FLAG_NO_PREDICTION)) {
-      // dense kernels are still enqueued: they return at once unless a prediction failed
-    } else {
-      tiles[L_SAMP] = 0;
-      tiles[L_CAND] = 0;
-    }
+    // the dense kernels are always enqueued: they return at once unless a prediction failed
     if (launch_compress(T, tiles, P.samp_total, stream) != cudaSuccess) return GD_ERR_CUDA;
     return GD_OK;
   } catch (const std::bad_alloc&) {
@@ -323,6 +346,36 @@ int gd_status(const void* workspace, void* stream) {
   gd_stats s;
   int rc = gd_get_stats(workspace, stream, &s);
   return rc != GD_OK ? rc : s.status;
+}
+
+int gd_profile_enable(int enable) {
+  g_profile_on = enable != 0;
+  if (!g_profile_on) g_ev_used = 0;
+  return GD_OK;
+}
+
+int gd_profile_collect(float* ms_out, uint32_t capacity, uint32_t* count_out) {
+  if (!count_out || (capacity && !ms_out)) return GD_ERR_INVALID_ARG;
+  uint32_t w = 0;
+  int rc = GD_OK;
+  for (uint32_t i = 0; i < g_ev_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(g_ev_end[i]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, g_ev_begin[i], g_ev_end[i]) != cudaSuccess) {
+      rc = GD_ERR_CUDA;
+      break;
+    }
+    if (w < capacity) ms_out[w++] = ms;
+  }
+  g_ev_used = 0;
+  *count_out = w;
+  return rc;
+}
+
+int gd_launch_count(uint64_t* count_out) {
+  if (!count_out) return GD_ERR_INVALID_ARG;
+  *count_out = g_launches;
+  return GD_OK;
 }
 
 int gd_step_host(const gd_compress_args* a, const gd_apply_args* apply, const gd_host_io* io, void* stream_v) {

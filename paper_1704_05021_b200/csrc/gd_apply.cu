@@ -131,6 +131,7 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
       A.means = p.means;
       apply_kernel<<<(unsigned)g_sm_count * 8u, kThreads, 0, stream>>>(A);
       if (cudaPeekAtLastError() != cudaSuccess) return GD_ERR_CUDA;
+      note_launches(1);
     }
     return GD_OK;
   } catch (const std::bad_alloc&) {

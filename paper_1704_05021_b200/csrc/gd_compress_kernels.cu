@@ -555,6 +555,7 @@ __global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constan
   do {                                            \
     cudaError_t e_ = cudaPeekAtLastError();       \
     if (e_ != cudaSuccess) return e_;             \
+    note_launches(1);                             \
   } while (0)
 
 cudaError_t launch_compress(const DevTables& T, const uint32_t* tiles, uint64_t samp_total, cudaStream_t stream) {
@@ -569,8 +570,10 @@ cudaError_t launch_compress(const DevTables& T, const uint32_t* tiles, uint64_t 
     }
   }
   if (tiles[L_EMIT]) {
+    profile_mark(stream, true);
     add_emit_kernel<<<tiles[L_EMIT], kThreads, 0, stream>>>(T);
     GD_LAUNCH_CHECK();
+    profile_mark(stream, false);
   }
   if (predict && tiles[L_CAND]) {
     for (int pass = 0; pass < 3; ++pass) {

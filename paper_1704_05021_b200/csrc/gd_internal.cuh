@@ -153,4 +153,8 @@ __device__ __forceinline__ bool predicted_ok(const DevTables& T, const ScopeDesc
 // Host-side entry points of the kernel groups (defined in the .cu files).
 cudaError_t launch_compress(const DevTables& T, const uint32_t* tiles_per_launch, uint64_t samp_total, cudaStream_t stream);
 
+// Measurement hooks (gd_api.cu): count a kernel launch; record an event of the pair around the fused pass.
+void note_launches(uint32_t count);
+void profile_mark(cudaStream_t stream, bool begin);
+
 }  // namespace gd

@@ -115,7 +115,8 @@ def _fill_laplace_with_outliers(out: torch.Tensor, gen, scale: float, p_out: flo
         hi = min(lo + _CHUNK, n)
         part = out[lo:hi]
         u = torch.rand(hi - lo, generator=gen, device=out.device, dtype=torch.float32) - 0.5
-        lap = -scale * torch.sign(u) * torch.log1p(-2.0 * u.abs())
+        # inverse CDF of Laplace(0, scale); the clamp keeps rand() == 0 finite (|x| <= ~17.3 * scale)
+        lap = -scale * torch.sign(u) * torch.log((1.0 - 2.0 * u.abs()).clamp_min(2.0 ** -25))
         pick = torch.rand(hi - lo, generator=gen, device=out.device, dtype=torch.float32) < p_out
         big = torch.randn(hi - lo, generator=gen, device=out.device, dtype=torch.float32) * std_out
         part.copy_(torch.where(pick, big, lap))

@@ -234,7 +234,6 @@ def test_config5_full_scale_properties(cuda_device):
     sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
     params = torch.zeros(w.n, dtype=torch.float32, device=cuda_device)
     views = sess.shard_views(params)
-    v_prev = torch.zeros(w.n, dtype=torch.float32, device=cuda_device)
     for step in range(2):
         g = W.make_gradient(w, step, cuda_device)
         v = g + sess.residual                       # the same single fp32 add, by the tensor library
@@ -271,4 +270,3 @@ def test_config5_full_scale_properties(cuda_device):
         p_before[idx] += val
         assert torch.equal(params.view(torch.int32), p_before.view(torch.int32))
         del v, keys, expect_res, p_before, g
-    del v_prev
