@@ -198,7 +198,7 @@ def run_cuda(args):
         dist.init_process_group("nccl", device_id=dev)
     B.load_library()
 
-    w = W.workload(args.config)
+    w = W.workload(args.config, scale_log2=args.scale_log2) if args.scale_log2 else W.workload(args.config)
     sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
                            B.GD_FLAG_NO_PREDICTION if args.no_prediction else 0, dev)
     params = W.make_params(w, dev)
@@ -347,6 +347,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--pool", type=int, default=10, help="distinct gradients kept on the device and cycled")
     ap.add_argument("--no-prediction", action="store_true", help="force the dense selection path")
+    ap.add_argument("--scale-log2", type=int, default=0,
+                    help="length 2^x for the flat workloads 1 and 5 (profiling on a smaller case)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

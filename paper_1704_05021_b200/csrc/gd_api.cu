@@ -55,6 +55,7 @@ struct Plan {
   uint32_t tiles[L_COUNT] = {0, 0, 0, 0, 0};
   uint64_t samp_total = 0, cand_total = 0, k_total = 0;
   uint32_t n_scopes = 0;
+  uint32_t emit_chunk_tiles = 1;
   // workspace layout (byte offsets)
   size_t off_ctl = 0, off_state = 0, off_hist = 0, off_sums = 0, off_cnts = 0, off_desc_emit = 0,
          off_desc_cand = 0, off_desc_dcomp = 0, zero_bytes = 0;
@@ -81,6 +82,13 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, i
   if (scope_mode != GD_SCOPE_GLOBAL && scope_mode != GD_SCOPE_PER_LAYER) return GD_ERR_INVALID_ARG;
   if (n > (1ull << 32)) return GD_ERR_TOO_LARGE;
   const bool predict = !(flags & GD_FLAG_NO_PREDICTION);
+  // The fused pass gives each CTA a chunk of 1, 2, 4 or 8 tiles: as large as still leaves about
+  // four waves of CTAs (4 per SM on 148 SMs) for the whole vector.
+  const uint64_t dense_tiles = (n + kTile - 1) / kTile;
+  uint32_t chunk_tiles = 8;
+  while (chunk_tiles > 1 && dense_tiles < (uint64_t)chunk_tiles * 2368u) chunk_tiles >>= 1;
+  P->emit_chunk_tiles = chunk_tiles;
+  const uint64_t CH = (uint64_t)chunk_tiles * kTile;
   const uint32_t ns_count = scope_mode == GD_SCOPE_GLOBAL ? 1u : n_layers;
   P->n_scopes = ns_count;
   P->scopes.resize(ns_count);
@@ -108,7 +116,7 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, i
     for (int l = 0; l < L_COUNT; ++l) P->tile0[l][s] = (uint32_t)tiles[l];
     P->samp_off[s] = d.samp_base;
     if (ns) {
-      tiles[L_EMIT] += (d.hi + kTile - 1) / kTile - d.lo / kTile;
+      tiles[L_EMIT] += (d.hi + CH - 1) / CH - d.lo / CH;
       tiles[L_DSEL] += (ns + kDenseSelTile - 1) / kDenseSelTile;
       tiles[L_DCOMP] += (ns + kTile - 1) / kTile;
     }
@@ -162,6 +170,17 @@ uint64_t g_launches = 0;
 }  // namespace
 
 void note_launches(uint32_t count) { g_launches += count; }
+
+int sm_count() {
+  static int cached = 0;
+  if (cached > 0) return cached;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return 148;   // B200; only sizes grids
+  cached = sms;
+  return cached;
+}
 
 void profile_mark(cudaStream_t stream, bool begin) {
   if (!g_profile_on) return;
@@ -288,6 +307,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     T.flags = a->flags;
     T.value_mode = a->value_mode;
     T.k_total = P.k_total;
+    T.emit_chunk_tiles = P.emit_chunk_tiles;
     T.ctl = (Ctl*)(ws + P.off_ctl);
     T.state = (ScopeState*)(ws + P.off_state);
     T.hist = (unsigned long long*)(ws + P.off_hist);
@@ -314,7 +334,16 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     uint32_t tiles[L_COUNT];
     for (int l = 0; l < L_COUNT; ++l) tiles[l] = P.tiles[l];
     // the dense kernels are always enqueued: they return at once unless a prediction failed
-    if (launch_compress(T, tiles, P.samp_total, stream) != cudaSuccess) return GD_ERR_CUDA;
+    const bool predict = !(a->flags & GD_FLAG_NO_PREDICTION);
+    if (predict && launch_sample_select(T, tiles, P.samp_total, stream) != cudaSuccess) return GD_ERR_CUDA;
+    if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+    if (predict) {
+      if (launch_candidate_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+      if (launch_compact(T, tiles, false, stream) != cudaSuccess) return GD_ERR_CUDA;
+    }
+    if (launch_dense_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+    if (launch_compact(T, tiles, true, stream) != cudaSuccess) return GD_ERR_CUDA;
+    if (launch_finalize(T, stream) != cudaSuccess) return GD_ERR_CUDA;
     return GD_OK;
   } catch (const std::bad_alloc&) {
     return GD_ERR_INVALID_ARG;

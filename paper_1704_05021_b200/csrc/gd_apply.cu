@@ -52,8 +52,6 @@ __global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__
   }
 }
 
-int g_sm_count = 0;
-
 }  // namespace
 
 }  // namespace gd
@@ -107,13 +105,6 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
     unsigned char* ws = (unsigned char*)a->workspace;
     if (cudaMemcpyAsync(ws, blob.data(), need, cudaMemcpyHostToDevice, stream) != cudaSuccess) return GD_ERR_CUDA;
 
-    if (g_sm_count == 0) {
-      int dev = 0, sms = 0;
-      if (cudaGetDevice(&dev) != cudaSuccess ||
-          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-        return GD_ERR_CUDA;
-      g_sm_count = sms;
-    }
     ApplyDev A;
     std::memset(&A, 0, sizeof(A));
     A.params = (float* const*)(ws + o_params);
@@ -129,7 +120,7 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
       A.val = p.val;
       A.cnt_off = p.shard_cnt_off;
       A.means = p.means;
-      apply_kernel<<<(unsigned)g_sm_count * 8u, kThreads, 0, stream>>>(A);
+      apply_kernel<<<(unsigned)sm_count() * 8u, kThreads, 0, stream>>>(A);
       if (cudaPeekAtLastError() != cudaSuccess) return GD_ERR_CUDA;
       note_launches(1);
     }

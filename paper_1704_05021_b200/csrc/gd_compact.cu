@@ -1,0 +1,232 @@
+// Survivor compaction of gd_compress (Algorithm 1, steps 3-5: mask, residual rewrite, sparse
+// output), the two-means sums of Section 5.4, and the kernel that finishes a call (thresholds,
+// shard offsets of Section 3, the means).
+#include "gd_scan.cuh"
+
+namespace gd {
+
+namespace {
+
+// Single-pass look-back scan with two counters per tile: keys above tau, and keys equal to tau.  An
+// element above tau goes to slot  (#above before it) + min(#ties before it, q); a tie is kept iff fewer
+// than q ties precede it.  VIEW == V_CAND walks the candidate list, V_DENSE the dense range itself.
+// CTAs take tiles from an atomic ticket until none is left.
+template <int VIEW>
+__global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
+  constexpr int LK = VIEW == V_CAND ? L_CAND : L_DCOMP;
+  constexpr int ROUNDS = kTile / kThreads;   // 16 elements per thread
+  __shared__ uint32_t s_tile;
+  __shared__ uint32_t s_wg[kWarps], s_we[kWarps];
+  __shared__ uint64_t s_exg, s_exe;
+  __shared__ int s_ok, s_single;
+  __shared__ uint32_t s_layer;
+  __shared__ double s_red[kWarps][2];
+  __shared__ uint32_t s_redc[kWarps][2];
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  if (VIEW == V_DENSE && !(T.flags & GD_FLAG_NO_PREDICTION) && T.ctl->dense_needed == 0u) return;
+  const uint32_t* tile0 = T.tile0[LK];
+  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
+  const uint32_t ltm = lanemask_lt();
+  uint4* desc = reinterpret_cast<uint4*>(VIEW == V_CAND ? T.desc_cand : T.desc_dcomp);
+
+  for (;;) {
+    __syncthreads();                       // previous tile is done with the shared variables
+    if (tid == 0) s_tile = atomicAdd(&T.ctl->ticket[LK], 1u);
+    __syncthreads();
+    const uint32_t t = s_tile;
+    if (t >= total_tiles) break;
+    const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
+    const ScopeDesc& d = T.scopes[s];
+    const ScopeState* st = T.state + s;
+    const bool pred = predicted_ok(T, d, *st);
+    if (VIEW == V_CAND ? !pred : pred) continue;    // the other view owns this scope
+    const uint32_t first = __ldg(tile0 + s);
+    const uint32_t lt = t - first;
+    const uint64_t len = VIEW == V_CAND ? st->cand_count : d.hi - d.lo;
+    const uint64_t beg = (uint64_t)lt * kTile;
+    if (beg >= len) continue;                       // trailing tiles of a short candidate list
+    const uint64_t end = (beg + kTile < len) ? beg + kTile : len;
+    const float* vals = VIEW == V_CAND ? T.cand_val + d.cand_base : T.residual + d.lo;
+    const uint32_t tau = st->tau;
+    const uint64_t q = st->q;
+
+    if (two_means && tid == 0) {
+      uint64_t i_first, i_last;
+      if (VIEW == V_CAND) {
+        i_first = T.cand_idx[d.cand_base + beg];
+        i_last = T.cand_idx[d.cand_base + end - 1];
+      } else {
+        i_first = d.lo + beg;
+        i_last = d.lo + end - 1;
+      }
+      const uint32_t l0 = range_of(T.layer_off, T.n_layers, i_first);
+      const uint32_t l1 = range_of(T.layer_off, T.n_layers, i_last);
+      s_layer = l0;
+      s_single = (l0 == l1) ? 1 : 0;
+    }
+
+    // phase 1: load, classify, count
+    const uint64_t wbeg = beg + (uint64_t)warp * (32u * ROUNDS) + lane;
+    uint32_t vb[ROUNDS];
+    uint32_t gtm = 0, eqm = 0, wg = 0, we = 0;
+#pragma unroll
+    for (int j = 0; j < ROUNDS; ++j) {
+      const uint64_t i = wbeg + (uint64_t)j * 32u;
+      uint32_t b = 0;
+      bool isgt = false, iseq = false;
+      if (i < end) {
+        b = __float_as_uint(vals[i]);
+        const uint32_t key = b & kAbsMask;
+        isgt = key > tau;
+        iseq = key == tau;
+      }
+      vb[j] = b;
+      gtm |= (isgt ? 1u : 0u) << j;
+      eqm |= (iseq ? 1u : 0u) << j;
+      wg += __popc(__ballot_sync(0xFFFFFFFFu, isgt));
+      we += __popc(__ballot_sync(0xFFFFFFFFu, iseq));
+    }
+    if (lane == 0) { s_wg[warp] = wg; s_we[warp] = we; }
+    __syncthreads();
+    uint32_t woff_g = 0, woff_e = 0, tot_g = 0, tot_e = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const uint32_t cg = s_wg[w], ce = s_we[w];
+      woff_g += (w < (int)warp) ? cg : 0u;
+      woff_e += (w < (int)warp) ? ce : 0u;
+      tot_g += cg;
+      tot_e += ce;
+    }
+    if (warp == 0) {
+      uint64_t ex_a, ex_b;
+      const bool ok = tile_lookback(desc, t, first, tot_g, tot_e, ex_a, ex_b, T.ctl);
+      if (lane == 0) { s_exg = ex_a; s_exe = ex_b; s_ok = ok ? 1 : 0; }
+    }
+    __syncthreads();
+    if (!s_ok) continue;
+
+    // phase 2: place the survivors
+    uint64_t rg = s_exg + woff_g, re = s_exe + woff_e;   // running counts before this warp's round
+    const bool single = two_means && s_single;
+    const uint32_t tile_layer = two_means ? s_layer : 0u;
+    double sum_p = 0.0, sum_n = 0.0;
+    uint32_t cnt_p = 0, cnt_n = 0;
+    bool bad = false;
+#pragma unroll
+    for (int j = 0; j < ROUNDS; ++j) {
+      const bool isgt = (gtm >> j) & 1u, iseq = (eqm >> j) & 1u;
+      const uint32_t mg = __ballot_sync(0xFFFFFFFFu, isgt), me = __ballot_sync(0xFFFFFFFFu, iseq);
+      if (isgt || iseq) {
+        const uint64_t gb = rg + __popc(mg & ltm), eb = re + __popc(me & ltm);
+        if (isgt || eb < q) {
+          const uint64_t pos = gb + (eb < q ? eb : q);
+          const uint64_t i = wbeg + (uint64_t)j * 32u;
+          const uint64_t idx = VIEW == V_CAND ? (uint64_t)T.cand_idx[d.cand_base + i] : d.lo + i;
+          if (pos < d.k && idx < T.n) {
+            const uint32_t b = vb[j];
+            T.residual[idx] = 0.0f;
+            if (two_means) {
+              const uint32_t sgn = b >> 31;
+              T.out_idx[d.out_base + pos] = (uint32_t)idx | (sgn << 31);
+              const double x = (double)__uint_as_float(b);
+              if (single) {
+                if (sgn) { sum_n += x; ++cnt_n; } else { sum_p += x; ++cnt_p; }
+              } else {
+                const uint32_t l = range_of(T.layer_off, T.n_layers, idx);
+                atomicAdd(T.sums + 2 * (size_t)l + sgn, x);
+                atomicAdd(T.cnts + 2 * (size_t)l + sgn, 1ull);
+              }
+            } else {
+              T.out_idx[d.out_base + pos] = (uint32_t)idx;
+              T.out_val[d.out_base + pos] = __uint_as_float(b);
+            }
+          } else {
+            bad = true;
+          }
+        }
+      }
+      rg += __popc(mg);
+      re += __popc(me);
+    }
+    if (bad) atomicCAS(&T.ctl->status, (int)GD_OK, (int)GD_ERR_INTERNAL);
+    if (single) {   // uniform over the CTA
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        sum_p += __shfl_xor_sync(0xFFFFFFFFu, sum_p, o);
+        sum_n += __shfl_xor_sync(0xFFFFFFFFu, sum_n, o);
+        cnt_p += __shfl_xor_sync(0xFFFFFFFFu, cnt_p, o);
+        cnt_n += __shfl_xor_sync(0xFFFFFFFFu, cnt_n, o);
+      }
+      if (lane == 0) { s_red[warp][0] = sum_p; s_red[warp][1] = sum_n; s_redc[warp][0] = cnt_p; s_redc[warp][1] = cnt_n; }
+      __syncthreads();
+      if (tid < 2) {
+        double sx = 0.0;
+        unsigned long long cx = 0;
+        for (int w = 0; w < kWarps; ++w) { sx += s_red[w][tid]; cx += s_redc[w][tid]; }
+        if (cx) {
+          atomicAdd(T.sums + 2 * (size_t)tile_layer + tid, sx);
+          atomicAdd(T.cnts + 2 * (size_t)tile_layer + tid, cx);
+        }
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constant__ DevTables T) {
+  const uint32_t tid = threadIdx.x;
+  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
+  uint32_t n_pred = 0, n_dense = 0;
+  unsigned long long n_cand = 0;
+  for (uint32_t s = tid; s < T.n_scopes; s += kThreads) {
+    const ScopeDesc& d = T.scopes[s];
+    const ScopeState& st = T.state[s];
+    if (T.out_tau) T.out_tau[s] = d.k == 0 ? 0xFFFFFFFFu : st.tau;
+    if (st.used_dense) ++n_dense; else ++n_pred;
+    n_cand += st.cand_count;
+  }
+  if (n_pred) atomicAdd(&T.ctl->n_scopes_predicted, n_pred);
+  if (n_dense) atomicAdd(&T.ctl->n_scopes_dense, n_dense);
+  if (n_cand) atomicAdd(reinterpret_cast<unsigned long long*>(&T.ctl->n_candidates), n_cand);
+  if (tid == 0) { T.ctl->n_scopes = T.n_scopes; T.ctl->n_kept = T.k_total; }
+  // survivors are in ascending index order: shard j starts at the first index >= shard_off[j]
+  for (uint32_t j = tid; j <= T.n_shards; j += kThreads) {
+    const uint64_t bound = T.shard_off[j];
+    uint64_t lo = 0, hi = T.k_total;
+    while (lo < hi) {
+      const uint64_t mid = (lo + hi) >> 1;
+      uint32_t w = T.out_idx[mid];
+      if (two_means) w &= kAbsMask;
+      if ((uint64_t)w < bound) lo = mid + 1; else hi = mid;
+    }
+    T.out_shard_cnt_off[j] = (uint32_t)lo;
+  }
+  if (two_means) {
+    for (uint32_t e = tid; e < 2 * T.n_layers; e += kThreads) {
+      const unsigned long long c = T.cnts[e];
+      T.out_means[e] = c ? (float)(T.sums[e] / (double)c) : 0.0f;
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, cudaStream_t stream) {
+  const uint32_t total = tiles[dense ? L_DCOMP : L_CAND];
+  if (!total) return cudaSuccess;
+  const uint32_t cap = (uint32_t)sm_count() * 8u;
+  const uint32_t grid = total < cap ? total : cap;
+  if (dense)
+    compact_kernel<V_DENSE><<<grid, kThreads, 0, stream>>>(T, total);
+  else
+    compact_kernel<V_CAND><<<grid, kThreads, 0, stream>>>(T, total);
+  GD_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+
+cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream) {
+  finalize_kernel<<<1, kThreads, 0, stream>>>(T);
+  GD_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+
+}  // namespace gd

@@ -1,0 +1,182 @@
+// The fused full pass of gd_compress: Algorithm 1, step 1 (grad += residuals) over the whole
+// gradient, fused with the emission of the threshold candidates.
+//
+// One CTA streams one chunk of C tiles (C * 4096 consecutive elements) of one scope:
+//   phase A  per tile: 128-bit loads of g and r, v = g + r, 128-bit store of v over r, and a
+//            16-bit mask per thread of the entries with |v| >= tau_lo (the predicted lower bound);
+//   scan     one decoupled look-back per chunk gives the number of candidates in all earlier
+//            chunks of the scope;
+//   phase B  threads that own candidates read their v back (their own stores) and append
+//            (index, v) to the scope's candidate list, in index order.
+// The look-back is per chunk, not per tile, so that its latency (a few L2 round trips) is paid
+// once per C * 48 KiB of traffic and the chain of prefixes never limits the streaming rate.
+#include "gd_scan.cuh"
+
+namespace gd {
+
+namespace {
+
+// Chunks are aligned to C * kTile elements of the flat vector; a chunk that straddles a scope
+// boundary is processed once per scope, each pass touching only its own scope's elements.  Inside a
+// tile, warp w owns 512 consecutive elements and reads them as four rounds of 128-bit accesses (lane
+// l, round j -> elements w*512 + j*128 + l*4 .. +3): candidate order inside a warp is (round, lane,
+// component), across warps (warp), across tiles (tile).
+template <int C>
+__global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_constant__ DevTables T) {
+  constexpr int E = C * kWarps;              // (tile, warp) counters of one chunk
+  constexpr int PER = (E + 31) / 32;
+  __shared__ uint32_t s_chunk;
+  __shared__ uint32_t s_cnt[E];              // per (tile, warp): count, then exclusive offset in the chunk
+  __shared__ uint64_t s_excl;
+  __shared__ uint32_t s_total;
+  __shared__ int s_ok;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  if (tid == 0) s_chunk = atomicAdd(&T.ctl->ticket[L_EMIT], 1u);
+  __syncthreads();
+  const uint32_t t = s_chunk;
+  const uint32_t* tile0 = T.tile0[L_EMIT];
+  const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
+  const ScopeDesc& d = T.scopes[s];
+  const uint64_t lo = d.lo, hi = d.hi;
+  const uint32_t first = __ldg(tile0 + s), nchunks = __ldg(tile0 + s + 1) - first;
+  const uint32_t lt = t - first;
+  constexpr uint64_t CH = (uint64_t)C * kTile;
+  const uint64_t cbase = (lo / CH + lt) * CH;
+  const uint32_t tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || d.k == 0) ? 0xFFFFFFFFu : T.state[s].tau_lo;
+  const uint64_t toff = (uint64_t)warp * 512u + lane * 4u;   // this thread's first element inside a tile
+
+  // ---- phase A
+  uint32_t cm[C];
+#pragma unroll
+  for (int i = 0; i < C; ++i) {
+    const uint64_t base = cbase + (uint64_t)i * kTile;
+    uint32_t cmask = 0;
+    if (base >= lo && base + kTile <= hi) {
+      const uint64_t e0 = base + toff;
+      float4 g4[4], r4[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) g4[j] = __ldcs(reinterpret_cast<const float4*>(T.grad + e0 + j * 128));
+#pragma unroll
+      for (int j = 0; j < 4; ++j) r4[j] = *reinterpret_cast<const float4*>(T.residual + e0 + j * 128);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float4 x;
+        x.x = __fadd_rn(g4[j].x, r4[j].x);
+        x.y = __fadd_rn(g4[j].y, r4[j].y);
+        x.z = __fadd_rn(g4[j].z, r4[j].z);
+        x.w = __fadd_rn(g4[j].w, r4[j].w);
+        *reinterpret_cast<float4*>(T.residual + e0 + j * 128) = x;
+        cmask |= ((__float_as_uint(x.x) & kAbsMask) >= tau_lo ? 1u : 0u) << (4 * j + 0);
+        cmask |= ((__float_as_uint(x.y) & kAbsMask) >= tau_lo ? 1u : 0u) << (4 * j + 1);
+        cmask |= ((__float_as_uint(x.z) & kAbsMask) >= tau_lo ? 1u : 0u) << (4 * j + 2);
+        cmask |= ((__float_as_uint(x.w) & kAbsMask) >= tau_lo ? 1u : 0u) << (4 * j + 3);
+      }
+    } else if (base < hi && base + kTile > lo) {   // tile cut by the scope (or by the end of the vector)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const uint64_t e = base + toff + j * 128 + c;
+          if (e >= lo && e < hi) {
+            const float x = __fadd_rn(__ldg(T.grad + e), T.residual[e]);
+            T.residual[e] = x;
+            cmask |= ((__float_as_uint(x) & kAbsMask) >= tau_lo ? 1u : 0u) << (4 * j + c);
+          }
+        }
+      }
+    }
+    cm[i] = cmask;
+    const uint32_t wc = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)__popc(cmask));
+    if (lane == 0) s_cnt[i * kWarps + warp] = wc;
+  }
+  __syncthreads();
+
+  // ---- scan: counts -> exclusive offsets inside the chunk, then one look-back for the chunk
+  if (warp == 0) {
+    uint32_t a[PER], sum = 0;
+#pragma unroll
+    for (int p = 0; p < PER; ++p) {
+      const int e = (int)lane * PER + p;
+      a[p] = e < E ? s_cnt[e] : 0u;
+      sum += a[p];
+    }
+    uint32_t inc = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+      if ((int)lane >= o) inc += y;
+    }
+    uint32_t run = inc - sum;
+#pragma unroll
+    for (int p = 0; p < PER; ++p) {
+      const int e = (int)lane * PER + p;
+      if (e < E) s_cnt[e] = run;
+      run += a[p];
+    }
+    const uint32_t total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+    uint64_t ex_a, ex_b;
+    const bool ok = tile_lookback(reinterpret_cast<uint4*>(T.desc_emit), t, first, total, 0, ex_a, ex_b, T.ctl);
+    if (lane == 0) { s_excl = ex_a; s_total = total; s_ok = ok ? 1 : 0; }
+  }
+  __syncthreads();
+  if (!s_ok) return;
+  const uint64_t excl = s_excl;
+
+  // ---- phase B: append this thread's candidates
+  const uint32_t ltm = lanemask_lt();
+  const uint64_t cap = d.cand_cap;
+  uint32_t* cidx = T.cand_idx + d.cand_base;
+  float* cval = T.cand_val + d.cand_base;
+#pragma unroll
+  for (int i = 0; i < C; ++i) {
+    const uint32_t cmask = cm[i];
+    if (!__any_sync(0xFFFFFFFFu, cmask != 0u)) continue;
+    uint64_t run = excl + s_cnt[i * kWarps + warp];
+    const uint64_t e0 = cbase + (uint64_t)i * kTile + toff;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t f = (cmask >> (4 * j)) & 15u;
+      if (!__any_sync(0xFFFFFFFFu, f != 0u)) continue;
+      const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, f & 1u), b1 = __ballot_sync(0xFFFFFFFFu, f & 2u);
+      const uint32_t b2 = __ballot_sync(0xFFFFFFFFu, f & 4u), b3 = __ballot_sync(0xFFFFFFFFu, f & 8u);
+      if (f) {
+        uint64_t pos = run + __popc(b0 & ltm) + __popc(b1 & ltm) + __popc(b2 & ltm) + __popc(b3 & ltm);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (f & (1u << c)) {
+            if (pos < cap) {
+              const uint64_t e = e0 + j * 128 + c;
+              cidx[pos] = (uint32_t)e;
+              cval[pos] = T.residual[e];      // v, as stored by this thread in phase A
+            }
+            ++pos;
+          }
+        }
+      }
+      run += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+    }
+  }
+  if (tid == 0 && lt == nchunks - 1) {
+    const uint64_t m = excl + s_total;
+    T.state[s].cand_count = m;
+    if (!(T.flags & GD_FLAG_NO_PREDICTION) && (m < d.k || m > cap)) atomicAdd(&T.ctl->dense_needed, 1u);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
+  if (!tiles[L_EMIT]) return cudaSuccess;
+  profile_mark(stream, true);
+  switch (T.emit_chunk_tiles) {
+    case 1: add_emit_kernel<1><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
+    case 2: add_emit_kernel<2><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
+    case 4: add_emit_kernel<4><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
+    default: add_emit_kernel<8><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
+  }
+  GD_LAUNCH_CHECK();
+  profile_mark(stream, false);
+  return cudaSuccess;
+}
+
+}  // namespace gd

@@ -24,6 +24,13 @@ enum Launch : int { L_EMIT = 0, L_SAMP = 1, L_CAND = 2, L_DSEL = 3, L_DCOMP = 4,
 // Views a selection can run over.
 enum View : int { V_SAMPLE = 0, V_CAND = 1, V_DENSE = 2 };
 
+#define GD_LAUNCH_CHECK()                         \
+  do {                                            \
+    cudaError_t e_ = cudaPeekAtLastError();       \
+    if (e_ != cudaSuccess) return e_;             \
+    note_launches(1);                             \
+  } while (0)
+
 // Look-back descriptor flags (low two bits of a 64-bit word; the count sits above them).
 enum : uint64_t { F_INVALID = 0, F_AGG = 1, F_PREFIX = 2, F_ABORT = 3 };
 
@@ -62,7 +69,7 @@ struct Ctl {             // zeroed at the start of every call
   uint32_t n_scopes;
   uint32_t n_scopes_predicted;
   uint32_t n_scopes_dense;
-  uint32_t pad;
+  uint32_t dense_needed;   // scopes whose prediction failed (set by the fused pass)
   uint64_t n_candidates;
   uint64_t n_kept;
 };
@@ -74,7 +81,7 @@ struct DevTables {       // passed by value to every kernel
   uint32_t n_scopes, n_layers, n_shards;
   uint32_t flags;
   int32_t value_mode;
-  uint32_t pad;
+  uint32_t emit_chunk_tiles;         // tiles of kTile elements one CTA of the fused pass streams (1, 2, 4 or 8)
   uint64_t k_total;
   // zeroed region
   Ctl* ctl;
@@ -150,8 +157,14 @@ __device__ __forceinline__ bool predicted_ok(const DevTables& T, const ScopeDesc
   return m >= d.k && m <= d.cand_cap;
 }
 
-// Host-side entry points of the kernel groups (defined in the .cu files).
-cudaError_t launch_compress(const DevTables& T, const uint32_t* tiles_per_launch, uint64_t samp_total, cudaStream_t stream);
+// Host-side launchers of the kernel groups (one per .cu file); `tiles` is indexed by Launch.
+cudaError_t launch_sample_select(const DevTables& T, const uint32_t* tiles, uint64_t samp_total, cudaStream_t stream);
+cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
+cudaError_t launch_candidate_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
+cudaError_t launch_dense_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
+cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, cudaStream_t stream);
+cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream);
+int sm_count();   // multiprocessors of the current device (0 on error)
 
 // Measurement hooks (gd_api.cu): count a kernel launch; record an event of the pair around the fused pass.
 void note_launches(uint32_t count);
