@@ -198,6 +198,38 @@ typedef struct gd_host_io {
 int gd_step_host(const gd_compress_args* args, const gd_apply_args* apply, const gd_host_io* io, void* stream);
 
 /*
+ * gd_compress_static - gd_compress for callers that cannot hand the library a workspace.
+ * (No counterpart in the paper: this is a packaging variant of gd_compress.)
+ *
+ * Some hosts of this library run inside a memory plan that is fixed before the first step - an
+ * inference or training runtime that has already carved up the whole device, a plug-in called from
+ * a context where cudaMalloc is forbidden or would synchronise the device, a pre-sized arena whose
+ * owner will not grow it.  Such a caller can still provide the gradient, the residual and the
+ * output buffers, because those are part of its own plan, but it has nowhere to put the scratch
+ * memory gd_compress wants.  For them the library carries a fixed scratch area of
+ * GD_STATIC_WORKSPACE_BYTES inside its own device image, and this entry point uses it in place of
+ * args->workspace (args->workspace and args->workspace_bytes are ignored).  Everything else -
+ * arguments, results, error codes - is exactly gd_compress.
+ *
+ * Limits and rules:
+ *   - the scratch is part of the loaded library: every GPU that loads libgd.so gives up
+ *     GD_STATIC_WORKSPACE_BYTES of device memory until the process exits, used or not;
+ *   - a call whose gd_workspace_bytes() exceeds GD_STATIC_WORKSPACE_BYTES is refused with
+ *     GD_ERR_TOO_LARGE before anything is enqueued (as a guide: one flat scope of 2^24 elements at a
+ *     99 % drop ratio needs about 7.4 MiB);
+ *   - the first call on each device looks up the scratch area's device address (once per device, with
+ *     that device current); make that first call outside any stream capture;
+ *   - no device memory is allocated or freed, here or in anything this entry point calls;
+ *   - all calls on one device share the one scratch area.  Each call clears the part that must
+ *     start at zero, but two calls that overlap on the GPU (different streams, no ordering between
+ *     them) would race on it: keep calls on one device ordered;
+ *   - *workspace_out (if workspace_out is not NULL) receives the scratch area's device address, the
+ *     value to pass to gd_status() and gd_get_stats() after the call.
+ */
+#define GD_STATIC_WORKSPACE_BYTES (16u << 20)
+int gd_compress_static(const gd_compress_args* args, void* stream, const void** workspace_out);
+
+/*
  * Measurement hooks (no counterpart in the paper).  While enabled, every gd_compress call records
  * a pair of CUDA events on its stream around the fused full pass (the kernel that streams the
  * dense gradient and residual once); gd_profile_collect waits for the recorded pairs, writes their

@@ -31,8 +31,9 @@ GD_FLAG_NO_PREDICTION = 1
 EXPORTS = [
     "gd_status_string", "gd_kept_count", "gd_total_kept", "gd_workspace_bytes", "gd_apply_workspace_bytes",
     "gd_compress", "gd_decompress_apply", "gd_residual_reset", "gd_status", "gd_get_stats", "gd_step_host",
-    "gd_profile_enable", "gd_profile_collect", "gd_launch_count",
+    "gd_profile_enable", "gd_profile_collect", "gd_launch_count", "gd_compress_static",
 ]
+GD_STATIC_WORKSPACE_BYTES = 16 << 20
 
 
 class GdError(RuntimeError):
@@ -106,6 +107,7 @@ def load_library():
     lib.gd_status.argtypes = [C.c_void_p, C.c_void_p]
     lib.gd_get_stats.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(_Stats)]
     lib.gd_step_host.argtypes = [C.POINTER(_CompressArgs), C.POINTER(_ApplyArgs), C.POINTER(_HostIo), C.c_void_p]
+    lib.gd_compress_static.argtypes = [C.POINTER(_CompressArgs), C.c_void_p, C.POINTER(C.c_void_p)]
     lib.gd_profile_enable.argtypes = [C.c_int]
     lib.gd_profile_collect.argtypes = [C.POINTER(C.c_float), C.c_uint32, C.POINTER(C.c_uint32)]
     lib.gd_launch_count.argtypes = [C.POINTER(C.c_uint64)]
@@ -264,3 +266,20 @@ def gd_launch_count() -> int:
     out = C.c_uint64(0)
     _check(load_library().gd_launch_count(C.byref(out)), "gd_launch_count")
     return out.value
+
+
+def gd_compress_static(call: CompressCall, stream=None) -> int:
+    """gd_compress on the library's built-in scratch area (for callers that cannot allocate a workspace).
+
+    The workspace stored in `call` is ignored.  Returns the device address of the scratch area, which
+    is what gd_status_at / gd_get_stats_at take.  Calls on one device must not overlap on the GPU.
+    """
+    out = C.c_void_p(0)
+    _check(load_library().gd_compress_static(C.byref(call.args), _stream_handle(stream), C.byref(out)),
+           "gd_compress_static")
+    return out.value or 0
+
+
+def gd_status_at(workspace_address: int, stream=None) -> int:
+    """gd_status for a workspace known by its device address (e.g. the one gd_compress_static returns)."""
+    return load_library().gd_status(C.c_void_p(workspace_address), _stream_handle(stream))

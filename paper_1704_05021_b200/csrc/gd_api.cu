@@ -377,6 +377,33 @@ int gd_status(const void* workspace, void* stream) {
   return rc != GD_OK ? rc : s.status;
 }
 
+// Scratch of gd_compress_static: lives in the library's device image, one copy per GPU that loads it.
+static __device__ __align__(256) unsigned char g_static_workspace[GD_STATIC_WORKSPACE_BYTES];
+
+int gd_compress_static(const gd_compress_args* a, void* stream, const void** workspace_out) {
+  if (!a) return GD_ERR_INVALID_ARG;
+  size_t need = 0;
+  int rc = gd_workspace_bytes(a->layer_off, a->n_layers, a->n_shards, a->scope_mode, a->drop_ppm, &need);
+  if (rc != GD_OK) return rc;
+  if (need > (size_t)GD_STATIC_WORKSPACE_BYTES) return GD_ERR_TOO_LARGE;
+  // In host code g_static_workspace is only a handle: its device address has to be asked for, once
+  // per device, with that device current.
+  constexpr int kMaxDevices = 64;
+  static void* scratch_of_device[kMaxDevices] = {nullptr};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GD_ERR_CUDA;
+  if (!scratch_of_device[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return GD_ERR_CUDA;
+    scratch_of_device[dev] = p;
+  }
+  gd_compress_args b = *a;
+  b.workspace = scratch_of_device[dev];
+  b.workspace_bytes = (size_t)GD_STATIC_WORKSPACE_BYTES;
+  if (workspace_out) *workspace_out = b.workspace;
+  return gd_compress(&b, stream);
+}
+
 int gd_profile_enable(int enable) {
   g_profile_on = enable != 0;
   if (!g_profile_on) g_ev_used = 0;
