@@ -179,6 +179,23 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------- replicas: the only multi-rank logic
+def max_over_ranks(local_value: float, device) -> float:
+    """The slowest rank's value (ranks are independent replicas; nothing else crosses ranks)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(local_value)
+    t = torch.tensor([local_value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_gbs(n_elements: int, steps: int, world: int, total_ms: float) -> float:
+    """Dense-gradient GB/s of the whole job: every replica moves 4 * n bytes per step."""
+    return world * 4.0 * n_elements * steps / (total_ms * 1e-3) / 1e9
+
+
 # ---------------------------------------------------------------- the CUDA arm
 def run_cuda(args):
     import torch
@@ -243,12 +260,9 @@ def run_cuda(args):
         raise RuntimeError(f"device status {stats['status']} in the timed region")
     total_ms = ev[0].elapsed_time(ev[-1])
     step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
-    value = world * 4.0 * w.n * args.steps / (total_ms * 1e-3) / 1e9
+    value = aggregate_gbs(w.n, args.steps, world, total_ms)
 
     # end to end through the host entry point: gradient in page-locked host memory, push read back
     e2e = None
@@ -275,12 +289,9 @@ def run_cuda(args):
                            means_host if two else None)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = max_over_ranks(dt, dev)
         d2h = 4 * (w.n_shards + 1) + 4 * k + (8 * (len(w.layer_off) - 1) if two else 4 * k)
-        e2e = {"value": world * 4.0 * w.n * e2e_steps / dt / 1e9, "unit": UNIT, "h2d_bytes_per_step": 4 * w.n,
+        e2e = {"value": aggregate_gbs(w.n, e2e_steps, world, dt * 1e3), "unit": UNIT, "h2d_bytes_per_step": 4 * w.n,
                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": 1e3 * dt / e2e_steps}
         del g_host, g_dev
 
