@@ -27,6 +27,7 @@ if ROOT not in sys.path:
 
 METRIC = "dense-gradient GB/s through compress+apply"
 UNIT = "GB/s"
+ADD_EMIT_DRAM_BYTES_PER_ELEMENT = 11.61   # ncu, see profiles/add_emit_kernel_flat_2p27.md
 
 
 def read_peaks():
@@ -311,16 +312,11 @@ def run_cuda(args):
         roofline["achieved"] = fused_bytes / (fused_avg_ms * 1e-3) / 1e9
         roofline["frac"] = roofline["achieved"] / peak
         roofline["avg_launch_ms"] = fused_avg_ms
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-    try:
-        with open(traffic_path) as fh:
-            tr = json.load(fh)
-        per_elt = tr.get(f"config{w.config}", tr.get("default"))
-        if per_elt is not None:
-            roofline["traffic"] = float(per_elt["add_emit_dram_bytes_per_element"]) * w.n
-            roofline["traffic_source"] = per_elt.get("source")
-    except Exception:
-        pass
+    # DRAM traffic of the fused pass from the ncu capture of the 2^27-element case of the same kernel
+    # (profiles/add_emit_kernel_flat_2p27.md): every element is read twice and written once, so the
+    # figure scales with n.
+    roofline["traffic"] = ADD_EMIT_DRAM_BYTES_PER_ELEMENT * w.n
+    roofline["traffic_source"] = "ncu dram__bytes_read.sum + dram__bytes_write.sum at n = 2^27, scaled by n"
     k_frac = sess.k_total / max(w.n, 1)
     per_surv = 16.0 if w.value_mode == B.GD_VALUES_TWO_MEANS else 24.0
     alg_step_bytes = (12.0 + per_surv * k_frac) * w.n

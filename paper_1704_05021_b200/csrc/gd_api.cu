@@ -159,6 +159,22 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, i
   return GD_OK;
 }
 
+// Start of a call in one launch: clears the control region of the workspace and writes the small
+// host-built tables, which travel as a kernel argument, behind it.
+constexpr size_t kSetupBlobBytes = 3584;
+struct SetupBlob {
+  unsigned char bytes[kSetupBlobBytes];
+};
+
+__global__ void __launch_bounds__(kThreads) setup_kernel(const __grid_constant__ SetupBlob blob, uint4* tables_dst,
+                                                         uint32_t tables_vec, uint4* zero_dst, uint64_t zero_vec) {
+  const uint64_t stride = (uint64_t)gridDim.x * kThreads;
+  const uint64_t g = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
+  for (uint64_t i = g; i < zero_vec; i += stride) zero_dst[i] = make_uint4(0u, 0u, 0u, 0u);
+  const uint4* src = reinterpret_cast<const uint4*>(blob.bytes);
+  for (uint64_t i = g; i < tables_vec; i += stride) tables_dst[i] = src[i];
+}
+
 // measurement hooks
 constexpr uint32_t kProfilePairs = 4096;
 bool g_profile_on = false;
@@ -170,6 +186,26 @@ uint64_t g_launches = 0;
 }  // namespace
 
 void note_launches(uint32_t count) { g_launches += count; }
+
+cudaError_t launch_setup(void* tables_dst, const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes,
+                         cudaStream_t stream) {
+  if (tables_bytes > kSetupBlobBytes) {   // many layers: the tables do not fit a kernel argument
+    cudaError_t e = cudaMemsetAsync(zero_dst, 0, zero_bytes, stream);
+    if (e != cudaSuccess) return e;
+    return cudaMemcpyAsync(tables_dst, tables_src, tables_bytes, cudaMemcpyHostToDevice, stream);
+  }
+  SetupBlob blob;
+  std::memcpy(blob.bytes, tables_src, tables_bytes);
+  const uint64_t zero_vec = zero_bytes / 16;   // both regions are 256-byte aligned and padded
+  uint64_t blocks = (zero_vec + kThreads * 8 - 1) / (kThreads * 8);
+  const uint64_t cap = (uint64_t)sm_count() * 4;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  setup_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(blob, (uint4*)tables_dst, (uint32_t)(tables_bytes / 16),
+                                                         (uint4*)zero_dst, zero_vec);
+  GD_LAUNCH_CHECK();
+  return cudaSuccess;
+}
 
 int sm_count() {
   static int cached = 0;
@@ -292,8 +328,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     std::memcpy(blob.data() + P.t_shard_off, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
 
     unsigned char* ws = (unsigned char*)a->workspace;
-    if (cudaMemsetAsync(ws, 0, P.zero_bytes, stream) != cudaSuccess) return GD_ERR_CUDA;
-    if (cudaMemcpyAsync(ws + P.off_tables, blob.data(), P.tables_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    if (launch_setup(ws + P.off_tables, blob.data(), P.tables_bytes, ws, P.zero_bytes, stream) != cudaSuccess)
       return GD_ERR_CUDA;
 
     DevTables T;
@@ -333,17 +368,17 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
 
     uint32_t tiles[L_COUNT];
     for (int l = 0; l < L_COUNT; ++l) tiles[l] = P.tiles[l];
-    // the dense kernels are always enqueued: they return at once unless a prediction failed
     const bool predict = !(a->flags & GD_FLAG_NO_PREDICTION);
-    if (predict && launch_sample_select(T, tiles, P.samp_total, stream) != cudaSuccess) return GD_ERR_CUDA;
+    if (predict && launch_sample_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
     if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+    // The dense kernels are always enqueued: they return at once unless a prediction failed.  The
+    // compaction that runs last also finishes the call (thresholds, shard offsets, means).
+    if (launch_dense_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+    if (launch_compact(T, tiles, true, !predict, stream) != cudaSuccess) return GD_ERR_CUDA;
     if (predict) {
       if (launch_candidate_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
-      if (launch_compact(T, tiles, false, stream) != cudaSuccess) return GD_ERR_CUDA;
+      if (launch_compact(T, tiles, false, true, stream) != cudaSuccess) return GD_ERR_CUDA;
     }
-    if (launch_dense_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
-    if (launch_compact(T, tiles, true, stream) != cudaSuccess) return GD_ERR_CUDA;
-    if (launch_finalize(T, stream) != cudaSuccess) return GD_ERR_CUDA;
     return GD_OK;
   } catch (const std::bad_alloc&) {
     return GD_ERR_INVALID_ARG;

@@ -27,12 +27,25 @@ struct ApplyDev {
   const float* means;
 };
 
+// Small shard / layer tables travel as a kernel argument (no copy to the device is needed then).
+constexpr uint32_t kInlineShards = 32, kInlineLayers = 64;
+struct ApplyInline {
+  float* params[kInlineShards];
+  uint64_t shard_off[kInlineShards + 1];
+  uint64_t layer_off[kInlineLayers + 1];
+};
+
 // Segmented scatter-add: the entries [cnt_off[0], cnt_off[n_shards]) of one push, one thread per
 // entry in a grid-stride loop.  Indices inside one push are unique, so a plain read-modify-write is
 // enough; pushes are separate launches in stream order.
-__global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__ ApplyDev A) {
+template <bool INLINE>
+__global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__ ApplyDev A,
+                                                         const __grid_constant__ ApplyInline I) {
+  float* const* params = INLINE ? I.params : A.params;
+  const uint64_t* shard_off = INLINE ? I.shard_off : A.shard_off;
+  const uint64_t* layer_off = INLINE ? I.layer_off : A.layer_off;
   const uint64_t begin = A.cnt_off[0], end = A.cnt_off[A.n_shards];
-  const uint64_t lo_all = A.shard_off[0], hi_all = A.shard_off[A.n_shards];
+  const uint64_t lo_all = shard_off[0], hi_all = shard_off[A.n_shards];
   const uint64_t stride = (uint64_t)gridDim.x * kThreads;
   for (uint64_t p = begin + (uint64_t)blockIdx.x * kThreads + threadIdx.x; p < end; p += stride) {
     const uint32_t w = __ldcs(A.idx + p);
@@ -40,14 +53,14 @@ __global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__
     float x;
     if (A.value_mode == GD_VALUES_TWO_MEANS) {
       pos = w & kAbsMask;
-      const uint32_t l = range_of(A.layer_off, A.n_layers, pos);
+      const uint32_t l = range_of(layer_off, A.n_layers, pos);
       x = __ldg(A.means + 2 * (size_t)l + (w >> 31));
     } else {
       x = __ldcs(A.val + p);
     }
     if (pos < lo_all || pos >= hi_all) continue;
-    const uint32_t j = range_of(A.shard_off, A.n_shards, pos);
-    float* dst = A.params[j] + (pos - A.shard_off[j]);
+    const uint32_t j = range_of(shard_off, A.n_shards, pos);
+    float* dst = params[j] + (pos - shard_off[j]);
     *dst = __fmaf_rn(A.alpha, x, *dst);
   }
 }
@@ -98,13 +111,21 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
     const size_t o_params = 0;
     const size_t o_shard = align_up_a(sizeof(float*) * (size_t)a->n_shards);
     const size_t o_layer = o_shard + align_up_a(sizeof(uint64_t) * ((size_t)a->n_shards + 1));
-    std::vector<unsigned char> blob(need, 0);
-    std::memcpy(blob.data() + o_params, a->params, sizeof(float*) * (size_t)a->n_shards);
-    std::memcpy(blob.data() + o_shard, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
-    if (two_means) std::memcpy(blob.data() + o_layer, a->layer_off, sizeof(uint64_t) * ((size_t)n_layers + 1));
     unsigned char* ws = (unsigned char*)a->workspace;
-    if (cudaMemcpyAsync(ws, blob.data(), need, cudaMemcpyHostToDevice, stream) != cudaSuccess) return GD_ERR_CUDA;
-
+    const bool use_inline = a->n_shards <= kInlineShards && n_layers <= kInlineLayers;
+    ApplyInline I;
+    std::memset(&I, 0, sizeof(I));
+    if (use_inline) {
+      std::memcpy(I.params, a->params, sizeof(float*) * (size_t)a->n_shards);
+      std::memcpy(I.shard_off, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
+      if (two_means) std::memcpy(I.layer_off, a->layer_off, sizeof(uint64_t) * ((size_t)n_layers + 1));
+    } else {
+      std::vector<unsigned char> blob(need, 0);
+      std::memcpy(blob.data() + o_params, a->params, sizeof(float*) * (size_t)a->n_shards);
+      std::memcpy(blob.data() + o_shard, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
+      if (two_means) std::memcpy(blob.data() + o_layer, a->layer_off, sizeof(uint64_t) * ((size_t)n_layers + 1));
+      if (cudaMemcpyAsync(ws, blob.data(), need, cudaMemcpyHostToDevice, stream) != cudaSuccess) return GD_ERR_CUDA;
+    }
     ApplyDev A;
     std::memset(&A, 0, sizeof(A));
     A.params = (float* const*)(ws + o_params);
@@ -114,13 +135,17 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
     A.n_layers = n_layers;
     A.value_mode = a->value_mode;
     A.alpha = a->alpha;
+    const unsigned grid = (unsigned)sm_count() * 8u;
     for (uint32_t w = 0; w < a->n_pushes; ++w) {
       const gd_push& p = a->pushes[w];
       A.idx = p.idx;
       A.val = p.val;
       A.cnt_off = p.shard_cnt_off;
       A.means = p.means;
-      apply_kernel<<<(unsigned)sm_count() * 8u, kThreads, 0, stream>>>(A);
+      if (use_inline)
+        apply_kernel<true><<<grid, kThreads, 0, stream>>>(A, I);
+      else
+        apply_kernel<false><<<grid, kThreads, 0, stream>>>(A, I);
       if (cudaPeekAtLastError() != cudaSuccess) return GD_ERR_CUDA;
       note_launches(1);
     }

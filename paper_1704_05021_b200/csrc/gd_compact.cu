@@ -7,12 +7,67 @@ namespace gd {
 
 namespace {
 
+// Finishes a call: thresholds, statistics, shard offsets (Section 3: the survivors, ascending in
+// index, are cut into one piece per server) and the two means (Section 5.4).  Run by one whole CTA
+// after every survivor has been written.
+__device__ void finalize_call(const DevTables& T) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
+  uint32_t n_pred = 0, n_dense = 0;
+  unsigned long long n_cand = 0;
+  for (uint32_t s = tid; s < T.n_scopes; s += kThreads) {
+    const ScopeDesc& d = T.scopes[s];
+    const ScopeState* st = T.state + s;
+    if (T.out_tau) T.out_tau[s] = d.k == 0 ? 0xFFFFFFFFu : __ldcg(&st->tau);
+    if (__ldcg(&st->used_dense)) ++n_dense; else ++n_pred;
+    n_cand += __ldcg(reinterpret_cast<const unsigned long long*>(&st->cand_count));
+  }
+  if (n_pred) atomicAdd(&T.ctl->n_scopes_predicted, n_pred);
+  if (n_dense) atomicAdd(&T.ctl->n_scopes_dense, n_dense);
+  if (n_cand) atomicAdd(reinterpret_cast<unsigned long long*>(&T.ctl->n_candidates), n_cand);
+  if (tid == 0) { T.ctl->n_scopes = T.n_scopes; T.ctl->n_kept = T.k_total; }
+  // shard j starts at the first survivor with index >= shard_off[j]: a 33-way search per warp
+  for (uint32_t j = warp; j <= T.n_shards; j += kWarps) {
+    const uint64_t bound = T.shard_off[j];
+    uint64_t lo = 0, hi = T.k_total;                 // answer in [lo, hi]
+    while (hi - lo > 32) {
+      const uint64_t span = hi - lo;
+      const uint64_t p = lo + span * (lane + 1) / 33;   // lo < p < hi, ascending in lane
+      uint32_t w = __ldcg(T.out_idx + p);
+      if (two_means) w &= kAbsMask;
+      const uint32_t c = __popc(__ballot_sync(0xFFFFFFFFu, (uint64_t)w < bound));   // probes 0..c-1 are below
+      const uint64_t nlo = c ? lo + span * c / 33 + 1 : lo;
+      const uint64_t nhi = c < 32 ? lo + span * (c + 1) / 33 : hi;
+      lo = nlo;
+      hi = nhi;
+    }
+    const uint64_t p = lo + lane;
+    bool below = false;
+    if (p < hi) {
+      uint32_t w = __ldcg(T.out_idx + p);
+      if (two_means) w &= kAbsMask;
+      below = (uint64_t)w < bound;
+    }
+    lo += __popc(__ballot_sync(0xFFFFFFFFu, below));
+    if (lane == 0) T.out_shard_cnt_off[j] = (uint32_t)lo;
+  }
+  if (two_means) {
+    for (uint32_t e = tid; e < 2 * T.n_layers; e += kThreads) {
+      const unsigned long long c = __ldcg(T.cnts + e);
+      T.out_means[e] = c ? (float)(__ldcg(T.sums + e) / (double)c) : 0.0f;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constant__ DevTables T) { finalize_call(T); }
+
 // Single-pass look-back scan with two counters per tile: keys above tau, and keys equal to tau.  An
 // element above tau goes to slot  (#above before it) + min(#ties before it, q); a tie is kept iff fewer
 // than q ties precede it.  VIEW == V_CAND walks the candidate list, V_DENSE the dense range itself.
 // CTAs take tiles from an atomic ticket until none is left.
 template <int VIEW>
-__global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
+__global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles,
+                                                           int do_finalize) {
   constexpr int LK = VIEW == V_CAND ? L_CAND : L_DCOMP;
   constexpr int ROUNDS = kTile / kThreads;   // 16 elements per thread
   __shared__ uint32_t s_tile;
@@ -22,6 +77,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   __shared__ uint32_t s_layer;
   __shared__ double s_red[kWarps][2];
   __shared__ uint32_t s_redc[kWarps][2];
+  __shared__ int s_last;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   if (VIEW == V_DENSE && !(T.flags & GD_FLAG_NO_PREDICTION) && T.ctl->dense_needed == 0u) return;
   const uint32_t* tile0 = T.tile0[LK];
@@ -170,61 +226,34 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
       }
     }
   }
-}
-
-__global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constant__ DevTables T) {
-  const uint32_t tid = threadIdx.x;
-  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
-  uint32_t n_pred = 0, n_dense = 0;
-  unsigned long long n_cand = 0;
-  for (uint32_t s = tid; s < T.n_scopes; s += kThreads) {
-    const ScopeDesc& d = T.scopes[s];
-    const ScopeState& st = T.state[s];
-    if (T.out_tau) T.out_tau[s] = d.k == 0 ? 0xFFFFFFFFu : st.tau;
-    if (st.used_dense) ++n_dense; else ++n_pred;
-    n_cand += st.cand_count;
-  }
-  if (n_pred) atomicAdd(&T.ctl->n_scopes_predicted, n_pred);
-  if (n_dense) atomicAdd(&T.ctl->n_scopes_dense, n_dense);
-  if (n_cand) atomicAdd(reinterpret_cast<unsigned long long*>(&T.ctl->n_candidates), n_cand);
-  if (tid == 0) { T.ctl->n_scopes = T.n_scopes; T.ctl->n_kept = T.k_total; }
-  // survivors are in ascending index order: shard j starts at the first index >= shard_off[j]
-  for (uint32_t j = tid; j <= T.n_shards; j += kThreads) {
-    const uint64_t bound = T.shard_off[j];
-    uint64_t lo = 0, hi = T.k_total;
-    while (lo < hi) {
-      const uint64_t mid = (lo + hi) >> 1;
-      uint32_t w = T.out_idx[mid];
-      if (two_means) w &= kAbsMask;
-      if ((uint64_t)w < bound) lo = mid + 1; else hi = mid;
-    }
-    T.out_shard_cnt_off[j] = (uint32_t)lo;
-  }
-  if (two_means) {
-    for (uint32_t e = tid; e < 2 * T.n_layers; e += kThreads) {
-      const unsigned long long c = T.cnts[e];
-      T.out_means[e] = c ? (float)(T.sums[e] / (double)c) : 0.0f;
-    }
-  }
+  if (!do_finalize) return;
+  // the last CTA to leave finishes the call
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&T.ctl->compact_done[VIEW == V_CAND ? 0 : 1], 1u) == gridDim.x - 1u) ? 1 : 0;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  finalize_call(T);
 }
 
 }  // namespace
 
-cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, cudaStream_t stream) {
-  const uint32_t total = tiles[dense ? L_DCOMP : L_CAND];
-  if (!total) return cudaSuccess;
-  const uint32_t cap = (uint32_t)sm_count() * 8u;
-  const uint32_t grid = total < cap ? total : cap;
-  if (dense)
-    compact_kernel<V_DENSE><<<grid, kThreads, 0, stream>>>(T, total);
-  else
-    compact_kernel<V_CAND><<<grid, kThreads, 0, stream>>>(T, total);
+cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream) {
+  finalize_kernel<<<1, kThreads, 0, stream>>>(T);
   GD_LAUNCH_CHECK();
   return cudaSuccess;
 }
 
-cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream) {
-  finalize_kernel<<<1, kThreads, 0, stream>>>(T);
+cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, bool finalize, cudaStream_t stream) {
+  const uint32_t total = tiles[dense ? L_DCOMP : L_CAND];
+  if (!total) return finalize ? launch_finalize(T, stream) : cudaSuccess;
+  const uint32_t cap = (uint32_t)sm_count() * 8u;
+  const uint32_t grid = total < cap ? total : cap;
+  if (dense)
+    compact_kernel<V_DENSE><<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
+  else
+    compact_kernel<V_CAND><<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
   GD_LAUNCH_CHECK();
   return cudaSuccess;
 }

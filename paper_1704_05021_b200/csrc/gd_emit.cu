@@ -2,12 +2,14 @@
 // gradient, fused with the emission of the threshold candidates.
 //
 // One CTA streams one chunk of C tiles (C * 4096 consecutive elements) of one scope:
-//   phase A  per tile: 128-bit loads of g and r, v = g + r, 128-bit store of v over r, and a
-//            16-bit mask per thread of the entries with |v| >= tau_lo (the predicted lower bound);
+//   phase A  per tile: 128-bit loads of g and r, v = g + r, 128-bit store of v over r; the rare
+//            entries with |v| >= tau_lo (the predicted lower bound) are appended, in order, to a
+//            small per-warp stash in shared memory;
 //   scan     one decoupled look-back per chunk gives the number of candidates in all earlier
 //            chunks of the scope;
-//   phase B  threads that own candidates read their v back (their own stores) and append
-//            (index, v) to the scope's candidate list, in index order.
+//   phase B  every warp copies its stash to the scope's candidate list at its final, index-ordered
+//            position.  A warp whose stash overflowed (a dense run of candidates) re-reads its own
+//            part of the chunk instead.
 // The look-back is per chunk, not per tile, so that its latency (a few L2 round trips) is paid
 // once per C * 48 KiB of traffic and the chain of prefixes never limits the streaming rate.
 #include "gd_scan.cuh"
@@ -15,6 +17,13 @@
 namespace gd {
 
 namespace {
+
+constexpr uint32_t kStash = 128;   // candidate slots per warp and chunk in shared memory
+
+struct StashEntry {
+  uint32_t idx;
+  float val;
+};
 
 // Chunks are aligned to C * kTile elements of the flat vector; a chunk that straddles a scope
 // boundary is processed once per scope, each pass touching only its own scope's elements.  Inside a
@@ -26,10 +35,12 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
   constexpr int E = C * kWarps;              // (tile, warp) counters of one chunk
   constexpr int PER = (E + 31) / 32;
   __shared__ uint32_t s_chunk;
-  __shared__ uint32_t s_cnt[E];              // per (tile, warp): count, then exclusive offset in the chunk
+  __shared__ uint32_t s_cnt[E];              // candidates per (tile, warp)
+  __shared__ uint32_t s_off[E];              // their exclusive offsets inside the chunk
   __shared__ uint64_t s_excl;
   __shared__ uint32_t s_total;
   __shared__ int s_ok;
+  __shared__ StashEntry s_stash[kWarps][kStash];
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   if (tid == 0) s_chunk = atomicAdd(&T.ctl->ticket[L_EMIT], 1u);
   __syncthreads();
@@ -44,13 +55,15 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
   const uint64_t cbase = (lo / CH + lt) * CH;
   const uint32_t tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || d.k == 0) ? 0xFFFFFFFFu : T.state[s].tau_lo;
   const uint64_t toff = (uint64_t)warp * 512u + lane * 4u;   // this thread's first element inside a tile
+  const uint32_t ltm = lanemask_lt();
+  StashEntry* stash = s_stash[warp];
 
   // ---- phase A
-  uint32_t cm[C];
-#pragma unroll
+  uint32_t fill = 0;                         // candidates of this warp so far in the chunk (warp-uniform)
+#pragma unroll 1
   for (int i = 0; i < C; ++i) {
     const uint64_t base = cbase + (uint64_t)i * kTile;
-    uint32_t cmask = 0;
+    uint32_t wc = 0;                         // candidates of this warp in this tile (warp-uniform)
     if (base >= lo && base + kTile <= hi) {
       const uint64_t e0 = base + toff;
       float4 g4[4], r4[4];
@@ -60,33 +73,63 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
       for (int j = 0; j < 4; ++j) r4[j] = *reinterpret_cast<const float4*>(T.residual + e0 + j * 128);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        float4 x;
-        x.x = __fadd_rn(g4[j].x, r4[j].x);
-        x.y = __fadd_rn(g4[j].y, r4[j].y);
-        x.z = __fadd_rn(g4[j].z, r4[j].z);
-        x.w = __fadd_rn(g4[j].w, r4[j].w);
-        *reinterpret_cast<float4*>(T.residual + e0 + j * 128) = x;
-        cmask |= ((__float_as_uint(x.x) & kAbsMask) >= tau_lo ? 1u : 0u) << (4 * j + 0);
-        cmask |= ((__float_as_uint(x.y) & kAbsMask) >= tau_lo ? 1u : 0u) << (4 * j + 1);
-        cmask |= ((__float_as_uint(x.z) & kAbsMask) >= tau_lo ? 1u : 0u) << (4 * j + 2);
-        cmask |= ((__float_as_uint(x.w) & kAbsMask) >= tau_lo ? 1u : 0u) << (4 * j + 3);
+        float x[4];
+        x[0] = __fadd_rn(g4[j].x, r4[j].x);
+        x[1] = __fadd_rn(g4[j].y, r4[j].y);
+        x[2] = __fadd_rn(g4[j].z, r4[j].z);
+        x[3] = __fadd_rn(g4[j].w, r4[j].w);
+        *reinterpret_cast<float4*>(T.residual + e0 + j * 128) = make_float4(x[0], x[1], x[2], x[3]);
+        uint32_t f = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) f |= ((__float_as_uint(x[c]) & kAbsMask) >= tau_lo ? 1u : 0u) << c;
+        if (__any_sync(0xFFFFFFFFu, f != 0u)) {
+          const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, f & 1u), b1 = __ballot_sync(0xFFFFFFFFu, f & 2u);
+          const uint32_t b2 = __ballot_sync(0xFFFFFFFFu, f & 4u), b3 = __ballot_sync(0xFFFFFFFFu, f & 8u);
+          if (f) {
+            uint32_t p = fill + wc + __popc(b0 & ltm) + __popc(b1 & ltm) + __popc(b2 & ltm) + __popc(b3 & ltm);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              if (f & (1u << c)) {
+                if (p < kStash) { stash[p].idx = (uint32_t)(e0 + j * 128 + c); stash[p].val = x[c]; }
+                ++p;
+              }
+            }
+          }
+          wc += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+        }
       }
     } else if (base < hi && base + kTile > lo) {   // tile cut by the scope (or by the end of the vector)
-#pragma unroll
+#pragma unroll 1
       for (int j = 0; j < 4; ++j) {
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+        uint32_t f = 0;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           const uint64_t e = base + toff + j * 128 + c;
           if (e >= lo && e < hi) {
-            const float x = __fadd_rn(__ldg(T.grad + e), T.residual[e]);
-            T.residual[e] = x;
-            cmask |= ((__float_as_uint(x) & kAbsMask) >= tau_lo ? 1u : 0u) << (4 * j + c);
+            x[c] = __fadd_rn(__ldg(T.grad + e), T.residual[e]);
+            T.residual[e] = x[c];
+            f |= ((__float_as_uint(x[c]) & kAbsMask) >= tau_lo ? 1u : 0u) << c;
           }
+        }
+        if (__any_sync(0xFFFFFFFFu, f != 0u)) {
+          const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, f & 1u), b1 = __ballot_sync(0xFFFFFFFFu, f & 2u);
+          const uint32_t b2 = __ballot_sync(0xFFFFFFFFu, f & 4u), b3 = __ballot_sync(0xFFFFFFFFu, f & 8u);
+          if (f) {
+            uint32_t p = fill + wc + __popc(b0 & ltm) + __popc(b1 & ltm) + __popc(b2 & ltm) + __popc(b3 & ltm);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              if (f & (1u << c)) {
+                if (p < kStash) { stash[p].idx = (uint32_t)(base + toff + j * 128 + c); stash[p].val = x[c]; }
+                ++p;
+              }
+            }
+          }
+          wc += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
         }
       }
     }
-    cm[i] = cmask;
-    const uint32_t wc = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)__popc(cmask));
+    fill += wc;
     if (lane == 0) s_cnt[i * kWarps + warp] = wc;
   }
   __syncthreads();
@@ -110,7 +153,7 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
 #pragma unroll
     for (int p = 0; p < PER; ++p) {
       const int e = (int)lane * PER + p;
-      if (e < E) s_cnt[e] = run;
+      if (e < E) s_off[e] = run;
       run += a[p];
     }
     const uint32_t total = __shfl_sync(0xFFFFFFFFu, inc, 31);
@@ -122,44 +165,63 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
   if (!s_ok) return;
   const uint64_t excl = s_excl;
 
-  // ---- phase B: append this thread's candidates
-  const uint32_t ltm = lanemask_lt();
-  const uint64_t cap = d.cand_cap;
-  uint32_t* cidx = T.cand_idx + d.cand_base;
-  float* cval = T.cand_val + d.cand_base;
+  // ---- phase B: this warp's candidates go to their final positions
+  if (fill) {
+    const uint64_t cap = d.cand_cap;
+    uint32_t* cidx = T.cand_idx + d.cand_base;
+    float* cval = T.cand_val + d.cand_base;
+    if (fill <= kStash) {
+      uint32_t a = 0;                        // first stash entry of tile i
+#pragma unroll 1
+      for (int i = 0; i < C; ++i) {
+        const uint32_t c = s_cnt[i * kWarps + warp];
+        const uint64_t dst = excl + s_off[i * kWarps + warp];
+        for (uint32_t e = lane; e < c; e += 32) {
+          const uint64_t pos = dst + e;
+          if (pos < cap) { cidx[pos] = stash[a + e].idx; cval[pos] = stash[a + e].val; }
+        }
+        a += c;
+      }
+    } else {
+      // more candidates than the stash holds: read this warp's elements back (they are v now)
+#pragma unroll 1
+      for (int i = 0; i < C; ++i) {
+        if (s_cnt[i * kWarps + warp] == 0u) continue;
+        uint64_t run = excl + s_off[i * kWarps + warp];
+        const uint64_t base = cbase + (uint64_t)i * kTile;
+#pragma unroll 1
+        for (int j = 0; j < 4; ++j) {
+          float x[4] = {0.f, 0.f, 0.f, 0.f};
+          uint32_t f = 0;
 #pragma unroll
-  for (int i = 0; i < C; ++i) {
-    const uint32_t cmask = cm[i];
-    if (!__any_sync(0xFFFFFFFFu, cmask != 0u)) continue;
-    uint64_t run = excl + s_cnt[i * kWarps + warp];
-    const uint64_t e0 = cbase + (uint64_t)i * kTile + toff;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint32_t f = (cmask >> (4 * j)) & 15u;
-      if (!__any_sync(0xFFFFFFFFu, f != 0u)) continue;
-      const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, f & 1u), b1 = __ballot_sync(0xFFFFFFFFu, f & 2u);
-      const uint32_t b2 = __ballot_sync(0xFFFFFFFFu, f & 4u), b3 = __ballot_sync(0xFFFFFFFFu, f & 8u);
-      if (f) {
-        uint64_t pos = run + __popc(b0 & ltm) + __popc(b1 & ltm) + __popc(b2 & ltm) + __popc(b3 & ltm);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          if (f & (1u << c)) {
-            if (pos < cap) {
-              const uint64_t e = e0 + j * 128 + c;
-              cidx[pos] = (uint32_t)e;
-              cval[pos] = T.residual[e];      // v, as stored by this thread in phase A
+          for (int c = 0; c < 4; ++c) {
+            const uint64_t e = base + toff + j * 128 + c;
+            if (e >= lo && e < hi) {
+              x[c] = T.residual[e];
+              f |= ((__float_as_uint(x[c]) & kAbsMask) >= tau_lo ? 1u : 0u) << c;
             }
-            ++pos;
           }
+          const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, f & 1u), b1 = __ballot_sync(0xFFFFFFFFu, f & 2u);
+          const uint32_t b2 = __ballot_sync(0xFFFFFFFFu, f & 4u), b3 = __ballot_sync(0xFFFFFFFFu, f & 8u);
+          if (f) {
+            uint64_t pos = run + __popc(b0 & ltm) + __popc(b1 & ltm) + __popc(b2 & ltm) + __popc(b3 & ltm);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              if (f & (1u << c)) {
+                if (pos < cap) { cidx[pos] = (uint32_t)(base + toff + j * 128 + c); cval[pos] = x[c]; }
+                ++pos;
+              }
+            }
+          }
+          run += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
         }
       }
-      run += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
     }
   }
   if (tid == 0 && lt == nchunks - 1) {
     const uint64_t m = excl + s_total;
     T.state[s].cand_count = m;
-    if (!(T.flags & GD_FLAG_NO_PREDICTION) && (m < d.k || m > cap)) atomicAdd(&T.ctl->dense_needed, 1u);
+    if (!(T.flags & GD_FLAG_NO_PREDICTION) && (m < d.k || m > d.cand_cap)) atomicAdd(&T.ctl->dense_needed, 1u);
   }
 }
 

@@ -70,6 +70,9 @@ struct Ctl {             // zeroed at the start of every call
   uint32_t n_scopes_predicted;
   uint32_t n_scopes_dense;
   uint32_t dense_needed;   // scopes whose prediction failed (set by the fused pass)
+  uint32_t barrier[3];     // grid barriers of the three selection kernels
+  uint32_t compact_done[2];// CTAs of each compaction kernel that have finished
+  uint32_t pad;
   uint64_t n_candidates;
   uint64_t n_kept;
 };
@@ -144,7 +147,7 @@ __device__ __forceinline__ uint32_t range_of(const uint64_t* __restrict__ off, u
   uint32_t lo = 0, hi = count;
   while (hi - lo > 1) {
     uint32_t mid = (lo + hi) >> 1;
-    if (__ldg(off + mid) <= x) lo = mid; else hi = mid;
+    if (off[mid] <= x) lo = mid; else hi = mid;
   }
   return lo;
 }
@@ -158,11 +161,13 @@ __device__ __forceinline__ bool predicted_ok(const DevTables& T, const ScopeDesc
 }
 
 // Host-side launchers of the kernel groups (one per .cu file); `tiles` is indexed by Launch.
-cudaError_t launch_sample_select(const DevTables& T, const uint32_t* tiles, uint64_t samp_total, cudaStream_t stream);
+cudaError_t launch_setup(void* tables_dst, const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes,
+                         cudaStream_t stream);
+cudaError_t launch_sample_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_candidate_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_dense_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
-cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, cudaStream_t stream);
+cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, bool finalize, cudaStream_t stream);
 cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream);
 int sm_count();   // multiprocessors of the current device (0 on error)
 

@@ -3,6 +3,11 @@
 //   the sample   -> tau_lo, the predicted lower bound used by the fused pass,
 //   the candidate list the fused pass emitted -> tau and the tie quota (the usual case),
 //   the dense range itself -> the same, for scopes whose prediction failed.
+//
+// One cooperative launch does a whole selection: per pass every CTA histograms one digit of the
+// 31-bit magnitude key (11 + 10 + 10 bits) over its share of the tiles, the grid meets at a
+// barrier, one CTA per scope turns the histogram into the next digit, and the grid meets again.
+// The barrier is a counter in the workspace; its wait is bounded like every other wait here.
 #include "gd_internal.cuh"
 
 namespace gd {
@@ -14,177 +19,239 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
   return x;
 }
 
-// One thread per sample: stratum li of scope s covers [a, b) of the scope and one position inside
-// it is read.  The sample only steers the prediction; any sample gives the same final result.
-__global__ void __launch_bounds__(kThreads) sample_gather_kernel(const __grid_constant__ DevTables T,
-                                                                 uint64_t samp_total) {
-  const uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
-  if (i >= samp_total) return;
-  const uint32_t s = range_of(T.samp_off, T.n_scopes, i);
-  const ScopeDesc& d = T.scopes[s];
-  const uint64_t li = i - d.samp_base;
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// All CTAs of a cooperative launch meet here.  `phase` counts the barriers this CTA has passed.
+// Returns false (after recording GD_ERR_DEVICE_TIMEOUT) if the others did not arrive in time.
+__device__ bool grid_barrier(uint32_t* counter, uint32_t& phase, Ctl* ctl) {
+  __shared__ int s_pass;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t target = (++phase) * gridDim.x;
+    __threadfence();
+    atomicAdd(counter, 1u);
+    uint32_t spins = 0;
+    int ok = 1;
+    while (ld_acquire_u32(counter) < target) {
+      if (++spins > kLookbackSpinLimit) { ok = 0; break; }
+      if (spins > 4) __nanosleep(40);
+    }
+    if (!ok) atomicCAS(&ctl->status, (int)GD_OK, (int)GD_ERR_DEVICE_TIMEOUT);
+    s_pass = ok;
+  } else {
+    ++phase;
+  }
+  __syncthreads();
+  return s_pass != 0;
+}
+
+// The value of sample i: stratum li of scope s covers [a, b) of the scope and one position inside it
+// is read.  The sample only steers the prediction; any sample gives the same final result.
+__device__ __forceinline__ float sample_value(const DevTables& T, const ScopeDesc& d, uint32_t s, uint64_t li) {
   const uint64_t ns = d.hi - d.lo, m = d.samp_m;
   const uint64_t a = (li * ns) / m, b = ((li + 1) * ns) / m;
   const uint64_t width = b - a;
   uint64_t pos = d.lo + a;
   if (width > 1) pos += mix32((uint32_t)li * 0x9E3779B9u + s) % width;
-  T.samp_val[i] = __fadd_rn(__ldg(T.grad + pos), T.residual[pos]);
+  return __fadd_rn(__ldg(T.grad + pos), T.residual[pos]);
 }
 
-// One pass histograms one digit of the 31-bit magnitude key among the elements that match the
-// digits fixed so far; the last CTA of a scope to finish turns the histogram into the next digit.
-// After three passes (11 + 10 + 10 bits) the state holds the rank-th largest key, the number of
-// keys above it and how many keys equal to it belong to the top `rank`.
 template <int VIEW>
-__global__ void __launch_bounds__(kThreads) select_pass_kernel(const __grid_constant__ DevTables T, int pass,
-                                                               uint32_t total_tiles) {
+__device__ __forceinline__ bool view_active(const DevTables& T, const ScopeDesc& d, const ScopeState* st) {
+  if (VIEW == V_SAMPLE) return d.samp_m != 0;
+  const bool pred = predicted_ok(T, d, *st);
+  return VIEW == V_CAND ? pred : !pred;
+}
+
+template <int VIEW>
+__global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
   constexpr int LK = VIEW == V_SAMPLE ? L_SAMP : (VIEW == V_CAND ? L_CAND : L_DSEL);
   constexpr uint32_t TILE = VIEW == V_DENSE ? kDenseSelTile : kTile;
+  constexpr int PASSES = VIEW == V_SAMPLE ? 2 : 3;   // the prediction needs 21 bits only
+  constexpr uint32_t NONE = 0xFFFFFFFFu;
   __shared__ uint32_t sh[kRadixBins0];
   __shared__ unsigned long long s_warp[kWarps];
-  __shared__ int s_last;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-  if (T.ctl->status != GD_OK) return;   // set only by an earlier kernel of this call
+  if (T.ctl->status != GD_OK) return;   // set only by an earlier kernel of this call: uniform over the grid
   if (VIEW == V_DENSE && !(T.flags & GD_FLAG_NO_PREDICTION) && T.ctl->dense_needed == 0u) return;
   const uint32_t* tile0 = T.tile0[LK];
-  const int shift = pass == 0 ? kShift0 : (pass == 1 ? kShift1 : kShift2);
-  const int bits = pass == 0 ? kRadixBits0 : 10;
-  const uint32_t nbins = 1u << bits;
-  const int pshift = pass == 1 ? kShift0 : kShift1;   // shift that exposes the digits fixed so far
+  const uint32_t per = (total_tiles + gridDim.x - 1) / gridDim.x;
+  const uint32_t t_beg = blockIdx.x * per;
+  const uint32_t t_end = (t_beg + per < total_tiles) ? t_beg + per : total_tiles;
+  uint32_t phase = 0;
 
-  for (uint32_t t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-    const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
-    const ScopeDesc& d = T.scopes[s];
-    ScopeState* st = T.state + s;
-    const uint32_t first = __ldg(tile0 + s), ntiles = __ldg(tile0 + s + 1) - first;
-    const uint32_t lt = t - first;
+  for (int pass = 0; pass < PASSES; ++pass) {
+    const int shift = pass == 0 ? kShift0 : (pass == 1 ? kShift1 : kShift2);
+    const int bits = pass == 0 ? kRadixBits0 : 10;
+    const uint32_t nbins = 1u << bits;
+    const int pshift = pass == 1 ? kShift0 : kShift1;   // shift that exposes the digits fixed so far
 
-    uint64_t len, rank;
-    const float* vals;
-    if (VIEW == V_SAMPLE) {
-      len = d.samp_m; vals = T.samp_val + d.samp_base; rank = d.samp_rank;
-    } else if (VIEW == V_CAND) {
-      if (!predicted_ok(T, d, *st)) continue;
-      len = st->cand_count; vals = T.cand_val + d.cand_base; rank = d.k;
-    } else {
-      if (predicted_ok(T, d, *st)) continue;
-      len = d.hi - d.lo; vals = T.residual + d.lo; rank = d.k;
-    }
-    uint32_t prefix = 0;
-    uint64_t gt = 0;
-    if (pass > 0) { prefix = st->sel[VIEW].prefix; rank = st->sel[VIEW].rank; gt = st->sel[VIEW].gt; }
-
-    __syncthreads();                       // previous iteration is done with sh / s_last
+    // ---- histogram of this CTA's tiles; flushed whenever the scope changes
     for (uint32_t b = tid; b < nbins; b += kThreads) sh[b] = 0;
     __syncthreads();
-    const uint64_t beg = (uint64_t)lt * TILE;
-    const uint64_t end = (beg + TILE < len) ? beg + TILE : len;
-    for (uint64_t i0 = beg + (tid & ~31u); i0 < end; i0 += kThreads) {   // warp-uniform trip count
-      const uint64_t i = i0 + lane;
-      uint32_t digit = 0xFFFFFFFFu;                                      // "does not count"
-      if (i < end) {
-        const uint32_t key = __float_as_uint(vals[i]) & kAbsMask;
-        if (pass == 0 || (key >> pshift) == prefix) digit = (key >> shift) & (nbins - 1u);
+    uint32_t cur = NONE;                                // scope the shared histogram belongs to
+    for (uint32_t t = t_beg; t < t_end; ++t) {
+      const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
+      const ScopeDesc& d = T.scopes[s];
+      ScopeState* st = T.state + s;
+      if (!view_active<VIEW>(T, d, st)) continue;
+      if (s != cur) {
+        if (cur != NONE) {
+          __syncthreads();
+          unsigned long long* gh = T.hist + (size_t)cur * kRadixBins0;
+          for (uint32_t b = tid; b < nbins; b += kThreads) {
+            const uint32_t c = sh[b];
+            if (c) atomicAdd(gh + b, (unsigned long long)c);
+            sh[b] = 0;
+          }
+          __syncthreads();
+        }
+        cur = s;
       }
-      const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, digit, 0);
-      if (__all_sync(0xFFFFFFFFu, digit == d0)) {        // whole warp in one bin: one add
-        if (lane == 0 && d0 != 0xFFFFFFFFu) atomicAdd(&sh[d0], 32u);
-      } else if (digit != 0xFFFFFFFFu) {
-        atomicAdd(&sh[digit], 1u);
+      const uint32_t lt = t - __ldg(tile0 + s);
+      uint64_t len;
+      const float* vals;
+      if (VIEW == V_SAMPLE) { len = d.samp_m; vals = T.samp_val + d.samp_base; }
+      else if (VIEW == V_CAND) { len = st->cand_count; vals = T.cand_val + d.cand_base; }
+      else { len = d.hi - d.lo; vals = T.residual + d.lo; }
+      const uint32_t prefix = pass > 0 ? __ldcg(&st->sel[VIEW].prefix) : 0u;
+      const uint64_t beg = (uint64_t)lt * TILE;
+      const uint64_t end = (beg + TILE < len) ? beg + TILE : len;
+      for (uint64_t i0 = beg + (tid & ~31u); i0 < end; i0 += kThreads) {   // warp-uniform trip count
+        const uint64_t i = i0 + lane;
+        uint32_t digit = NONE;                                             // "does not count"
+        if (i < end) {
+          float x;
+          if (VIEW == V_SAMPLE && pass == 0) {
+            x = sample_value(T, d, s, i);
+            T.samp_val[d.samp_base + i] = x;
+          } else {
+            x = vals[i];
+          }
+          const uint32_t key = __float_as_uint(x) & kAbsMask;
+          if (pass == 0 || (key >> pshift) == prefix) digit = (key >> shift) & (nbins - 1u);
+        }
+        // one shared-memory add per distinct digit in the warp
+        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
+        if (digit != NONE && lane == (uint32_t)__ffs((int)peers) - 1u) atomicAdd(&sh[digit], (uint32_t)__popc(peers));
       }
     }
     __syncthreads();
-    unsigned long long* ghist = T.hist + (size_t)s * kRadixBins0;
-    for (uint32_t b = tid; b < nbins; b += kThreads) {
-      const uint32_t c = sh[b];
-      if (c) atomicAdd(ghist + b, (unsigned long long)c);
+    if (cur != NONE) {
+      unsigned long long* gh = T.hist + (size_t)cur * kRadixBins0;
+      for (uint32_t b = tid; b < nbins; b += kThreads) {
+        const uint32_t c = sh[b];
+        if (c) atomicAdd(gh + b, (unsigned long long)c);
+      }
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(&st->done[VIEW][pass], 1u) == ntiles - 1u) ? 1 : 0;
-    __syncthreads();
-    if (!s_last) continue;
-    __threadfence();
+    if (!grid_barrier(&T.ctl->barrier[VIEW], phase, T.ctl)) return;
 
-    // Last CTA of the scope: thread x owns the bins [top - C + 1, top], top = nbins - 1 - x * C.
-    const uint32_t C = nbins / kThreads;
-    const uint32_t top = nbins - 1u - tid * C;
-    unsigned long long cs = 0;
-    for (uint32_t j = 0; j < C; ++j) cs += __ldcg(ghist + top - j);
-    unsigned long long inc = cs;
+    // ---- one CTA per scope: histogram -> next digit.  Thread x owns the bins [top - C + 1, top].
+    for (uint32_t s = blockIdx.x; s < T.n_scopes; s += gridDim.x) {
+      const ScopeDesc& d = T.scopes[s];
+      ScopeState* st = T.state + s;
+      if (!view_active<VIEW>(T, d, st)) continue;
+      uint64_t rank = VIEW == V_SAMPLE ? d.samp_rank : d.k;
+      uint32_t prefix = 0;
+      uint64_t gt = 0;
+      if (pass > 0) {
+        prefix = __ldcg(&st->sel[VIEW].prefix);
+        rank = __ldcg(&st->sel[VIEW].rank);
+        gt = __ldcg(&st->sel[VIEW].gt);
+      }
+      unsigned long long* gh = T.hist + (size_t)s * kRadixBins0;
+      const uint32_t C = nbins / kThreads;                 // 8 or 4 bins per thread
+      const uint32_t top = nbins - 1u - tid * C;
+      unsigned long long bin[8];
+      unsigned long long cs = 0;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-      if ((int)lane >= o) inc += y;
-    }
-    if (lane == 31) s_warp[warp] = inc;
-    __syncthreads();
-    unsigned long long above = inc - cs;
-    for (uint32_t w = 0; w < warp; ++w) above += s_warp[w];
-    if (tid == kThreads - 1 && above + cs < rank) atomicCAS(&T.ctl->status, (int)GD_OK, (int)GD_ERR_INTERNAL);
-    const bool owner = rank == 0 ? (tid == 0) : (above < rank && rank <= above + cs);
-    if (owner) {
-      uint32_t digit = nbins - 1u;
-      unsigned long long acc = 0;
-      if (rank != 0) {
-        acc = above;
-        for (uint32_t j = 0; j < C; ++j) {
-          const unsigned long long c = __ldcg(ghist + top - j);
-          if (acc + c >= rank) { digit = top - j; break; }
-          acc += c;
+      for (uint32_t j = 0; j < 8; ++j) {
+        bin[j] = j < C ? __ldcg(gh + top - j) : 0ull;
+        cs += bin[j];
+      }
+      unsigned long long inc = cs;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if ((int)lane >= o) inc += y;
+      }
+      __syncthreads();                                     // s_warp free again
+      if (lane == 31) s_warp[warp] = inc;
+      __syncthreads();
+      unsigned long long above = inc - cs;
+      for (uint32_t w = 0; w < warp; ++w) above += s_warp[w];
+      if (tid == kThreads - 1 && above + cs < rank) atomicCAS(&T.ctl->status, (int)GD_OK, (int)GD_ERR_INTERNAL);
+      const bool owner = rank == 0 ? (tid == 0) : (above < rank && rank <= above + cs);
+      if (owner) {
+        uint32_t digit = nbins - 1u;
+        unsigned long long acc = 0;
+        if (rank != 0) {
+          acc = above;
+#pragma unroll
+          for (uint32_t j = 0; j < 8; ++j) {
+            if (j < C) {
+              if (acc + bin[j] >= rank) { digit = top - j; break; }
+              acc += bin[j];
+            }
+          }
+        }
+        const uint32_t nprefix = (prefix << bits) | digit;
+        const uint64_t nrank = rank - acc, ngt = gt + acc;
+        st->sel[VIEW].prefix = nprefix;
+        st->sel[VIEW].rank = nrank;
+        st->sel[VIEW].gt = ngt;
+        if (pass == PASSES - 1) {
+          if (VIEW == V_SAMPLE) {
+            st->tau_lo = nprefix << kShift1;               // lower edge of the 21-bit bucket
+          } else {
+            st->tau = nprefix; st->q = nrank; st->gt = ngt;
+            if (VIEW == V_DENSE) st->used_dense = 1u;
+          }
         }
       }
-      const uint32_t nprefix = (prefix << bits) | digit;
-      const uint64_t nrank = rank - acc, ngt = gt + acc;
-      st->sel[VIEW].prefix = nprefix;
-      st->sel[VIEW].rank = nrank;
-      st->sel[VIEW].gt = ngt;
-      if (pass == 2) {
-        if (VIEW == V_SAMPLE) {
-          st->tau_lo = nprefix;
-        } else {
-          st->tau = nprefix; st->q = nrank; st->gt = ngt;
-          if (VIEW == V_DENSE) st->used_dense = 1u;
-        }
-      }
+      for (uint32_t b = tid; b < nbins; b += kThreads) gh[b] = 0ull;   // ready for the next pass
     }
-    __syncthreads();
-    for (uint32_t b = tid; b < nbins; b += kThreads) ghist[b] = 0ull;   // ready for the next pass
+    if (pass + 1 < PASSES && !grid_barrier(&T.ctl->barrier[VIEW], phase, T.ctl)) return;
   }
+}
+
+template <int VIEW>
+cudaError_t launch_select(const DevTables& T, uint32_t total_tiles, uint32_t ctas_per_sm, cudaStream_t stream) {
+  if (!total_tiles) return cudaSuccess;
+  static int resident = 0;                                 // co-resident CTAs per SM of this kernel
+  if (resident == 0) {
+    int r = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, select_kernel<VIEW>, kThreads, 0) != cudaSuccess || r <= 0)
+      return cudaErrorLaunchFailure;
+    resident = r;
+  }
+  const uint32_t per_sm = ctas_per_sm < (uint32_t)resident ? ctas_per_sm : (uint32_t)resident;
+  uint32_t grid = (uint32_t)sm_count() * per_sm;
+  if (grid > total_tiles) grid = total_tiles;
+  DevTables Tc = T;
+  void* args[] = {(void*)&Tc, (void*)&total_tiles};
+  cudaError_t e = cudaLaunchCooperativeKernel((const void*)select_kernel<VIEW>, dim3(grid), dim3(kThreads), args, 0, stream);
+  if (e != cudaSuccess) return e;
+  note_launches(1);
+  return cudaSuccess;
 }
 
 }  // namespace
 
-cudaError_t launch_sample_select(const DevTables& T, const uint32_t* tiles, uint64_t samp_total, cudaStream_t stream) {
-  if (!samp_total) return cudaSuccess;
-  const uint32_t blocks = (uint32_t)((samp_total + kThreads - 1) / kThreads);
-  sample_gather_kernel<<<blocks, kThreads, 0, stream>>>(T, samp_total);
-  GD_LAUNCH_CHECK();
-  for (int pass = 0; pass < 3; ++pass) {
-    select_pass_kernel<V_SAMPLE><<<tiles[L_SAMP], kThreads, 0, stream>>>(T, pass, tiles[L_SAMP]);
-    GD_LAUNCH_CHECK();
-  }
-  return cudaSuccess;
+cudaError_t launch_sample_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
+  return launch_select<V_SAMPLE>(T, tiles[L_SAMP], 2, stream);
 }
 
 cudaError_t launch_candidate_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
-  if (!tiles[L_CAND]) return cudaSuccess;
-  for (int pass = 0; pass < 3; ++pass) {
-    select_pass_kernel<V_CAND><<<tiles[L_CAND], kThreads, 0, stream>>>(T, pass, tiles[L_CAND]);
-    GD_LAUNCH_CHECK();
-  }
-  return cudaSuccess;
+  return launch_select<V_CAND>(T, tiles[L_CAND], 2, stream);
 }
 
 cudaError_t launch_dense_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
-  if (!tiles[L_DSEL]) return cudaSuccess;
-  const uint32_t cap = (uint32_t)sm_count() * 8u;
-  const uint32_t grid = tiles[L_DSEL] < cap ? tiles[L_DSEL] : cap;
-  for (int pass = 0; pass < 3; ++pass) {
-    select_pass_kernel<V_DENSE><<<grid, kThreads, 0, stream>>>(T, pass, tiles[L_DSEL]);
-    GD_LAUNCH_CHECK();
-  }
-  return cudaSuccess;
+  return launch_select<V_DENSE>(T, tiles[L_DSEL], 8, stream);
 }
 
 }  // namespace gd

@@ -270,3 +270,16 @@ def test_config5_full_scale_properties(cuda_device):
         p_before[idx] += val
         assert torch.equal(params.view(torch.int32), p_before.view(torch.int32))
         del v, keys, expect_res, p_before, g
+
+
+@pytest.mark.parametrize("value_mode", [B.GD_VALUES_FP32, B.GD_VALUES_TWO_MEANS])
+def test_many_layers_and_shards(cuda_device, value_mode):
+    """More layers and shards than fit a kernel argument: the tables go through the workspace instead."""
+    rng = np.random.default_rng(99)
+    sizes = [int(x) for x in rng.integers(0, 9000, size=70)]
+    sizes[5] = 0
+    sizes[17] = 70_000
+    for scope_mode in (B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER):
+        w = W.small_layered(len(sizes), sizes, 980_000, scope_mode, value_mode, 40)
+        grads = [torch.from_numpy(rng.laplace(0, 1e-3, w.n).astype(np.float32)) for _ in range(2)]
+        run_steps(w, cuda_device, 2, grads=grads)
