@@ -230,14 +230,17 @@ int gd_step_host(const gd_compress_args* args, const gd_apply_args* apply, const
 int gd_compress_static(const gd_compress_args* args, void* stream, const void** workspace_out);
 
 /*
- * Measurement hooks (no counterpart in the paper).  While enabled, every gd_compress call records
- * a pair of CUDA events on its stream around the fused full pass (the kernel that streams the
- * dense gradient and residual once); gd_profile_collect waits for the recorded pairs, writes their
- * durations in milliseconds (oldest first, at most `capacity`) and forgets them.  At most 4096
- * pairs are held between two collects; later launches are not recorded.  Not thread-safe.
+ * Measurement hooks (no counterpart in the paper).  gd_profile_enable(1) makes every gd_compress
+ * record a pair of CUDA events on its stream around the fused full pass (the kernel that streams
+ * the dense gradient and residual once); gd_profile_enable(2) brackets every kernel the library
+ * launches; 0 switches the hooks off.  gd_profile_collect waits for the recorded pairs, writes their
+ * durations in milliseconds (oldest first, at most `capacity`) and, if tags_out is not NULL, which
+ * kernel each belongs to (0 setup, 1 sample selection, 2 fused pass, 3 dense selection, 4 dense
+ * compaction, 5 candidate selection, 6 candidate compaction, 7 finalize, 8 apply), then forgets them.
+ * At most 4096 pairs are held between two collects; later launches are not recorded.  Not thread-safe.
  */
-int gd_profile_enable(int enable);
-int gd_profile_collect(float* ms_out, uint32_t capacity, uint32_t* count_out);
+int gd_profile_enable(int mode);
+int gd_profile_collect(float* ms_out, uint32_t* tags_out, uint32_t capacity, uint32_t* count_out);
 
 /* Number of kernels this library has launched in this process (memsets and copies not counted). */
 int gd_launch_count(uint64_t* count_out);

@@ -109,7 +109,7 @@ def load_library():
     lib.gd_step_host.argtypes = [C.POINTER(_CompressArgs), C.POINTER(_ApplyArgs), C.POINTER(_HostIo), C.c_void_p]
     lib.gd_compress_static.argtypes = [C.POINTER(_CompressArgs), C.c_void_p, C.POINTER(C.c_void_p)]
     lib.gd_profile_enable.argtypes = [C.c_int]
-    lib.gd_profile_collect.argtypes = [C.POINTER(C.c_float), C.c_uint32, C.POINTER(C.c_uint32)]
+    lib.gd_profile_collect.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_uint32), C.c_uint32, C.POINTER(C.c_uint32)]
     lib.gd_launch_count.argtypes = [C.POINTER(C.c_uint64)]
     for name in EXPORTS:
         if name != "gd_status_string":
@@ -251,14 +251,22 @@ def gd_step_host(call: CompressCall, apply: Optional[ApplyCall], grad_host: torc
     _check(load_library().gd_step_host(C.byref(call.args), ap, C.byref(io), _stream_handle(stream)), "gd_step_host")
 
 
-def gd_profile_enable(enable: bool) -> None:
-    _check(load_library().gd_profile_enable(1 if enable else 0), "gd_profile_enable")
+PROFILE_TAGS = ["setup", "sample_select", "add_emit", "dense_select", "dense_compact", "cand_select", "cand_compact",
+                "finalize", "apply"]
 
 
-def gd_profile_collect(capacity: int = 4096) -> list:
+def gd_profile_enable(mode) -> None:
+    """0 / False: off; 1 / True: time the fused pass of every gd_compress; 2: time every kernel."""
+    _check(load_library().gd_profile_enable(int(mode)), "gd_profile_enable")
+
+
+def gd_profile_collect(capacity: int = 4096, with_tags: bool = False):
     buf = (C.c_float * capacity)()
+    tags = (C.c_uint32 * capacity)()
     cnt = C.c_uint32(0)
-    _check(load_library().gd_profile_collect(buf, capacity, C.byref(cnt)), "gd_profile_collect")
+    _check(load_library().gd_profile_collect(buf, tags, capacity, C.byref(cnt)), "gd_profile_collect")
+    if with_tags:
+        return [(PROFILE_TAGS[tags[i]], buf[i]) for i in range(cnt.value)]
     return [buf[i] for i in range(cnt.value)]
 
 

@@ -14,6 +14,9 @@ namespace {
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
+// Sample size per scope: kSampleFactor expected samples above the threshold, within [min, max].
+constexpr double kSampleFactor = 256.0, kSampleMin = 16384.0, kSampleMax = 262144.0;
+
 inline uint64_t kept_count(uint64_t n, uint32_t drop_ppm) {
   return n - (n * (uint64_t)drop_ppm) / 1000000ull;   // n <= 2^32, drop_ppm <= 1e6: no overflow
 }
@@ -26,9 +29,9 @@ inline uint64_t kept_count(uint64_t n, uint32_t drop_ppm) {
 // affects results: a scope whose prediction fails is selected densely.
 void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint64_t* cap) {
   if (k == 0 || ns == 0) { *m = 0; *rank = 0; *cap = 0; return; }
-  double target = 1024.0 * (double)ns / (double)k;
-  if (target < 32768.0) target = 32768.0;
-  if (target > 1048576.0) target = 1048576.0;
+  double target = kSampleFactor * (double)ns / (double)k;
+  if (target < kSampleMin) target = kSampleMin;
+  if (target > kSampleMax) target = kSampleMax;
   const uint64_t mt = (uint64_t)target;
   if (mt * 2 >= ns) {
     *m = ns;
@@ -136,7 +139,7 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, i
   size_t off = 0;
   P->off_ctl = off;          off = align_up(off + sizeof(Ctl));
   P->off_state = off;        off = align_up(off + sizeof(ScopeState) * ns_count);
-  P->off_hist = off;         off = align_up(off + sizeof(unsigned long long) * kRadixBins0 * (size_t)ns_count);
+  P->off_hist = off;         off = align_up(off + sizeof(unsigned long long) * kHistBinsPerScope * (size_t)ns_count);
   P->off_sums = off;         off = align_up(off + sizeof(double) * 2 * (size_t)n_layers);
   P->off_cnts = off;         off = align_up(off + sizeof(unsigned long long) * 2 * (size_t)n_layers);
   P->off_desc_emit = off;    off = align_up(off + 16 * (size_t)P->tiles[L_EMIT]);
@@ -177,8 +180,9 @@ __global__ void __launch_bounds__(kThreads) setup_kernel(const __grid_constant__
 
 // measurement hooks
 constexpr uint32_t kProfilePairs = 4096;
-bool g_profile_on = false;
+int g_profile_mode = 0;   // 0 off, 1 the fused pass only, 2 every kernel
 cudaEvent_t g_ev_begin[kProfilePairs], g_ev_end[kProfilePairs];
+uint32_t g_ev_tag[kProfilePairs];
 uint32_t g_ev_created = 0, g_ev_used = 0;
 bool g_pair_open = false;
 uint64_t g_launches = 0;
@@ -194,6 +198,7 @@ cudaError_t launch_setup(void* tables_dst, const void* tables_src, size_t tables
     if (e != cudaSuccess) return e;
     return cudaMemcpyAsync(tables_dst, tables_src, tables_bytes, cudaMemcpyHostToDevice, stream);
   }
+  ProfileScope prof(stream, PT_SETUP);
   SetupBlob blob;
   std::memcpy(blob.bytes, tables_src, tables_bytes);
   const uint64_t zero_vec = zero_bytes / 16;   // both regions are 256-byte aligned and padded
@@ -218,8 +223,8 @@ int sm_count() {
   return cached;
 }
 
-void profile_mark(cudaStream_t stream, bool begin) {
-  if (!g_profile_on) return;
+void profile_mark(cudaStream_t stream, bool begin, uint32_t tag) {
+  if (g_profile_mode == 0 || (g_profile_mode == 1 && tag != PT_ADD_EMIT)) return;
   if (begin) {
     g_pair_open = false;
     if (g_ev_used >= kProfilePairs) return;
@@ -231,6 +236,7 @@ void profile_mark(cudaStream_t stream, bool begin) {
     if (cudaEventRecord(g_ev_begin[g_ev_used], stream) == cudaSuccess) g_pair_open = true;
   } else if (g_pair_open) {
     cudaEventRecord(g_ev_end[g_ev_used], stream);
+    g_ev_tag[g_ev_used] = tag;
     ++g_ev_used;
     g_pair_open = false;
   }
@@ -439,13 +445,14 @@ int gd_compress_static(const gd_compress_args* a, void* stream, const void** wor
   return gd_compress(&b, stream);
 }
 
-int gd_profile_enable(int enable) {
-  g_profile_on = enable != 0;
-  if (!g_profile_on) g_ev_used = 0;
+int gd_profile_enable(int mode) {
+  if (mode < 0 || mode > 2) return GD_ERR_INVALID_ARG;
+  g_profile_mode = mode;
+  if (mode == 0) g_ev_used = 0;
   return GD_OK;
 }
 
-int gd_profile_collect(float* ms_out, uint32_t capacity, uint32_t* count_out) {
+int gd_profile_collect(float* ms_out, uint32_t* tags_out, uint32_t capacity, uint32_t* count_out) {
   if (!count_out || (capacity && !ms_out)) return GD_ERR_INVALID_ARG;
   uint32_t w = 0;
   int rc = GD_OK;
@@ -456,7 +463,11 @@ int gd_profile_collect(float* ms_out, uint32_t capacity, uint32_t* count_out) {
       rc = GD_ERR_CUDA;
       break;
     }
-    if (w < capacity) ms_out[w++] = ms;
+    if (w < capacity) {
+      ms_out[w] = ms;
+      if (tags_out) tags_out[w] = g_ev_tag[i];
+      ++w;
+    }
   }
   g_ev_used = 0;
   *count_out = w;

@@ -142,6 +142,7 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
       A.val = p.val;
       A.cnt_off = p.shard_cnt_off;
       A.means = p.means;
+      ProfileScope prof(stream, PT_APPLY);
       if (use_inline)
         apply_kernel<true><<<grid, kThreads, 0, stream>>>(A, I);
       else

@@ -80,7 +80,10 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   __shared__ int s_last;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   if (VIEW == V_DENSE && !(T.flags & GD_FLAG_NO_PREDICTION) && T.ctl->dense_needed == 0u) return;
-  const uint32_t* tile0 = T.tile0[LK];
+  __shared__ SmemTables s_tab;
+  const ScopeDesc* scopes;
+  const uint32_t* tile0;
+  load_tables(T, LK, &s_tab, &scopes, &tile0);
   const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
   const uint32_t ltm = lanemask_lt();
   uint4* desc = reinterpret_cast<uint4*>(VIEW == V_CAND ? T.desc_cand : T.desc_dcomp);
@@ -92,11 +95,11 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
     const uint32_t t = s_tile;
     if (t >= total_tiles) break;
     const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
-    const ScopeDesc& d = T.scopes[s];
+    const ScopeDesc& d = scopes[s];
     const ScopeState* st = T.state + s;
     const bool pred = predicted_ok(T, d, *st);
     if (VIEW == V_CAND ? !pred : pred) continue;    // the other view owns this scope
-    const uint32_t first = __ldg(tile0 + s);
+    const uint32_t first = tile0[s];
     const uint32_t lt = t - first;
     const uint64_t len = VIEW == V_CAND ? st->cand_count : d.hi - d.lo;
     const uint64_t beg = (uint64_t)lt * kTile;
@@ -123,8 +126,13 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
 
     // phase 1: load, classify, count
     const uint64_t wbeg = beg + (uint64_t)warp * (32u * ROUNDS) + lane;
-    uint32_t vb[ROUNDS];
+    uint32_t vb[ROUNDS], ib[ROUNDS];
     uint32_t gtm = 0, eqm = 0, wg = 0, we = 0;
+#pragma unroll
+    for (int j = 0; j < ROUNDS; ++j) {   // the candidates' indices travel with their values: loaded up front
+      const uint64_t i = wbeg + (uint64_t)j * 32u;
+      ib[j] = (VIEW == V_CAND && i < end) ? T.cand_idx[d.cand_base + i] : 0u;
+    }
 #pragma unroll
     for (int j = 0; j < ROUNDS; ++j) {
       const uint64_t i = wbeg + (uint64_t)j * 32u;
@@ -177,7 +185,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
         if (isgt || eb < q) {
           const uint64_t pos = gb + (eb < q ? eb : q);
           const uint64_t i = wbeg + (uint64_t)j * 32u;
-          const uint64_t idx = VIEW == V_CAND ? (uint64_t)T.cand_idx[d.cand_base + i] : d.lo + i;
+          const uint64_t idx = VIEW == V_CAND ? (uint64_t)ib[j] : d.lo + i;
           if (pos < d.k && idx < T.n) {
             const uint32_t b = vb[j];
             T.residual[idx] = 0.0f;
@@ -240,6 +248,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
 }  // namespace
 
 cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream) {
+  ProfileScope prof(stream, PT_FINALIZE);
   finalize_kernel<<<1, kThreads, 0, stream>>>(T);
   GD_LAUNCH_CHECK();
   return cudaSuccess;
@@ -248,6 +257,7 @@ cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream) {
 cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, bool finalize, cudaStream_t stream) {
   const uint32_t total = tiles[dense ? L_DCOMP : L_CAND];
   if (!total) return finalize ? launch_finalize(T, stream) : cudaSuccess;
+  ProfileScope prof(stream, dense ? PT_DENSE_COMPACT : PT_CAND_COMPACT);
   const uint32_t cap = (uint32_t)sm_count() * 8u;
   const uint32_t grid = total < cap ? total : cap;
   if (dense)

@@ -41,15 +41,18 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
   __shared__ uint32_t s_total;
   __shared__ int s_ok;
   __shared__ StashEntry s_stash[kWarps][kStash];
+  __shared__ SmemTables s_tab;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   if (tid == 0) s_chunk = atomicAdd(&T.ctl->ticket[L_EMIT], 1u);
+  const ScopeDesc* scopes;
+  const uint32_t* tile0;
+  load_tables(T, L_EMIT, &s_tab, &scopes, &tile0);
   __syncthreads();
   const uint32_t t = s_chunk;
-  const uint32_t* tile0 = T.tile0[L_EMIT];
   const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
-  const ScopeDesc& d = T.scopes[s];
+  const ScopeDesc& d = scopes[s];
   const uint64_t lo = d.lo, hi = d.hi;
-  const uint32_t first = __ldg(tile0 + s), nchunks = __ldg(tile0 + s + 1) - first;
+  const uint32_t first = tile0[s], nchunks = tile0[s + 1] - first;
   const uint32_t lt = t - first;
   constexpr uint64_t CH = (uint64_t)C * kTile;
   const uint64_t cbase = (lo / CH + lt) * CH;
@@ -229,7 +232,7 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
 
 cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
   if (!tiles[L_EMIT]) return cudaSuccess;
-  profile_mark(stream, true);
+  ProfileScope prof(stream, PT_ADD_EMIT);
   switch (T.emit_chunk_tiles) {
     case 1: add_emit_kernel<1><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
     case 2: add_emit_kernel<2><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
@@ -237,7 +240,6 @@ cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStrea
     default: add_emit_kernel<8><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
   }
   GD_LAUNCH_CHECK();
-  profile_mark(stream, false);
   return cudaSuccess;
 }
 

@@ -16,6 +16,7 @@ constexpr uint32_t kDenseSelTile = 32768;  // elements per CTA in the dense hist
 constexpr int kRadixBits0 = 11;         // 31-bit magnitude key = 11 + 10 + 10 bits
 constexpr int kRadixBins0 = 1 << kRadixBits0;
 constexpr int kShift0 = 20, kShift1 = 10, kShift2 = 0;
+constexpr uint32_t kHistBinsPerScope = 2048 + 1024 + 2048 + 1024 + 1024;   // sample: 2 passes; selection: 3
 constexpr uint32_t kAbsMask = 0x7FFFFFFFu;
 constexpr uint32_t kLookbackSpinLimit = 1u << 21;  // polls before a look-back wait gives up
 
@@ -89,7 +90,7 @@ struct DevTables {       // passed by value to every kernel
   // zeroed region
   Ctl* ctl;
   ScopeState* state;
-  unsigned long long* hist;          // [n_scopes][kRadixBins0]
+  unsigned long long* hist;          // [n_scopes][kHistBinsPerScope]
   double* sums;                      // [n_layers][2]
   unsigned long long* cnts;          // [n_layers][2]
   uint64_t* desc_emit;               // [tiles(L_EMIT)]
@@ -130,13 +131,40 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
 }
 __device__ __forceinline__ uint64_t pack_desc(uint64_t flag, uint64_t value) { return (value << 2) | flag; }
 
+// Copy of the small per-call tables in shared memory: scope descriptors and the tile -> scope table
+// of one launch kind.  With few scopes (the usual case) every later lookup is a shared-memory read
+// instead of a chain of dependent global loads.
+constexpr uint32_t kSmemScopes = 32;
+struct SmemTables {
+  ScopeDesc scopes[kSmemScopes];
+  uint32_t tile0[kSmemScopes + 1];
+};
+
+// Called by all threads of a CTA; the caller synchronises before using the result.  Returns the
+// tables to use: the shared copy when the scopes fit, else the global ones.
+__device__ __forceinline__ void load_tables(const DevTables& T, int launch_kind, SmemTables* sm,
+                                            const ScopeDesc** scopes, const uint32_t** tile0) {
+  if (T.n_scopes <= kSmemScopes) {
+    const uint32_t words = T.n_scopes * (uint32_t)(sizeof(ScopeDesc) / 8);
+    const uint64_t* src = reinterpret_cast<const uint64_t*>(T.scopes);
+    uint64_t* dst = reinterpret_cast<uint64_t*>(sm->scopes);
+    for (uint32_t i = threadIdx.x; i < words; i += blockDim.x) dst[i] = src[i];
+    for (uint32_t i = threadIdx.x; i <= T.n_scopes; i += blockDim.x) sm->tile0[i] = T.tile0[launch_kind][i];
+    *scopes = sm->scopes;
+    *tile0 = sm->tile0;
+  } else {
+    *scopes = T.scopes;
+    *tile0 = T.tile0[launch_kind];
+  }
+}
+
 // Largest s in [0, n_scopes) with tile0[s] <= t (tile0 has n_scopes + 1 entries, ascending; scopes
 // without tiles repeat their successor's value, so the scope found is the one that owns tile t).
 __device__ __forceinline__ uint32_t scope_of_tile(const uint32_t* __restrict__ tile0, uint32_t n_scopes, uint32_t t) {
   uint32_t lo = 0, hi = n_scopes;  // invariant: tile0[lo] <= t < tile0[hi]
   while (hi - lo > 1) {
     uint32_t mid = (lo + hi) >> 1;
-    if (__ldg(tile0 + mid) <= t) lo = mid; else hi = mid;
+    if (tile0[mid] <= t) lo = mid; else hi = mid;
   }
   return lo;
 }
@@ -173,6 +201,15 @@ int sm_count();   // multiprocessors of the current device (0 on error)
 
 // Measurement hooks (gd_api.cu): count a kernel launch; record an event of the pair around the fused pass.
 void note_launches(uint32_t count);
-void profile_mark(cudaStream_t stream, bool begin);
+// Kernel tags of the measurement hooks, in the order a step launches them.
+enum ProfileTag : uint32_t { PT_SETUP = 0, PT_SAMPLE_SELECT = 1, PT_ADD_EMIT = 2, PT_DENSE_SELECT = 3, PT_DENSE_COMPACT = 4,
+                             PT_CAND_SELECT = 5, PT_CAND_COMPACT = 6, PT_FINALIZE = 7, PT_APPLY = 8 };
+void profile_mark(cudaStream_t stream, bool begin, uint32_t tag);
+struct ProfileScope {   // records an event pair around the launches made during its lifetime
+  cudaStream_t stream;
+  uint32_t tag;
+  ProfileScope(cudaStream_t s, uint32_t t) : stream(s), tag(t) { profile_mark(stream, true, tag); }
+  ~ProfileScope() { profile_mark(stream, false, tag); }
+};
 
 }  // namespace gd

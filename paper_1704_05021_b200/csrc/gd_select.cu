@@ -6,8 +6,8 @@
 //
 // One cooperative launch does a whole selection: per pass every CTA histograms one digit of the
 // 31-bit magnitude key (11 + 10 + 10 bits) over its share of the tiles, the grid meets at a
-// barrier, one CTA per scope turns the histogram into the next digit, and the grid meets again.
-// The barrier is a counter in the workspace; its wait is bounded like every other wait here.
+// barrier, and every CTA works out the next digit of the scopes it touches from the finished
+// histogram.  The barrier is a counter in the workspace; its wait is bounded like every other wait.
 #include "gd_internal.cuh"
 
 namespace gd {
@@ -67,6 +67,87 @@ __device__ __forceinline__ bool view_active(const DevTables& T, const ScopeDesc&
   return VIEW == V_CAND ? pred : !pred;
 }
 
+// Running state of a radix selection: the digits fixed so far, the rank still to find inside that
+// bucket, and the number of keys above the bucket.
+struct SelRun {
+  uint32_t prefix;
+  uint64_t rank, gt;
+};
+
+// Histograms of one scope: the sample's two passes, then the three passes of the candidate (or
+// dense) selection.  Each is filled once per call and never cleared inside a call.
+__device__ __forceinline__ unsigned long long* hist_of(const DevTables& T, uint32_t s, int view, int pass) {
+  unsigned long long* base = T.hist + (size_t)s * kHistBinsPerScope;
+  if (view == V_SAMPLE) return base + (pass == 0 ? 0 : 2048);
+  return base + (pass == 0 ? 3072 : (pass == 1 ? 5120 : 6144));
+}
+
+// Run by a whole CTA after the grid barrier that completes histogram `gh`: walks it from the top
+// bin down and fixes the next digit.  Every CTA that needs the digit computes it for itself, so no
+// second barrier is needed to hand it around.
+__device__ SelRun next_digit(const unsigned long long* gh, int bits, SelRun in, Ctl* ctl) {
+  __shared__ unsigned long long s_warp[kWarps];
+  __shared__ unsigned long long s_acc;
+  __shared__ uint32_t s_digit;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const uint32_t nbins = 1u << bits;
+  const uint32_t C = nbins / kThreads;                 // 8 or 4 bins per thread: [top - C + 1, top]
+  const uint32_t top = nbins - 1u - tid * C;
+  unsigned long long bin[8];
+  unsigned long long cs = 0;
+#pragma unroll
+  for (uint32_t j = 0; j < 8; ++j) {
+    bin[j] = j < C ? __ldcg(gh + top - j) : 0ull;
+    cs += bin[j];
+  }
+  unsigned long long inc = cs;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+    if ((int)lane >= o) inc += y;
+  }
+  __syncthreads();                                     // the shared scratch is free again
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  unsigned long long above = inc - cs;
+  for (uint32_t w = 0; w < warp; ++w) above += s_warp[w];
+  if (tid == kThreads - 1 && above + cs < in.rank) atomicCAS(&ctl->status, (int)GD_OK, (int)GD_ERR_INTERNAL);
+  const bool owner = in.rank == 0 ? (tid == 0) : (above < in.rank && in.rank <= above + cs);
+  if (owner) {
+    uint32_t digit = nbins - 1u;
+    unsigned long long acc = 0;
+    if (in.rank != 0) {
+      acc = above;
+#pragma unroll
+      for (uint32_t j = 0; j < 8; ++j) {
+        if (j < C) {
+          if (acc + bin[j] >= in.rank) { digit = top - j; break; }
+          acc += bin[j];
+        }
+      }
+    }
+    s_digit = digit;
+    s_acc = acc;
+  }
+  __syncthreads();
+  SelRun out;
+  out.prefix = (in.prefix << bits) | s_digit;
+  out.rank = in.rank - s_acc;
+  out.gt = in.gt + s_acc;
+  return out;
+}
+
+// State of scope s before pass `pass`, recomputed from the finished histograms of the earlier passes.
+template <int VIEW>
+__device__ SelRun state_before(const DevTables& T, const ScopeDesc& d, uint32_t s, int pass) {
+  SelRun r;
+  r.prefix = 0;
+  r.rank = VIEW == V_SAMPLE ? d.samp_rank : d.k;
+  r.gt = 0;
+  for (int p = 0; p < pass; ++p) r = next_digit(hist_of(T, s, VIEW, p), p == 0 ? kRadixBits0 : 10, r, T.ctl);
+  return r;
+}
+
 template <int VIEW>
 __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
   constexpr int LK = VIEW == V_SAMPLE ? L_SAMP : (VIEW == V_CAND ? L_CAND : L_DSEL);
@@ -74,35 +155,67 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
   constexpr int PASSES = VIEW == V_SAMPLE ? 2 : 3;   // the prediction needs 21 bits only
   constexpr uint32_t NONE = 0xFFFFFFFFu;
   __shared__ uint32_t sh[kRadixBins0];
-  __shared__ unsigned long long s_warp[kWarps];
-  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  __shared__ SmemTables s_tab;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
   if (T.ctl->status != GD_OK) return;   // set only by an earlier kernel of this call: uniform over the grid
   if (VIEW == V_DENSE && !(T.flags & GD_FLAG_NO_PREDICTION) && T.ctl->dense_needed == 0u) return;
-  const uint32_t* tile0 = T.tile0[LK];
+  const ScopeDesc* scopes;
+  const uint32_t* tile0;
+  load_tables(T, LK, &s_tab, &scopes, &tile0);
   const uint32_t per = (total_tiles + gridDim.x - 1) / gridDim.x;
   const uint32_t t_beg = blockIdx.x * per;
   const uint32_t t_end = (t_beg + per < total_tiles) ? t_beg + per : total_tiles;
   uint32_t phase = 0;
 
-  for (int pass = 0; pass < PASSES; ++pass) {
+  for (int pass = 0; pass <= PASSES; ++pass) {
     const int shift = pass == 0 ? kShift0 : (pass == 1 ? kShift1 : kShift2);
     const int bits = pass == 0 ? kRadixBits0 : 10;
     const uint32_t nbins = 1u << bits;
     const int pshift = pass == 1 ? kShift0 : kShift1;   // shift that exposes the digits fixed so far
 
-    // ---- histogram of this CTA's tiles; flushed whenever the scope changes
-    for (uint32_t b = tid; b < nbins; b += kThreads) sh[b] = 0;
+    for (uint32_t b = tid; b < kRadixBins0; b += kThreads) sh[b] = 0;
     __syncthreads();
     uint32_t cur = NONE;                                // scope the shared histogram belongs to
+    uint32_t seen = NONE;                               // scope whose values are cached below
+    bool active = false, have_run = false;
+    uint64_t len = 0;
+    uint32_t prefix = 0;
+    const float* vals = nullptr;
     for (uint32_t t = t_beg; t < t_end; ++t) {
-      const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
-      const ScopeDesc& d = T.scopes[s];
-      ScopeState* st = T.state + s;
-      if (!view_active<VIEW>(T, d, st)) continue;
+      const uint32_t s = (seen != NONE && t < tile0[seen + 1]) ? seen : scope_of_tile(tile0, T.n_scopes, t);
+      const ScopeDesc& d = scopes[s];
+      const uint32_t lt = t - tile0[s];
+      if (s != seen) {                                  // per-scope values, worked out once per scope
+        seen = s;
+        ScopeState* st = T.state + s;
+        active = view_active<VIEW>(T, d, st);
+        if (VIEW == V_SAMPLE) { len = d.samp_m; vals = T.samp_val + d.samp_base; }
+        else if (VIEW == V_CAND) { len = st->cand_count; vals = T.cand_val + d.cand_base; }
+        else { len = d.hi - d.lo; vals = T.residual + d.lo; }
+        have_run = false;
+      }
+      if (!active) continue;
+      const uint64_t beg = (uint64_t)lt * TILE;
+      if (pass == PASSES ? lt != 0 : beg >= len) continue;
+      if (pass > 0 && !have_run) {                      // digits fixed by the earlier passes
+        const SelRun run = state_before<VIEW>(T, d, s, pass);
+        have_run = true;
+        prefix = run.prefix;
+        if (pass == PASSES && tid == 0) {               // the CTA with the scope's first tile records the result
+          ScopeState* st = T.state + s;
+          if (VIEW == V_SAMPLE) {
+            st->tau_lo = run.prefix << kShift1;         // lower edge of the 21-bit bucket
+          } else {
+            st->tau = run.prefix; st->q = run.rank; st->gt = run.gt;
+            if (VIEW == V_DENSE) st->used_dense = 1u;
+          }
+        }
+      }
+      if (pass == PASSES) continue;
       if (s != cur) {
         if (cur != NONE) {
           __syncthreads();
-          unsigned long long* gh = T.hist + (size_t)cur * kRadixBins0;
+          unsigned long long* gh = hist_of(T, cur, VIEW, pass);
           for (uint32_t b = tid; b < nbins; b += kThreads) {
             const uint32_t c = sh[b];
             if (c) atomicAdd(gh + b, (unsigned long long)c);
@@ -112,116 +225,52 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
         }
         cur = s;
       }
-      const uint32_t lt = t - __ldg(tile0 + s);
-      uint64_t len;
-      const float* vals;
-      if (VIEW == V_SAMPLE) { len = d.samp_m; vals = T.samp_val + d.samp_base; }
-      else if (VIEW == V_CAND) { len = st->cand_count; vals = T.cand_val + d.cand_base; }
-      else { len = d.hi - d.lo; vals = T.residual + d.lo; }
-      const uint32_t prefix = pass > 0 ? __ldcg(&st->sel[VIEW].prefix) : 0u;
-      const uint64_t beg = (uint64_t)lt * TILE;
       const uint64_t end = (beg + TILE < len) ? beg + TILE : len;
-      for (uint64_t i0 = beg + (tid & ~31u); i0 < end; i0 += kThreads) {   // warp-uniform trip count
-        const uint64_t i = i0 + lane;
-        uint32_t digit = NONE;                                             // "does not count"
-        if (i < end) {
-          float x;
-          if (VIEW == V_SAMPLE && pass == 0) {
-            x = sample_value(T, d, s, i);
-            T.samp_val[d.samp_base + i] = x;
-          } else {
-            x = vals[i];
+      // batches of 16 elements per thread: all loads of a batch are in flight before the first is used
+      for (uint64_t b0 = beg; b0 < end; b0 += kTile) {
+        uint32_t keys[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const uint64_t i = b0 + (uint64_t)j * kThreads + tid;
+          float x = 0.f;
+          if (i < end) {
+            if (VIEW == V_SAMPLE && pass == 0) x = sample_value(T, d, s, i);
+            else x = vals[i];
           }
-          const uint32_t key = __float_as_uint(x) & kAbsMask;
-          if (pass == 0 || (key >> pshift) == prefix) digit = (key >> shift) & (nbins - 1u);
+          keys[j] = __float_as_uint(x);
         }
-        // one shared-memory add per distinct digit in the warp
-        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
-        if (digit != NONE && lane == (uint32_t)__ffs((int)peers) - 1u) atomicAdd(&sh[digit], (uint32_t)__popc(peers));
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const uint64_t i = b0 + (uint64_t)j * kThreads + tid;
+          uint32_t digit = NONE;                                           // "does not count"
+          if (i < end) {
+            if (VIEW == V_SAMPLE && pass == 0) T.samp_val[d.samp_base + i] = __uint_as_float(keys[j]);
+            const uint32_t key = keys[j] & kAbsMask;
+            if (pass == 0 || (key >> pshift) == prefix) digit = (key >> shift) & (nbins - 1u);
+          }
+          // one shared-memory add per distinct digit in the warp
+          const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
+          if (digit != NONE && lane == (uint32_t)__ffs((int)peers) - 1u) atomicAdd(&sh[digit], (uint32_t)__popc(peers));
+        }
       }
     }
+    if (pass == PASSES) break;
     __syncthreads();
     if (cur != NONE) {
-      unsigned long long* gh = T.hist + (size_t)cur * kRadixBins0;
+      unsigned long long* gh = hist_of(T, cur, VIEW, pass);
       for (uint32_t b = tid; b < nbins; b += kThreads) {
         const uint32_t c = sh[b];
         if (c) atomicAdd(gh + b, (unsigned long long)c);
       }
     }
     if (!grid_barrier(&T.ctl->barrier[VIEW], phase, T.ctl)) return;
-
-    // ---- one CTA per scope: histogram -> next digit.  Thread x owns the bins [top - C + 1, top].
-    for (uint32_t s = blockIdx.x; s < T.n_scopes; s += gridDim.x) {
-      const ScopeDesc& d = T.scopes[s];
-      ScopeState* st = T.state + s;
-      if (!view_active<VIEW>(T, d, st)) continue;
-      uint64_t rank = VIEW == V_SAMPLE ? d.samp_rank : d.k;
-      uint32_t prefix = 0;
-      uint64_t gt = 0;
-      if (pass > 0) {
-        prefix = __ldcg(&st->sel[VIEW].prefix);
-        rank = __ldcg(&st->sel[VIEW].rank);
-        gt = __ldcg(&st->sel[VIEW].gt);
-      }
-      unsigned long long* gh = T.hist + (size_t)s * kRadixBins0;
-      const uint32_t C = nbins / kThreads;                 // 8 or 4 bins per thread
-      const uint32_t top = nbins - 1u - tid * C;
-      unsigned long long bin[8];
-      unsigned long long cs = 0;
-#pragma unroll
-      for (uint32_t j = 0; j < 8; ++j) {
-        bin[j] = j < C ? __ldcg(gh + top - j) : 0ull;
-        cs += bin[j];
-      }
-      unsigned long long inc = cs;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-        if ((int)lane >= o) inc += y;
-      }
-      __syncthreads();                                     // s_warp free again
-      if (lane == 31) s_warp[warp] = inc;
-      __syncthreads();
-      unsigned long long above = inc - cs;
-      for (uint32_t w = 0; w < warp; ++w) above += s_warp[w];
-      if (tid == kThreads - 1 && above + cs < rank) atomicCAS(&T.ctl->status, (int)GD_OK, (int)GD_ERR_INTERNAL);
-      const bool owner = rank == 0 ? (tid == 0) : (above < rank && rank <= above + cs);
-      if (owner) {
-        uint32_t digit = nbins - 1u;
-        unsigned long long acc = 0;
-        if (rank != 0) {
-          acc = above;
-#pragma unroll
-          for (uint32_t j = 0; j < 8; ++j) {
-            if (j < C) {
-              if (acc + bin[j] >= rank) { digit = top - j; break; }
-              acc += bin[j];
-            }
-          }
-        }
-        const uint32_t nprefix = (prefix << bits) | digit;
-        const uint64_t nrank = rank - acc, ngt = gt + acc;
-        st->sel[VIEW].prefix = nprefix;
-        st->sel[VIEW].rank = nrank;
-        st->sel[VIEW].gt = ngt;
-        if (pass == PASSES - 1) {
-          if (VIEW == V_SAMPLE) {
-            st->tau_lo = nprefix << kShift1;               // lower edge of the 21-bit bucket
-          } else {
-            st->tau = nprefix; st->q = nrank; st->gt = ngt;
-            if (VIEW == V_DENSE) st->used_dense = 1u;
-          }
-        }
-      }
-      for (uint32_t b = tid; b < nbins; b += kThreads) gh[b] = 0ull;   // ready for the next pass
-    }
-    if (pass + 1 < PASSES && !grid_barrier(&T.ctl->barrier[VIEW], phase, T.ctl)) return;
   }
 }
 
 template <int VIEW>
 cudaError_t launch_select(const DevTables& T, uint32_t total_tiles, uint32_t ctas_per_sm, cudaStream_t stream) {
   if (!total_tiles) return cudaSuccess;
+  ProfileScope prof(stream, VIEW == V_SAMPLE ? PT_SAMPLE_SELECT : (VIEW == V_CAND ? PT_CAND_SELECT : PT_DENSE_SELECT));
   static int resident = 0;                                 // co-resident CTAs per SM of this kernel
   if (resident == 0) {
     int r = 0;
