@@ -39,7 +39,7 @@ typedef enum {
 } gd_status_t;
 
 enum { GD_SCOPE_GLOBAL = 0, GD_SCOPE_PER_LAYER = 1 };
-enum { GD_VALUES_FP32 = 0, GD_VALUES_TWO_MEANS = 1 };
+enum { GD_VALUES_FP32 = 0, GD_VALUES_TWO_MEANS = 1, GD_VALUES_THRESHOLD = 2 };
 
 /* gd_compress_args.flags */
 enum {
@@ -88,6 +88,11 @@ int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes
  *              (fp64 accumulation, rounded to fp32, +0.0f for an empty group); out_idx[t] carries
  *              index | signbit << 31 and out_val is not written.  The residual is unchanged by the
  *              value mode: it holds the dropped mass only.
+ *   threshold mode (Section 5.4, the quantisation that maps "all surviving values to the dropping
+ *              threshold, effectively the minimum surviving absolute value"): same packing as two-means
+ *              mode; out_means[l] = (+t, -t) with t the float whose bit pattern is the tau of the scope
+ *              that holds layer l (+0, -0 if that scope keeps nothing), so that a push decodes exactly
+ *              like a two-means push.
  *
  * Results are bit-exact functions of (grad, residual, offsets, drop_ppm) except the two means,
  * whose fp64 partial sums are combined in an unspecified order.  Non-finite inputs are ordered by
@@ -98,7 +103,7 @@ int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes
 typedef struct gd_compress_args {
   const float* grad;          /* device, n fp32, 16-byte aligned, read-only */
   float* residual;            /* device, n fp32, 16-byte aligned, in/out */
-  uint64_t n;                 /* <= 2^32 (GD_VALUES_FP32) or <= 2^31 (GD_VALUES_TWO_MEANS) */
+  uint64_t n;                 /* <= 2^32 (GD_VALUES_FP32) or <= 2^31 (the packed modes) */
   const uint64_t* layer_off;  /* HOST, n_layers + 1 ascending offsets, [0] = 0, last = n */
   uint32_t n_layers;          /* >= 1 */
   uint32_t n_shards;          /* >= 1 */
@@ -111,7 +116,7 @@ typedef struct gd_compress_args {
   float* out_val;             /* device, gd_total_kept() fp32; may be NULL in two-means mode */
   uint32_t* out_shard_cnt_off;/* device, n_shards + 1 words */
   uint32_t* out_tau;          /* device, one word per scope (1, or n_layers); may be NULL */
-  float* out_means;           /* device, n_layers x 2 fp32 (mu+, mu-); two-means mode only */
+  float* out_means;           /* device, n_layers x 2 fp32 (mu+, mu-); two-means and threshold modes */
   void* workspace;            /* device, 256-byte aligned, >= gd_workspace_bytes() */
   size_t workspace_bytes;
 } gd_compress_args;
@@ -126,9 +131,9 @@ int gd_compress(const gd_compress_args* args, void* stream);
  */
 typedef struct gd_push {
   const uint32_t* idx;
-  const float* val;              /* NULL in two-means mode */
+  const float* val;              /* NULL in the packed modes */
   const uint32_t* shard_cnt_off;
-  const float* means;            /* n_layers x 2, two-means mode only */
+  const float* means;            /* n_layers x 2, packed modes only */
 } gd_push;
 
 /*
@@ -136,7 +141,7 @@ typedef struct gd_push {
  * and adds the pushed pieces into it.  For every push in array order and every entry of it
  * whose index lies in a shard [shard_off[j], shard_off[j+1]):
  *     params[j][index - shard_off[j]] += alpha * value
- * with value = val[t] (fp32 mode) or the mean of the entry's layer and sign (two-means mode).
+ * with value = val[t] (fp32 mode) or means[layer of the entry][sign] (two-means and threshold modes).
  * One fused multiply-add in fp32 per entry; with alpha = 1 the result is fl32(p + value).
  * Pushes are applied one after another in stream order; indices inside one push are unique.
  * Entries whose index lies outside every shard are skipped.  The optimiser is not part of
@@ -150,7 +155,7 @@ typedef struct gd_apply_args {
   const gd_push* pushes;       /* HOST array of n_pushes */
   int32_t value_mode;          /* GD_VALUES_* */
   float alpha;
-  const uint64_t* layer_off;   /* HOST, n_layers + 1; two-means mode only */
+  const uint64_t* layer_off;   /* HOST, n_layers + 1; packed modes only */
   uint32_t n_layers;
   uint32_t reserved;
   void* workspace;             /* device, 256-byte aligned, >= gd_apply_workspace_bytes() */
@@ -241,6 +246,18 @@ int gd_compress_static(const gd_compress_args* args, void* stream, const void** 
  */
 int gd_profile_enable(int mode);
 int gd_profile_collect(float* ms_out, uint32_t* tags_out, uint32_t capacity, uint32_t* count_out);
+
+/*
+ * Self-test of the bounded device-side waits (no counterpart in the paper).  Every wait in the
+ * library's kernels - on a predecessor tile of a scan, on a grid barrier - gives up after a fixed
+ * number of polls, marks its tile aborted so that nothing waits on it, and records
+ * GD_ERR_DEVICE_TIMEOUT in the workspace.  This call enqueues a one-warp kernel that waits, for at
+ * most spin_limit polls, on a tile nothing will ever publish, and then lets a second tile meet the
+ * aborted one.  Afterwards gd_status(workspace) is GD_ERR_DEVICE_TIMEOUT and gd_get_stats reports
+ * n_scopes = 1 if the first wait gave up (as it must) and n_scopes_predicted = 1 if the second tile
+ * aborted without waiting.  The context stays usable.  workspace: device, 256-byte aligned, >= 512 bytes.
+ */
+int gd_selftest_bounded_wait(void* workspace, size_t workspace_bytes, uint32_t spin_limit, void* stream);
 
 /* Number of kernels this library has launched in this process (memsets and copies not counted). */
 int gd_launch_count(uint64_t* count_out);

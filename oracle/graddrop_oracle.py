@@ -26,6 +26,9 @@ Readings taken where the paper is silent:
   * two-value quantisation (Section 5.4, "averages of values being quantized"): one pair
     (mean of kept entries with sign bit 0, mean of kept entries with sign bit 1) per layer,
     survivors packed as index | signbit << 31; the residual still holds only the dropped mass;
+  * threshold quantisation (Section 5.4: every surviving value is mapped to the dropping
+    threshold, "effectively the minimum surviving absolute value"): same packing; the pair of a
+    layer is (+t, -t) with t the float whose bit pattern is the tau of the scope holding the layer;
   * the server applies a push as p[idx - shard_start] += alpha * value (Section 3: a server
     owns 1/N of the parameters); this oracle evaluates that sum in fp64.
 """
@@ -37,6 +40,7 @@ SCOPE_GLOBAL = 0
 SCOPE_PER_LAYER = 1
 VALUES_FP32 = 0
 VALUES_TWO_MEANS = 1
+VALUES_THRESHOLD = 2
 
 _ABS_MASK = np.uint32(0x7FFFFFFF)
 TAU_NONE = 0xFFFFFFFF
@@ -158,6 +162,19 @@ def compress(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GL
             means = np.where(cnts > 0, sums / np.maximum(cnts, 1), 0.0).astype(np.float32)
         out["idx"] = (kept.astype(np.uint32) | (sign.astype(np.uint32) << np.uint32(31)))
         out["means"], out["counts"], out["sums"] = means, cnts, sums
+    elif value_mode == VALUES_THRESHOLD:
+        if n > (1 << 31):
+            raise ValueError("threshold packing needs n <= 2^31")
+        n_layers = len(layer_off) - 1
+        sign = (val.view(np.uint32) >> np.uint32(31))
+        means = np.zeros((n_layers, 2), dtype=np.float32)
+        for l in range(n_layers):
+            tau = taus[0] if scope_mode == SCOPE_GLOBAL else taus[l]
+            bits = np.uint32(0 if tau == TAU_NONE else tau)
+            means[l, 0] = bits.view(np.float32)                       # +t: the smallest kept |v| of the scope
+            means[l, 1] = (bits | np.uint32(0x80000000)).view(np.float32)
+        out["idx"] = kept.astype(np.uint32) | (sign << np.uint32(31))
+        out["means"] = means
     elif value_mode != VALUES_FP32:
         raise ValueError("bad value_mode")
     return out

@@ -26,12 +26,14 @@ GD_SCOPE_GLOBAL = 0
 GD_SCOPE_PER_LAYER = 1
 GD_VALUES_FP32 = 0
 GD_VALUES_TWO_MEANS = 1
+GD_VALUES_THRESHOLD = 2
 GD_FLAG_NO_PREDICTION = 1
 
 EXPORTS = [
     "gd_status_string", "gd_kept_count", "gd_total_kept", "gd_workspace_bytes", "gd_apply_workspace_bytes",
     "gd_compress", "gd_decompress_apply", "gd_residual_reset", "gd_status", "gd_get_stats", "gd_step_host",
     "gd_profile_enable", "gd_profile_collect", "gd_launch_count", "gd_compress_static",
+    "gd_selftest_bounded_wait",
 ]
 GD_STATIC_WORKSPACE_BYTES = 16 << 20
 
@@ -108,6 +110,7 @@ def load_library():
     lib.gd_get_stats.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(_Stats)]
     lib.gd_step_host.argtypes = [C.POINTER(_CompressArgs), C.POINTER(_ApplyArgs), C.POINTER(_HostIo), C.c_void_p]
     lib.gd_compress_static.argtypes = [C.POINTER(_CompressArgs), C.c_void_p, C.POINTER(C.c_void_p)]
+    lib.gd_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_size_t, C.c_uint32, C.c_void_p]
     lib.gd_profile_enable.argtypes = [C.c_int]
     lib.gd_profile_collect.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_uint32), C.c_uint32, C.POINTER(C.c_uint32)]
     lib.gd_launch_count.argtypes = [C.POINTER(C.c_uint64)]
@@ -291,3 +294,8 @@ def gd_compress_static(call: CompressCall, stream=None) -> int:
 def gd_status_at(workspace_address: int, stream=None) -> int:
     """gd_status for a workspace known by its device address (e.g. the one gd_compress_static returns)."""
     return load_library().gd_status(C.c_void_p(workspace_address), _stream_handle(stream))
+
+
+def gd_selftest_bounded_wait(workspace: torch.Tensor, spin_limit: int = 2000, stream=None) -> None:
+    _check(load_library().gd_selftest_bounded_wait(workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                                   spin_limit, _stream_handle(stream)), "gd_selftest_bounded_wait")

@@ -312,15 +312,15 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     if (rc != GD_OK) return rc;
     const uint64_t n = a->layer_off[a->n_layers];
     if (n_sh != n || a->n != n) return GD_ERR_INVALID_ARG;
-    if (a->value_mode != GD_VALUES_FP32 && a->value_mode != GD_VALUES_TWO_MEANS) return GD_ERR_INVALID_ARG;
-    if (a->value_mode == GD_VALUES_TWO_MEANS && n > (1ull << 31)) return GD_ERR_TOO_LARGE;
+    if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_THRESHOLD) return GD_ERR_INVALID_ARG;
+    if (a->value_mode != GD_VALUES_FP32 && n > (1ull << 31)) return GD_ERR_TOO_LARGE;
     if (a->flags & ~(uint32_t)GD_FLAG_NO_PREDICTION) return GD_ERR_INVALID_ARG;
     if (n && (!a->grad || !a->residual)) return GD_ERR_INVALID_ARG;
     if (((uintptr_t)a->grad | (uintptr_t)a->residual) & 15u) return GD_ERR_INVALID_ARG;
     if (!a->out_shard_cnt_off) return GD_ERR_INVALID_ARG;
     if (P.k_total && !a->out_idx) return GD_ERR_INVALID_ARG;
     if (P.k_total && a->value_mode == GD_VALUES_FP32 && !a->out_val) return GD_ERR_INVALID_ARG;
-    if (a->value_mode == GD_VALUES_TWO_MEANS && !a->out_means) return GD_ERR_INVALID_ARG;
+    if (a->value_mode != GD_VALUES_FP32 && !a->out_means) return GD_ERR_INVALID_ARG;
     if (!a->workspace || ((uintptr_t)a->workspace & (kAlign - 1))) return GD_ERR_WORKSPACE;
     if (a->workspace_bytes < P.total_bytes) return GD_ERR_WORKSPACE;
 
@@ -474,6 +474,13 @@ int gd_profile_collect(float* ms_out, uint32_t* tags_out, uint32_t capacity, uin
   return rc;
 }
 
+int gd_selftest_bounded_wait(void* workspace, size_t workspace_bytes, uint32_t spin_limit, void* stream) {
+  if (!workspace || ((uintptr_t)workspace & (kAlign - 1)) || workspace_bytes < 512) return GD_ERR_WORKSPACE;
+  if (spin_limit == 0 || spin_limit > kLookbackSpinLimit) return GD_ERR_INVALID_ARG;
+  if (launch_bounded_wait_selftest(workspace, spin_limit, (cudaStream_t)stream) != cudaSuccess) return GD_ERR_CUDA;
+  return GD_OK;
+}
+
 int gd_launch_count(uint64_t* count_out) {
   if (!count_out) return GD_ERR_INVALID_ARG;
   *count_out = g_launches;
@@ -503,7 +510,7 @@ int gd_step_host(const gd_compress_args* a, const gd_apply_args* apply, const gd
   if (e == cudaSuccess && io->shard_cnt_off_host)
     e = cudaMemcpyAsync(io->shard_cnt_off_host, a->out_shard_cnt_off, sizeof(uint32_t) * ((size_t)a->n_shards + 1),
                         cudaMemcpyDeviceToHost, stream);
-  if (e == cudaSuccess && io->means_host && a->value_mode == GD_VALUES_TWO_MEANS)
+  if (e == cudaSuccess && io->means_host && a->value_mode != GD_VALUES_FP32)
     e = cudaMemcpyAsync(io->means_host, a->out_means, sizeof(float) * 2 * (size_t)a->n_layers, cudaMemcpyDeviceToHost,
                         stream);
   if (e != cudaSuccess) return GD_ERR_CUDA;

@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__
     const uint32_t w = __ldcs(A.idx + p);
     uint64_t pos = w;
     float x;
-    if (A.value_mode == GD_VALUES_TWO_MEANS) {
+    if (A.value_mode != GD_VALUES_FP32) {
       pos = w & kAbsMask;
       const uint32_t l = range_of(layer_off, A.n_layers, pos);
       x = __ldg(A.means + 2 * (size_t)l + (w >> 31));
@@ -85,8 +85,8 @@ int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes
 int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
   if (!a || !a->params || !a->shard_off || a->n_shards == 0) return GD_ERR_INVALID_ARG;
   if (a->n_pushes && !a->pushes) return GD_ERR_INVALID_ARG;
-  if (a->value_mode != GD_VALUES_FP32 && a->value_mode != GD_VALUES_TWO_MEANS) return GD_ERR_INVALID_ARG;
-  const bool two_means = a->value_mode == GD_VALUES_TWO_MEANS;
+  if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_THRESHOLD) return GD_ERR_INVALID_ARG;
+  const bool two_means = a->value_mode != GD_VALUES_FP32;   // the packed modes decode through the means table
   if (two_means && (!a->layer_off || a->n_layers == 0)) return GD_ERR_INVALID_ARG;
   for (uint32_t j = 0; j < a->n_shards; ++j) {
     if (a->shard_off[j + 1] < a->shard_off[j]) return GD_ERR_INVALID_ARG;

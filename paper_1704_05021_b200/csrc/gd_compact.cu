@@ -13,6 +13,7 @@ namespace {
 __device__ void finalize_call(const DevTables& T) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
+  const bool packed = T.value_mode != GD_VALUES_FP32;
   uint32_t n_pred = 0, n_dense = 0;
   unsigned long long n_cand = 0;
   for (uint32_t s = tid; s < T.n_scopes; s += kThreads) {
@@ -34,7 +35,7 @@ __device__ void finalize_call(const DevTables& T) {
       const uint64_t span = hi - lo;
       const uint64_t p = lo + span * (lane + 1) / 33;   // lo < p < hi, ascending in lane
       uint32_t w = __ldcg(T.out_idx + p);
-      if (two_means) w &= kAbsMask;
+      if (packed) w &= kAbsMask;
       const uint32_t c = __popc(__ballot_sync(0xFFFFFFFFu, (uint64_t)w < bound));   // probes 0..c-1 are below
       const uint64_t nlo = c ? lo + span * c / 33 + 1 : lo;
       const uint64_t nhi = c < 32 ? lo + span * (c + 1) / 33 : hi;
@@ -45,7 +46,7 @@ __device__ void finalize_call(const DevTables& T) {
     bool below = false;
     if (p < hi) {
       uint32_t w = __ldcg(T.out_idx + p);
-      if (two_means) w &= kAbsMask;
+      if (packed) w &= kAbsMask;
       below = (uint64_t)w < bound;
     }
     lo += __popc(__ballot_sync(0xFFFFFFFFu, below));
@@ -55,6 +56,14 @@ __device__ void finalize_call(const DevTables& T) {
     for (uint32_t e = tid; e < 2 * T.n_layers; e += kThreads) {
       const unsigned long long c = __ldcg(T.cnts + e);
       T.out_means[e] = c ? (float)(__ldcg(T.sums + e) / (double)c) : 0.0f;
+    }
+  } else if (T.value_mode == GD_VALUES_THRESHOLD) {
+    // every survivor of layer l stands for +-t, t = the threshold of the scope that holds the layer
+    for (uint32_t l = tid; l < T.n_layers; l += kThreads) {
+      const uint32_t s = T.n_scopes == 1 ? 0u : l;
+      const uint32_t tau = T.scopes[s].k == 0 ? 0u : __ldcg(&T.state[s].tau);
+      T.out_means[2 * l] = __uint_as_float(tau);
+      T.out_means[2 * l + 1] = __uint_as_float(tau | 0x80000000u);
     }
   }
 }
@@ -85,6 +94,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   const uint32_t* tile0;
   load_tables(T, LK, &s_tab, &scopes, &tile0);
   const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
+  const bool packed = T.value_mode != GD_VALUES_FP32;
   const uint32_t ltm = lanemask_lt();
   uint4* desc = reinterpret_cast<uint4*>(VIEW == V_CAND ? T.desc_cand : T.desc_dcomp);
 
@@ -189,11 +199,13 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
           if (pos < d.k && idx < T.n) {
             const uint32_t b = vb[j];
             T.residual[idx] = 0.0f;
-            if (two_means) {
+            if (packed) {
               const uint32_t sgn = b >> 31;
               T.out_idx[d.out_base + pos] = (uint32_t)idx | (sgn << 31);
               const double x = (double)__uint_as_float(b);
-              if (single) {
+              if (!two_means) {
+                // threshold mode: the value is implied by the scope's tau
+              } else if (single) {
                 if (sgn) { sum_n += x; ++cnt_n; } else { sum_p += x; ++cnt_p; }
               } else {
                 const uint32_t l = range_of(T.layer_off, T.n_layers, idx);
@@ -245,7 +257,27 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   finalize_call(T);
 }
 
+// Self-test kernel of the bounded waits: tile 1 waits on tile 0, which nothing publishes; tile 2
+// then meets the aborted tile 1.
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(Ctl* ctl, uint4* desc, uint32_t spin_limit) {
+  uint64_t ex_a, ex_b;
+  const bool ok1 = tile_lookback(desc, 1, 0, 5, 0, ex_a, ex_b, ctl, spin_limit);
+  const bool ok2 = tile_lookback(desc, 2, 0, 7, 0, ex_a, ex_b, ctl, spin_limit);
+  if (lane_id() == 0) {
+    ctl->n_scopes = ok1 ? 0u : 1u;
+    ctl->n_scopes_predicted = ok2 ? 0u : 1u;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream) {
+  cudaError_t e = cudaMemsetAsync(workspace, 0, 512, stream);
+  if (e != cudaSuccess) return e;
+  bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>((Ctl*)workspace, (uint4*)((unsigned char*)workspace + 256), spin_limit);
+  GD_LAUNCH_CHECK();
+  return cudaSuccess;
+}
 
 cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream) {
   ProfileScope prof(stream, PT_FINALIZE);

@@ -197,6 +197,7 @@ cudaError_t launch_candidate_select(const DevTables& T, const uint32_t* tiles, c
 cudaError_t launch_dense_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, bool finalize, cudaStream_t stream);
 cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream);
+cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream);
 int sm_count();   // multiprocessors of the current device (0 on error)
 
 // Measurement hooks (gd_api.cu): count a kernel launch; record an event of the pair around the fused pass.

@@ -29,7 +29,8 @@ __device__ __forceinline__ uint64_t warp_sum(uint64_t x) {
 // GD_ERR_DEVICE_TIMEOUT and returns false; a tile that meets an aborted predecessor aborts too, so
 // nothing waits on a tile that gave up.
 __device__ __forceinline__ bool tile_lookback(uint4* desc, uint32_t t, uint32_t first, uint64_t tot_a, uint64_t tot_b,
-                                              uint64_t& ex_a, uint64_t& ex_b, Ctl* ctl) {
+                                              uint64_t& ex_a, uint64_t& ex_b, Ctl* ctl,
+                                              uint32_t spin_limit = kLookbackSpinLimit) {
   const uint32_t lane = lane_id();
   ex_a = 0;
   ex_b = 0;
@@ -53,7 +54,7 @@ __device__ __forceinline__ bool tile_lookback(uint4* desc, uint32_t t, uint32_t 
       nearest = stop ? (uint32_t)__ffs((int)stop) - 1u : 32u;
       const uint32_t need = nearest >= 32u ? 0xFFFFFFFFu : ((1u << nearest) - 1u);
       if ((inv & need) == 0u) break;
-      if (++spins > kLookbackSpinLimit) { ok = false; break; }
+      if (++spins > spin_limit) { ok = false; break; }
       if (spins > 8) __nanosleep(64);
     }
     if (!ok) break;

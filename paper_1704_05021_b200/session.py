@@ -64,7 +64,7 @@ class GradDropSession:
     def push(self) -> dict:
         """The last compress call's output as a push record for ApplyCall."""
         p = {"idx": self.out_idx, "shard_cnt_off": self.out_shard_cnt_off}
-        if self.value_mode == B.GD_VALUES_TWO_MEANS:
+        if self.value_mode != B.GD_VALUES_FP32:
             p["means"] = self.out_means
         else:
             p["val"] = self.out_val
@@ -72,7 +72,7 @@ class GradDropSession:
 
     def apply_call(self, params: List[torch.Tensor], alpha: float = 1.0, pushes=None) -> B.ApplyCall:
         pushes = [self.push()] if pushes is None else pushes
-        lo = self.layer_off if self.value_mode == B.GD_VALUES_TWO_MEANS else None
+        lo = self.layer_off if self.value_mode != B.GD_VALUES_FP32 else None
         return B.ApplyCall(params, self.shard_off, pushes, self.value_mode, alpha, self.apply_workspace, lo)
 
     def apply(self, params: List[torch.Tensor], alpha: float = 1.0, stream=None) -> None:

@@ -29,6 +29,7 @@ SCOPE_GLOBAL = 0
 SCOPE_PER_LAYER = 1
 VALUES_FP32 = 0
 VALUES_TWO_MEANS = 1
+VALUES_THRESHOLD = 2
 
 _CHUNK = 1 << 24  # elements generated per call of the random generator (bounds temporaries)
 

@@ -35,6 +35,8 @@ def compare_step(sess: GradDropSession, exp: dict, tag: str):
     if sess.value_mode == B.GD_VALUES_FP32:
         got_val = _np_u32(sess.out_val)[:k]
         assert np.array_equal(got_val, exp["val"].view(np.uint32)), f"{tag}: val bits differ"
+    elif sess.value_mode == B.GD_VALUES_THRESHOLD:
+        assert np.array_equal(_np_u32(sess.out_means), exp["means"].view(np.uint32)), f"{tag}: +-tau pairs differ"
     else:
         got_means = sess.out_means.cpu().numpy().astype(np.float64)
         ref = np.where(exp["counts"] > 0, exp["sums"] / np.maximum(exp["counts"], 1), 0.0)
@@ -114,7 +116,7 @@ def test_empty_gradient(cuda_device):
 
 @pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
 @pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
-@pytest.mark.parametrize("value_mode", [B.GD_VALUES_FP32, B.GD_VALUES_TWO_MEANS])
+@pytest.mark.parametrize("value_mode", [B.GD_VALUES_FP32, B.GD_VALUES_TWO_MEANS, B.GD_VALUES_THRESHOLD])
 def test_ragged_layers(cuda_device, flags, scope_mode, value_mode):
     sizes = [10, 0, 37, 1, 4096 + 5, 5, 100_003, 3, 8192, 2]      # unaligned starts, tiny and empty layers
     rng = np.random.default_rng(7)
@@ -176,7 +178,25 @@ def test_integer_gradients_conserve_mass(cuda_device):
 # ---------------------------------------------------------------- workloads 2, 3, 4 (shapes of the paper's models)
 @pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
 def test_config2_mnist_shaped(cuda_device, scope_mode):
-    run_steps(W.workload(2, scope_mode=scope_mode), cuda_device, 3, method="select", expect_dense=False)
+    steps = 20 if scope_mode == B.GD_SCOPE_PER_LAYER else 5        # the workload's 20 steps, error feedback carried
+    run_steps(W.workload(2, scope_mode=scope_mode), cuda_device, steps, method="select", expect_dense=False)
+
+
+def test_config3_threshold_quantisation(cuda_device):
+    w = W.workload(4)
+    w.value_mode = B.GD_VALUES_THRESHOLD
+    run_steps(w, cuda_device, 1, method="select")
+
+
+def test_bounded_wait_gives_up_and_context_survives(cuda_device):
+    """A wait on a tile that nothing publishes runs out of polls, reports a timeout, and the next call works."""
+    ws = torch.zeros(4096, dtype=torch.uint8, device=cuda_device)
+    B.gd_selftest_bounded_wait(ws, spin_limit=2000)
+    st = B.gd_get_stats(ws)
+    assert st["status"] == B.GD_ERR_DEVICE_TIMEOUT
+    assert st["n_scopes"] == 1            # the first wait gave up
+    assert st["n_scopes_predicted"] == 1  # the tile behind it aborted instead of waiting
+    run_steps(W.workload(1), cuda_device, 1)
 
 
 def test_config2_no_prediction(cuda_device):
@@ -186,7 +206,7 @@ def test_config2_no_prediction(cuda_device):
 
 @pytest.mark.parametrize("config", [3, 4])
 def test_config34_nmt_shaped(cuda_device, config):
-    run_steps(W.workload(config), cuda_device, 2, method="select")
+    run_steps(W.workload(config), cuda_device, 4 if config == 3 else 2, method="select")
 
 
 def test_config4_matches_config3_sets(cuda_device):

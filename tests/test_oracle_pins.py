@@ -368,3 +368,25 @@ def test_apply_two_means_decode():
     ref, _ = orc.apply_pushes(np.ones(6, np.float32), 4, [{"idx": idx, "means": means}],
                               value_mode=orc.VALUES_TWO_MEANS, layer_off=layer_off)
     assert ref.tolist() == [-2.0, 1.0, 1.0, 1.0, 1.0, 3.0]
+
+
+# ---------------------------------------------------------------- threshold quantisation
+def test_threshold_quantisation_values():
+    """Every survivor stands for +-(the smallest kept magnitude of its scope), written out by hand."""
+    layer_off = [0, 4, 10]
+    g = np.array([0.5, -3.0, 0.25, 2.0,   -0.125, 7.0, -6.0, 0.0625, 5.0, -0.03125], dtype=np.float32)
+    r = np.full(10, -0.0, dtype=np.float32)
+    out = orc.compress(g, r, layer_off, [0, 10], 500_000, scope_mode=orc.SCOPE_PER_LAYER,
+                       value_mode=orc.VALUES_THRESHOLD)
+    # layer 0 keeps 2 of 4: -3.0, 2.0 -> t = 2.0 ; layer 1 keeps 3 of 6: 7.0, -6.0, 5.0 -> t = 5.0
+    assert (out["idx"] & np.uint32(0x7FFFFFFF)).tolist() == [1, 3, 5, 6, 8]
+    assert (out["idx"] >> np.uint32(31)).tolist() == [1, 0, 0, 1, 0]
+    assert out["means"].tolist() == [[2.0, -2.0], [5.0, -5.0]]
+    pos, val = orc.decode_push(out["idx"], None, orc.VALUES_THRESHOLD, out["means"], layer_off)
+    assert val.tolist() == [-2.0, 2.0, 5.0, -5.0, 5.0]
+    assert np.all(np.abs(val) <= np.abs(g[pos]))          # never larger than the value it stands for
+    glob = orc.compress(g, r, layer_off, [0, 10], 500_000, scope_mode=orc.SCOPE_GLOBAL,
+                        value_mode=orc.VALUES_THRESHOLD)
+    assert glob["means"].tolist() == [[2.0, -2.0], [2.0, -2.0]]     # one global threshold: 7, -6, 5, -3, 2 kept
+    none = orc.compress(g, r, layer_off, [0, 10], 1_000_000, value_mode=orc.VALUES_THRESHOLD)
+    assert none["idx"].size == 0 and np.all(none["means"].view(np.uint32) == [[0, 0x80000000]] * 2)
