@@ -121,7 +121,7 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, i
     if (ns) {
       tiles[L_EMIT] += (d.hi + CH - 1) / CH - d.lo / CH;
       tiles[L_DSEL] += (ns + kDenseSelTile - 1) / kDenseSelTile;
-      tiles[L_DCOMP] += (ns + kTile - 1) / kTile;
+      tiles[L_DCOMP] += (ns + kDenseChunkTiles * kTile - 1) / (kDenseChunkTiles * kTile);
     }
     tiles[L_SAMP] += (m + kTile - 1) / kTile;
     tiles[L_CAND] += (cap + kTile - 1) / kTile;

@@ -257,6 +257,205 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   finalize_call(T);
 }
 
+// Compaction over the dense range itself, for scopes whose prediction failed.  Same placement rule
+// as above, but one ticket covers a chunk of kDenseChunkTiles tiles (512 KiB of values) and the chunk does
+// one look-back: at 4 bytes per element the chain of look-backs would otherwise have to advance about a
+// hundred tiles per microsecond, which the L2 round trips between CTAs cannot sustain.
+// The classification masks stay in registers; the values of the (few) survivors are read again.
+__global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid_constant__ DevTables T,
+                                                                    uint32_t total_chunks, int do_finalize) {
+  constexpr int CD = (int)kDenseChunkTiles;
+  constexpr int ROUNDS = kTile / kThreads;   // 16 elements per thread and tile
+  constexpr int E = CD * kWarps;             // (tile, warp) counters of one chunk: 32
+  __shared__ uint32_t s_chunk;
+  __shared__ uint32_t s_cg[E], s_ce[E], s_og[E], s_oe[E];
+  __shared__ uint64_t s_exg, s_exe;
+  __shared__ int s_ok, s_single, s_last;
+  __shared__ uint32_t s_layer;
+  __shared__ double s_red[kWarps][2];
+  __shared__ uint32_t s_redc[kWarps][2];
+  __shared__ SmemTables s_tab;
+  __shared__ uint32_t s_mask[CD][kThreads];   // per tile and thread; low 16 bits: key > tau, high 16: key == tau
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  if (!(T.flags & GD_FLAG_NO_PREDICTION) && T.ctl->dense_needed == 0u) return;
+  const ScopeDesc* scopes;
+  const uint32_t* tile0;
+  load_tables(T, L_DCOMP, &s_tab, &scopes, &tile0);
+  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
+  const bool packed = T.value_mode != GD_VALUES_FP32;
+  const uint32_t ltm = lanemask_lt();
+  uint4* desc = reinterpret_cast<uint4*>(T.desc_dcomp);
+
+  for (;;) {
+    __syncthreads();                       // previous chunk is done with the shared variables
+    if (tid == 0) s_chunk = atomicAdd(&T.ctl->ticket[L_DCOMP], 1u);
+    __syncthreads();
+    const uint32_t t = s_chunk;
+    if (t >= total_chunks) break;
+    const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
+    const ScopeDesc& d = scopes[s];
+    const ScopeState* st = T.state + s;
+    if (predicted_ok(T, d, *st)) continue;          // the candidate list owns this scope
+    const uint32_t first = tile0[s];
+    const uint32_t lt = t - first;
+    const uint64_t len = d.hi - d.lo;
+    const uint64_t beg = (uint64_t)lt * (CD * kTile);
+    const uint64_t end = (beg + CD * kTile < len) ? beg + CD * kTile : len;
+    const float* vals = T.residual + d.lo;
+    const uint32_t tau = st->tau;
+    const uint64_t q = st->q;
+    if (two_means && tid == 0) {
+      const uint32_t l0 = range_of(T.layer_off, T.n_layers, d.lo + beg);
+      const uint32_t l1 = range_of(T.layer_off, T.n_layers, d.lo + end - 1);
+      s_layer = l0;
+      s_single = (l0 == l1) ? 1 : 0;
+    }
+
+    // phase 1: classify every element of the chunk, count per (tile, warp)
+#pragma unroll 1
+    for (int c = 0; c < CD; ++c) {
+      if (beg + (uint64_t)c * kTile >= end) {       // the scope ends inside this chunk (uniform over the CTA)
+        s_mask[c][tid] = 0;
+        if (lane == 0) { s_cg[c * kWarps + warp] = 0; s_ce[c * kWarps + warp] = 0; }
+        continue;
+      }
+      const uint64_t wbeg = beg + (uint64_t)c * kTile + (uint64_t)warp * (32u * ROUNDS) + lane;
+      uint32_t vb[ROUNDS];
+#pragma unroll
+      for (int j = 0; j < ROUNDS; ++j) {
+        const uint64_t i = wbeg + (uint64_t)j * 32u;
+        vb[j] = i < end ? __float_as_uint(vals[i]) : 0xFFFFFFFFu;
+      }
+      uint32_t m = 0, wg = 0, we = 0;
+#pragma unroll
+      for (int j = 0; j < ROUNDS; ++j) {
+        const uint64_t i = wbeg + (uint64_t)j * 32u;
+        const uint32_t key = vb[j] & kAbsMask;
+        const bool isgt = i < end && key > tau, iseq = i < end && key == tau;
+        m |= (isgt ? 1u : 0u) << j;
+        m |= (iseq ? 1u : 0u) << (16 + j);
+        wg += __popc(__ballot_sync(0xFFFFFFFFu, isgt));
+        we += __popc(__ballot_sync(0xFFFFFFFFu, iseq));
+      }
+      s_mask[c][tid] = m;
+      if (lane == 0) { s_cg[c * kWarps + warp] = wg; s_ce[c * kWarps + warp] = we; }
+    }
+    __syncthreads();
+    if (warp == 0) {                                // E counter pairs, PER consecutive ones per lane
+      constexpr int PER = E / 32;
+      uint32_t ag[PER], ae[PER], sg = 0, se = 0;
+#pragma unroll
+      for (int p = 0; p < PER; ++p) {
+        ag[p] = s_cg[lane * PER + p];
+        ae[p] = s_ce[lane * PER + p];
+        sg += ag[p];
+        se += ae[p];
+      }
+      uint32_t ig = sg, ie = se;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t yg = __shfl_up_sync(0xFFFFFFFFu, ig, o), ye = __shfl_up_sync(0xFFFFFFFFu, ie, o);
+        if ((int)lane >= o) { ig += yg; ie += ye; }
+      }
+      uint32_t rg0 = ig - sg, re0 = ie - se;
+#pragma unroll
+      for (int p = 0; p < PER; ++p) {
+        s_og[lane * PER + p] = rg0;
+        s_oe[lane * PER + p] = re0;
+        rg0 += ag[p];
+        re0 += ae[p];
+      }
+      const uint32_t tot_g = __shfl_sync(0xFFFFFFFFu, ig, 31), tot_e = __shfl_sync(0xFFFFFFFFu, ie, 31);
+      uint64_t ex_a, ex_b;
+      const bool ok = tile_lookback(desc, t, first, tot_g, tot_e, ex_a, ex_b, T.ctl);
+      if (lane == 0) { s_exg = ex_a; s_exe = ex_b; s_ok = ok ? 1 : 0; }
+    }
+    __syncthreads();
+    if (!s_ok) continue;
+
+    // phase 2: place the survivors
+    const bool single = two_means && s_single;
+    const uint32_t tile_layer = two_means ? s_layer : 0u;
+    double sum_p = 0.0, sum_n = 0.0;
+    uint32_t cnt_p = 0, cnt_n = 0;
+    bool bad = false;
+#pragma unroll 1
+    for (int c = 0; c < CD; ++c) {
+      const uint32_t m = s_mask[c][tid];
+      if (!__any_sync(0xFFFFFFFFu, m != 0u)) continue;
+      const uint64_t wbeg = beg + (uint64_t)c * kTile + (uint64_t)warp * (32u * ROUNDS) + lane;
+      uint64_t rg = s_exg + s_og[c * kWarps + warp], re = s_exe + s_oe[c * kWarps + warp];
+#pragma unroll
+      for (int j = 0; j < ROUNDS; ++j) {
+        const bool isgt = (m >> j) & 1u, iseq = (m >> (16 + j)) & 1u;
+        const uint32_t mg = __ballot_sync(0xFFFFFFFFu, isgt), me = __ballot_sync(0xFFFFFFFFu, iseq);
+        if (isgt || iseq) {
+          const uint64_t gb = rg + __popc(mg & ltm), eb = re + __popc(me & ltm);
+          if (isgt || eb < q) {
+            const uint64_t pos = gb + (eb < q ? eb : q);
+            const uint64_t i = wbeg + (uint64_t)j * 32u;
+            const uint64_t idx = d.lo + i;
+            if (pos < d.k && idx < T.n) {
+              const uint32_t b = __float_as_uint(vals[i]);   // read again: only survivors get here
+              T.residual[idx] = 0.0f;
+              if (packed) {
+                const uint32_t sgn = b >> 31;
+                T.out_idx[d.out_base + pos] = (uint32_t)idx | (sgn << 31);
+                const double x = (double)__uint_as_float(b);
+                if (!two_means) {
+                  // threshold mode: the value is implied by the scope's tau
+                } else if (single) {
+                  if (sgn) { sum_n += x; ++cnt_n; } else { sum_p += x; ++cnt_p; }
+                } else {
+                  const uint32_t l = range_of(T.layer_off, T.n_layers, idx);
+                  atomicAdd(T.sums + 2 * (size_t)l + sgn, x);
+                  atomicAdd(T.cnts + 2 * (size_t)l + sgn, 1ull);
+                }
+              } else {
+                T.out_idx[d.out_base + pos] = (uint32_t)idx;
+                T.out_val[d.out_base + pos] = __uint_as_float(b);
+              }
+            } else {
+              bad = true;
+            }
+          }
+        }
+        rg += __popc(mg);
+        re += __popc(me);
+      }
+    }
+    if (bad) atomicCAS(&T.ctl->status, (int)GD_OK, (int)GD_ERR_INTERNAL);
+    if (single) {   // uniform over the CTA
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        sum_p += __shfl_xor_sync(0xFFFFFFFFu, sum_p, o);
+        sum_n += __shfl_xor_sync(0xFFFFFFFFu, sum_n, o);
+        cnt_p += __shfl_xor_sync(0xFFFFFFFFu, cnt_p, o);
+        cnt_n += __shfl_xor_sync(0xFFFFFFFFu, cnt_n, o);
+      }
+      if (lane == 0) { s_red[warp][0] = sum_p; s_red[warp][1] = sum_n; s_redc[warp][0] = cnt_p; s_redc[warp][1] = cnt_n; }
+      __syncthreads();
+      if (tid < 2) {
+        double sx = 0.0;
+        unsigned long long cx = 0;
+        for (int w = 0; w < kWarps; ++w) { sx += s_red[w][tid]; cx += s_redc[w][tid]; }
+        if (cx) {
+          atomicAdd(T.sums + 2 * (size_t)tile_layer + tid, sx);
+          atomicAdd(T.cnts + 2 * (size_t)tile_layer + tid, cx);
+        }
+      }
+    }
+  }
+  if (!do_finalize) return;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&T.ctl->compact_done[1], 1u) == gridDim.x - 1u) ? 1 : 0;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  finalize_call(T);
+}
+
 // Self-test kernel of the bounded waits: tile 1 waits on tile 0, which nothing publishes; tile 2
 // then meets the aborted tile 1.
 __global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(Ctl* ctl, uint4* desc, uint32_t spin_limit) {
@@ -290,10 +489,10 @@ cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense
   const uint32_t total = tiles[dense ? L_DCOMP : L_CAND];
   if (!total) return finalize ? launch_finalize(T, stream) : cudaSuccess;
   ProfileScope prof(stream, dense ? PT_DENSE_COMPACT : PT_CAND_COMPACT);
-  const uint32_t cap = (uint32_t)sm_count() * 8u;
+  const uint32_t cap = (uint32_t)sm_count() * (dense ? 3u : 8u);
   const uint32_t grid = total < cap ? total : cap;
   if (dense)
-    compact_kernel<V_DENSE><<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
+    compact_dense_kernel<<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
   else
     compact_kernel<V_CAND><<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
   GD_LAUNCH_CHECK();

@@ -56,7 +56,11 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
   const uint32_t lt = t - first;
   constexpr uint64_t CH = (uint64_t)C * kTile;
   const uint64_t cbase = (lo / CH + lt) * CH;
-  const uint32_t tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || d.k == 0) ? 0xFFFFFFFFu : T.state[s].tau_lo;
+  // Zeros are never candidates: when the prediction is 0 the list holds the non-zero entries, and if
+  // there are fewer than k of them the threshold is 0 and the zeros that are kept are found by the
+  // dense compaction alone (no dense selection is needed to know tau = 0).
+  uint32_t tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || d.k == 0) ? 0xFFFFFFFFu : T.state[s].tau_lo;
+  if (tau_lo == 0u) tau_lo = 1u;
   const uint64_t toff = (uint64_t)warp * 512u + lane * 4u;   // this thread's first element inside a tile
   const uint32_t ltm = lanemask_lt();
   StashEntry* stash = s_stash[warp];

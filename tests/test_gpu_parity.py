@@ -303,3 +303,33 @@ def test_many_layers_and_shards(cuda_device, value_mode):
         w = W.small_layered(len(sizes), sizes, 980_000, scope_mode, value_mode, 40)
         grads = [torch.from_numpy(rng.laplace(0, 1e-3, w.n).astype(np.float32)) for _ in range(2)]
         run_steps(w, cuda_device, 2, grads=grads)
+
+
+# ---------------------------------------------------------------- other drop ratios (Section 5.1: 90 %, 99 %, 99.9 %)
+@pytest.mark.parametrize("drop_ppm", [900_000, 999_000])
+@pytest.mark.parametrize("config", [2, 3])
+def test_drop_ratio_sweep(cuda_device, config, drop_ppm):
+    """The paper's other two drop ratios on the MNIST- and NMT-shaped sets (at 90 % the push is 10x larger,
+    most warps of the fused pass overflow their stash, and the apply matters)."""
+    w = W.workload(config, scope_mode=B.GD_SCOPE_PER_LAYER)
+    w.drop_ppm = drop_ppm
+    run_steps(w, cuda_device, 2, method="select")
+
+
+def test_more_kept_than_nonzero(cuda_device):
+    """Row-sparse layers whose non-zero entries number fewer than k: the threshold is 0 and the lowest-index
+    zeros fill the quota (the NMT embeddings at a 90 % drop ratio)."""
+    rng = np.random.default_rng(5)
+    sizes = [200_000, 64, 300_001]
+    grads = []
+    for _ in range(2):
+        g = np.zeros(sum(sizes), np.float32)
+        rows = rng.choice(sizes[0] // 500, 12, replace=False)
+        for r_ in rows:
+            g[r_ * 500:(r_ + 1) * 500] = rng.standard_normal(500) * 1e-3
+        g[sizes[0] + sizes[1]:] = np.where(rng.random(sizes[2]) < 0.03, rng.standard_normal(sizes[2]), 0)
+        grads.append(torch.from_numpy(g))
+    for scope_mode in (B.GD_SCOPE_PER_LAYER, B.GD_SCOPE_GLOBAL):
+        w = W.small_layered(3, sizes, 900_000, scope_mode, B.GD_VALUES_FP32, 3)
+        sess = run_steps(w, cuda_device, 2, grads=grads)
+        assert sess.stats()["n_scopes_dense"] >= 1
