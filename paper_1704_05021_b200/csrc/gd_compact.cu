@@ -312,7 +312,7 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
     }
 
     // phase 1: classify every element of the chunk, count per (tile, warp)
-#pragma unroll 1
+#pragma unroll 2
     for (int c = 0; c < CD; ++c) {
       if (beg + (uint64_t)c * kTile >= end) {       // the scope ends inside this chunk (uniform over the CTA)
         s_mask[c][tid] = 0;

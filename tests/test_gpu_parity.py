@@ -333,3 +333,52 @@ def test_more_kept_than_nonzero(cuda_device):
         w = W.small_layered(3, sizes, 900_000, scope_mode, B.GD_VALUES_FP32, 3)
         sess = run_steps(w, cuda_device, 2, grads=grads)
         assert sess.stats()["n_scopes_dense"] >= 1
+
+
+# ---------------------------------------------------------------- several workers pushing into one server shard
+@pytest.mark.parametrize("value_mode", [B.GD_VALUES_FP32, B.GD_VALUES_TWO_MEANS])
+def test_three_workers_push_into_each_server(cuda_device, value_mode):
+    """Section 3: every server owns 1/N of the parameters and receives one piece from every worker.  Three
+    workers compress their own gradients; each of the 4 servers applies the three pieces of its shard in
+    one call (pushes collide on many indices and are applied in order)."""
+    rng = np.random.default_rng(17)
+    sizes = [30_000, 11, 50_001]
+    w = W.small_layered(3, sizes, 950_000, B.GD_SCOPE_PER_LAYER, value_mode, 4)
+    workers, expected = [], []
+    for _ in range(3):
+        sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
+        g = rng.laplace(0, 1e-3, w.n).astype(np.float32)
+        g[rng.integers(0, w.n, 2000)] *= 50.0                      # shared hot spots are unlikely; force some
+        g[:500] += 0.5
+        exp = orc.compress(g, orc.residual_reset(w.n), w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode)
+        sess.compress(torch.from_numpy(g).to(cuda_device))
+        compare_step(sess, exp, "worker")
+        workers.append(sess)
+        expected.append(exp)
+    p0 = (rng.standard_normal(w.n) * 0.01).astype(np.float32)
+    params = torch.from_numpy(p0).to(cuda_device)
+    aws = torch.empty(B.gd_apply_workspace_bytes(1, len(sizes)), dtype=torch.uint8, device=cuda_device)
+    for j in range(w.n_shards):                                    # server j: its shard only, pieces j of all workers
+        lo, hi = w.shard_off[j], w.shard_off[j + 1]
+        pushes = []
+        for sess in workers:
+            p = {"idx": sess.out_idx, "shard_cnt_off": sess.out_shard_cnt_off[j:j + 2]}
+            if value_mode == B.GD_VALUES_FP32:
+                p["val"] = sess.out_val
+            else:
+                p["means"] = sess.out_means
+            pushes.append(p)
+        call = B.ApplyCall([params[lo:hi]], [lo, hi], pushes, value_mode, 0.25, aws,
+                           w.layer_off if value_mode != B.GD_VALUES_FP32 else None)
+        B.gd_decompress_apply(call)
+    torch.cuda.synchronize()
+    got = params.cpu().numpy().astype(np.float64)
+    collisions = 0
+    for j in range(w.n_shards):
+        lo, hi = w.shard_off[j], w.shard_off[j + 1]
+        ref, bound = orc.apply_pushes(p0[lo:hi], lo, expected, alpha=0.25, value_mode=value_mode, layer_off=w.layer_off)
+        assert np.all(np.abs(got[lo:hi] - ref) <= REL_TOL * bound + 1e-45), f"server {j}"
+    hits = np.zeros(w.n, np.int32)
+    for exp in expected:
+        hits[(exp["idx"] & np.uint32(0x7FFFFFFF)).astype(np.int64)] += 1
+    assert (hits >= 2).sum() > 100                                 # the pushes really collide
