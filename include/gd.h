@@ -94,6 +94,18 @@ int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes
  *              that holds layer l (+0, -0 if that scope keeps nothing), so that a push decodes exactly
  *              like a two-means push.
  *
+ *   delta mode (delta_base != NULL; Section 4, third paragraph: the same function is applied to
+ *              parameter pulls "encoded as deltas from the last version pulled by the client", the
+ *              server keeping that last version): grad holds the server's current parameters,
+ *              delta_base the copy the client is known to hold, and
+ *                  v[i] = grad[i] - delta_base[i]          (one fp32 subtraction)
+ *              takes the place of grad + residual; the residual's old contents are not read.  After the
+ *              selection delta_base[i] <- delta_base[i] + v[i] (one fp32 add) for every survivor, which is
+ *              exactly what gd_decompress_apply with alpha = 1 does to the client's copy, so the two
+ *              copies stay equal bit for bit; what was dropped stays in the next delta by itself.  The
+ *              residual buffer is used as scratch and returns v where dropped, +0 where kept.  Delta
+ *              mode needs GD_VALUES_FP32.
+ *
  * Results are bit-exact functions of (grad, residual, offsets, drop_ppm) except the two means,
  * whose fp64 partial sums are combined in an unspecified order.  Non-finite inputs are ordered by
  * their bit pattern (NaN above Inf above finite); NaN payloads follow the device's fp32 add.
@@ -119,6 +131,7 @@ typedef struct gd_compress_args {
   float* out_means;           /* device, n_layers x 2 fp32 (mu+, mu-); two-means and threshold modes */
   void* workspace;            /* device, 256-byte aligned, >= gd_workspace_bytes() */
   size_t workspace_bytes;
+  float* delta_base;          /* device, n fp32, 16-byte aligned, in/out, or NULL (see "delta mode" above) */
 } gd_compress_args;
 
 int gd_compress(const gd_compress_args* args, void* stream);

@@ -97,6 +97,28 @@ def _kept_in_scope(keys: np.ndarray, k: int, method: str):
     return local, tau
 
 
+def compress_delta(params, last_pulled, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GLOBAL, method="sort"):
+    """GradDrop applied to a parameter pull (Section 4, third paragraph).
+
+    The server keeps `last_pulled`, the copy the client is known to hold, and sends the dropped
+    delta  v = params - last_pulled  (one fp32 subtraction per element).  Whatever is sent is added
+    to last_pulled with one fp32 add, which is exactly what the client does to its own copy, so the
+    two stay equal; what is dropped stays inside the next delta, so no separate residual is read.
+    Returns the dict of compress() (its "residual" is v where dropped, +0 where kept) plus
+    "last_pulled", the updated copy.
+    """
+    p = np.ascontiguousarray(params, dtype=np.float32)
+    last = np.ascontiguousarray(last_pulled, dtype=np.float32)
+    v = p - last
+    out = compress(v, np.full_like(v, -0.0), layer_off, shard_off, drop_ppm, scope_mode, VALUES_FP32, method)
+    # (v + -0.0 is v bit for bit, so compress() selects on v itself)
+    new_last = last.copy()
+    kept = out["idx"].astype(np.int64)
+    new_last[kept] = last[kept] + out["val"]
+    out["last_pulled"] = new_last
+    return out
+
+
 def compress(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GLOBAL,
              value_mode=VALUES_FP32, method="sort"):
     """One GradDrop call (Algorithm 1) for one worker's flat fp32 gradient.

@@ -52,7 +52,7 @@ class _CompressArgs(C.Structure):
         ("value_mode", C.c_int32), ("flags", C.c_uint32),
         ("out_idx", C.c_void_p), ("out_val", C.c_void_p), ("out_shard_cnt_off", C.c_void_p),
         ("out_tau", C.c_void_p), ("out_means", C.c_void_p),
-        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("delta_base", C.c_void_p),
     ]
 
 
@@ -175,8 +175,8 @@ class CompressCall:
     """The marshalled argument block of one gd_compress call (kept so it can be re-issued cheaply)."""
 
     def __init__(self, grad, residual, layer_off, shard_off, drop_ppm, scope_mode, value_mode, out_idx, out_val,
-                 out_shard_cnt_off, out_tau, out_means, workspace, flags=0):
-        self._keep = (grad, residual, out_idx, out_val, out_shard_cnt_off, out_tau, out_means, workspace)
+                 out_shard_cnt_off, out_tau, out_means, workspace, flags=0, delta_base=None):
+        self._keep = (grad, residual, out_idx, out_val, out_shard_cnt_off, out_tau, out_means, workspace, delta_base)
         self._layer_off = _u64_array(layer_off)
         self._shard_off = _u64_array(shard_off)
         a = _CompressArgs()
@@ -188,6 +188,7 @@ class CompressCall:
         a.out_tau, a.out_means = _ptr(out_tau), _ptr(out_means)
         a.workspace = _ptr(workspace)
         a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        a.delta_base = _ptr(delta_base)
         self.args = a
 
     def set_grad(self, grad: torch.Tensor):

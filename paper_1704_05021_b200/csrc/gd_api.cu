@@ -317,6 +317,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     if (a->flags & ~(uint32_t)GD_FLAG_NO_PREDICTION) return GD_ERR_INVALID_ARG;
     if (n && (!a->grad || !a->residual)) return GD_ERR_INVALID_ARG;
     if (((uintptr_t)a->grad | (uintptr_t)a->residual) & 15u) return GD_ERR_INVALID_ARG;
+    if (a->delta_base && (a->value_mode != GD_VALUES_FP32 || ((uintptr_t)a->delta_base & 15u))) return GD_ERR_INVALID_ARG;
     if (!a->out_shard_cnt_off) return GD_ERR_INVALID_ARG;
     if (P.k_total && !a->out_idx) return GD_ERR_INVALID_ARG;
     if (P.k_total && a->value_mode == GD_VALUES_FP32 && !a->out_val) return GD_ERR_INVALID_ARG;
@@ -341,6 +342,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     std::memset(&T, 0, sizeof(T));
     T.grad = a->grad;
     T.residual = a->residual;
+    T.delta_base = a->delta_base;
     T.n = n;
     T.n_scopes = P.n_scopes;
     T.n_layers = a->n_layers;

@@ -215,6 +215,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
             } else {
               T.out_idx[d.out_base + pos] = (uint32_t)idx;
               T.out_val[d.out_base + pos] = __uint_as_float(b);
+              if (T.delta_base) T.delta_base[idx] = __fadd_rn(T.delta_base[idx], __uint_as_float(b));
             }
           } else {
             bad = true;
@@ -414,6 +415,7 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
               } else {
                 T.out_idx[d.out_base + pos] = (uint32_t)idx;
                 T.out_val[d.out_base + pos] = __uint_as_float(b);
+                if (T.delta_base) T.delta_base[idx] = __fadd_rn(T.delta_base[idx], __uint_as_float(b));
               }
             } else {
               bad = true;

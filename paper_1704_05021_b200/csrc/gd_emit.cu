@@ -64,6 +64,8 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
   const uint64_t toff = (uint64_t)warp * 512u + lane * 4u;   // this thread's first element inside a tile
   const uint32_t ltm = lanemask_lt();
   StashEntry* stash = s_stash[warp];
+  const bool delta = T.delta_base != nullptr;            // v = g - base instead of g + r
+  const float* second = delta ? T.delta_base : T.residual;
 
   // ---- phase A
   uint32_t fill = 0;                         // candidates of this warp so far in the chunk (warp-uniform)
@@ -77,14 +79,14 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
 #pragma unroll
       for (int j = 0; j < 4; ++j) g4[j] = __ldcs(reinterpret_cast<const float4*>(T.grad + e0 + j * 128));
 #pragma unroll
-      for (int j = 0; j < 4; ++j) r4[j] = *reinterpret_cast<const float4*>(T.residual + e0 + j * 128);
+      for (int j = 0; j < 4; ++j) r4[j] = *reinterpret_cast<const float4*>(second + e0 + j * 128);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         float x[4];
-        x[0] = __fadd_rn(g4[j].x, r4[j].x);
-        x[1] = __fadd_rn(g4[j].y, r4[j].y);
-        x[2] = __fadd_rn(g4[j].z, r4[j].z);
-        x[3] = __fadd_rn(g4[j].w, r4[j].w);
+        x[0] = delta ? __fsub_rn(g4[j].x, r4[j].x) : __fadd_rn(g4[j].x, r4[j].x);
+        x[1] = delta ? __fsub_rn(g4[j].y, r4[j].y) : __fadd_rn(g4[j].y, r4[j].y);
+        x[2] = delta ? __fsub_rn(g4[j].z, r4[j].z) : __fadd_rn(g4[j].z, r4[j].z);
+        x[3] = delta ? __fsub_rn(g4[j].w, r4[j].w) : __fadd_rn(g4[j].w, r4[j].w);
         *reinterpret_cast<float4*>(T.residual + e0 + j * 128) = make_float4(x[0], x[1], x[2], x[3]);
         uint32_t f = 0;
 #pragma unroll
@@ -114,7 +116,7 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
         for (int c = 0; c < 4; ++c) {
           const uint64_t e = base + toff + j * 128 + c;
           if (e >= lo && e < hi) {
-            x[c] = __fadd_rn(__ldg(T.grad + e), T.residual[e]);
+            x[c] = delta ? __fsub_rn(__ldg(T.grad + e), second[e]) : __fadd_rn(__ldg(T.grad + e), second[e]);
             T.residual[e] = x[c];
             f |= ((__float_as_uint(x[c]) & kAbsMask) >= tau_lo ? 1u : 0u) << c;
           }

@@ -82,6 +82,7 @@ struct Ctl {             // zeroed at the start of every call
 struct DevTables {       // passed by value to every kernel
   const float* grad;
   float* residual;
+  float* delta_base;                 // delta mode: v = grad - delta_base, survivors are added back to it
   uint64_t n;
   uint32_t n_scopes, n_layers, n_shards;
   uint32_t flags;

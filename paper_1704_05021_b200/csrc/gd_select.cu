@@ -57,7 +57,7 @@ __device__ __forceinline__ float sample_value(const DevTables& T, const ScopeDes
   const uint64_t width = b - a;
   uint64_t pos = d.lo + a;
   if (width > 1) pos += mix32((uint32_t)li * 0x9E3779B9u + s) % width;
-  return __fadd_rn(__ldg(T.grad + pos), T.residual[pos]);
+  return T.delta_base ? __fsub_rn(__ldg(T.grad + pos), T.delta_base[pos]) : __fadd_rn(__ldg(T.grad + pos), T.residual[pos]);
 }
 
 template <int VIEW>

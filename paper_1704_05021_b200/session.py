@@ -61,6 +61,14 @@ class GradDropSession:
     def compress(self, grad: torch.Tensor, stream=None) -> None:
         B.gd_compress(self.compress_call(grad), stream)
 
+    def compress_delta(self, params: torch.Tensor, last_pulled: torch.Tensor, stream=None) -> None:
+        """Server side of a pull: GradDrop of params - last_pulled; the survivors are added to last_pulled."""
+        assert last_pulled.is_cuda and last_pulled.dtype == torch.float32 and last_pulled.numel() == self.n
+        call = B.CompressCall(params, self.residual, self.layer_off, self.shard_off, self.drop_ppm, self.scope_mode,
+                              self.value_mode, self.out_idx, self.out_val, self.out_shard_cnt_off, self.out_tau,
+                              self.out_means, self.workspace, self.flags, delta_base=last_pulled)
+        B.gd_compress(call, stream)
+
     def push(self) -> dict:
         """The last compress call's output as a push record for ApplyCall."""
         p = {"idx": self.out_idx, "shard_cnt_off": self.out_shard_cnt_off}

@@ -382,3 +382,32 @@ def test_three_workers_push_into_each_server(cuda_device, value_mode):
     for exp in expected:
         hits[(exp["idx"] & np.uint32(0x7FFFFFFF)).astype(np.int64)] += 1
     assert (hits >= 2).sum() > 100                                 # the pushes really collide
+
+
+# ---------------------------------------------------------------- parameter pulls as dropped deltas
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
+def test_delta_pull_matches_oracle_and_client_copy(cuda_device, flags):
+    """Section 4, third paragraph: the server sends GradDrop(params - last pulled copy).  The library's
+    delta mode must equal the oracle bit for bit, and the server's record of the client's copy must stay
+    identical to what the client holds after applying the pull with alpha = 1."""
+    rng = np.random.default_rng(23)
+    sizes = [70_000, 9, 4096, 130_003]
+    w = W.small_layered(len(sizes), sizes, 980_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 2)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, flags, cuda_device)
+    p_host = (rng.standard_normal(w.n) * 0.1).astype(np.float32)
+    last_host = np.zeros(w.n, dtype=np.float32)
+    last_dev = torch.zeros(w.n, dtype=torch.float32, device=cuda_device)
+    client = torch.zeros(w.n, dtype=torch.float32, device=cuda_device)
+    client_views = sess.shard_views(client)
+    for step in range(4):
+        p_host = p_host + rng.laplace(0, 1e-3, w.n).astype(np.float32)
+        p_dev = torch.from_numpy(p_host).to(cuda_device)
+        exp = orc.compress_delta(p_host, last_host, w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode)
+        sess.compress_delta(p_dev, last_dev)
+        compare_step(sess, exp, f"pull {step} flags {flags}")
+        assert np.array_equal(_np_u32(last_dev), exp["last_pulled"].view(np.uint32)), f"pull {step}: last pulled copy"
+        assert torch.equal(p_dev.cpu(), torch.from_numpy(p_host)), "parameters were modified"
+        sess.apply(client_views, 1.0)
+        torch.cuda.synchronize()
+        assert torch.equal(client.view(torch.int32), last_dev.view(torch.int32)), f"pull {step}: client copy differs"
+        last_host = exp["last_pulled"]

@@ -390,3 +390,36 @@ def test_threshold_quantisation_values():
     assert glob["means"].tolist() == [[2.0, -2.0], [2.0, -2.0]]     # one global threshold: 7, -6, 5, -3, 2 kept
     none = orc.compress(g, r, layer_off, [0, 10], 1_000_000, value_mode=orc.VALUES_THRESHOLD)
     assert none["idx"].size == 0 and np.all(none["means"].view(np.uint32) == [[0, 0x80000000]] * 2)
+
+
+# ---------------------------------------------------------------- parameter pulls as dropped deltas
+def test_delta_pull_by_hand_and_invariants():
+    # by hand: delta = p - last = [0.5, -4, 0.25, 3, 0, -1]; keep 2 of 6 (drop 2/3): -4 and 3
+    p = np.array([1.5, -3.0, 0.25, 5.0, 2.0, 0.0], dtype=np.float32)
+    last = np.array([1.0, 1.0, 0.0, 2.0, 2.0, 1.0], dtype=np.float32)
+    out = orc.compress_delta(p, last, [0, 6], [0, 3, 6], 666_667)
+    assert out["idx"].tolist() == [1, 3] and out["val"].tolist() == [-4.0, 3.0]
+    assert out["last_pulled"].tolist() == [1.0, -3.0, 0.0, 5.0, 2.0, 1.0]
+    assert out["residual"].tolist() == [0.5, 0.0, 0.25, 0.0, 0.0, -1.0]
+    assert out["shard_cnt_off"].tolist() == [0, 1, 2]
+
+    rng = np.random.default_rng(31)
+    n = 3000
+    layer_off, shard_off = [0, 1000, n], [0, n]
+    p = rng.integers(-500, 500, n).astype(np.float32)              # integer-valued: every fp32 op is exact
+    last = np.zeros(n, dtype=np.float32)
+    client = np.zeros(n, dtype=np.float32)
+    for step in range(6):
+        p = p + rng.integers(-50, 51, n).astype(np.float32)
+        out = orc.compress_delta(p, last, layer_off, shard_off, 900_000, scope_mode=orc.SCOPE_PER_LAYER)
+        v = [float(a) - float(b) for a, b in zip(p, last)]
+        want = []
+        for lo, hi in ((0, 1000), (1000, n)):
+            want += [lo + i for i in brute_force_kept(v[lo:hi], orc.kept_count(hi - lo, 900_000))]
+        assert out["idx"].tolist() == want
+        client[out["idx"]] = client[out["idx"]] + out["val"]       # what the client does with the pull
+        last = out["last_pulled"]
+        assert np.array_equal(client.view(np.uint32), last.view(np.uint32))      # server's record == client's copy
+        assert np.array_equal(p - last, out["residual"])           # nothing lost: the rest is the next delta
+    out = orc.compress_delta(p, last, layer_off, shard_off, 0)     # R = 0: the client catches up completely
+    assert np.array_equal(out["last_pulled"], p)
