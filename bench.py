@@ -218,7 +218,8 @@ def run_cuda(args):
 
     w = W.workload(args.config, scale_log2=args.scale_log2) if args.scale_log2 else W.workload(args.config)
     sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
-                           B.GD_FLAG_NO_PREDICTION if args.no_prediction else 0, dev)
+                           (B.GD_FLAG_NO_PREDICTION if args.no_prediction else 0) |
+                           (B.GD_FLAG_SAMPLED_THRESHOLD if args.sampled else 0), dev)
     params = W.make_params(w, dev)
     views = sess.shard_views(params)
     pool = max(1, min(args.steps + args.warmup, args.pool))
@@ -325,7 +326,7 @@ def run_cuda(args):
     # figure scales with n.
     roofline["traffic"] = ADD_EMIT_DRAM_BYTES_PER_ELEMENT * w.n
     roofline["traffic_source"] = "ncu dram__bytes_read.sum + dram__bytes_write.sum at n = 2^27, scaled by n"
-    k_frac = sess.k_total / max(w.n, 1)
+    k_frac = (stats["n_kept"] if args.sampled else sess.k_total) / max(w.n, 1)
     per_surv = 16.0 if w.value_mode == B.GD_VALUES_TWO_MEANS else 24.0
     alg_step_bytes = (12.0 + per_surv * k_frac) * w.n
     step_frac = (alg_step_bytes / (ms_per_step * 1e-3) / 1e9) / peak
@@ -342,7 +343,8 @@ def run_cuda(args):
         "config": workload_config(w, {
             "l2": "L2 flushed between timed steps (512 MiB write), steps timed one by one" if flush
                   else "inputs larger than L2 (gradient + residual stream 8 bytes per element per step)",
-            "gradient_pool": pool, "prediction": not args.no_prediction}),
+            "gradient_pool": pool, "prediction": not args.no_prediction,
+            "threshold": "sampled (0.1 % sample, approximate)" if args.sampled else "exact"}),
         "step_ms": {"min": min(step_ms), "median": statistics.median(step_ms), "max": max(step_ms)},
         "step_roofline": {"algorithmic_bytes_per_step": alg_step_bytes, "frac_of_peak": step_frac,
                           "frac_of_8000": (alg_step_bytes / (ms_per_step * 1e-3) / 1e9) / 8000.0},
@@ -365,6 +367,8 @@ def main():
     ap.add_argument("--no-prediction", action="store_true", help="force the dense selection path")
     ap.add_argument("--scale-log2", type=int, default=0,
                     help="length 2^x for the flat workloads 1 and 5 (profiling on a smaller case)")
+    ap.add_argument("--sampled", action="store_true",
+                    help="threshold selected on a 0.1 %% sample (the paper's approximation); survivor count varies")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

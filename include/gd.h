@@ -35,7 +35,8 @@ typedef enum {
   GD_ERR_WORKSPACE = -3,      /* workspace missing or smaller than gd_workspace_bytes() */
   GD_ERR_CUDA = -4,           /* a CUDA runtime call failed (launch, memset, copy) */
   GD_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait gave up; outputs of that call are invalid */
-  GD_ERR_INTERNAL = -6        /* device-side consistency check failed; outputs of that call are invalid */
+  GD_ERR_INTERNAL = -6,       /* device-side consistency check failed; outputs of that call are invalid */
+  GD_ERR_OVERFLOW = -7        /* sampled-threshold mode: more survivors than gd_sampled_capacity(); outputs invalid */
 } gd_status_t;
 
 enum { GD_SCOPE_GLOBAL = 0, GD_SCOPE_PER_LAYER = 1 };
@@ -43,8 +44,10 @@ enum { GD_VALUES_FP32 = 0, GD_VALUES_TWO_MEANS = 1, GD_VALUES_THRESHOLD = 2 };
 
 /* gd_compress_args.flags */
 enum {
-  GD_FLAG_NO_PREDICTION = 1u  /* do not predict the threshold from a sample: always select over the
+  GD_FLAG_NO_PREDICTION = 1u, /* do not predict the threshold from a sample: always select over the
                                  whole dense vector (same results, more memory traffic) */
+  GD_FLAG_SAMPLED_THRESHOLD = 2u /* the approximation of Section 4: the threshold is selected on a 0.1 %
+                                 sample and every entry at or above it is kept (see gd_compress) */
 };
 
 const char* gd_status_string(int status);
@@ -65,6 +68,13 @@ int gd_kept_count(uint64_t n_scope, uint32_t drop_ppm, uint64_t* k_out);
  */
 int gd_total_kept(const uint64_t* layer_off, uint32_t n_layers, int scope_mode, uint32_t drop_ppm,
                   uint64_t* k_total_out);
+
+/*
+ * Size, in entries, that out_idx / out_val must have for GD_FLAG_SAMPLED_THRESHOLD, where the number of
+ * survivors is not known in advance: per scope min(n_s, 4 k_s + 8192), summed.
+ */
+int gd_sampled_capacity(const uint64_t* layer_off, uint32_t n_layers, int scope_mode, uint32_t drop_ppm,
+                        uint64_t* capacity_out);
 
 /* Bytes of device workspace gd_compress needs for these arguments (same meaning as in gd_compress_args). */
 int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, int scope_mode,
@@ -105,6 +115,18 @@ int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes
  *              copies stay equal bit for bit; what was dropped stays in the next delta by itself.  The
  *              residual buffer is used as scratch and returns v where dropped, +0 where kept.  Delta
  *              mode needs GD_VALUES_FP32.
+ *
+ *   sampled-threshold mode (GD_FLAG_SAMPLED_THRESHOLD; Section 4, fourth paragraph: "We sample 0.1% of
+ *              the gradient and obtain the threshold by running selection on the samples"): per scope,
+ *              m = n_s if n_s <= 4096, else max(4096, ceil(n_s / 1000)) positions are sampled, one in each
+ *              of m equal strata (position of sample i of scope s: a + (h mod (b - a)), a = floor(i n_s / m),
+ *              b = floor((i + 1) n_s / m), h = mix(i * 0x9E3779B9 + s) in 32-bit arithmetic with
+ *              mix(x): x ^= x >> 16; x *= 0x7FEB352D; x ^= x >> 15; x *= 0x846CA68B; x ^= x >> 16);
+ *              the threshold key t is the (m - floor(m * drop_ppm / 1e6))-th largest sample key and EVERY
+ *              entry of the scope with key >= t is kept, so the number of survivors varies: out_idx and
+ *              out_val must hold gd_sampled_capacity() entries, the count is out_shard_cnt_off[n_shards],
+ *              out_tau[s] = t, and a scope with more than min(n_s, 4 k_s + 8192) survivors makes the call
+ *              end with GD_ERR_OVERFLOW in the status word.  Needs GD_VALUES_FP32.
  *
  * Results are bit-exact functions of (grad, residual, offsets, drop_ppm) except the two means,
  * whose fp64 partial sums are combined in an unspecified order.  Non-finite inputs are ordered by
@@ -203,7 +225,8 @@ int gd_get_stats(const void* workspace, void* stream, gd_stats* out);
  * to the device buffer args->grad, runs gd_compress and then gd_decompress_apply (apply may be
  * NULL), and copies the push (indices, values or means, shard offsets) back to the host buffers.
  * Synchronises the stream before returning.  Host buffers should be page-locked for full copy
- * bandwidth.  k_total = gd_total_kept() entries are copied to idx_host / val_host.
+ * bandwidth.  gd_total_kept() entries (gd_sampled_capacity() with GD_FLAG_SAMPLED_THRESHOLD) are copied to
+ * idx_host / val_host.
  */
 typedef struct gd_host_io {
   const float* grad_host;        /* HOST, n fp32 */

@@ -97,6 +97,74 @@ def _kept_in_scope(keys: np.ndarray, k: int, method: str):
     return local, tau
 
 
+def _mix32(x: np.ndarray) -> np.ndarray:
+    """A fixed 32-bit integer mix (the position hash of the sampled-threshold mode), in uint32 arithmetic."""
+    x = x.astype(np.uint32)
+    x = x ^ (x >> np.uint32(16))
+    x = (x * np.uint32(0x7FEB352D)).astype(np.uint32)
+    x = x ^ (x >> np.uint32(15))
+    x = (x * np.uint32(0x846CA68B)).astype(np.uint32)
+    x = x ^ (x >> np.uint32(16))
+    return x
+
+
+def sampled_positions(lo: int, hi: int, scope_index: int) -> np.ndarray:
+    """Positions read by the sampled-threshold mode in scope [lo, hi) (Section 4: "We sample 0.1% of the gradient").
+
+    m = n_s if n_s <= 4096 else max(4096, ceil(n_s / 1000)); the scope is cut into m strata
+    [floor(i n_s / m), floor((i + 1) n_s / m)) and stratum i contributes the position
+    a + (mix32(i * 0x9E3779B9 + scope_index) mod width).  The rule is part of this mode's definition,
+    which is why the CUDA library restates it; nothing else is shared.
+    """
+    ns = hi - lo
+    m = ns if ns <= 4096 else max(4096, -(-ns // 1000))
+    i = np.arange(m, dtype=np.uint64)
+    a = (i * np.uint64(ns)) // np.uint64(max(m, 1))
+    b = ((i + np.uint64(1)) * np.uint64(ns)) // np.uint64(max(m, 1))
+    width = b - a
+    with np.errstate(over="ignore"):
+        h = _mix32((i.astype(np.uint32) * np.uint32(0x9E3779B9) + np.uint32(scope_index)).astype(np.uint32))
+    off = np.where(width > 1, h.astype(np.uint64) % np.maximum(width, np.uint64(1)), np.uint64(0))
+    return (np.uint64(lo) + a + off).astype(np.int64)
+
+
+def compress_sampled(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GLOBAL):
+    """GradDrop with the threshold selected on a sample (Section 4, fourth paragraph).
+
+    Per scope: the threshold key t is the k_m-th largest key among the sampled entries,
+    k_m = m - floor(m * drop_ppm / 1e6), and every entry of the scope with key >= t is kept
+    (nothing if k_m = 0).  The number of survivors therefore varies from call to call.
+    """
+    g = np.ascontiguousarray(grad, dtype=np.float32)
+    r = np.ascontiguousarray(residual, dtype=np.float32)
+    n = g.shape[0]
+    v = g + r
+    keys = magnitude_keys(v)
+    kept_parts, taus = [], []
+    for si, (lo, hi) in enumerate(scopes_of(layer_off, scope_mode)):
+        pos = sampled_positions(lo, hi, si)
+        m = pos.shape[0]
+        k_m = kept_count(m, drop_ppm)
+        if k_m == 0:
+            taus.append(TAU_NONE)
+            continue
+        t = np.sort(keys[pos])[m - k_m]                      # the k_m-th largest sample key
+        taus.append(int(t))
+        kept_parts.append(lo + np.flatnonzero(keys[lo:hi] >= t))
+    kept = np.concatenate(kept_parts).astype(np.int64) if kept_parts else np.empty(0, dtype=np.int64)
+    new_residual = v.copy()
+    new_residual[kept] = np.float32(0.0)
+    return {
+        "idx": kept.astype(np.uint32),
+        "val": v[kept],
+        "residual": new_residual,
+        "tau": np.asarray(taus, dtype=np.uint32),
+        "shard_cnt_off": np.searchsorted(kept, np.asarray([int(x) for x in shard_off], dtype=np.int64),
+                                         side="left").astype(np.uint32),
+        "v": v,
+    }
+
+
 def compress_delta(params, last_pulled, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GLOBAL, method="sort"):
     """GradDrop applied to a parameter pull (Section 4, third paragraph).
 

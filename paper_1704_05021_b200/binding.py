@@ -28,12 +28,14 @@ GD_VALUES_FP32 = 0
 GD_VALUES_TWO_MEANS = 1
 GD_VALUES_THRESHOLD = 2
 GD_FLAG_NO_PREDICTION = 1
+GD_FLAG_SAMPLED_THRESHOLD = 2
+GD_ERR_OVERFLOW = -7
 
 EXPORTS = [
     "gd_status_string", "gd_kept_count", "gd_total_kept", "gd_workspace_bytes", "gd_apply_workspace_bytes",
     "gd_compress", "gd_decompress_apply", "gd_residual_reset", "gd_status", "gd_get_stats", "gd_step_host",
     "gd_profile_enable", "gd_profile_collect", "gd_launch_count", "gd_compress_static",
-    "gd_selftest_bounded_wait",
+    "gd_selftest_bounded_wait", "gd_sampled_capacity",
 ]
 GD_STATIC_WORKSPACE_BYTES = 16 << 20
 
@@ -111,6 +113,7 @@ def load_library():
     lib.gd_step_host.argtypes = [C.POINTER(_CompressArgs), C.POINTER(_ApplyArgs), C.POINTER(_HostIo), C.c_void_p]
     lib.gd_compress_static.argtypes = [C.POINTER(_CompressArgs), C.c_void_p, C.POINTER(C.c_void_p)]
     lib.gd_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_size_t, C.c_uint32, C.c_void_p]
+    lib.gd_sampled_capacity.argtypes = [C.POINTER(C.c_uint64), C.c_uint32, C.c_int, C.c_uint32, C.POINTER(C.c_uint64)]
     lib.gd_profile_enable.argtypes = [C.c_int]
     lib.gd_profile_collect.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_uint32), C.c_uint32, C.POINTER(C.c_uint32)]
     lib.gd_launch_count.argtypes = [C.POINTER(C.c_uint64)]
@@ -256,7 +259,7 @@ def gd_step_host(call: CompressCall, apply: Optional[ApplyCall], grad_host: torc
 
 
 PROFILE_TAGS = ["setup", "sample_select", "add_emit", "dense_select", "dense_compact", "cand_select", "cand_compact",
-                "finalize", "apply"]
+                "finalize", "apply", "pack_sampled"]
 
 
 def gd_profile_enable(mode) -> None:
@@ -300,3 +303,11 @@ def gd_status_at(workspace_address: int, stream=None) -> int:
 def gd_selftest_bounded_wait(workspace: torch.Tensor, spin_limit: int = 2000, stream=None) -> None:
     _check(load_library().gd_selftest_bounded_wait(workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                                    spin_limit, _stream_handle(stream)), "gd_selftest_bounded_wait")
+
+
+def gd_sampled_capacity(layer_off: Sequence[int], scope_mode: int, drop_ppm: int) -> int:
+    out = C.c_uint64(0)
+    arr = _u64_array(layer_off)
+    _check(load_library().gd_sampled_capacity(arr, len(layer_off) - 1, scope_mode, drop_ppm, C.byref(out)),
+           "gd_sampled_capacity")
+    return out.value

@@ -51,6 +51,17 @@ void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint6
   *cap = c < ns ? c : ns;
 }
 
+// Sampled-threshold mode (Section 4): sample size and output capacity of one scope.
+inline uint64_t sampled_m(uint64_t ns) {
+  if (ns <= 4096) return ns;
+  const uint64_t m = (ns + 999) / 1000;
+  return m < 4096 ? 4096 : m;
+}
+inline uint64_t sampled_cap(uint64_t ns, uint64_t k) {
+  const uint64_t c = 4 * k + 8192;
+  return c < ns ? c : ns;
+}
+
 struct Plan {
   std::vector<ScopeDesc> scopes;
   std::vector<uint32_t> tile0[L_COUNT];
@@ -85,6 +96,7 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, i
   if (scope_mode != GD_SCOPE_GLOBAL && scope_mode != GD_SCOPE_PER_LAYER) return GD_ERR_INVALID_ARG;
   if (n > (1ull << 32)) return GD_ERR_TOO_LARGE;
   const bool predict = !(flags & GD_FLAG_NO_PREDICTION);
+  const bool sampled = (flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
   // The fused pass gives each CTA a chunk of 1, 2, 4 or 8 tiles: as large as still leaves about
   // four waves of CTAs (4 per SM on 148 SMs) for the whole vector.
   const uint64_t dense_tiles = (n + kTile - 1) / kTile;
@@ -108,7 +120,13 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, i
     d.out_base = out_base;
     out_base += d.k;
     uint64_t m = 0, rank = 0, cap = 0;
-    if (predict) plan_prediction(ns, d.k, &m, &rank, &cap);
+    if (sampled) {
+      m = sampled_m(ns);
+      rank = kept_count(m, drop_ppm);
+      cap = sampled_cap(ns, d.k);
+    } else if (predict) {
+      plan_prediction(ns, d.k, &m, &rank, &cap);
+    }
     d.cand_base = cand_base;
     d.cand_cap = cap;
     cand_base += (cap + 3) / 4 * 4;
@@ -257,6 +275,7 @@ const char* gd_status_string(int status) {
     case GD_ERR_CUDA: return "CUDA runtime error";
     case GD_ERR_DEVICE_TIMEOUT: return "bounded device-side wait timed out";
     case GD_ERR_INTERNAL: return "device-side consistency check failed";
+    case GD_ERR_OVERFLOW: return "more survivors than the sampled-threshold capacity";
     default: return "unknown status";
   }
 }
@@ -286,14 +305,30 @@ int gd_total_kept(const uint64_t* layer_off, uint32_t n_layers, int scope_mode, 
   return GD_OK;
 }
 
+int gd_sampled_capacity(const uint64_t* layer_off, uint32_t n_layers, int scope_mode, uint32_t drop_ppm,
+                        uint64_t* capacity_out) {
+  if (!capacity_out) return GD_ERR_INVALID_ARG;
+  try {
+    Plan P;
+    int rc = make_plan(layer_off, n_layers, 1, scope_mode, drop_ppm, GD_FLAG_SAMPLED_THRESHOLD, &P);
+    if (rc != GD_OK) return rc;
+    *capacity_out = P.cand_total;
+    return GD_OK;
+  } catch (const std::bad_alloc&) {
+    return GD_ERR_INVALID_ARG;
+  }
+}
+
 int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, int scope_mode,
                        uint32_t drop_ppm, size_t* bytes_out) {
   if (!bytes_out) return GD_ERR_INVALID_ARG;
   try {
-    Plan P;
+    Plan P, Q;
     int rc = make_plan(layer_off, n_layers, n_shards, scope_mode, drop_ppm, 0u, &P);
     if (rc != GD_OK) return rc;
-    *bytes_out = P.total_bytes;
+    rc = make_plan(layer_off, n_layers, n_shards, scope_mode, drop_ppm, GD_FLAG_SAMPLED_THRESHOLD, &Q);
+    if (rc != GD_OK) return rc;
+    *bytes_out = P.total_bytes > Q.total_bytes ? P.total_bytes : Q.total_bytes;   // whichever mode is used
     return GD_OK;
   } catch (const std::bad_alloc&) {
     return GD_ERR_INVALID_ARG;
@@ -314,12 +349,14 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     if (n_sh != n || a->n != n) return GD_ERR_INVALID_ARG;
     if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_THRESHOLD) return GD_ERR_INVALID_ARG;
     if (a->value_mode != GD_VALUES_FP32 && n > (1ull << 31)) return GD_ERR_TOO_LARGE;
-    if (a->flags & ~(uint32_t)GD_FLAG_NO_PREDICTION) return GD_ERR_INVALID_ARG;
+    if (a->flags & ~(uint32_t)(GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD)) return GD_ERR_INVALID_ARG;
+    const bool sampled = (a->flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
+    if (sampled && ((a->flags & GD_FLAG_NO_PREDICTION) || a->value_mode != GD_VALUES_FP32)) return GD_ERR_INVALID_ARG;
     if (n && (!a->grad || !a->residual)) return GD_ERR_INVALID_ARG;
     if (((uintptr_t)a->grad | (uintptr_t)a->residual) & 15u) return GD_ERR_INVALID_ARG;
     if (a->delta_base && (a->value_mode != GD_VALUES_FP32 || ((uintptr_t)a->delta_base & 15u))) return GD_ERR_INVALID_ARG;
     if (!a->out_shard_cnt_off) return GD_ERR_INVALID_ARG;
-    if (P.k_total && !a->out_idx) return GD_ERR_INVALID_ARG;
+    if ((P.k_total || (sampled && P.cand_total)) && !a->out_idx) return GD_ERR_INVALID_ARG;
     if (P.k_total && a->value_mode == GD_VALUES_FP32 && !a->out_val) return GD_ERR_INVALID_ARG;
     if (a->value_mode != GD_VALUES_FP32 && !a->out_means) return GD_ERR_INVALID_ARG;
     if (!a->workspace || ((uintptr_t)a->workspace & (kAlign - 1))) return GD_ERR_WORKSPACE;
@@ -351,6 +388,8 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     T.value_mode = a->value_mode;
     T.k_total = P.k_total;
     T.emit_chunk_tiles = P.emit_chunk_tiles;
+    T.sample_passes = sampled ? 3u : 2u;
+    if (sampled) T.k_total = P.cand_total;   // capacity of the outputs; the count is found on the device
     T.ctl = (Ctl*)(ws + P.off_ctl);
     T.state = (ScopeState*)(ws + P.off_state);
     T.hist = (unsigned long long*)(ws + P.off_hist);
@@ -376,6 +415,12 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
 
     uint32_t tiles[L_COUNT];
     for (int l = 0; l < L_COUNT; ++l) tiles[l] = P.tiles[l];
+    if (sampled) {
+      if (launch_sample_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+      if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+      if (launch_pack_sampled(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+      return GD_OK;
+    }
     const bool predict = !(a->flags & GD_FLAG_NO_PREDICTION);
     if (predict && launch_sample_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
     if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
@@ -493,7 +538,9 @@ int gd_step_host(const gd_compress_args* a, const gd_apply_args* apply, const gd
   if (!a || !io || !io->grad_host) return GD_ERR_INVALID_ARG;
   cudaStream_t stream = (cudaStream_t)stream_v;
   uint64_t k_total = 0;
-  int rc = gd_total_kept(a->layer_off, a->n_layers, a->scope_mode, a->drop_ppm, &k_total);
+  int rc = (a->flags & GD_FLAG_SAMPLED_THRESHOLD)
+               ? gd_sampled_capacity(a->layer_off, a->n_layers, a->scope_mode, a->drop_ppm, &k_total)
+               : gd_total_kept(a->layer_off, a->n_layers, a->scope_mode, a->drop_ppm, &k_total);
   if (rc != GD_OK) return rc;
   if (a->n && cudaMemcpyAsync((void*)a->grad, io->grad_host, sizeof(float) * a->n, cudaMemcpyHostToDevice, stream) !=
                   cudaSuccess)

@@ -10,7 +10,7 @@ namespace {
 // Finishes a call: thresholds, statistics, shard offsets (Section 3: the survivors, ascending in
 // index, are cut into one piece per server) and the two means (Section 5.4).  Run by one whole CTA
 // after every survivor has been written.
-__device__ void finalize_call(const DevTables& T) {
+__device__ void finalize_call(const DevTables& T, uint64_t k_total) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
   const bool packed = T.value_mode != GD_VALUES_FP32;
@@ -26,11 +26,11 @@ __device__ void finalize_call(const DevTables& T) {
   if (n_pred) atomicAdd(&T.ctl->n_scopes_predicted, n_pred);
   if (n_dense) atomicAdd(&T.ctl->n_scopes_dense, n_dense);
   if (n_cand) atomicAdd(reinterpret_cast<unsigned long long*>(&T.ctl->n_candidates), n_cand);
-  if (tid == 0) { T.ctl->n_scopes = T.n_scopes; T.ctl->n_kept = T.k_total; }
+  if (tid == 0) { T.ctl->n_scopes = T.n_scopes; T.ctl->n_kept = k_total; }
   // shard j starts at the first survivor with index >= shard_off[j]: a 33-way search per warp
   for (uint32_t j = warp; j <= T.n_shards; j += kWarps) {
     const uint64_t bound = T.shard_off[j];
-    uint64_t lo = 0, hi = T.k_total;                 // answer in [lo, hi]
+    uint64_t lo = 0, hi = k_total;                   // answer in [lo, hi]
     while (hi - lo > 32) {
       const uint64_t span = hi - lo;
       const uint64_t p = lo + span * (lane + 1) / 33;   // lo < p < hi, ascending in lane
@@ -68,7 +68,7 @@ __device__ void finalize_call(const DevTables& T) {
   }
 }
 
-__global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constant__ DevTables T) { finalize_call(T); }
+__global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constant__ DevTables T) { finalize_call(T, T.k_total); }
 
 // Single-pass look-back scan with two counters per tile: keys above tau, and keys equal to tau.  An
 // element above tau goes to slot  (#above before it) + min(#ties before it, q); a tie is kept iff fewer
@@ -255,7 +255,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  finalize_call(T);
+  finalize_call(T, T.k_total);
 }
 
 // Compaction over the dense range itself, for scopes whose prediction failed.  Same placement rule
@@ -455,7 +455,76 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  finalize_call(T);
+  finalize_call(T, T.k_total);
+}
+
+// Sampled-threshold mode: the candidate lists ARE the survivors.  Copies every scope's list to its
+// place in the output (scopes concatenated in index order), clears the survivors' residual slots,
+// and lets the last CTA finish the call with the survivor count found here.
+__global__ void __launch_bounds__(kThreads) pack_sampled_kernel(const __grid_constant__ DevTables T) {
+  __shared__ unsigned long long s_part[kWarps];
+  __shared__ unsigned long long s_off;
+  __shared__ int s_last;
+  __shared__ SmemTables s_tab;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const ScopeDesc* scopes;
+  const uint32_t* tile0;
+  load_tables(T, L_CAND, &s_tab, &scopes, &tile0);
+  __syncthreads();
+  const uint32_t t = blockIdx.x;
+  const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
+  const ScopeDesc& d = scopes[s];
+  // survivors of the scopes before s (and, for the last CTA, of all scopes)
+  auto count_before = [&](uint32_t upto) -> unsigned long long {
+    unsigned long long part = 0;
+    for (uint32_t x = tid; x < upto; x += kThreads) {
+      const unsigned long long m = T.state[x].cand_count, c = scopes[x].cand_cap;
+      part += m < c ? m : c;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+    __syncthreads();
+    if (lane == 0) s_part[warp] = part;
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long tot = 0;
+      for (int w = 0; w < kWarps; ++w) tot += s_part[w];
+      s_off = tot;
+    }
+    __syncthreads();
+    return s_off;
+  };
+  const unsigned long long m_all = T.state[s].cand_count;
+  const uint64_t m = m_all < d.cand_cap ? m_all : d.cand_cap;
+  const uint64_t beg = (uint64_t)(t - tile0[s]) * kTile;
+  if (beg < m) {
+    const uint64_t out_off = count_before(s);
+    const uint64_t end = (beg + kTile < m) ? beg + kTile : m;
+    uint32_t ib[16], vb[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const uint64_t i = beg + (uint64_t)j * kThreads + tid;
+      ib[j] = i < end ? T.cand_idx[d.cand_base + i] : 0u;
+      vb[j] = i < end ? __float_as_uint(T.cand_val[d.cand_base + i]) : 0u;
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const uint64_t i = beg + (uint64_t)j * kThreads + tid;
+      if (i < end && ib[j] < T.n && out_off + i < T.k_total) {
+        T.out_idx[out_off + i] = ib[j];
+        T.out_val[out_off + i] = __uint_as_float(vb[j]);
+        T.residual[ib[j]] = 0.0f;
+        if (T.delta_base) T.delta_base[ib[j]] = __fadd_rn(T.delta_base[ib[j]], __uint_as_float(vb[j]));
+      }
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&T.ctl->compact_done[0], 1u) == gridDim.x - 1u) ? 1 : 0;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  finalize_call(T, count_before(T.n_scopes));
 }
 
 // Self-test kernel of the bounded waits: tile 1 waits on tile 0, which nothing publishes; tile 2
@@ -483,6 +552,14 @@ cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, c
 cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream) {
   ProfileScope prof(stream, PT_FINALIZE);
   finalize_kernel<<<1, kThreads, 0, stream>>>(T);
+  GD_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+
+cudaError_t launch_pack_sampled(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
+  if (!tiles[L_CAND]) return launch_finalize(T, stream);   // nothing can survive: finish with count 0
+  ProfileScope prof(stream, PT_PACK_SAMPLED);
+  pack_sampled_kernel<<<tiles[L_CAND], kThreads, 0, stream>>>(T);
   GD_LAUNCH_CHECK();
   return cudaSuccess;
 }

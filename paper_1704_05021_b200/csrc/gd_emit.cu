@@ -60,7 +60,8 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
   // there are fewer than k of them the threshold is 0 and the zeros that are kept are found by the
   // dense compaction alone (no dense selection is needed to know tau = 0).
   uint32_t tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || d.k == 0) ? 0xFFFFFFFFu : T.state[s].tau_lo;
-  if (tau_lo == 0u) tau_lo = 1u;
+  const bool sampled = (T.flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;   // tau_lo is the threshold itself: keep key >= tau_lo
+  if (tau_lo == 0u && !sampled) tau_lo = 1u;
   const uint64_t toff = (uint64_t)warp * 512u + lane * 4u;   // this thread's first element inside a tile
   const uint32_t ltm = lanemask_lt();
   StashEntry* stash = s_stash[warp];
@@ -230,7 +231,11 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
   if (tid == 0 && lt == nchunks - 1) {
     const uint64_t m = excl + s_total;
     T.state[s].cand_count = m;
-    if (!(T.flags & GD_FLAG_NO_PREDICTION) && (m < d.k || m > d.cand_cap)) atomicAdd(&T.ctl->dense_needed, 1u);
+    if (sampled) {
+      if (m > d.cand_cap) atomicCAS(&T.ctl->status, (int)GD_OK, (int)GD_ERR_OVERFLOW);
+    } else if (!(T.flags & GD_FLAG_NO_PREDICTION) && (m < d.k || m > d.cand_cap)) {
+      atomicAdd(&T.ctl->dense_needed, 1u);
+    }
   }
 }
 

@@ -17,7 +17,7 @@ constexpr uint32_t kDenseChunkTiles = 32;  // tiles per ticket (and per look-bac
 constexpr int kRadixBits0 = 11;         // 31-bit magnitude key = 11 + 10 + 10 bits
 constexpr int kRadixBins0 = 1 << kRadixBits0;
 constexpr int kShift0 = 20, kShift1 = 10, kShift2 = 0;
-constexpr uint32_t kHistBinsPerScope = 2048 + 1024 + 2048 + 1024 + 1024;   // sample: 2 passes; selection: 3
+constexpr uint32_t kHistBinsPerScope = 2 * (2048 + 1024 + 1024);   // three passes over the sample, three over the list
 constexpr uint32_t kAbsMask = 0x7FFFFFFFu;
 constexpr uint32_t kLookbackSpinLimit = 1u << 21;  // polls before a look-back wait gives up
 
@@ -88,6 +88,8 @@ struct DevTables {       // passed by value to every kernel
   uint32_t flags;
   int32_t value_mode;
   uint32_t emit_chunk_tiles;         // tiles of kTile elements one CTA of the fused pass streams (1, 2, 4 or 8)
+  uint32_t sample_passes;            // radix passes over the sample: 2 (prediction, 21 bits) or 3 (sampled-threshold mode)
+  uint32_t pad1;
   uint64_t k_total;
   // zeroed region
   Ctl* ctl;
@@ -199,13 +201,14 @@ cudaError_t launch_candidate_select(const DevTables& T, const uint32_t* tiles, c
 cudaError_t launch_dense_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, bool finalize, cudaStream_t stream);
 cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream);
+cudaError_t launch_pack_sampled(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream);
 int sm_count();   // multiprocessors of the current device (0 on error)
 
 // Measurement hooks (gd_api.cu): count a kernel launch; record an event of the pair around the fused pass.
 void note_launches(uint32_t count);
 // Kernel tags of the measurement hooks, in the order a step launches them.
-enum ProfileTag : uint32_t { PT_SETUP = 0, PT_SAMPLE_SELECT = 1, PT_ADD_EMIT = 2, PT_DENSE_SELECT = 3, PT_DENSE_COMPACT = 4,
+enum ProfileTag : uint32_t { PT_SETUP = 0, PT_PACK_SAMPLED = 9, PT_SAMPLE_SELECT = 1, PT_ADD_EMIT = 2, PT_DENSE_SELECT = 3, PT_DENSE_COMPACT = 4,
                              PT_CAND_SELECT = 5, PT_CAND_COMPACT = 6, PT_FINALIZE = 7, PT_APPLY = 8 };
 void profile_mark(cudaStream_t stream, bool begin, uint32_t tag);
 struct ProfileScope {   // records an event pair around the launches made during its lifetime

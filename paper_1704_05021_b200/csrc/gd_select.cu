@@ -74,12 +74,12 @@ struct SelRun {
   uint64_t rank, gt;
 };
 
-// Histograms of one scope: the sample's two passes, then the three passes of the candidate (or
-// dense) selection.  Each is filled once per call and never cleared inside a call.
+// Histograms of one scope: up to three passes over the sample, then the three passes of the candidate
+// (or dense) selection.  Each is filled once per call and never cleared inside a call.
 __device__ __forceinline__ unsigned long long* hist_of(const DevTables& T, uint32_t s, int view, int pass) {
   unsigned long long* base = T.hist + (size_t)s * kHistBinsPerScope;
-  if (view == V_SAMPLE) return base + (pass == 0 ? 0 : 2048);
-  return base + (pass == 0 ? 3072 : (pass == 1 ? 5120 : 6144));
+  const uint32_t off = pass == 0 ? 0u : (pass == 1 ? 2048u : 3072u);   // 2048 + 1024 + 1024 bins
+  return base + (view == V_SAMPLE ? 0u : 4096u) + off;
 }
 
 // Run by a whole CTA after the grid barrier that completes histogram `gh`: walks it from the top
@@ -152,7 +152,7 @@ template <int VIEW>
 __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
   constexpr int LK = VIEW == V_SAMPLE ? L_SAMP : (VIEW == V_CAND ? L_CAND : L_DSEL);
   constexpr uint32_t TILE = VIEW == V_DENSE ? kDenseSelTile : kTile;
-  constexpr int PASSES = VIEW == V_SAMPLE ? 2 : 3;   // the prediction needs 21 bits only
+  const int PASSES = VIEW == V_SAMPLE ? (int)T.sample_passes : 3;   // the prediction needs 21 bits only
   constexpr uint32_t NONE = 0xFFFFFFFFu;
   __shared__ uint32_t sh[kRadixBins0];
   __shared__ SmemTables s_tab;
@@ -215,7 +215,9 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
         if (pass == PASSES && tid == 0) {               // the CTA with the scope's first tile records the result
           ScopeState* st = T.state + s;
           if (VIEW == V_SAMPLE) {
-            st->tau_lo = run.prefix << kShift1;         // lower edge of the 21-bit bucket
+            // prediction: lower edge of the 21-bit bucket; sampled-threshold mode: the full key, which is the result
+            st->tau_lo = PASSES == 3 ? run.prefix : run.prefix << kShift1;
+            if (PASSES == 3) st->tau = run.prefix;
           } else {
             st->tau = run.prefix; st->q = run.rank; st->gt = run.gt;
             if (VIEW == V_DENSE) st->used_dense = 1u;

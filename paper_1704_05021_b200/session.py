@@ -28,7 +28,10 @@ class GradDropSession:
         self.n_shards = len(self.shard_off) - 1
         self.drop_ppm, self.scope_mode, self.value_mode, self.flags = drop_ppm, scope_mode, value_mode, flags
         self.n_scopes = 1 if scope_mode == B.GD_SCOPE_GLOBAL else self.n_layers
-        self.k_total = B.gd_total_kept(self.layer_off, scope_mode, drop_ppm)
+        self.sampled = bool(flags & B.GD_FLAG_SAMPLED_THRESHOLD)
+        # exact modes: the survivor count is known; sampled-threshold mode: the capacity of the outputs
+        self.k_total = (B.gd_sampled_capacity(self.layer_off, scope_mode, drop_ppm) if self.sampled
+                        else B.gd_total_kept(self.layer_off, scope_mode, drop_ppm))
         dev = self.device
         self.residual = torch.empty(self.n, dtype=torch.float32, device=dev)
         self.out_idx = torch.zeros(max(self.k_total, 1), dtype=torch.int32, device=dev)
@@ -90,6 +93,10 @@ class GradDropSession:
 
     def shard_views(self, flat_params: torch.Tensor) -> List[torch.Tensor]:
         return [flat_params[self.shard_off[j]:self.shard_off[j + 1]] for j in range(self.n_shards)]
+
+    def kept(self) -> int:
+        """Survivors of the last compress call (a device read in sampled-threshold mode)."""
+        return int(self.out_shard_cnt_off[-1].item()) if self.sampled else self.k_total
 
     def status(self) -> int:
         return B.gd_status(self.workspace)

@@ -411,3 +411,67 @@ def test_delta_pull_matches_oracle_and_client_copy(cuda_device, flags):
         torch.cuda.synchronize()
         assert torch.equal(client.view(torch.int32), last_dev.view(torch.int32)), f"pull {step}: client copy differs"
         last_host = exp["last_pulled"]
+
+
+# ---------------------------------------------------------------- sampled threshold (Section 4: select on a 0.1 % sample)
+def compare_sampled(sess, exp, tag):
+    assert sess.status() == B.GD_OK, f"{tag}: device status {sess.status()}"
+    K = exp["idx"].shape[0]
+    assert sess.kept() == K, f"{tag}: kept {sess.kept()} vs {K}"
+    assert K <= sess.k_total
+    assert np.array_equal(_np_u32(sess.out_tau), exp["tau"]), f"{tag}: thresholds"
+    assert np.array_equal(_np_u32(sess.out_idx)[:K], exp["idx"]), f"{tag}: indices"
+    assert np.array_equal(_np_u32(sess.out_val)[:K], exp["val"].view(np.uint32)), f"{tag}: values"
+    assert np.array_equal(_np_u32(sess.residual), exp["residual"].view(np.uint32)), f"{tag}: residual"
+    assert np.array_equal(_np_u32(sess.out_shard_cnt_off), exp["shard_cnt_off"]), f"{tag}: shard offsets"
+
+
+@pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
+def test_sampled_threshold_matches_oracle(cuda_device, scope_mode):
+    rng = np.random.default_rng(61)
+    sizes = [3000, 0, 4096, 4097, 10, 700_001, 64_000]           # whole-scope samples, 4096-sample scopes, a 0.1 % scope
+    for ppm in (990_000, 900_000, 1_000_000):
+        w = W.small_layered(len(sizes), sizes, ppm, scope_mode, B.GD_VALUES_FP32, 3)
+        sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
+                               B.GD_FLAG_SAMPLED_THRESHOLD, cuda_device)
+        params = torch.zeros(w.n, dtype=torch.float32, device=cuda_device)
+        views = sess.shard_views(params)
+        r_host = orc.residual_reset(w.n)
+        sent = np.zeros(w.n, np.float32)
+        for step in range(3):
+            g = rng.laplace(0, 1e-3, w.n).astype(np.float32)
+            g[rng.random(w.n) < 0.2] = 0.0
+            exp = orc.compress_sampled(g, r_host, w.layer_off, w.shard_off, ppm, scope_mode)
+            sess.compress(torch.from_numpy(g).to(cuda_device))
+            compare_sampled(sess, exp, f"sampled ppm {ppm} step {step}")
+            sess.apply(views)
+            sent[exp["idx"]] += exp["val"]
+            r_host = exp["residual"]
+        torch.cuda.synchronize()
+        assert np.array_equal(_np_u32(params), sent.view(np.uint32))
+
+
+def test_sampled_threshold_on_workload_shapes(cuda_device):
+    for cfg, scale in ((2, None), (5, 24)):
+        w = W.workload(cfg, scale_log2=scale) if scale else W.workload(cfg, scope_mode=B.GD_SCOPE_PER_LAYER)
+        sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
+                               B.GD_FLAG_SAMPLED_THRESHOLD, cuda_device)
+        r_host = orc.residual_reset(w.n)
+        for step in range(2):
+            g = W.make_gradient(w, step, cuda_device)
+            exp = orc.compress_sampled(g.cpu().numpy(), r_host, w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode)
+            sess.compress(g)
+            compare_sampled(sess, exp, f"sampled workload {cfg} step {step}")
+            r_host = exp["residual"]
+            k_exact = B.gd_total_kept(w.layer_off, w.scope_mode, w.drop_ppm)
+            assert 0.5 * k_exact < sess.kept() < 2.0 * k_exact       # about the requested fraction
+
+
+def test_sampled_threshold_overflow_is_reported(cuda_device):
+    n = 1_000_000                                                   # every entry ties with the threshold: all are kept
+    w = W.small_layered(1, [n], 990_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 1)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
+                           B.GD_FLAG_SAMPLED_THRESHOLD, cuda_device)
+    sess.compress(torch.full((n,), 0.25, device=cuda_device))
+    assert sess.status() == B.GD_ERR_OVERFLOW
+    run_steps(W.workload(1), cuda_device, 1)                        # the context is fine afterwards

@@ -423,3 +423,65 @@ def test_delta_pull_by_hand_and_invariants():
         assert np.array_equal(p - last, out["residual"])           # nothing lost: the rest is the next delta
     out = orc.compress_delta(p, last, layer_off, shard_off, 0)     # R = 0: the client catches up completely
     assert np.array_equal(out["last_pulled"], p)
+
+
+# ---------------------------------------------------------------- sampled threshold (Section 4)
+def _mix32_py(x):
+    x &= 0xFFFFFFFF
+    x ^= x >> 16
+    x = (x * 0x7FEB352D) & 0xFFFFFFFF
+    x ^= x >> 15
+    x = (x * 0x846CA68B) & 0xFFFFFFFF
+    x ^= x >> 16
+    return x
+
+
+def test_sampled_positions_are_one_per_stratum():
+    for lo, hi, si in ((0, 10, 0), (5, 4101, 3), (100, 100 + 4097, 1), (0, 5_000_000, 7), (17, 17 + 123_457, 2)):
+        ns = hi - lo
+        pos = orc.sampled_positions(lo, hi, si)
+        m = ns if ns <= 4096 else max(4096, -(-ns // 1000))
+        assert pos.shape[0] == m
+        for i in (0, 1, m // 2, m - 1):                         # pure-Python restatement on a few strata
+            a, b = (i * ns) // m, ((i + 1) * ns) // m
+            want = lo + a + (_mix32_py(i * 0x9E3779B9 + si) % (b - a) if b - a > 1 else 0)
+            assert int(pos[i]) == want
+        assert np.all(np.diff(pos) > 0) and pos[0] >= lo and pos[-1] < hi      # distinct, ordered, in range
+    assert orc.sampled_positions(3, 3 + 4096, 0).tolist() == list(range(3, 3 + 4096))   # small scopes: everything
+
+
+def test_sampled_threshold_small_scope_is_exact_selection_with_all_ties():
+    rng = np.random.default_rng(41)
+    n = 3000                                                   # <= 4096: the sample is the whole scope
+    g = rng.choice(np.array([0.0, 0.5, -0.5, 1.0, -2.0, 3.0], np.float32), n)
+    r = np.full(n, -0.0, np.float32)
+    for ppm in (500_000, 900_000, 990_000, 1_000_000, 0):
+        out = orc.compress_sampled(g, r, [0, n], [0, n // 2, n], ppm)
+        exact = orc.compress(g, r, [0, n], [0, n // 2, n], ppm)
+        assert int(out["tau"][0]) == int(exact["tau"][0])
+        if ppm == 1_000_000:
+            assert out["idx"].size == 0
+            continue
+        keys = g.view(np.uint32) & np.uint32(0x7FFFFFFF)
+        want = np.flatnonzero(keys >= out["tau"][0])           # the exact set plus every tie at tau
+        assert np.array_equal(out["idx"].astype(np.int64), want)
+        assert set(exact["idx"].tolist()) <= set(out["idx"].tolist())
+        assert out["shard_cnt_off"].tolist() == [0, int((want < n // 2).sum()), want.size]
+
+
+def test_sampled_threshold_keeps_about_the_requested_fraction():
+    rng = np.random.default_rng(43)
+    n = 4_000_000
+    g = rng.laplace(0, 1e-3, n).astype(np.float32)
+    r = np.zeros(n, np.float32)
+    out = orc.compress_sampled(g, r, [0, n], [0, n], 990_000)
+    m = 4096                                                   # ceil(n / 1000) = 4000 < 4096
+    pos = orc.sampled_positions(0, n, 0)
+    assert pos.shape[0] == m
+    k_m = m - (m * 990_000) // 1_000_000
+    t = sorted((f32_bits(x) & 0x7FFFFFFF for x in g[pos]), reverse=True)[k_m - 1]
+    assert int(out["tau"][0]) == t
+    frac = out["idx"].size / n
+    assert abs(frac - 0.01) < 6 * 0.01 / math.sqrt(k_m)        # sampling error of a quantile from k_m tail samples
+    assert np.array_equal(out["val"], g[out["idx"]])
+    assert not out["residual"][out["idx"]].any()
