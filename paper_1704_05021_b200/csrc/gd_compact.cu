@@ -70,14 +70,13 @@ __device__ void finalize_call(const DevTables& T, uint64_t k_total) {
 
 __global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constant__ DevTables T) { finalize_call(T, T.k_total); }
 
-// Single-pass look-back scan with two counters per tile: keys above tau, and keys equal to tau.  An
-// element above tau goes to slot  (#above before it) + min(#ties before it, q); a tie is kept iff fewer
-// than q ties precede it.  VIEW == V_CAND walks the candidate list, V_DENSE the dense range itself.
-// CTAs take tiles from an atomic ticket until none is left.
-template <int VIEW>
+// Compaction over the candidate list: a single-pass look-back scan with two counters per tile, keys
+// above tau and keys equal to tau.  An element above tau goes to slot  (#above before it) +
+// min(#ties before it, q); a tie is kept iff fewer than q ties precede it.  CTAs take tiles from an
+// atomic ticket until none is left; the last CTA to leave finishes the call.
 __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles,
                                                            int do_finalize) {
-  constexpr int LK = VIEW == V_CAND ? L_CAND : L_DCOMP;
+  constexpr int LK = L_CAND;
   constexpr int ROUNDS = kTile / kThreads;   // 16 elements per thread
   __shared__ uint32_t s_tile;
   __shared__ uint32_t s_wg[kWarps], s_we[kWarps];
@@ -88,7 +87,6 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   __shared__ uint32_t s_redc[kWarps][2];
   __shared__ int s_last;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-  if (VIEW == V_DENSE && !(T.flags & GD_FLAG_NO_PREDICTION) && T.ctl->dense_needed == 0u) return;
   __shared__ SmemTables s_tab;
   const ScopeDesc* scopes;
   const uint32_t* tile0;
@@ -96,7 +94,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
   const bool packed = T.value_mode != GD_VALUES_FP32;
   const uint32_t ltm = lanemask_lt();
-  uint4* desc = reinterpret_cast<uint4*>(VIEW == V_CAND ? T.desc_cand : T.desc_dcomp);
+  uint4* desc = reinterpret_cast<uint4*>(T.desc_cand);
 
   for (;;) {
     __syncthreads();                       // previous tile is done with the shared variables
@@ -107,27 +105,20 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
     const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
     const ScopeDesc& d = scopes[s];
     const ScopeState* st = T.state + s;
-    const bool pred = predicted_ok(T, d, *st);
-    if (VIEW == V_CAND ? !pred : pred) continue;    // the other view owns this scope
+    if (!predicted_ok(T, d, *st)) continue;         // the dense kernels own this scope
     const uint32_t first = tile0[s];
     const uint32_t lt = t - first;
-    const uint64_t len = VIEW == V_CAND ? st->cand_count : d.hi - d.lo;
+    const uint64_t len = st->cand_count;
     const uint64_t beg = (uint64_t)lt * kTile;
     if (beg >= len) continue;                       // trailing tiles of a short candidate list
     const uint64_t end = (beg + kTile < len) ? beg + kTile : len;
-    const float* vals = VIEW == V_CAND ? T.cand_val + d.cand_base : T.residual + d.lo;
+    const float* vals = T.cand_val + d.cand_base;
     const uint32_t tau = st->tau;
     const uint64_t q = st->q;
 
     if (two_means && tid == 0) {
-      uint64_t i_first, i_last;
-      if (VIEW == V_CAND) {
-        i_first = T.cand_idx[d.cand_base + beg];
-        i_last = T.cand_idx[d.cand_base + end - 1];
-      } else {
-        i_first = d.lo + beg;
-        i_last = d.lo + end - 1;
-      }
+      const uint64_t i_first = T.cand_idx[d.cand_base + beg];
+      const uint64_t i_last = T.cand_idx[d.cand_base + end - 1];
       const uint32_t l0 = range_of(T.layer_off, T.n_layers, i_first);
       const uint32_t l1 = range_of(T.layer_off, T.n_layers, i_last);
       s_layer = l0;
@@ -141,7 +132,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
 #pragma unroll
     for (int j = 0; j < ROUNDS; ++j) {   // the candidates' indices travel with their values: loaded up front
       const uint64_t i = wbeg + (uint64_t)j * 32u;
-      ib[j] = (VIEW == V_CAND && i < end) ? T.cand_idx[d.cand_base + i] : 0u;
+      ib[j] = i < end ? T.cand_idx[d.cand_base + i] : 0u;
     }
 #pragma unroll
     for (int j = 0; j < ROUNDS; ++j) {
@@ -194,8 +185,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
         const uint64_t gb = rg + __popc(mg & ltm), eb = re + __popc(me & ltm);
         if (isgt || eb < q) {
           const uint64_t pos = gb + (eb < q ? eb : q);
-          const uint64_t i = wbeg + (uint64_t)j * 32u;
-          const uint64_t idx = VIEW == V_CAND ? (uint64_t)ib[j] : d.lo + i;
+          const uint64_t idx = ib[j];
           if (pos < d.k && idx < T.n) {
             const uint32_t b = vb[j];
             T.residual[idx] = 0.0f;
@@ -251,7 +241,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   // the last CTA to leave finishes the call
   __threadfence();
   __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(&T.ctl->compact_done[VIEW == V_CAND ? 0 : 1], 1u) == gridDim.x - 1u) ? 1 : 0;
+  if (tid == 0) s_last = (atomicAdd(&T.ctl->compact_done[0], 1u) == gridDim.x - 1u) ? 1 : 0;
   __syncthreads();
   if (!s_last) return;
   __threadfence();
@@ -573,7 +563,7 @@ cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense
   if (dense)
     compact_dense_kernel<<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
   else
-    compact_kernel<V_CAND><<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
+    compact_kernel<<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
   GD_LAUNCH_CHECK();
   return cudaSuccess;
 }

@@ -475,3 +475,57 @@ def test_sampled_threshold_overflow_is_reported(cuda_device):
     sess.compress(torch.full((n,), 0.25, device=cuda_device))
     assert sess.status() == B.GD_ERR_OVERFLOW
     run_steps(W.workload(1), cuda_device, 1)                        # the context is fine afterwards
+
+
+# ---------------------------------------------------------------- beyond 2^31 elements (64-bit offsets, full uint32 indices)
+def test_more_than_2_31_elements(cuda_device):
+    """n = 2^31 + 2^20 + 5: byte offsets pass 2^33 and indices pass 2^31.  The oracle's sort does not fit here, so
+    the result is pinned by what defines it: tau is the k-th largest key iff #{key > tau} < k <= #{key >= tau};
+    the kept set is every key above tau plus the lowest-index ties; values and residual reassemble v."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 * (1 << 30):
+        pytest.skip("needs 60 GiB of free device memory")
+    n = (1 << 31) + (1 << 20) + 5
+    w = W.small_layered(1, [n], 999_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 3)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
+    gen = torch.Generator(device=cuda_device).manual_seed(2031)
+    g = torch.empty(n, dtype=torch.float32, device=cuda_device)
+    chunk = 1 << 26
+    for lo in range(0, n, chunk):
+        hi = min(lo + chunk, n)
+        g[lo:hi] = torch.randn(hi - lo, generator=gen, device=cuda_device) * 1e-3
+    g[n - 3:] = torch.tensor([5.0, -6.0, 7.0], device=cuda_device)          # the very last entries must be kept
+    g[(1 << 31) - 1] = -8.0
+    g[1 << 31] = 9.0
+    k = sess.k_total
+    for step in range(2):
+        r_before = sess.residual.clone()
+        sess.compress(g)
+        assert sess.status() == B.GD_OK
+        assert sess.stats()["n_scopes_dense"] == 0
+        tau = int(_np_u32(sess.out_tau)[0])
+        idx = sess.out_idx[:k].to(torch.int64) & 0xFFFFFFFF
+        assert bool((idx[1:] > idx[:-1]).all()) and int(idx[-1]) == n - 1
+        n_gt = n_eq = 0
+        kept_mask_count = 0
+        for lo in range(0, n, chunk):                                      # chunked: no tensor larger than 2^26 here
+            hi = min(lo + chunk, n)
+            v = g[lo:hi] + r_before[lo:hi]
+            keys = v.view(torch.int32) & 0x7FFFFFFF
+            n_gt += int((keys > tau).sum())
+            n_eq += int((keys == tau).sum())
+            sel = idx[(idx >= lo) & (idx < hi)] - lo
+            kept = torch.zeros(hi - lo, dtype=torch.bool, device=cuda_device)
+            kept[sel] = True
+            kept_mask_count += int(kept.sum())
+            assert bool((keys[kept] >= tau).all()) and bool((keys[~kept] <= tau).all())
+            want_res = torch.where(kept, torch.zeros_like(v), v)
+            assert torch.equal(sess.residual[lo:hi].view(torch.int32), want_res.view(torch.int32))
+        assert n_gt < k <= n_gt + n_eq and kept_mask_count == k
+        v_kept = g[idx] + r_before[idx]
+        assert torch.equal(sess.out_val[:k].view(torch.int32), v_kept.view(torch.int32))
+        for probe in ((1 << 31) - 1, 1 << 31, n - 3, n - 2, n - 1):
+            assert bool((idx == probe).any())                              # the planted large entries, both sides of 2^31
+        bounds = torch.tensor(w.shard_off, device=cuda_device)
+        assert torch.equal(torch.searchsorted(idx, bounds).to(torch.int32), sess.out_shard_cnt_off)
+        del r_before
