@@ -19,6 +19,12 @@ namespace gd {
 namespace {
 
 constexpr uint32_t kStash = 128;   // candidate slots per warp and chunk in shared memory
+#ifndef GD_EMIT_WARPS
+#define GD_EMIT_WARPS 8
+#endif
+constexpr int kEmitWarps = GD_EMIT_WARPS;            // warps per CTA of the fused pass
+constexpr int kEmitThreads = 32 * kEmitWarps;
+constexpr uint32_t kEmitTile = 512u * kEmitWarps;    // elements one CTA handles per round trip: 512 per warp
 
 struct StashEntry {
   uint32_t idx;
@@ -31,8 +37,9 @@ struct StashEntry {
 // l, round j -> elements w*512 + j*128 + l*4 .. +3): candidate order inside a warp is (round, lane,
 // component), across warps (warp), across tiles (tile).
 template <int C>
-__global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_constant__ DevTables T) {
-  constexpr int E = C * kWarps;              // (tile, warp) counters of one chunk
+__global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_kernel(const __grid_constant__ DevTables T) {
+  constexpr int CT = C * (int)(kTile / kEmitTile);   // tiles of kEmitTile elements per chunk
+  constexpr int E = CT * kEmitWarps;         // (tile, warp) counters of one chunk
   constexpr int PER = (E + 31) / 32;
   __shared__ uint32_t s_chunk;
   __shared__ uint32_t s_cnt[E];              // candidates per (tile, warp)
@@ -40,7 +47,7 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
   __shared__ uint64_t s_excl;
   __shared__ uint32_t s_total;
   __shared__ int s_ok;
-  __shared__ StashEntry s_stash[kWarps][kStash];
+  __shared__ StashEntry s_stash[kEmitWarps][kStash];
   __shared__ SmemTables s_tab;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   if (tid == 0) s_chunk = atomicAdd(&T.ctl->ticket[L_EMIT], 1u);
@@ -71,10 +78,10 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
   // ---- phase A
   uint32_t fill = 0;                         // candidates of this warp so far in the chunk (warp-uniform)
 #pragma unroll 1
-  for (int i = 0; i < C; ++i) {
-    const uint64_t base = cbase + (uint64_t)i * kTile;
+  for (int i = 0; i < CT; ++i) {
+    const uint64_t base = cbase + (uint64_t)i * kEmitTile;
     uint32_t wc = 0;                         // candidates of this warp in this tile (warp-uniform)
-    if (base >= lo && base + kTile <= hi) {
+    if (base >= lo && base + kEmitTile <= hi) {
       const uint64_t e0 = base + toff;
       float4 g4[4], r4[4];
 #pragma unroll
@@ -108,7 +115,7 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
           wc += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
         }
       }
-    } else if (base < hi && base + kTile > lo) {   // tile cut by the scope (or by the end of the vector)
+    } else if (base < hi && base + kEmitTile > lo) {   // tile cut by the scope (or by the end of the vector)
 #pragma unroll 1
       for (int j = 0; j < 4; ++j) {
         float x[4] = {0.f, 0.f, 0.f, 0.f};
@@ -140,7 +147,7 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
       }
     }
     fill += wc;
-    if (lane == 0) s_cnt[i * kWarps + warp] = wc;
+    if (lane == 0) s_cnt[i * kEmitWarps + warp] = wc;
   }
   __syncthreads();
 
@@ -183,9 +190,9 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
     if (fill <= kStash) {
       uint32_t a = 0;                        // first stash entry of tile i
 #pragma unroll 1
-      for (int i = 0; i < C; ++i) {
-        const uint32_t c = s_cnt[i * kWarps + warp];
-        const uint64_t dst = excl + s_off[i * kWarps + warp];
+      for (int i = 0; i < CT; ++i) {
+        const uint32_t c = s_cnt[i * kEmitWarps + warp];
+        const uint64_t dst = excl + s_off[i * kEmitWarps + warp];
         for (uint32_t e = lane; e < c; e += 32) {
           const uint64_t pos = dst + e;
           if (pos < cap) { cidx[pos] = stash[a + e].idx; cval[pos] = stash[a + e].val; }
@@ -195,10 +202,10 @@ __global__ void __launch_bounds__(kThreads, 4) add_emit_kernel(const __grid_cons
     } else {
       // more candidates than the stash holds: read this warp's elements back (they are v now)
 #pragma unroll 1
-      for (int i = 0; i < C; ++i) {
-        if (s_cnt[i * kWarps + warp] == 0u) continue;
-        uint64_t run = excl + s_off[i * kWarps + warp];
-        const uint64_t base = cbase + (uint64_t)i * kTile;
+      for (int i = 0; i < CT; ++i) {
+        if (s_cnt[i * kEmitWarps + warp] == 0u) continue;
+        uint64_t run = excl + s_off[i * kEmitWarps + warp];
+        const uint64_t base = cbase + (uint64_t)i * kEmitTile;
 #pragma unroll 1
         for (int j = 0; j < 4; ++j) {
           float x[4] = {0.f, 0.f, 0.f, 0.f};
@@ -245,10 +252,10 @@ cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStrea
   if (!tiles[L_EMIT]) return cudaSuccess;
   ProfileScope prof(stream, PT_ADD_EMIT);
   switch (T.emit_chunk_tiles) {
-    case 1: add_emit_kernel<1><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
-    case 2: add_emit_kernel<2><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
-    case 4: add_emit_kernel<4><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
-    default: add_emit_kernel<8><<<tiles[L_EMIT], kThreads, 0, stream>>>(T); break;
+    case 1: add_emit_kernel<1><<<tiles[L_EMIT], kEmitThreads, 0, stream>>>(T); break;
+    case 2: add_emit_kernel<2><<<tiles[L_EMIT], kEmitThreads, 0, stream>>>(T); break;
+    case 4: add_emit_kernel<4><<<tiles[L_EMIT], kEmitThreads, 0, stream>>>(T); break;
+    default: add_emit_kernel<8><<<tiles[L_EMIT], kEmitThreads, 0, stream>>>(T); break;
   }
   GD_LAUNCH_CHECK();
   return cudaSuccess;
