@@ -40,7 +40,7 @@ typedef enum {
 } gd_status_t;
 
 enum { GD_SCOPE_GLOBAL = 0, GD_SCOPE_PER_LAYER = 1 };
-enum { GD_VALUES_FP32 = 0, GD_VALUES_TWO_MEANS = 1, GD_VALUES_THRESHOLD = 2 };
+enum { GD_VALUES_FP32 = 0, GD_VALUES_TWO_MEANS = 1, GD_VALUES_THRESHOLD = 2, GD_VALUES_COLUMN_MEANS = 3 };
 
 /* gd_compress_args.flags */
 enum {
@@ -76,12 +76,21 @@ int gd_total_kept(const uint64_t* layer_off, uint32_t n_layers, int scope_mode, 
 int gd_sampled_capacity(const uint64_t* layer_off, uint32_t n_layers, int scope_mode, uint32_t drop_ppm,
                         uint64_t* capacity_out);
 
-/* Bytes of device workspace gd_compress needs for these arguments (same meaning as in gd_compress_args). */
-int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, int scope_mode,
-                       uint32_t drop_ppm, size_t* bytes_out);
+/*
+ * Bytes of device workspace gd_compress needs for these arguments (same meaning as in gd_compress_args).
+ * layer_cols may be NULL unless GD_VALUES_COLUMN_MEANS will be used.
+ */
+int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* layer_cols, uint32_t n_shards,
+                       int scope_mode, uint32_t drop_ppm, size_t* bytes_out);
 
 /* Bytes of device workspace gd_decompress_apply needs. */
 int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes_out);
+
+/*
+ * Number of (mu+, mu-) pairs of a push: n_layers for GD_VALUES_TWO_MEANS and GD_VALUES_THRESHOLD, the
+ * sum of layer_cols for GD_VALUES_COLUMN_MEANS, 0 for GD_VALUES_FP32.  out_means holds 2 floats per pair.
+ */
+int gd_means_pairs(uint32_t n_layers, const uint32_t* layer_cols, int value_mode, uint64_t* pairs_out);
 
 /*
  * gd_compress - Algorithm 1 (GradDrop) for one worker's flat fp32 gradient.
@@ -98,6 +107,11 @@ int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes
  *              (fp64 accumulation, rounded to fp32, +0.0f for an empty group); out_idx[t] carries
  *              index | signbit << 31 and out_val is not written.  The residual is unchanged by the
  *              value mode: it holds the dropped mass only.
+ *   column-means mode (Section 5.4: the averages are taken "at the column level, rather than choosing
+ *              centers globally"): layer l is a row-major matrix with layer_cols[l] columns (its size must
+ *              be a multiple of layer_cols[l]; 1 = one pair for the whole layer, as in two-means mode), and
+ *              every column c gets its own pair: pair index = sum of layer_cols of the earlier layers + c,
+ *              out_means[2 * pair] = mu+, out_means[2 * pair + 1] = mu-.  Packing as in two-means mode.
  *   threshold mode (Section 5.4, the quantisation that maps "all surviving values to the dropping
  *              threshold, effectively the minimum surviving absolute value"): same packing as two-means
  *              mode; out_means[l] = (+t, -t) with t the float whose bit pattern is the tau of the scope
@@ -150,10 +164,11 @@ typedef struct gd_compress_args {
   float* out_val;             /* device, gd_total_kept() fp32; may be NULL in two-means mode */
   uint32_t* out_shard_cnt_off;/* device, n_shards + 1 words */
   uint32_t* out_tau;          /* device, one word per scope (1, or n_layers); may be NULL */
-  float* out_means;           /* device, n_layers x 2 fp32 (mu+, mu-); two-means and threshold modes */
+  float* out_means;           /* device, gd_means_pairs() x 2 fp32 (mu+, mu-); the packed modes */
   void* workspace;            /* device, 256-byte aligned, >= gd_workspace_bytes() */
   size_t workspace_bytes;
   float* delta_base;          /* device, n fp32, 16-byte aligned, in/out, or NULL (see "delta mode" above) */
+  const uint32_t* layer_cols; /* HOST, n_layers column counts; GD_VALUES_COLUMN_MEANS only, else may be NULL */
 } gd_compress_args;
 
 int gd_compress(const gd_compress_args* args, void* stream);
@@ -168,7 +183,7 @@ typedef struct gd_push {
   const uint32_t* idx;
   const float* val;              /* NULL in the packed modes */
   const uint32_t* shard_cnt_off;
-  const float* means;            /* n_layers x 2, packed modes only */
+  const float* means;            /* gd_means_pairs() x 2, packed modes only */
 } gd_push;
 
 /*
@@ -176,7 +191,8 @@ typedef struct gd_push {
  * and adds the pushed pieces into it.  For every push in array order and every entry of it
  * whose index lies in a shard [shard_off[j], shard_off[j+1]):
  *     params[j][index - shard_off[j]] += alpha * value
- * with value = val[t] (fp32 mode) or means[layer of the entry][sign] (two-means and threshold modes).
+ * with value = val[t] (fp32 mode) or means[pair of the entry][sign] (the packed modes; the pair is the
+ * entry's layer, or its layer and column in column-means mode).
  * One fused multiply-add in fp32 per entry; with alpha = 1 the result is fl32(p + value).
  * Pushes are applied one after another in stream order; indices inside one push are unique.
  * Entries whose index lies outside every shard are skipped.  The optimiser is not part of
@@ -195,6 +211,7 @@ typedef struct gd_apply_args {
   uint32_t reserved;
   void* workspace;             /* device, 256-byte aligned, >= gd_apply_workspace_bytes() */
   size_t workspace_bytes;
+  const uint32_t* layer_cols;  /* HOST, n_layers column counts; GD_VALUES_COLUMN_MEANS only, else may be NULL */
 } gd_apply_args;
 
 int gd_decompress_apply(const gd_apply_args* args, void* stream);

@@ -26,6 +26,8 @@ Readings taken where the paper is silent:
   * two-value quantisation (Section 5.4, "averages of values being quantized"): one pair
     (mean of kept entries with sign bit 0, mean of kept entries with sign bit 1) per layer,
     survivors packed as index | signbit << 31; the residual still holds only the dropped mass;
+  * column-wise averages (Section 5.4: centres chosen "at the column level" rather than per tensor):
+    a layer is a row-major matrix with layer_cols[l] columns and every column has its own pair;
   * threshold quantisation (Section 5.4: every surviving value is mapped to the dropping
     threshold, "effectively the minimum surviving absolute value"): same packing; the pair of a
     layer is (+t, -t) with t the float whose bit pattern is the tau of the scope holding the layer;
@@ -41,6 +43,7 @@ SCOPE_PER_LAYER = 1
 VALUES_FP32 = 0
 VALUES_TWO_MEANS = 1
 VALUES_THRESHOLD = 2
+VALUES_COLUMN_MEANS = 3
 
 _ABS_MASK = np.uint32(0x7FFFFFFF)
 TAU_NONE = 0xFFFFFFFF
@@ -187,8 +190,19 @@ def compress_delta(params, last_pulled, layer_off, shard_off, drop_ppm, scope_mo
     return out
 
 
+def pair_index(pos, layer_off, layer_cols=None):
+    """The (mean+, mean-) pair each position belongs to: its layer, or its layer and column."""
+    lo = np.asarray([int(x) for x in layer_off], dtype=np.int64)
+    n_layers = lo.shape[0] - 1
+    cols = np.ones(n_layers, dtype=np.int64) if layer_cols is None else np.asarray(layer_cols, dtype=np.int64)
+    pair_off = np.concatenate([[0], np.cumsum(cols)])
+    pos = np.asarray(pos, dtype=np.int64)
+    layer = np.searchsorted(lo, pos, side="right") - 1
+    return pair_off[layer] + (pos - lo[layer]) % cols[layer], int(pair_off[-1])
+
+
 def compress(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GLOBAL,
-             value_mode=VALUES_FP32, method="sort"):
+             value_mode=VALUES_FP32, method="sort", layer_cols=None):
     """One GradDrop call (Algorithm 1) for one worker's flat fp32 gradient.
 
     grad, residual : float32 arrays of n elements (not modified).
@@ -237,17 +251,20 @@ def compress(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GL
         "shard_cnt_off": shard_cnt_off,
         "v": v,
     }
-    if value_mode == VALUES_TWO_MEANS:
+    if value_mode in (VALUES_TWO_MEANS, VALUES_COLUMN_MEANS):
         if n > (1 << 31):
-            raise ValueError("two-means packing needs n <= 2^31")
-        n_layers = len(layer_off) - 1
-        sums = np.zeros((n_layers, 2), dtype=np.float64)
-        cnts = np.zeros((n_layers, 2), dtype=np.int64)
+            raise ValueError("packed indices need n <= 2^31")
+        if value_mode == VALUES_COLUMN_MEANS:
+            assert layer_cols is not None
+            for l in range(len(layer_off) - 1):
+                assert layer_cols[l] >= 1 and (layer_off[l + 1] - layer_off[l]) % layer_cols[l] == 0
+        pair, n_pairs = pair_index(kept, layer_off, layer_cols if value_mode == VALUES_COLUMN_MEANS else None)
+        sums = np.zeros((n_pairs, 2), dtype=np.float64)
+        cnts = np.zeros((n_pairs, 2), dtype=np.int64)
         sign = (val.view(np.uint32) >> np.uint32(31)).astype(np.int64)
-        layer = np.searchsorted(np.asarray(layer_off, dtype=np.int64), kept, side="right") - 1
         # unbuffered accumulation: one fp64 add per survivor, in ascending index order
-        np.add.at(sums, (layer, sign), val.astype(np.float64))
-        np.add.at(cnts, (layer, sign), 1)
+        np.add.at(sums, (pair, sign), val.astype(np.float64))
+        np.add.at(cnts, (pair, sign), 1)
         with np.errstate(invalid="ignore", divide="ignore"):
             means = np.where(cnts > 0, sums / np.maximum(cnts, 1), 0.0).astype(np.float32)
         out["idx"] = (kept.astype(np.uint32) | (sign.astype(np.uint32) << np.uint32(31)))
@@ -270,18 +287,18 @@ def compress(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GL
     return out
 
 
-def decode_push(push_idx, push_val, value_mode=VALUES_FP32, means=None, layer_off=None):
+def decode_push(push_idx, push_val, value_mode=VALUES_FP32, means=None, layer_off=None, layer_cols=None):
     """Positions and fp32 values a push stands for (the server-side decompress)."""
     idx = np.asarray(push_idx, dtype=np.uint32)
     if value_mode == VALUES_FP32:
         return idx.astype(np.int64), np.asarray(push_val, dtype=np.float32)
     pos = (idx & _ABS_MASK).astype(np.int64)
     sign = (idx >> np.uint32(31)).astype(np.int64)
-    layer = np.searchsorted(np.asarray(layer_off, dtype=np.int64), pos, side="right") - 1
-    return pos, np.asarray(means, dtype=np.float32)[layer, sign]
+    pair, _ = pair_index(pos, layer_off, layer_cols if value_mode == VALUES_COLUMN_MEANS else None)
+    return pos, np.asarray(means, dtype=np.float32)[pair, sign]
 
 
-def apply_pushes(params, shard_start, pushes, alpha=1.0, value_mode=VALUES_FP32, layer_off=None):
+def apply_pushes(params, shard_start, pushes, alpha=1.0, value_mode=VALUES_FP32, layer_off=None, layer_cols=None):
     """fp64 reference of the server-side scatter-add into one parameter shard (Section 3).
 
     params  : float32[shard_len], the shard's parameters before the pushes.
@@ -297,7 +314,7 @@ def apply_pushes(params, shard_start, pushes, alpha=1.0, value_mode=VALUES_FP32,
     lo, hi = int(shard_start), int(shard_start) + p0.shape[0]
     for push in pushes:
         pos, val = decode_push(push["idx"], push.get("val"), value_mode, push.get("means"),
-                               layer_off)
+                               layer_off, layer_cols)
         m = (pos >= lo) & (pos < hi)
         contrib = a * val[m].astype(np.float64)
         np.add.at(ref, pos[m] - lo, contrib)

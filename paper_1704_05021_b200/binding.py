@@ -27,6 +27,7 @@ GD_SCOPE_PER_LAYER = 1
 GD_VALUES_FP32 = 0
 GD_VALUES_TWO_MEANS = 1
 GD_VALUES_THRESHOLD = 2
+GD_VALUES_COLUMN_MEANS = 3
 GD_FLAG_NO_PREDICTION = 1
 GD_FLAG_SAMPLED_THRESHOLD = 2
 GD_ERR_OVERFLOW = -7
@@ -35,7 +36,7 @@ EXPORTS = [
     "gd_status_string", "gd_kept_count", "gd_total_kept", "gd_workspace_bytes", "gd_apply_workspace_bytes",
     "gd_compress", "gd_decompress_apply", "gd_residual_reset", "gd_status", "gd_get_stats", "gd_step_host",
     "gd_profile_enable", "gd_profile_collect", "gd_launch_count", "gd_compress_static",
-    "gd_selftest_bounded_wait", "gd_sampled_capacity",
+    "gd_selftest_bounded_wait", "gd_sampled_capacity", "gd_means_pairs",
 ]
 GD_STATIC_WORKSPACE_BYTES = 16 << 20
 
@@ -55,6 +56,7 @@ class _CompressArgs(C.Structure):
         ("out_idx", C.c_void_p), ("out_val", C.c_void_p), ("out_shard_cnt_off", C.c_void_p),
         ("out_tau", C.c_void_p), ("out_means", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("delta_base", C.c_void_p),
+        ("layer_cols", C.POINTER(C.c_uint32)),
     ]
 
 
@@ -68,7 +70,7 @@ class _ApplyArgs(C.Structure):
         ("n_shards", C.c_uint32), ("n_pushes", C.c_uint32), ("pushes", C.POINTER(_Push)),
         ("value_mode", C.c_int32), ("alpha", C.c_float),
         ("layer_off", C.POINTER(C.c_uint64)), ("n_layers", C.c_uint32), ("reserved", C.c_uint32),
-        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("layer_cols", C.POINTER(C.c_uint32)),
     ]
 
 
@@ -102,8 +104,9 @@ def load_library():
     lib.gd_status_string.argtypes = [C.c_int]
     lib.gd_kept_count.argtypes = [C.c_uint64, C.c_uint32, C.POINTER(C.c_uint64)]
     lib.gd_total_kept.argtypes = [C.POINTER(C.c_uint64), C.c_uint32, C.c_int, C.c_uint32, C.POINTER(C.c_uint64)]
-    lib.gd_workspace_bytes.argtypes = [C.POINTER(C.c_uint64), C.c_uint32, C.c_uint32, C.c_int, C.c_uint32,
-                                       C.POINTER(C.c_size_t)]
+    lib.gd_workspace_bytes.argtypes = [C.POINTER(C.c_uint64), C.c_uint32, C.POINTER(C.c_uint32), C.c_uint32, C.c_int,
+                                       C.c_uint32, C.POINTER(C.c_size_t)]
+    lib.gd_means_pairs.argtypes = [C.c_uint32, C.POINTER(C.c_uint32), C.c_int, C.POINTER(C.c_uint64)]
     lib.gd_apply_workspace_bytes.argtypes = [C.c_uint32, C.c_uint32, C.POINTER(C.c_size_t)]
     lib.gd_compress.argtypes = [C.POINTER(_CompressArgs), C.c_void_p]
     lib.gd_decompress_apply.argtypes = [C.POINTER(_ApplyArgs), C.c_void_p]
@@ -160,11 +163,22 @@ def gd_total_kept(layer_off: Sequence[int], scope_mode: int, drop_ppm: int) -> i
     return out.value
 
 
-def gd_workspace_bytes(layer_off: Sequence[int], n_shards: int, scope_mode: int, drop_ppm: int) -> int:
+def _u32_array(values: Optional[Sequence[int]]):
+    return None if values is None else (C.c_uint32 * len(values))(*[int(v) for v in values])
+
+
+def gd_workspace_bytes(layer_off: Sequence[int], n_shards: int, scope_mode: int, drop_ppm: int,
+                       layer_cols: Optional[Sequence[int]] = None) -> int:
     out = C.c_size_t(0)
     arr = _u64_array(layer_off)
-    _check(load_library().gd_workspace_bytes(arr, len(layer_off) - 1, n_shards, scope_mode, drop_ppm, C.byref(out)),
-           "gd_workspace_bytes")
+    _check(load_library().gd_workspace_bytes(arr, len(layer_off) - 1, _u32_array(layer_cols), n_shards, scope_mode,
+                                             drop_ppm, C.byref(out)), "gd_workspace_bytes")
+    return out.value
+
+
+def gd_means_pairs(n_layers: int, layer_cols: Optional[Sequence[int]], value_mode: int) -> int:
+    out = C.c_uint64(0)
+    _check(load_library().gd_means_pairs(n_layers, _u32_array(layer_cols), value_mode, C.byref(out)), "gd_means_pairs")
     return out.value
 
 
@@ -178,7 +192,7 @@ class CompressCall:
     """The marshalled argument block of one gd_compress call (kept so it can be re-issued cheaply)."""
 
     def __init__(self, grad, residual, layer_off, shard_off, drop_ppm, scope_mode, value_mode, out_idx, out_val,
-                 out_shard_cnt_off, out_tau, out_means, workspace, flags=0, delta_base=None):
+                 out_shard_cnt_off, out_tau, out_means, workspace, flags=0, delta_base=None, layer_cols=None):
         self._keep = (grad, residual, out_idx, out_val, out_shard_cnt_off, out_tau, out_means, workspace, delta_base)
         self._layer_off = _u64_array(layer_off)
         self._shard_off = _u64_array(shard_off)
@@ -192,6 +206,9 @@ class CompressCall:
         a.workspace = _ptr(workspace)
         a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
         a.delta_base = _ptr(delta_base)
+        self._layer_cols = _u32_array(layer_cols)
+        if self._layer_cols is not None:
+            a.layer_cols = self._layer_cols
         self.args = a
 
     def set_grad(self, grad: torch.Tensor):
@@ -203,7 +220,7 @@ class ApplyCall:
     """The marshalled argument block of one gd_decompress_apply call."""
 
     def __init__(self, params: Sequence[torch.Tensor], shard_off, pushes, value_mode, alpha, workspace,
-                 layer_off=None):
+                 layer_off=None, layer_cols=None):
         self._keep = (list(params), pushes, workspace)
         n_shards = len(shard_off) - 1
         self._params = (C.c_void_p * n_shards)(*[p.data_ptr() if p.numel() else None for p in params])
@@ -223,6 +240,9 @@ class ApplyCall:
             a.layer_off, a.n_layers = self._layer_off, len(layer_off) - 1
         a.workspace = _ptr(workspace)
         a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        self._layer_cols = _u32_array(layer_cols)
+        if self._layer_cols is not None:
+            a.layer_cols = self._layer_cols
         self.args = a
 
 

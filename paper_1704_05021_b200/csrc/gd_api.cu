@@ -74,7 +74,11 @@ struct Plan {
   size_t off_ctl = 0, off_state = 0, off_hist = 0, off_sums = 0, off_cnts = 0, off_desc_emit = 0,
          off_desc_cand = 0, off_desc_dcomp = 0, zero_bytes = 0;
   size_t off_tables = 0, tables_bytes = 0;
-  size_t t_scopes = 0, t_tile0[L_COUNT] = {0, 0, 0, 0, 0}, t_samp_off = 0, t_layer_off = 0, t_shard_off = 0;
+  size_t t_scopes = 0, t_tile0[L_COUNT] = {0, 0, 0, 0, 0}, t_samp_off = 0, t_layer_off = 0, t_shard_off = 0,
+         t_pair_off = 0, t_layer_cols = 0;
+  std::vector<uint64_t> pair_off;
+  std::vector<uint32_t> layer_cols;
+  uint64_t n_pairs = 0;
   size_t off_samp = 0, off_cand_idx = 0, off_cand_val = 0, total_bytes = 0;
 };
 
@@ -87,8 +91,9 @@ int check_offsets(const uint64_t* off, uint32_t count, uint64_t* n_out) {
   return GD_OK;
 }
 
-int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, int scope_mode, uint32_t drop_ppm,
-              uint32_t flags, Plan* P) {
+// layer_cols == NULL: one (mu+, mu-) pair per layer.
+int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* layer_cols, uint32_t n_shards, int scope_mode,
+              uint32_t drop_ppm, uint32_t flags, Plan* P) {
   uint64_t n = 0;
   int rc = check_offsets(layer_off, n_layers, &n);
   if (rc != GD_OK) return rc;
@@ -97,6 +102,16 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, i
   if (n > (1ull << 32)) return GD_ERR_TOO_LARGE;
   const bool predict = !(flags & GD_FLAG_NO_PREDICTION);
   const bool sampled = (flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
+  P->pair_off.assign((size_t)n_layers + 1, 0);
+  P->layer_cols.assign(n_layers, 1);
+  for (uint32_t l = 0; l < n_layers; ++l) {
+    const uint64_t size = layer_off[l + 1] - layer_off[l];
+    uint32_t cols = layer_cols ? layer_cols[l] : 1u;
+    if (cols == 0 || (size % cols) != 0) return GD_ERR_INVALID_ARG;   // a layer is rows x cols, row-major
+    P->layer_cols[l] = cols;
+    P->pair_off[l + 1] = P->pair_off[l] + cols;
+  }
+  P->n_pairs = P->pair_off[n_layers];
   // The fused pass gives each CTA a chunk of 1, 2, 4 or 8 tiles: as large as still leaves about
   // four waves of CTAs (4 per SM on 148 SMs) for the whole vector.
   const uint64_t dense_tiles = (n + kTile - 1) / kTile;
@@ -158,19 +173,23 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, i
   P->off_ctl = off;          off = align_up(off + sizeof(Ctl));
   P->off_state = off;        off = align_up(off + sizeof(ScopeState) * ns_count);
   P->off_hist = off;         off = align_up(off + sizeof(unsigned long long) * kHistBinsPerScope * (size_t)ns_count);
-  P->off_sums = off;         off = align_up(off + sizeof(double) * 2 * (size_t)n_layers);
-  P->off_cnts = off;         off = align_up(off + sizeof(unsigned long long) * 2 * (size_t)n_layers);
+  P->off_sums = off;         off = align_up(off + sizeof(double) * 2 * (size_t)P->n_pairs);
+  P->off_cnts = off;         off = align_up(off + sizeof(unsigned long long) * 2 * (size_t)P->n_pairs);
   P->off_desc_emit = off;    off = align_up(off + 16 * (size_t)P->tiles[L_EMIT]);
   P->off_desc_cand = off;    off = align_up(off + 16 * (size_t)P->tiles[L_CAND]);
   P->off_desc_dcomp = off;   off = align_up(off + 16 * (size_t)P->tiles[L_DCOMP]);
   P->zero_bytes = off;
   P->off_tables = off;
   size_t t = 0;
-  P->t_scopes = t;           t = align_up(t + sizeof(ScopeDesc) * ns_count);
-  for (int l = 0; l < L_COUNT; ++l) { P->t_tile0[l] = t; t = align_up(t + sizeof(uint32_t) * (ns_count + 1)); }
-  P->t_samp_off = t;         t = align_up(t + sizeof(uint64_t) * (ns_count + 1));
-  P->t_layer_off = t;        t = align_up(t + sizeof(uint64_t) * ((size_t)n_layers + 1));
-  P->t_shard_off = t;        t = align_up(t + sizeof(uint64_t) * ((size_t)n_shards + 1));
+  auto sub = [](size_t x) { return (x + 15) / 16 * 16; };   // tables are packed at 16-byte steps
+  P->t_scopes = t;           t = sub(t + sizeof(ScopeDesc) * ns_count);
+  for (int l = 0; l < L_COUNT; ++l) { P->t_tile0[l] = t; t = sub(t + sizeof(uint32_t) * (ns_count + 1)); }
+  P->t_samp_off = t;         t = sub(t + sizeof(uint64_t) * (ns_count + 1));
+  P->t_layer_off = t;        t = sub(t + sizeof(uint64_t) * ((size_t)n_layers + 1));
+  P->t_shard_off = t;        t = sub(t + sizeof(uint64_t) * ((size_t)n_shards + 1));
+  P->t_pair_off = t;         t = sub(t + sizeof(uint64_t) * ((size_t)n_layers + 1));
+  P->t_layer_cols = t;       t = sub(t + sizeof(uint32_t) * (size_t)n_layers);
+  t = align_up(t);
   P->tables_bytes = t;
   off += t;
   P->off_samp = off;         off = align_up(off + sizeof(float) * P->samp_total);
@@ -310,7 +329,7 @@ int gd_sampled_capacity(const uint64_t* layer_off, uint32_t n_layers, int scope_
   if (!capacity_out) return GD_ERR_INVALID_ARG;
   try {
     Plan P;
-    int rc = make_plan(layer_off, n_layers, 1, scope_mode, drop_ppm, GD_FLAG_SAMPLED_THRESHOLD, &P);
+    int rc = make_plan(layer_off, n_layers, nullptr, 1, scope_mode, drop_ppm, GD_FLAG_SAMPLED_THRESHOLD, &P);
     if (rc != GD_OK) return rc;
     *capacity_out = P.cand_total;
     return GD_OK;
@@ -319,14 +338,28 @@ int gd_sampled_capacity(const uint64_t* layer_off, uint32_t n_layers, int scope_
   }
 }
 
-int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, uint32_t n_shards, int scope_mode,
-                       uint32_t drop_ppm, size_t* bytes_out) {
+int gd_means_pairs(uint32_t n_layers, const uint32_t* layer_cols, int value_mode, uint64_t* pairs_out) {
+  if (!pairs_out) return GD_ERR_INVALID_ARG;
+  if (value_mode == GD_VALUES_FP32) { *pairs_out = 0; return GD_OK; }
+  if (value_mode == GD_VALUES_TWO_MEANS || value_mode == GD_VALUES_THRESHOLD) { *pairs_out = n_layers; return GD_OK; }
+  if (value_mode != GD_VALUES_COLUMN_MEANS || !layer_cols) return GD_ERR_INVALID_ARG;
+  uint64_t total = 0;
+  for (uint32_t l = 0; l < n_layers; ++l) {
+    if (layer_cols[l] == 0) return GD_ERR_INVALID_ARG;
+    total += layer_cols[l];
+  }
+  *pairs_out = total;
+  return GD_OK;
+}
+
+int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* layer_cols, uint32_t n_shards,
+                       int scope_mode, uint32_t drop_ppm, size_t* bytes_out) {
   if (!bytes_out) return GD_ERR_INVALID_ARG;
   try {
     Plan P, Q;
-    int rc = make_plan(layer_off, n_layers, n_shards, scope_mode, drop_ppm, 0u, &P);
+    int rc = make_plan(layer_off, n_layers, layer_cols, n_shards, scope_mode, drop_ppm, 0u, &P);
     if (rc != GD_OK) return rc;
-    rc = make_plan(layer_off, n_layers, n_shards, scope_mode, drop_ppm, GD_FLAG_SAMPLED_THRESHOLD, &Q);
+    rc = make_plan(layer_off, n_layers, layer_cols, n_shards, scope_mode, drop_ppm, GD_FLAG_SAMPLED_THRESHOLD, &Q);
     if (rc != GD_OK) return rc;
     *bytes_out = P.total_bytes > Q.total_bytes ? P.total_bytes : Q.total_bytes;   // whichever mode is used
     return GD_OK;
@@ -340,14 +373,16 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
   cudaStream_t stream = (cudaStream_t)stream_v;
   try {
     Plan P;
-    int rc = make_plan(a->layer_off, a->n_layers, a->n_shards, a->scope_mode, a->drop_ppm, a->flags, &P);
+    if (a->value_mode == GD_VALUES_COLUMN_MEANS && !a->layer_cols) return GD_ERR_INVALID_ARG;
+    int rc = make_plan(a->layer_off, a->n_layers, a->value_mode == GD_VALUES_COLUMN_MEANS ? a->layer_cols : nullptr,
+                       a->n_shards, a->scope_mode, a->drop_ppm, a->flags, &P);
     if (rc != GD_OK) return rc;
     uint64_t n_sh = 0;
     rc = check_offsets(a->shard_off, a->n_shards, &n_sh);
     if (rc != GD_OK) return rc;
     const uint64_t n = a->layer_off[a->n_layers];
     if (n_sh != n || a->n != n) return GD_ERR_INVALID_ARG;
-    if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_THRESHOLD) return GD_ERR_INVALID_ARG;
+    if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_COLUMN_MEANS) return GD_ERR_INVALID_ARG;
     if (a->value_mode != GD_VALUES_FP32 && n > (1ull << 31)) return GD_ERR_TOO_LARGE;
     if (a->flags & ~(uint32_t)(GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD)) return GD_ERR_INVALID_ARG;
     const bool sampled = (a->flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
@@ -370,6 +405,8 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     std::memcpy(blob.data() + P.t_samp_off, P.samp_off.data(), sizeof(uint64_t) * (P.n_scopes + 1));
     std::memcpy(blob.data() + P.t_layer_off, a->layer_off, sizeof(uint64_t) * ((size_t)a->n_layers + 1));
     std::memcpy(blob.data() + P.t_shard_off, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
+    std::memcpy(blob.data() + P.t_pair_off, P.pair_off.data(), sizeof(uint64_t) * ((size_t)a->n_layers + 1));
+    std::memcpy(blob.data() + P.t_layer_cols, P.layer_cols.data(), sizeof(uint32_t) * (size_t)a->n_layers);
 
     unsigned char* ws = (unsigned char*)a->workspace;
     if (launch_setup(ws + P.off_tables, blob.data(), P.tables_bytes, ws, P.zero_bytes, stream) != cudaSuccess)
@@ -404,6 +441,9 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     T.samp_off = (const uint64_t*)(tb + P.t_samp_off);
     T.layer_off = (const uint64_t*)(tb + P.t_layer_off);
     T.shard_off = (const uint64_t*)(tb + P.t_shard_off);
+    T.pair_off = (const uint64_t*)(tb + P.t_pair_off);
+    T.layer_cols = (const uint32_t*)(tb + P.t_layer_cols);
+    T.n_pairs = P.n_pairs;
     T.samp_val = (float*)(ws + P.off_samp);
     T.cand_idx = (uint32_t*)(ws + P.off_cand_idx);
     T.cand_val = (float*)(ws + P.off_cand_val);
@@ -432,6 +472,9 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
       if (launch_candidate_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
       if (launch_compact(T, tiles, false, true, stream) != cudaSuccess) return GD_ERR_CUDA;
     }
+    if ((a->value_mode == GD_VALUES_TWO_MEANS || a->value_mode == GD_VALUES_COLUMN_MEANS) && P.n_pairs > kInlineMeansPairs &&
+        launch_means(T, stream) != cudaSuccess)
+      return GD_ERR_CUDA;
     return GD_OK;
   } catch (const std::bad_alloc&) {
     return GD_ERR_INVALID_ARG;
@@ -471,7 +514,8 @@ static __device__ __align__(256) unsigned char g_static_workspace[GD_STATIC_WORK
 int gd_compress_static(const gd_compress_args* a, void* stream, const void** workspace_out) {
   if (!a) return GD_ERR_INVALID_ARG;
   size_t need = 0;
-  int rc = gd_workspace_bytes(a->layer_off, a->n_layers, a->n_shards, a->scope_mode, a->drop_ppm, &need);
+  int rc = gd_workspace_bytes(a->layer_off, a->n_layers, a->value_mode == GD_VALUES_COLUMN_MEANS ? a->layer_cols : nullptr,
+                              a->n_shards, a->scope_mode, a->drop_ppm, &need);
   if (rc != GD_OK) return rc;
   if (need > (size_t)GD_STATIC_WORKSPACE_BYTES) return GD_ERR_TOO_LARGE;
   // In host code g_static_workspace is only a handle: its device address has to be asked for, once
@@ -559,9 +603,10 @@ int gd_step_host(const gd_compress_args* a, const gd_apply_args* apply, const gd
   if (e == cudaSuccess && io->shard_cnt_off_host)
     e = cudaMemcpyAsync(io->shard_cnt_off_host, a->out_shard_cnt_off, sizeof(uint32_t) * ((size_t)a->n_shards + 1),
                         cudaMemcpyDeviceToHost, stream);
+  uint64_t pairs = 0;
+  if (io->means_host && gd_means_pairs(a->n_layers, a->layer_cols, a->value_mode, &pairs) != GD_OK) return GD_ERR_INVALID_ARG;
   if (e == cudaSuccess && io->means_host && a->value_mode != GD_VALUES_FP32)
-    e = cudaMemcpyAsync(io->means_host, a->out_means, sizeof(float) * 2 * (size_t)a->n_layers, cudaMemcpyDeviceToHost,
-                        stream);
+    e = cudaMemcpyAsync(io->means_host, a->out_means, sizeof(float) * 2 * (size_t)pairs, cudaMemcpyDeviceToHost, stream);
   if (e != cudaSuccess) return GD_ERR_CUDA;
   return gd_status(a->workspace, stream_v);
 }

@@ -17,7 +17,9 @@ inline size_t align_up_a(size_t x) { return (x + kAlignA - 1) / kAlignA * kAlign
 struct ApplyDev {
   float* const* params;        // [n_shards] device pointers
   const uint64_t* shard_off;   // [n_shards + 1]
-  const uint64_t* layer_off;   // [n_layers + 1] (two-means mode)
+  const uint64_t* layer_off;   // [n_layers + 1] (packed modes)
+  const uint64_t* pair_off;    // [n_layers + 1]
+  const uint32_t* layer_cols;  // [n_layers]
   uint32_t n_shards, n_layers;
   int32_t value_mode;
   float alpha;
@@ -33,6 +35,8 @@ struct ApplyInline {
   float* params[kInlineShards];
   uint64_t shard_off[kInlineShards + 1];
   uint64_t layer_off[kInlineLayers + 1];
+  uint64_t pair_off[kInlineLayers + 1];
+  uint32_t layer_cols[kInlineLayers];
 };
 
 // Segmented scatter-add: the entries [cnt_off[0], cnt_off[n_shards]) of one push, one thread per
@@ -44,6 +48,8 @@ __global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__
   float* const* params = INLINE ? I.params : A.params;
   const uint64_t* shard_off = INLINE ? I.shard_off : A.shard_off;
   const uint64_t* layer_off = INLINE ? I.layer_off : A.layer_off;
+  const uint64_t* pair_off = INLINE ? I.pair_off : A.pair_off;
+  const uint32_t* layer_cols = INLINE ? I.layer_cols : A.layer_cols;
   const uint64_t begin = A.cnt_off[0], end = A.cnt_off[A.n_shards];
   const uint64_t lo_all = shard_off[0], hi_all = shard_off[A.n_shards];
   const uint64_t stride = (uint64_t)gridDim.x * kThreads;
@@ -53,8 +59,8 @@ __global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__
     float x;
     if (A.value_mode != GD_VALUES_FP32) {
       pos = w & kAbsMask;
-      const uint32_t l = range_of(layer_off, A.n_layers, pos);
-      x = __ldg(A.means + 2 * (size_t)l + (w >> 31));
+      const uint64_t pr = pair_of(layer_off, pair_off, layer_cols, A.n_layers, pos);
+      x = __ldg(A.means + 2 * pr + (w >> 31));
     } else {
       x = __ldcs(A.val + p);
     }
@@ -77,7 +83,8 @@ int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes
   if (!bytes_out || n_shards == 0) return GD_ERR_INVALID_ARG;
   size_t b = align_up_a(sizeof(float*) * (size_t)n_shards);
   b += align_up_a(sizeof(uint64_t) * ((size_t)n_shards + 1));
-  b += align_up_a(sizeof(uint64_t) * ((size_t)n_layers + 1));
+  b += 2 * align_up_a(sizeof(uint64_t) * ((size_t)n_layers + 1));   // layer offsets, pair offsets
+  b += align_up_a(sizeof(uint32_t) * ((size_t)n_layers + 1));        // columns per layer
   *bytes_out = b;
   return GD_OK;
 }
@@ -85,7 +92,8 @@ int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes
 int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
   if (!a || !a->params || !a->shard_off || a->n_shards == 0) return GD_ERR_INVALID_ARG;
   if (a->n_pushes && !a->pushes) return GD_ERR_INVALID_ARG;
-  if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_THRESHOLD) return GD_ERR_INVALID_ARG;
+  if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_COLUMN_MEANS) return GD_ERR_INVALID_ARG;
+  if (a->value_mode == GD_VALUES_COLUMN_MEANS && !a->layer_cols) return GD_ERR_INVALID_ARG;
   const bool two_means = a->value_mode != GD_VALUES_FP32;   // the packed modes decode through the means table
   if (two_means && (!a->layer_off || a->n_layers == 0)) return GD_ERR_INVALID_ARG;
   for (uint32_t j = 0; j < a->n_shards; ++j) {
@@ -111,19 +119,39 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
     const size_t o_params = 0;
     const size_t o_shard = align_up_a(sizeof(float*) * (size_t)a->n_shards);
     const size_t o_layer = o_shard + align_up_a(sizeof(uint64_t) * ((size_t)a->n_shards + 1));
+    const size_t o_pair = o_layer + align_up_a(sizeof(uint64_t) * ((size_t)n_layers + 1));
+    const size_t o_cols = o_pair + align_up_a(sizeof(uint64_t) * ((size_t)n_layers + 1));
     unsigned char* ws = (unsigned char*)a->workspace;
+    // pairs: one per layer, or one per column of every layer (column-means mode)
+    std::vector<uint64_t> pair_off((size_t)n_layers + 1, 0);
+    std::vector<uint32_t> cols(n_layers, 1u);
+    for (uint32_t l = 0; l < n_layers; ++l) {
+      if (a->value_mode == GD_VALUES_COLUMN_MEANS) {
+        cols[l] = a->layer_cols[l];
+        if (cols[l] == 0 || ((a->layer_off[l + 1] - a->layer_off[l]) % cols[l]) != 0) return GD_ERR_INVALID_ARG;
+      }
+      pair_off[l + 1] = pair_off[l] + cols[l];
+    }
     const bool use_inline = a->n_shards <= kInlineShards && n_layers <= kInlineLayers;
     ApplyInline I;
     std::memset(&I, 0, sizeof(I));
     if (use_inline) {
       std::memcpy(I.params, a->params, sizeof(float*) * (size_t)a->n_shards);
       std::memcpy(I.shard_off, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
-      if (two_means) std::memcpy(I.layer_off, a->layer_off, sizeof(uint64_t) * ((size_t)n_layers + 1));
+      if (two_means) {
+        std::memcpy(I.layer_off, a->layer_off, sizeof(uint64_t) * ((size_t)n_layers + 1));
+        std::memcpy(I.pair_off, pair_off.data(), sizeof(uint64_t) * ((size_t)n_layers + 1));
+        std::memcpy(I.layer_cols, cols.data(), sizeof(uint32_t) * (size_t)n_layers);
+      }
     } else {
       std::vector<unsigned char> blob(need, 0);
       std::memcpy(blob.data() + o_params, a->params, sizeof(float*) * (size_t)a->n_shards);
       std::memcpy(blob.data() + o_shard, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
-      if (two_means) std::memcpy(blob.data() + o_layer, a->layer_off, sizeof(uint64_t) * ((size_t)n_layers + 1));
+      if (two_means) {
+        std::memcpy(blob.data() + o_layer, a->layer_off, sizeof(uint64_t) * ((size_t)n_layers + 1));
+        std::memcpy(blob.data() + o_pair, pair_off.data(), sizeof(uint64_t) * ((size_t)n_layers + 1));
+        std::memcpy(blob.data() + o_cols, cols.data(), sizeof(uint32_t) * (size_t)n_layers);
+      }
       if (cudaMemcpyAsync(ws, blob.data(), need, cudaMemcpyHostToDevice, stream) != cudaSuccess) return GD_ERR_CUDA;
     }
     ApplyDev A;
@@ -131,6 +159,8 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
     A.params = (float* const*)(ws + o_params);
     A.shard_off = (const uint64_t*)(ws + o_shard);
     A.layer_off = (const uint64_t*)(ws + o_layer);
+    A.pair_off = (const uint64_t*)(ws + o_pair);
+    A.layer_cols = (const uint32_t*)(ws + o_cols);
     A.n_shards = a->n_shards;
     A.n_layers = n_layers;
     A.value_mode = a->value_mode;

@@ -12,7 +12,7 @@ namespace {
 // after every survivor has been written.
 __device__ void finalize_call(const DevTables& T, uint64_t k_total) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
+  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS || T.value_mode == GD_VALUES_COLUMN_MEANS;
   const bool packed = T.value_mode != GD_VALUES_FP32;
   uint32_t n_pred = 0, n_dense = 0;
   unsigned long long n_cand = 0;
@@ -53,9 +53,11 @@ __device__ void finalize_call(const DevTables& T, uint64_t k_total) {
     if (lane == 0) T.out_shard_cnt_off[j] = (uint32_t)lo;
   }
   if (two_means) {
-    for (uint32_t e = tid; e < 2 * T.n_layers; e += kThreads) {
-      const unsigned long long c = __ldcg(T.cnts + e);
-      T.out_means[e] = c ? (float)(__ldcg(T.sums + e) / (double)c) : 0.0f;
+    if (T.n_pairs <= kInlineMeansPairs) {              // otherwise a kernel of its own divides the sums
+      for (uint32_t e = tid; e < 2 * T.n_pairs; e += kThreads) {
+        const unsigned long long c = __ldcg(T.cnts + e);
+        T.out_means[e] = c ? (float)(__ldcg(T.sums + e) / (double)c) : 0.0f;
+      }
     }
   } else if (T.value_mode == GD_VALUES_THRESHOLD) {
     // every survivor of layer l stands for +-t, t = the threshold of the scope that holds the layer
@@ -91,7 +93,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   const ScopeDesc* scopes;
   const uint32_t* tile0;
   load_tables(T, LK, &s_tab, &scopes, &tile0);
-  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
+  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS || T.value_mode == GD_VALUES_COLUMN_MEANS;   // sums are kept
   const bool packed = T.value_mode != GD_VALUES_FP32;
   const uint32_t ltm = lanemask_lt();
   uint4* desc = reinterpret_cast<uint4*>(T.desc_cand);
@@ -121,8 +123,8 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
       const uint64_t i_last = T.cand_idx[d.cand_base + end - 1];
       const uint32_t l0 = range_of(T.layer_off, T.n_layers, i_first);
       const uint32_t l1 = range_of(T.layer_off, T.n_layers, i_last);
-      s_layer = l0;
-      s_single = (l0 == l1) ? 1 : 0;
+      s_layer = (uint32_t)T.pair_off[l0];              // the one pair of the tile, if it has only one
+      s_single = (l0 == l1 && T.layer_cols[l0] == 1u) ? 1 : 0;
     }
 
     // phase 1: load, classify, count
@@ -198,9 +200,9 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
               } else if (single) {
                 if (sgn) { sum_n += x; ++cnt_n; } else { sum_p += x; ++cnt_p; }
               } else {
-                const uint32_t l = range_of(T.layer_off, T.n_layers, idx);
-                atomicAdd(T.sums + 2 * (size_t)l + sgn, x);
-                atomicAdd(T.cnts + 2 * (size_t)l + sgn, 1ull);
+                const uint64_t pr = pair_of(T.layer_off, T.pair_off, T.layer_cols, T.n_layers, idx);
+                atomicAdd(T.sums + 2 * pr + sgn, x);
+                atomicAdd(T.cnts + 2 * pr + sgn, 1ull);
               }
             } else {
               T.out_idx[d.out_base + pos] = (uint32_t)idx;
@@ -272,7 +274,7 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
   const ScopeDesc* scopes;
   const uint32_t* tile0;
   load_tables(T, L_DCOMP, &s_tab, &scopes, &tile0);
-  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS;
+  const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS || T.value_mode == GD_VALUES_COLUMN_MEANS;   // sums are kept
   const bool packed = T.value_mode != GD_VALUES_FP32;
   const uint32_t ltm = lanemask_lt();
   uint4* desc = reinterpret_cast<uint4*>(T.desc_dcomp);
@@ -298,8 +300,8 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
     if (two_means && tid == 0) {
       const uint32_t l0 = range_of(T.layer_off, T.n_layers, d.lo + beg);
       const uint32_t l1 = range_of(T.layer_off, T.n_layers, d.lo + end - 1);
-      s_layer = l0;
-      s_single = (l0 == l1) ? 1 : 0;
+      s_layer = (uint32_t)T.pair_off[l0];              // the one pair of the chunk, if it has only one
+      s_single = (l0 == l1 && T.layer_cols[l0] == 1u) ? 1 : 0;
     }
 
     // phase 1: classify every element of the chunk, count per (tile, warp)
@@ -398,9 +400,9 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
                 } else if (single) {
                   if (sgn) { sum_n += x; ++cnt_n; } else { sum_p += x; ++cnt_p; }
                 } else {
-                  const uint32_t l = range_of(T.layer_off, T.n_layers, idx);
-                  atomicAdd(T.sums + 2 * (size_t)l + sgn, x);
-                  atomicAdd(T.cnts + 2 * (size_t)l + sgn, 1ull);
+                  const uint64_t pr = pair_of(T.layer_off, T.pair_off, T.layer_cols, T.n_layers, idx);
+                  atomicAdd(T.sums + 2 * pr + sgn, x);
+                  atomicAdd(T.cnts + 2 * pr + sgn, 1ull);
                 }
               } else {
                 T.out_idx[d.out_base + pos] = (uint32_t)idx;
@@ -517,6 +519,15 @@ __global__ void __launch_bounds__(kThreads) pack_sampled_kernel(const __grid_con
   finalize_call(T, count_before(T.n_scopes));
 }
 
+// Divides the accumulated sums by their counts when there are too many pairs for the finishing CTA.
+__global__ void __launch_bounds__(kThreads) means_kernel(const __grid_constant__ DevTables T) {
+  const uint64_t stride = (uint64_t)gridDim.x * kThreads;
+  for (uint64_t e = (uint64_t)blockIdx.x * kThreads + threadIdx.x; e < 2 * T.n_pairs; e += stride) {
+    const unsigned long long c = T.cnts[e];
+    T.out_means[e] = c ? (float)(T.sums[e] / (double)c) : 0.0f;
+  }
+}
+
 // Self-test kernel of the bounded waits: tile 1 waits on tile 0, which nothing publishes; tile 2
 // then meets the aborted tile 1.
 __global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(Ctl* ctl, uint4* desc, uint32_t spin_limit) {
@@ -542,6 +553,16 @@ cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, c
 cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream) {
   ProfileScope prof(stream, PT_FINALIZE);
   finalize_kernel<<<1, kThreads, 0, stream>>>(T);
+  GD_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+
+cudaError_t launch_means(const DevTables& T, cudaStream_t stream) {
+  ProfileScope prof(stream, PT_MEANS);
+  uint64_t blocks = (2 * T.n_pairs + kThreads - 1) / kThreads;
+  const uint64_t cap = (uint64_t)sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  means_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(T);
   GD_LAUNCH_CHECK();
   return cudaSuccess;
 }

@@ -20,6 +20,7 @@ constexpr int kShift0 = 20, kShift1 = 10, kShift2 = 0;
 constexpr uint32_t kHistBinsPerScope = 2 * (2048 + 1024 + 1024);   // three passes over the sample, three over the list
 constexpr uint32_t kAbsMask = 0x7FFFFFFFu;
 constexpr uint32_t kLookbackSpinLimit = 1u << 21;  // polls before a look-back wait gives up
+constexpr uint64_t kInlineMeansPairs = 2048;       // up to this many pairs the finishing CTA divides the sums itself
 
 // Kinds of tiled launches; each has its own tile -> scope table.
 enum Launch : int { L_EMIT = 0, L_SAMP = 1, L_CAND = 2, L_DSEL = 3, L_DCOMP = 4, L_COUNT = 5 };
@@ -95,8 +96,8 @@ struct DevTables {       // passed by value to every kernel
   Ctl* ctl;
   ScopeState* state;
   unsigned long long* hist;          // [n_scopes][kHistBinsPerScope]
-  double* sums;                      // [n_layers][2]
-  unsigned long long* cnts;          // [n_layers][2]
+  double* sums;                      // [n_pairs][2]
+  unsigned long long* cnts;          // [n_pairs][2]
   uint64_t* desc_emit;               // [tiles(L_EMIT)]
   uint64_t* desc_cand;               // [tiles(L_CAND)][2]
   uint64_t* desc_dcomp;              // [tiles(L_DCOMP)][2]
@@ -106,6 +107,9 @@ struct DevTables {       // passed by value to every kernel
   const uint64_t* samp_off;          // [n_scopes + 1]
   const uint64_t* layer_off;         // [n_layers + 1]
   const uint64_t* shard_off;         // [n_shards + 1]
+  const uint64_t* pair_off;          // [n_layers + 1] first (mu+, mu-) pair of each layer
+  const uint32_t* layer_cols;        // [n_layers] columns per layer (1 unless column-means mode)
+  uint64_t n_pairs;                  // pairs in total
   // buffers
   float* samp_val;
   uint32_t* cand_idx;
@@ -176,6 +180,14 @@ __device__ __forceinline__ uint32_t range_of(const uint64_t* __restrict__ off, u
   return lo;
 }
 
+// The (mu+, mu-) pair an index belongs to: its layer, or its layer and column (row-major layers).
+__device__ __forceinline__ uint64_t pair_of(const uint64_t* __restrict__ layer_off, const uint64_t* __restrict__ pair_off,
+                                            const uint32_t* __restrict__ layer_cols, uint32_t n_layers, uint64_t idx) {
+  const uint32_t l = range_of(layer_off, n_layers, idx);
+  const uint32_t cols = layer_cols[l];
+  return pair_off[l] + (cols > 1 ? (idx - layer_off[l]) % cols : 0ull);
+}
+
 // True when the scope's result comes from the candidate list the fused pass emitted: the
 // prediction was a valid lower bound (at least k candidates) and the list did not overflow.
 __device__ __forceinline__ bool predicted_ok(const DevTables& T, const ScopeDesc& d, const ScopeState& st) {
@@ -193,6 +205,7 @@ cudaError_t launch_candidate_select(const DevTables& T, const uint32_t* tiles, c
 cudaError_t launch_dense_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, bool finalize, cudaStream_t stream);
 cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream);
+cudaError_t launch_means(const DevTables& T, cudaStream_t stream);
 cudaError_t launch_pack_sampled(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream);
 int sm_count();   // multiprocessors of the current device (0 on error)
@@ -200,7 +213,7 @@ int sm_count();   // multiprocessors of the current device (0 on error)
 // Measurement hooks (gd_api.cu): count a kernel launch; record an event of the pair around the fused pass.
 void note_launches(uint32_t count);
 // Kernel tags of the measurement hooks, in the order a step launches them.
-enum ProfileTag : uint32_t { PT_SETUP = 0, PT_PACK_SAMPLED = 9, PT_SAMPLE_SELECT = 1, PT_ADD_EMIT = 2, PT_DENSE_SELECT = 3, PT_DENSE_COMPACT = 4,
+enum ProfileTag : uint32_t { PT_SETUP = 0, PT_PACK_SAMPLED = 9, PT_MEANS = 10, PT_SAMPLE_SELECT = 1, PT_ADD_EMIT = 2, PT_DENSE_SELECT = 3, PT_DENSE_COMPACT = 4,
                              PT_CAND_SELECT = 5, PT_CAND_COMPACT = 6, PT_FINALIZE = 7, PT_APPLY = 8 };
 void profile_mark(cudaStream_t stream, bool begin, uint32_t tag);
 struct ProfileScope {   // records an event pair around the launches made during its lifetime

@@ -17,7 +17,7 @@ class GradDropSession:
 
     def __init__(self, layer_off: Sequence[int], shard_off: Sequence[int], drop_ppm: int,
                  scope_mode: int = B.GD_SCOPE_GLOBAL, value_mode: int = B.GD_VALUES_FP32, flags: int = 0,
-                 device="cuda:0"):
+                 device="cuda:0", layer_cols: Optional[Sequence[int]] = None):
         self.device = torch.device(device)
         if self.device.type != "cuda":
             raise RuntimeError("GradDropSession needs a CUDA device: the library has no CPU path")
@@ -27,6 +27,8 @@ class GradDropSession:
         self.n_layers = len(self.layer_off) - 1
         self.n_shards = len(self.shard_off) - 1
         self.drop_ppm, self.scope_mode, self.value_mode, self.flags = drop_ppm, scope_mode, value_mode, flags
+        self.layer_cols = [int(c) for c in layer_cols] if value_mode == B.GD_VALUES_COLUMN_MEANS else None
+        self.n_pairs = B.gd_means_pairs(self.n_layers, self.layer_cols, value_mode)
         self.n_scopes = 1 if scope_mode == B.GD_SCOPE_GLOBAL else self.n_layers
         self.sampled = bool(flags & B.GD_FLAG_SAMPLED_THRESHOLD)
         # exact modes: the survivor count is known; sampled-threshold mode: the capacity of the outputs
@@ -38,8 +40,8 @@ class GradDropSession:
         self.out_val = torch.zeros(max(self.k_total, 1), dtype=torch.float32, device=dev)
         self.out_shard_cnt_off = torch.zeros(self.n_shards + 1, dtype=torch.int32, device=dev)
         self.out_tau = torch.zeros(self.n_scopes, dtype=torch.int32, device=dev)
-        self.out_means = torch.zeros(self.n_layers, 2, dtype=torch.float32, device=dev)
-        ws_bytes = B.gd_workspace_bytes(self.layer_off, self.n_shards, scope_mode, drop_ppm)
+        self.out_means = torch.zeros(max(self.n_pairs, 1), 2, dtype=torch.float32, device=dev)
+        ws_bytes = B.gd_workspace_bytes(self.layer_off, self.n_shards, scope_mode, drop_ppm, self.layer_cols)
         self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
         aws = B.gd_apply_workspace_bytes(self.n_shards, self.n_layers)
         self.apply_workspace = torch.empty(aws, dtype=torch.uint8, device=dev)
@@ -56,7 +58,7 @@ class GradDropSession:
             self._compress_call = B.CompressCall(
                 grad, self.residual, self.layer_off, self.shard_off, self.drop_ppm, self.scope_mode, self.value_mode,
                 self.out_idx, self.out_val, self.out_shard_cnt_off, self.out_tau, self.out_means, self.workspace,
-                self.flags)
+                self.flags, layer_cols=self.layer_cols)
         else:
             self._compress_call.set_grad(grad)
         return self._compress_call
@@ -84,7 +86,8 @@ class GradDropSession:
     def apply_call(self, params: List[torch.Tensor], alpha: float = 1.0, pushes=None) -> B.ApplyCall:
         pushes = [self.push()] if pushes is None else pushes
         lo = self.layer_off if self.value_mode != B.GD_VALUES_FP32 else None
-        return B.ApplyCall(params, self.shard_off, pushes, self.value_mode, alpha, self.apply_workspace, lo)
+        return B.ApplyCall(params, self.shard_off, pushes, self.value_mode, alpha, self.apply_workspace, lo,
+                           self.layer_cols)
 
     def apply(self, params: List[torch.Tensor], alpha: float = 1.0, stream=None) -> None:
         if self._apply_call is None or self._apply_call._keep[0] is not params:

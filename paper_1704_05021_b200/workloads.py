@@ -30,6 +30,7 @@ SCOPE_PER_LAYER = 1
 VALUES_FP32 = 0
 VALUES_TWO_MEANS = 1
 VALUES_THRESHOLD = 2
+VALUES_COLUMN_MEANS = 3
 
 _CHUNK = 1 << 24  # elements generated per call of the random generator (bounds temporaries)
 
@@ -63,6 +64,11 @@ class Workload:
     @property
     def n(self) -> int:
         return self.layer_off[-1]
+
+    @property
+    def layer_cols(self) -> List[int]:
+        """Columns of each layer seen as a row-major matrix (1 for vectors): the last dimension of its shape."""
+        return [int(shp[-1]) if len(shp) > 1 else 1 for shp in self.layer_shapes]
 
     def seed(self, step: int) -> int:
         return step if self.config == 1 else 1000 * self.config + step

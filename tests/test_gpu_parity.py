@@ -50,11 +50,12 @@ def compare_step(sess: GradDropSession, exp: dict, tag: str):
 
 def check_apply(sess: GradDropSession, exp: dict, p_before: np.ndarray, params: torch.Tensor, alpha: float, tag: str):
     push = {"idx": exp["idx"], "val": exp.get("val"), "means": exp.get("means")}
+    cols = sess.layer_cols
     got = params.cpu().numpy()
     for j in range(sess.n_shards):
         lo, hi = sess.shard_off[j], sess.shard_off[j + 1]
         ref, bound = orc.apply_pushes(p_before[lo:hi], lo, [push], alpha=alpha, value_mode=sess.value_mode,
-                                      layer_off=sess.layer_off)
+                                      layer_off=sess.layer_off, layer_cols=cols)
         err = np.abs(got[lo:hi].astype(np.float64) - ref)
         assert np.all(err <= REL_TOL * bound + 1e-45), f"{tag}: shard {j} max err {err.max()}"
         if alpha == 1.0 and sess.value_mode == B.GD_VALUES_FP32:     # one push, alpha 1: exactly fl32(p + v)
@@ -64,8 +65,10 @@ def check_apply(sess: GradDropSession, exp: dict, p_before: np.ndarray, params: 
             assert np.array_equal(got[lo:hi].view(np.uint32), want.view(np.uint32)), f"{tag}: shard {j} not exact"
 
 
-def run_steps(w, device, steps, flags=0, method="sort", grads=None, alpha=1.0, with_apply=True, expect_dense=None):
-    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, flags, device)
+def run_steps(w, device, steps, flags=0, method="sort", grads=None, alpha=1.0, with_apply=True, expect_dense=None,
+              layer_cols=None):
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, flags, device,
+                           layer_cols=layer_cols)
     r_host = orc.residual_reset(w.n)
     params = W.make_params(w, device) if with_apply else None
     views = sess.shard_views(params) if with_apply else None
@@ -73,7 +76,7 @@ def run_steps(w, device, steps, flags=0, method="sort", grads=None, alpha=1.0, w
         g = grads[step].to(device) if grads is not None else W.make_gradient(w, step, device)
         g_host = g.cpu().numpy()
         exp = orc.compress(g_host, r_host, w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
-                           method=method)
+                           method=method, layer_cols=layer_cols)
         g_before = g.clone()
         sess.compress(g)
         tag = f"{w.name} step {step} flags {flags}"
@@ -529,3 +532,23 @@ def test_more_than_2_31_elements(cuda_device):
         bounds = torch.tensor(w.shard_off, device=cuda_device)
         assert torch.equal(torch.searchsorted(idx, bounds).to(torch.int32), sess.out_shard_cnt_off)
         del r_before
+
+
+# ---------------------------------------------------------------- column-wise averages (Section 5.4)
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
+@pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
+def test_column_means_small_matrices(cuda_device, flags, scope_mode):
+    shapes = [(300, 40), (17,), (64, 500), (1, 33), (2000, 3)]
+    sizes = [int(np.prod(s_)) for s_ in shapes]
+    cols = [s_[-1] if len(s_) > 1 else 1 for s_ in shapes]
+    rng = np.random.default_rng(88)
+    w = W.small_layered(len(sizes), sizes, 950_000, scope_mode, B.GD_VALUES_COLUMN_MEANS, 3)
+    grads = [torch.from_numpy(rng.laplace(0, 1e-3, w.n).astype(np.float32)) for _ in range(2)]
+    run_steps(w, cuda_device, 2, flags=flags, grads=grads, layer_cols=cols, alpha=0.5)
+
+
+def test_column_means_on_the_nmt_shapes(cuda_device):
+    w = W.workload(4)
+    w.value_mode = B.GD_VALUES_COLUMN_MEANS
+    sess = run_steps(w, cuda_device, 1, method="select", layer_cols=w.layer_cols)
+    assert sess.n_pairs == sum(w.layer_cols) == 500 + 500 + 85000 + 1 + 8 * 1000

@@ -485,3 +485,41 @@ def test_sampled_threshold_keeps_about_the_requested_fraction():
     assert abs(frac - 0.01) < 6 * 0.01 / math.sqrt(k_m)        # sampling error of a quantile from k_m tail samples
     assert np.array_equal(out["val"], g[out["idx"]])
     assert not out["residual"][out["idx"]].any()
+
+
+# ---------------------------------------------------------------- column-wise averages (Section 5.4)
+def test_column_means_by_hand_and_against_two_means():
+    # one 3 x 4 matrix (row-major) followed by a vector of 4; keep 6 of 12 and 2 of 4
+    m = np.array([[4.0, -1.0, 0.5, 6.0],
+                  [-5.0, 0.25, 3.0, -0.125],
+                  [7.0, -8.0, 0.0625, -9.0]], dtype=np.float32)
+    vec = np.array([0.5, -2.0, 3.0, 0.25], dtype=np.float32)
+    g = np.concatenate([m.ravel(), vec])
+    r = np.full(g.shape[0], -0.0, np.float32)
+    layer_off, cols = [0, 12, 16], [4, 1]
+    out = orc.compress(g, r, layer_off, [0, 16], 500_000, scope_mode=orc.SCOPE_PER_LAYER,
+                       value_mode=orc.VALUES_COLUMN_MEANS, layer_cols=cols)
+    # matrix keeps |.| in {9, 8, 7, 6, 5, 4}: col 0: 4, -5, 7 ; col 1: -8 ; col 2: none ; col 3: 6, -9.  vector keeps 3, -2
+    assert (out["idx"] & np.uint32(0x7FFFFFFF)).tolist() == [0, 3, 4, 8, 9, 11, 13, 14]
+    want = [[5.5, -5.0], [0.0, -8.0], [0.0, 0.0], [6.0, -9.0], [3.0, -2.0]]
+    assert out["means"].tolist() == want
+    assert out["counts"].tolist() == [[2, 1], [0, 1], [0, 0], [1, 1], [1, 1]]
+    pos, val = orc.decode_push(out["idx"], None, orc.VALUES_COLUMN_MEANS, out["means"], layer_off, cols)
+    assert val.tolist() == [5.5, 6.0, -5.0, 5.5, -8.0, -9.0, -2.0, 3.0]
+    # with one column per layer the pairs are the two-means pairs
+    rng = np.random.default_rng(77)
+    g2 = rng.laplace(0, 1e-3, 16).astype(np.float32)
+    a = orc.compress(g2, r, layer_off, [0, 16], 500_000, value_mode=orc.VALUES_COLUMN_MEANS, layer_cols=[1, 1])
+    b = orc.compress(g2, r, layer_off, [0, 16], 500_000, value_mode=orc.VALUES_TWO_MEANS)
+    assert np.array_equal(a["means"], b["means"]) and np.array_equal(a["idx"], b["idx"])
+    # a column mean never leaves the range of the values it stands for
+    big = rng.standard_normal(40 * 25).astype(np.float32)
+    o = orc.compress(big, np.full(1000, -0.0, np.float32), [0, 1000], [0, 1000], 800_000,
+                     value_mode=orc.VALUES_COLUMN_MEANS, layer_cols=[25])
+    pos, val = orc.decode_push(o["idx"], None, orc.VALUES_COLUMN_MEANS, o["means"], [0, 1000], [25])
+    for c in range(25):
+        for sg, sel in ((0, big[pos] >= 0), (1, big[pos] < 0)):
+            mine = big[pos][(pos % 25 == c) & sel]
+            if mine.size:
+                assert mine.min() - 1e-6 <= o["means"][c, sg] <= mine.max() + 1e-6
+                assert abs(float(o["means"][c, sg]) - math.fsum(float(x) for x in mine) / mine.size) <= 1e-6 * abs(float(o["means"][c, sg]))
