@@ -274,7 +274,7 @@ int gd_step_host(const gd_compress_args* args, const gd_apply_args* apply, const
  *     GD_STATIC_WORKSPACE_BYTES of device memory until the process exits, used or not;
  *   - a call whose gd_workspace_bytes() exceeds GD_STATIC_WORKSPACE_BYTES is refused with
  *     GD_ERR_TOO_LARGE before anything is enqueued (as a guide: one flat scope of 2^24 elements at a
- *     99 % drop ratio needs about 7.4 MiB);
+ *     99 % drop ratio needs about 5.4 MiB, 2^25 elements about 10.6 MiB);
  *   - the first call on each device looks up the scratch area's device address (once per device, with
  *     that device current); make that first call outside any stream capture;
  *   - no device memory is allocated or freed, here or in anything this entry point calls;

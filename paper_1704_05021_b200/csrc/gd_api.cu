@@ -36,7 +36,7 @@ void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint6
   if (mt * 2 >= ns) {
     *m = ns;
     *rank = k;
-    uint64_t c = 2 * k + 1024;
+    uint64_t c = 3 * k + 1024;
     *cap = c < ns ? c : ns;
     return;
   }
@@ -47,7 +47,7 @@ void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint6
   if (r > mt) r = mt;
   if (r < 1) r = 1;
   *rank = r;
-  uint64_t c = 2 * k + 128 * (ns / mt) + 1024;
+  uint64_t c = 3 * k + 128 * (ns / mt) + 1024;
   *cap = c < ns ? c : ns;
 }
 
