@@ -552,3 +552,45 @@ def test_column_means_on_the_nmt_shapes(cuda_device):
     w.value_mode = B.GD_VALUES_COLUMN_MEANS
     sess = run_steps(w, cuda_device, 1, method="select", layer_cols=w.layer_cols)
     assert sess.n_pairs == sum(w.layer_cols) == 500 + 500 + 85000 + 1 + 8 * 1000
+
+
+# ---------------------------------------------------------------- randomised layouts
+@pytest.mark.parametrize("seed", range(12))
+def test_random_layouts_and_modes(cuda_device, seed):
+    """Random layer structures (tiny, empty, unaligned, large), drop ratios, scopes, value modes, shard counts and
+    value distributions, three steps each with the residual carried; everything compared with the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    n_layers = int(rng.integers(1, 9))
+    sizes = []
+    for _ in range(n_layers):
+        kind = rng.integers(0, 5)
+        sizes.append(int([0, rng.integers(1, 40), rng.integers(40, 5000), rng.integers(5000, 70_000),
+                          rng.integers(70_000, 400_000)][kind]))
+    if sum(sizes) == 0:
+        sizes[0] = 1234
+    ppm = int(rng.choice([0, 300_000, 900_000, 984_000, 990_000, 999_000, 999_999, 1_000_000]))
+    scope_mode = int(rng.integers(0, 2))
+    value_mode = int(rng.choice([B.GD_VALUES_FP32, B.GD_VALUES_TWO_MEANS, B.GD_VALUES_THRESHOLD, B.GD_VALUES_COLUMN_MEANS]))
+    flags = int(rng.choice([0, 0, B.GD_FLAG_NO_PREDICTION]))
+    shards = int(rng.integers(1, 7))
+    cols = None
+    if value_mode == B.GD_VALUES_COLUMN_MEANS:
+        cols = []
+        for s_ in sizes:
+            divs = [c for c in (1, 2, 3, 5, 8, 16, 50, 64) if s_ % c == 0] or [1]
+            cols.append(int(rng.choice(divs)))
+    w = W.small_layered(n_layers, sizes, ppm, scope_mode, value_mode, shards)
+    dist = int(rng.integers(0, 4))
+    grads = []
+    for _ in range(3):
+        if dist == 0:
+            g = rng.laplace(0, 1e-3, w.n)
+        elif dist == 1:
+            g = rng.standard_normal(w.n) * 10.0 ** rng.integers(-6, 1, w.n)
+        elif dist == 2:
+            g = np.where(rng.random(w.n) < 0.02, rng.standard_normal(w.n), 0.0)         # mostly exact zeros
+        else:
+            g = rng.choice(np.array([0.0, 0.25, -0.25, 0.5, 1.0, -2.0]), w.n)           # few distinct values
+        grads.append(torch.from_numpy(g.astype(np.float32)))
+    run_steps(w, cuda_device, 3, flags=flags, grads=grads, layer_cols=cols,
+              alpha=float(rng.choice([1.0, 0.5, -1.25])))
