@@ -160,8 +160,8 @@ typedef struct gd_compress_args {
   int32_t scope_mode;         /* GD_SCOPE_* */
   int32_t value_mode;         /* GD_VALUES_* */
   uint32_t flags;             /* GD_FLAG_* */
-  uint32_t* out_idx;          /* device, gd_total_kept() words */
-  float* out_val;             /* device, gd_total_kept() fp32; may be NULL in two-means mode */
+  uint32_t* out_idx;          /* device, gd_total_kept() words (gd_sampled_capacity() in sampled-threshold mode) */
+  float* out_val;             /* device, as many fp32; may be NULL in the packed modes */
   uint32_t* out_shard_cnt_off;/* device, n_shards + 1 words */
   uint32_t* out_tau;          /* device, one word per scope (1, or n_layers); may be NULL */
   float* out_means;           /* device, gd_means_pairs() x 2 fp32 (mu+, mu-); the packed modes */
