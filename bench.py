@@ -214,6 +214,11 @@ def run_cuda(args):
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    from paper_1704_05021_b200 import build as gd_build
+    if rank == 0:
+        gd_build.build_library()          # no-op when libgd.so is up to date; there is no other code path
+    if world > 1:
+        dist.barrier()
     B.load_library()
 
     w = W.workload(args.config, scale_log2=args.scale_log2) if args.scale_log2 else W.workload(args.config)

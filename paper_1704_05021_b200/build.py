@@ -36,7 +36,13 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     """Compiles the CUDA sources into paper_1704_05021_b200/libgd.so and returns its path."""
     if not force and not needs_build():
         return LIB_PATH
-    cmd = [_nvcc(), *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC]
+    try:
+        nvcc = _nvcc()
+    except RuntimeError:
+        if not force and os.path.exists(LIB_PATH):
+            return LIB_PATH          # no compiler here: use the library that was built with the sources
+        raise
+    cmd = [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB_PATH]

@@ -18,3 +18,10 @@ def cuda_device():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     return torch.device("cuda:0")
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_library():
+    """libgd.so is built in-tree before any test needs it (a no-op when it is up to date)."""
+    from paper_1704_05021_b200 import build as gd_build
+    return gd_build.build_library()
