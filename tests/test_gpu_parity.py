@@ -594,3 +594,23 @@ def test_random_layouts_and_modes(cuda_device, seed):
         grads.append(torch.from_numpy(g.astype(np.float32)))
     run_steps(w, cuda_device, 3, flags=flags, grads=grads, layer_cols=cols,
               alpha=float(rng.choice([1.0, 0.5, -1.25])))
+
+
+def test_config5_full_scale_against_the_oracle(cuda_device):
+    """One step of workload 5 at its full 2^30 elements, compared with the oracle itself (selection on the
+    composite keys: tens of GB of host memory, about a minute of host time)."""
+    import psutil
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * (1 << 30) or psutil.virtual_memory().available < 90 * (1 << 30):
+        pytest.skip("needs 40 GiB of device memory and 90 GiB of host memory")
+    w = W.workload(5)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
+    g = W.make_gradient(w, 0, cuda_device)
+    r0 = W.make_gradient(w, 7, cuda_device) * 0.25                 # a non-trivial residual to start from
+    sess.residual.copy_(r0)
+    exp = orc.compress(g.cpu().numpy(), r0.cpu().numpy(), w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode,
+                       method="select")
+    del r0
+    sess.compress(g)
+    compare_step(sess, exp, "workload 5, 2^30 elements, oracle")
+    assert sess.stats()["n_scopes_dense"] == 0
