@@ -16,6 +16,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Sample size per scope: kSampleFactor expected samples above the threshold, within [min, max].
 constexpr double kSampleFactor = 256.0, kSampleMin = 16384.0, kSampleMax = 262144.0;
+constexpr uint64_t kAutoDenseMax = 1ull << 21;   // vectors up to this length skip the prediction (measured crossover: 2^22)
 
 inline uint64_t kept_count(uint64_t n, uint32_t drop_ppm) {
   return n - (n * (uint64_t)drop_ppm) / 1000000ull;   // n <= 2^32, drop_ppm <= 1e6: no overflow
@@ -69,7 +70,8 @@ struct Plan {
   uint32_t tiles[L_COUNT] = {0, 0, 0, 0, 0};
   uint64_t samp_total = 0, cand_total = 0, k_total = 0;
   uint32_t n_scopes = 0;
-  uint32_t emit_chunk_tiles = 1;
+  bool predict = true;
+  uint32_t emit_chunk_tiles = 1, dense_sel_tile = kDenseSelTileMax, dense_chunk_tiles = kDenseChunkTilesMax;
   // workspace layout (byte offsets)
   size_t off_ctl = 0, off_state = 0, off_hist = 0, off_sums = 0, off_cnts = 0, off_desc_emit = 0,
          off_desc_cand = 0, off_desc_dcomp = 0, zero_bytes = 0;
@@ -100,8 +102,11 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
   if (n_shards == 0 || drop_ppm > 1000000u) return GD_ERR_INVALID_ARG;
   if (scope_mode != GD_SCOPE_GLOBAL && scope_mode != GD_SCOPE_PER_LAYER) return GD_ERR_INVALID_ARG;
   if (n > (1ull << 32)) return GD_ERR_TOO_LARGE;
-  const bool predict = !(flags & GD_FLAG_NO_PREDICTION);
   const bool sampled = (flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
+  // Short vectors are selected densely right away: below about 2^21 elements the three dense passes
+  // run out of L2 and cost less than sampling, predicting and selecting among candidates.
+  const bool predict = !(flags & GD_FLAG_NO_PREDICTION) && (sampled || n > kAutoDenseMax);
+  P->predict = predict;
   P->pair_off.assign((size_t)n_layers + 1, 0);
   P->layer_cols.assign(n_layers, 1);
   for (uint32_t l = 0; l < n_layers; ++l) {
@@ -119,6 +124,14 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
   while (chunk_tiles > 1 && dense_tiles < (uint64_t)chunk_tiles * 2368u) chunk_tiles >>= 1;
   P->emit_chunk_tiles = chunk_tiles;
   const uint64_t CH = (uint64_t)chunk_tiles * kTile;
+  // The dense kernels (used when a prediction fails) take large tiles on long vectors, where the
+  // chain of look-backs and the flushes of histograms must stay rare, and small ones on short
+  // vectors, which otherwise would not fill the GPU.
+  uint32_t sel_tile = kDenseSelTileMax, dchunk = kDenseChunkTilesMax;
+  while (sel_tile > kTile && n / sel_tile < 592u) sel_tile >>= 1;
+  while (dchunk > 1 && n / ((uint64_t)dchunk * kTile) < 888u) dchunk >>= 1;
+  P->dense_sel_tile = sel_tile;
+  P->dense_chunk_tiles = dchunk;
   const uint32_t ns_count = scope_mode == GD_SCOPE_GLOBAL ? 1u : n_layers;
   P->n_scopes = ns_count;
   P->scopes.resize(ns_count);
@@ -153,8 +166,8 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
     P->samp_off[s] = d.samp_base;
     if (ns) {
       tiles[L_EMIT] += (d.hi + CH - 1) / CH - d.lo / CH;
-      tiles[L_DSEL] += (ns + kDenseSelTile - 1) / kDenseSelTile;
-      tiles[L_DCOMP] += (ns + kDenseChunkTiles * kTile - 1) / (kDenseChunkTiles * kTile);
+      tiles[L_DSEL] += (ns + sel_tile - 1) / sel_tile;
+      tiles[L_DCOMP] += (ns + (uint64_t)dchunk * kTile - 1) / ((uint64_t)dchunk * kTile);
     }
     tiles[L_SAMP] += (m + kTile - 1) / kTile;
     tiles[L_CAND] += (cap + kTile - 1) / kTile;
@@ -421,11 +434,13 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     T.n_scopes = P.n_scopes;
     T.n_layers = a->n_layers;
     T.n_shards = a->n_shards;
-    T.flags = a->flags;
+    T.flags = P.predict ? a->flags : (a->flags | GD_FLAG_NO_PREDICTION);
     T.value_mode = a->value_mode;
     T.k_total = P.k_total;
     T.emit_chunk_tiles = P.emit_chunk_tiles;
     T.sample_passes = sampled ? 3u : 2u;
+    T.dense_sel_tile = P.dense_sel_tile;
+    T.dense_chunk_tiles = P.dense_chunk_tiles;
     if (sampled) T.k_total = P.cand_total;   // capacity of the outputs; the count is found on the device
     T.ctl = (Ctl*)(ws + P.off_ctl);
     T.state = (ScopeState*)(ws + P.off_state);
@@ -461,7 +476,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
       if (launch_pack_sampled(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
       return GD_OK;
     }
-    const bool predict = !(a->flags & GD_FLAG_NO_PREDICTION);
+    const bool predict = P.predict;
     if (predict && launch_sample_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
     if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
     // The dense kernels are always enqueued: they return at once unless a prediction failed.  The

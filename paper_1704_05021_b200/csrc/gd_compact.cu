@@ -251,13 +251,14 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
 }
 
 // Compaction over the dense range itself, for scopes whose prediction failed.  Same placement rule
-// as above, but one ticket covers a chunk of kDenseChunkTiles tiles (512 KiB of values) and the chunk does
+// as above, but one ticket covers a chunk of up to 32 tiles (512 KiB of values on long vectors) and the chunk does
 // one look-back: at 4 bytes per element the chain of look-backs would otherwise have to advance about a
 // hundred tiles per microsecond, which the L2 round trips between CTAs cannot sustain.
 // The classification masks stay in registers; the values of the (few) survivors are read again.
 __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid_constant__ DevTables T,
                                                                     uint32_t total_chunks, int do_finalize) {
-  constexpr int CD = (int)kDenseChunkTiles;
+  constexpr int CD = (int)kDenseChunkTilesMax;   // shared arrays are sized for the largest chunk
+  const int cd = (int)T.dense_chunk_tiles;        // tiles per chunk in this call
   constexpr int ROUNDS = kTile / kThreads;   // 16 elements per thread and tile
   constexpr int E = CD * kWarps;             // (tile, warp) counters of one chunk: 32
   __shared__ uint32_t s_chunk;
@@ -292,8 +293,9 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
     const uint32_t first = tile0[s];
     const uint32_t lt = t - first;
     const uint64_t len = d.hi - d.lo;
-    const uint64_t beg = (uint64_t)lt * (CD * kTile);
-    const uint64_t end = (beg + CD * kTile < len) ? beg + CD * kTile : len;
+    const uint64_t span = (uint64_t)cd * kTile;
+    const uint64_t beg = (uint64_t)lt * span;
+    const uint64_t end = (beg + span < len) ? beg + span : len;
     const float* vals = T.residual + d.lo;
     const uint32_t tau = st->tau;
     const uint64_t q = st->q;
@@ -307,7 +309,7 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
     // phase 1: classify every element of the chunk, count per (tile, warp)
 #pragma unroll 2
     for (int c = 0; c < CD; ++c) {
-      if (beg + (uint64_t)c * kTile >= end) {       // the scope ends inside this chunk (uniform over the CTA)
+      if (c >= cd || beg + (uint64_t)c * kTile >= end) {   // past the chunk, or the scope ends inside it (uniform)
         s_mask[c][tid] = 0;
         if (lane == 0) { s_cg[c * kWarps + warp] = 0; s_ce[c * kWarps + warp] = 0; }
         continue;
@@ -373,7 +375,7 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
     uint32_t cnt_p = 0, cnt_n = 0;
     bool bad = false;
 #pragma unroll 1
-    for (int c = 0; c < CD; ++c) {
+    for (int c = 0; c < cd; ++c) {
       const uint32_t m = s_mask[c][tid];
       if (!__any_sync(0xFFFFFFFFu, m != 0u)) continue;
       const uint64_t wbeg = beg + (uint64_t)c * kTile + (uint64_t)warp * (32u * ROUNDS) + lane;

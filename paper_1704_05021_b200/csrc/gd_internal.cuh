@@ -12,8 +12,8 @@ namespace gd {
 constexpr int kThreads = 256;           // threads per CTA in every tiled kernel
 constexpr int kWarps = kThreads / 32;
 constexpr uint32_t kTile = 4096;        // elements per tile of the streaming kernels
-constexpr uint32_t kDenseSelTile = 32768;  // elements per CTA in the dense histogram passes
-constexpr uint32_t kDenseChunkTiles = 32;  // tiles per ticket (and per look-back) in the dense compaction
+constexpr uint32_t kDenseSelTileMax = 32768;  // most elements per tile in the dense histogram passes
+constexpr uint32_t kDenseChunkTilesMax = 32;  // most tiles per ticket (and per look-back) in the dense compaction
 constexpr int kRadixBits0 = 11;         // 31-bit magnitude key = 11 + 10 + 10 bits
 constexpr int kRadixBins0 = 1 << kRadixBits0;
 constexpr int kShift0 = 20, kShift1 = 10, kShift2 = 0;
@@ -90,6 +90,8 @@ struct DevTables {       // passed by value to every kernel
   int32_t value_mode;
   uint32_t emit_chunk_tiles;         // tiles of kTile elements one CTA of the fused pass streams (1, 2, 4 or 8)
   uint32_t sample_passes;            // radix passes over the sample: 2 (prediction, 21 bits) or 3 (sampled-threshold mode)
+  uint32_t dense_sel_tile;           // elements per tile of the dense selection (4096 .. 32768, by vector length)
+  uint32_t dense_chunk_tiles;        // tiles per chunk of the dense compaction (1 .. 32, by vector length)
   uint32_t pad1;
   uint64_t k_total;
   // zeroed region

@@ -97,7 +97,13 @@ def run_steps(w, device, steps, flags=0, method="sort", grads=None, alpha=1.0, w
 # ---------------------------------------------------------------- workload 1: 2^20 flat, 5 steps
 @pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
 def test_config1_five_steps(cuda_device, flags):
-    run_steps(W.workload(1), cuda_device, 5, flags=flags, expect_dense=bool(flags))
+    run_steps(W.workload(1), cuda_device, 5, flags=flags, expect_dense=True)     # short vectors are selected densely
+
+
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
+def test_config1_shape_at_2_23(cuda_device, flags):
+    """The same distribution just above the length where the prediction is switched on."""
+    run_steps(W.workload(1, scale_log2=23), cuda_device, 3, flags=flags, method="select", expect_dense=bool(flags))
 
 
 # ---------------------------------------------------------------- edge sizes and drop ratios
