@@ -133,8 +133,9 @@ int gd_means_pairs(uint32_t n_layers, const uint32_t* layer_cols, int value_mode
  *   sampled-threshold mode (GD_FLAG_SAMPLED_THRESHOLD; Section 4, fourth paragraph: "We sample 0.1% of
  *              the gradient and obtain the threshold by running selection on the samples"): per scope,
  *              m = n_s if n_s <= 4096, else max(4096, ceil(n_s / 1000)) positions are sampled, one in each
- *              of m equal strata (position of sample i of scope s: a + (h mod (b - a)), a = floor(i n_s / m),
- *              b = floor((i + 1) n_s / m), h = mix(i * 0x9E3779B9 + s) in 32-bit arithmetic with
+ *              of m strata (with w = floor(n_s / m) and rem = n_s mod m, stratum i starts at
+ *              a = i w + min(i, rem) and has w + 1 elements if i < rem, else w; sample i of scope s is at
+ *              a + (h mod width), h = mix(i * 0x9E3779B9 + s) in 32-bit arithmetic with
  *              mix(x): x ^= x >> 16; x *= 0x7FEB352D; x ^= x >> 15; x *= 0x846CA68B; x ^= x >> 16);
  *              the threshold key t is the (m - floor(m * drop_ppm / 1e6))-th largest sample key and EVERY
  *              entry of the scope with key >= t is kept, so the number of survivors varies: out_idx and

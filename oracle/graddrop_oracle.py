@@ -114,17 +114,19 @@ def _mix32(x: np.ndarray) -> np.ndarray:
 def sampled_positions(lo: int, hi: int, scope_index: int) -> np.ndarray:
     """Positions read by the sampled-threshold mode in scope [lo, hi) (Section 4: "We sample 0.1% of the gradient").
 
-    m = n_s if n_s <= 4096 else max(4096, ceil(n_s / 1000)); the scope is cut into m strata
-    [floor(i n_s / m), floor((i + 1) n_s / m)) and stratum i contributes the position
-    a + (mix32(i * 0x9E3779B9 + scope_index) mod width).  The rule is part of this mode's definition,
-    which is why the CUDA library restates it; nothing else is shared.
+    m = n_s if n_s <= 4096 else max(4096, ceil(n_s / 1000)); the scope is cut into m strata, the first
+    (n_s mod m) of floor(n_s / m) + 1 elements and the rest of floor(n_s / m), and stratum i contributes
+    the position  start_i + (mix32(i * 0x9E3779B9 + scope_index) mod width_i).  The rule is part of this
+    mode's definition, which is why the CUDA library restates it; nothing else is shared.
     """
     ns = hi - lo
     m = ns if ns <= 4096 else max(4096, -(-ns // 1000))
+    if m == 0:
+        return np.empty(0, dtype=np.int64)
+    w, rem = ns // m, ns % m
     i = np.arange(m, dtype=np.uint64)
-    a = (i * np.uint64(ns)) // np.uint64(max(m, 1))
-    b = ((i + np.uint64(1)) * np.uint64(ns)) // np.uint64(max(m, 1))
-    width = b - a
+    a = i * np.uint64(w) + np.minimum(i, np.uint64(rem))
+    width = np.uint64(w) + (i < np.uint64(rem)).astype(np.uint64)
     with np.errstate(over="ignore"):
         h = _mix32((i.astype(np.uint32) * np.uint32(0x9E3779B9) + np.uint32(scope_index)).astype(np.uint32))
     off = np.where(width > 1, h.astype(np.uint64) % np.maximum(width, np.uint64(1)), np.uint64(0))

@@ -161,6 +161,8 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
     d.samp_base = samp_base;
     d.samp_m = m;
     d.samp_rank = rank;
+    d.samp_w = m ? ns / m : 0;
+    d.samp_rem = m ? ns % m : 0;
     samp_base += m;
     for (int l = 0; l < L_COUNT; ++l) P->tile0[l][s] = (uint32_t)tiles[l];
     P->samp_off[s] = d.samp_base;

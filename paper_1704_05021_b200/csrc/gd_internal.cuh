@@ -46,6 +46,8 @@ struct ScopeDesc {       // built on the host for every call, read-only on the d
   uint64_t samp_base;    // first slot of the scope in the sample buffer
   uint64_t samp_m;       // samples drawn from the scope
   uint64_t samp_rank;    // the prediction is the samp_rank-th largest sample key
+  uint64_t samp_w;       // floor(n_s / samp_m): width of a stratum (the first samp_rem strata are one wider)
+  uint64_t samp_rem;     // n_s mod samp_m
 };
 
 struct SelState {        // running state of one radix selection

@@ -49,12 +49,12 @@ __device__ bool grid_barrier(uint32_t* counter, uint32_t& phase, Ctl* ctl) {
   return s_pass != 0;
 }
 
-// The value of sample i: stratum li of scope s covers [a, b) of the scope and one position inside it
+// The value of sample li of scope s: the scope is cut into m strata and one position inside stratum li
 // is read.  The sample only steers the prediction; any sample gives the same final result.
 __device__ __forceinline__ float sample_value(const DevTables& T, const ScopeDesc& d, uint32_t s, uint64_t li) {
-  const uint64_t ns = d.hi - d.lo, m = d.samp_m;
-  const uint64_t a = (li * ns) / m, b = ((li + 1) * ns) / m;
-  const uint64_t width = b - a;
+  // m strata: the first (n_s mod m) have floor(n_s / m) + 1 elements, the others floor(n_s / m)
+  const uint64_t a = li * d.samp_w + (li < d.samp_rem ? li : d.samp_rem);
+  const uint32_t width = (uint32_t)d.samp_w + (li < d.samp_rem ? 1u : 0u);
   uint64_t pos = d.lo + a;
   if (width > 1) pos += mix32((uint32_t)li * 0x9E3779B9u + s) % width;
   return T.delta_base ? __fsub_rn(__ldg(T.grad + pos), T.delta_base[pos]) : __fadd_rn(__ldg(T.grad + pos), T.residual[pos]);
@@ -162,9 +162,16 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
   const ScopeDesc* scopes;
   const uint32_t* tile0;
   load_tables(T, LK, &s_tab, &scopes, &tile0);
+  // Each CTA takes a contiguous run of tiles (one flush of its histogram, and one pass over the finished
+  // histograms, per scope it touches), except for a single list: its tiles beyond its length (the capacity
+  // is a multiple of what it holds) are empty, and dealing the tiles out round-robin spreads the real ones
+  // over all CTAs.  (With several scopes, round-robin and block-cyclic splits were measured and lose more
+  // to the extra scope changes than they gain in balance.)
+  const bool round_robin = VIEW != V_DENSE && T.n_scopes == 1u;
   const uint32_t per = (total_tiles + gridDim.x - 1) / gridDim.x;
-  const uint32_t t_beg = blockIdx.x * per;
-  const uint32_t t_end = (t_beg + per < total_tiles) ? t_beg + per : total_tiles;
+  const uint32_t t_beg = round_robin ? blockIdx.x : blockIdx.x * per;
+  const uint32_t t_end = round_robin ? total_tiles : ((t_beg + per < total_tiles) ? t_beg + per : total_tiles);
+  const uint32_t t_step = round_robin ? gridDim.x : 1u;
   uint32_t phase = 0;
 
   for (int pass = 0; pass <= PASSES; ++pass) {
@@ -181,7 +188,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
     uint64_t len = 0;
     uint32_t prefix = 0;
     const float* vals = nullptr;
-    for (uint32_t t = t_beg; t < t_end; ++t) {
+    for (uint32_t t = t_beg; t < t_end; t += t_step) {
       const uint32_t s = (seen != NONE && t < tile0[seen + 1]) ? seen : scope_of_tile(tile0, T.n_scopes, t);
       const ScopeDesc& d = scopes[s];
       const uint32_t lt = t - tile0[s];

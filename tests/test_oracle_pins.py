@@ -442,9 +442,14 @@ def test_sampled_positions_are_one_per_stratum():
         pos = orc.sampled_positions(lo, hi, si)
         m = ns if ns <= 4096 else max(4096, -(-ns // 1000))
         assert pos.shape[0] == m
+        w_, rem = ns // m, ns % m
+        starts = [0]
+        for i in range(m):                                      # strata laid end to end: rem wide ones, then the rest
+            starts.append(starts[-1] + w_ + (1 if i < rem else 0))
+        assert starts[-1] == ns
         for i in (0, 1, m // 2, m - 1):                         # pure-Python restatement on a few strata
-            a, b = (i * ns) // m, ((i + 1) * ns) // m
-            want = lo + a + (_mix32_py(i * 0x9E3779B9 + si) % (b - a) if b - a > 1 else 0)
+            width = starts[i + 1] - starts[i]
+            want = lo + starts[i] + (_mix32_py(i * 0x9E3779B9 + si) % width if width > 1 else 0)
             assert int(pos[i]) == want
         assert np.all(np.diff(pos) > 0) and pos[0] >= lo and pos[-1] < hi      # distinct, ordered, in range
     assert orc.sampled_positions(3, 3 + 4096, 0).tolist() == list(range(3, 3 + 4096))   # small scopes: everything
