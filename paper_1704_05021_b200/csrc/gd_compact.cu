@@ -97,6 +97,23 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   const bool packed = T.value_mode != GD_VALUES_FP32;
   const uint32_t ltm = lanemask_lt();
   uint4* desc = reinterpret_cast<uint4*>(T.desc_cand);
+  // The lists' capacities are a multiple of what they hold.  With few scopes only the tiles that hold
+  // candidates are numbered (in list order), so that no ticket is spent on an empty tile.
+  __shared__ uint32_t s_vt0[kSmemScopes + 1];
+  const bool compacted = T.n_scopes <= kSmemScopes;
+  if (compacted) {
+    __syncthreads();                       // the table copy is complete
+    if (tid < T.n_scopes) {                 // one thread per scope reads its count, then a short serial prefix
+      const ScopeState* sx = T.state + tid;
+      s_vt0[tid + 1] = predicted_ok(T, scopes[tid], *sx) ? (uint32_t)((sx->cand_count + kTile - 1) / kTile) : 0u;
+    }
+    if (tid == 0) s_vt0[0] = 0;
+    __syncthreads();
+    if (tid == 0)
+      for (uint32_t x = 0; x < T.n_scopes; ++x) s_vt0[x + 1] += s_vt0[x];
+    __syncthreads();
+    total_tiles = s_vt0[T.n_scopes];
+  }
 
   for (;;) {
     __syncthreads();                       // previous tile is done with the shared variables
@@ -104,11 +121,18 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
     __syncthreads();
     const uint32_t t = s_tile;
     if (t >= total_tiles) break;
-    const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
+    uint32_t s, first;
+    if (compacted) {
+      s = 0;
+      while (t >= s_vt0[s + 1]) ++s;
+      first = s_vt0[s];
+    } else {
+      s = scope_of_tile(tile0, T.n_scopes, t);
+      first = tile0[s];
+    }
     const ScopeDesc& d = scopes[s];
     const ScopeState* st = T.state + s;
     if (!predicted_ok(T, d, *st)) continue;         // the dense kernels own this scope
-    const uint32_t first = tile0[s];
     const uint32_t lt = t - first;
     const uint64_t len = st->cand_count;
     const uint64_t beg = (uint64_t)lt * kTile;

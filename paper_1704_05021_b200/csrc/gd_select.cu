@@ -172,6 +172,27 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
   const uint32_t t_beg = round_robin ? blockIdx.x : blockIdx.x * per;
   const uint32_t t_end = round_robin ? total_tiles : ((t_beg + per < total_tiles) ? t_beg + per : total_tiles);
   const uint32_t t_step = round_robin ? gridDim.x : 1u;
+  // Several candidate lists: their capacities are a multiple of what they hold, so only the tiles that
+  // hold candidates are numbered (in list order) and split evenly, a contiguous run per CTA.
+  __shared__ uint32_t s_vt0[kSmemScopes + 1];
+  const bool compacted = VIEW == V_CAND && T.n_scopes > 1u && T.n_scopes <= kSmemScopes;
+  uint32_t v_beg = 0, v_end = 0;
+  if (compacted) {
+    __syncthreads();                                    // the table copy is complete
+    if (tid < T.n_scopes) {                 // one thread per scope reads its count, then a short serial prefix
+      const ScopeState* sx = T.state + tid;
+      s_vt0[tid + 1] = predicted_ok(T, scopes[tid], *sx) ? (uint32_t)((sx->cand_count + kTile - 1) / kTile) : 0u;
+    }
+    if (tid == 0) s_vt0[0] = 0;
+    __syncthreads();
+    if (tid == 0)
+      for (uint32_t x = 0; x < T.n_scopes; ++x) s_vt0[x + 1] += s_vt0[x];
+    __syncthreads();
+    const uint32_t valid = s_vt0[T.n_scopes];
+    const uint32_t per_v = (valid + gridDim.x - 1) / gridDim.x;
+    v_beg = blockIdx.x * per_v;
+    v_end = (v_beg + per_v < valid) ? v_beg + per_v : valid;
+  }
   uint32_t phase = 0;
 
   for (int pass = 0; pass <= PASSES; ++pass) {
@@ -188,10 +209,17 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
     uint64_t len = 0;
     uint32_t prefix = 0;
     const float* vals = nullptr;
-    for (uint32_t t = t_beg; t < t_end; t += t_step) {
-      const uint32_t s = (seen != NONE && t < tile0[seen + 1]) ? seen : scope_of_tile(tile0, T.n_scopes, t);
+    for (uint32_t t = compacted ? v_beg : t_beg; t < (compacted ? v_end : t_end); t += (compacted ? 1u : t_step)) {
+      uint32_t s, lt;
+      if (compacted) {                                  // t numbers the tiles that hold candidates
+        s = seen != NONE ? seen : 0u;
+        while (t >= s_vt0[s + 1]) ++s;
+        lt = t - s_vt0[s];
+      } else {
+        s = (seen != NONE && t < tile0[seen + 1]) ? seen : scope_of_tile(tile0, T.n_scopes, t);
+        lt = t - tile0[s];
+      }
       const ScopeDesc& d = scopes[s];
-      const uint32_t lt = t - tile0[s];
       if (s != seen) {                                  // per-scope values, worked out once per scope
         seen = s;
         ScopeState* st = T.state + s;
