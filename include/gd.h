@@ -46,8 +46,14 @@ enum { GD_VALUES_FP32 = 0, GD_VALUES_TWO_MEANS = 1, GD_VALUES_THRESHOLD = 2, GD_
 enum {
   GD_FLAG_NO_PREDICTION = 1u, /* do not predict the threshold from a sample: always select over the
                                  whole dense vector (same results, more memory traffic) */
-  GD_FLAG_SAMPLED_THRESHOLD = 2u /* the approximation of Section 4: the threshold is selected on a 0.1 %
+  GD_FLAG_SAMPLED_THRESHOLD = 2u, /* the approximation of Section 4: the threshold is selected on a 0.1 %
                                  sample and every entry at or above it is kept (see gd_compress) */
+  GD_FLAG_QUANT_ERROR_FEEDBACK = 4u /* 1-bit value modes only (Section 5.4).  The paper does not say whether
+                                 the error of the 1-bit quantisation is kept; Algorithm 1 keeps only the
+                                 dropped mass, which is the default here.  With this flag the residual of a
+                                 KEPT entry is v minus the fp32 value the receiver will decode for it (one
+                                 fp32 subtraction), as in the error feedback of 1-bit SGD that Section 2
+                                 describes, instead of +0; dropped entries are unchanged. */
 };
 
 const char* gd_status_string(int status);
@@ -295,7 +301,8 @@ int gd_compress_static(const gd_compress_args* args, void* stream, const void** 
  * launches; 0 switches the hooks off.  gd_profile_collect waits for the recorded pairs, writes their
  * durations in milliseconds (oldest first, at most `capacity`) and, if tags_out is not NULL, which
  * kernel each belongs to (0 setup, 1 sample selection, 2 fused pass, 3 dense selection, 4 dense
- * compaction, 5 candidate selection, 6 candidate compaction, 7 finalize, 8 apply), then forgets them.
+ * compaction, 5 candidate selection, 6 candidate compaction, 7 finalize, 8 apply, 9 sampled-mode pack,
+ * 10 means division, 11 quantisation-error feedback), then forgets them.
  * At most 4096 pairs are held between two collects; later launches are not recorded.  Not thread-safe.
  */
 int gd_profile_enable(int mode);

@@ -204,7 +204,7 @@ def pair_index(pos, layer_off, layer_cols=None):
 
 
 def compress(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GLOBAL,
-             value_mode=VALUES_FP32, method="sort", layer_cols=None):
+             value_mode=VALUES_FP32, method="sort", layer_cols=None, error_feedback=False):
     """One GradDrop call (Algorithm 1) for one worker's flat fp32 gradient.
 
     grad, residual : float32 arrays of n elements (not modified).
@@ -218,6 +218,10 @@ def compress(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GL
       shard_cnt_off uint32[n_shards+1] survivors with index below each shard boundary
       means     float32[n_layers, 2], counts int64[n_layers, 2], sums float64[n_layers, 2]
                 (two-means mode; column 0 = sign bit clear, column 1 = sign bit set)
+    error_feedback (1-bit value modes only): the paper is silent on whether the error of the 1-bit
+    quantisation stays local; Algorithm 1 keeps the dropped mass only (the default).  With the option
+    a kept entry leaves v minus its decoded fp32 value in the residual (one fp32 subtraction), the
+    error feedback of 1-bit SGD that Section 2 describes.
     """
     g = np.ascontiguousarray(grad, dtype=np.float32)
     r = np.ascontiguousarray(residual, dtype=np.float32)
@@ -286,6 +290,11 @@ def compress(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GL
         out["means"] = means
     elif value_mode != VALUES_FP32:
         raise ValueError("bad value_mode")
+    if error_feedback:
+        if value_mode == VALUES_FP32:
+            raise ValueError("error feedback needs a 1-bit value mode")
+        _, decoded = decode_push(out["idx"], None, value_mode, out["means"], layer_off, layer_cols)
+        new_residual[kept] = val - decoded          # fp32 - fp32, rounded once
     return out
 
 

@@ -30,6 +30,7 @@ GD_VALUES_THRESHOLD = 2
 GD_VALUES_COLUMN_MEANS = 3
 GD_FLAG_NO_PREDICTION = 1
 GD_FLAG_SAMPLED_THRESHOLD = 2
+GD_FLAG_QUANT_ERROR_FEEDBACK = 4
 GD_ERR_OVERFLOW = -7
 
 EXPORTS = [
@@ -279,7 +280,7 @@ def gd_step_host(call: CompressCall, apply: Optional[ApplyCall], grad_host: torc
 
 
 PROFILE_TAGS = ["setup", "sample_select", "add_emit", "dense_select", "dense_compact", "cand_select", "cand_compact",
-                "finalize", "apply", "pack_sampled"]
+                "finalize", "apply", "pack_sampled", "means", "feedback"]
 
 
 def gd_profile_enable(mode) -> None:

@@ -399,7 +399,9 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     if (n_sh != n || a->n != n) return GD_ERR_INVALID_ARG;
     if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_COLUMN_MEANS) return GD_ERR_INVALID_ARG;
     if (a->value_mode != GD_VALUES_FP32 && n > (1ull << 31)) return GD_ERR_TOO_LARGE;
-    if (a->flags & ~(uint32_t)(GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD)) return GD_ERR_INVALID_ARG;
+    if (a->flags & ~(uint32_t)(GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD | GD_FLAG_QUANT_ERROR_FEEDBACK))
+      return GD_ERR_INVALID_ARG;
+    if ((a->flags & GD_FLAG_QUANT_ERROR_FEEDBACK) && a->value_mode == GD_VALUES_FP32) return GD_ERR_INVALID_ARG;
     const bool sampled = (a->flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
     if (sampled && ((a->flags & GD_FLAG_NO_PREDICTION) || a->value_mode != GD_VALUES_FP32)) return GD_ERR_INVALID_ARG;
     if (n && (!a->grad || !a->residual)) return GD_ERR_INVALID_ARG;
@@ -492,6 +494,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     if ((a->value_mode == GD_VALUES_TWO_MEANS || a->value_mode == GD_VALUES_COLUMN_MEANS) && P.n_pairs > kInlineMeansPairs &&
         launch_means(T, stream) != cudaSuccess)
       return GD_ERR_CUDA;
+    if ((a->flags & GD_FLAG_QUANT_ERROR_FEEDBACK) && launch_feedback(T, stream) != cudaSuccess) return GD_ERR_CUDA;
     return GD_OK;
   } catch (const std::bad_alloc&) {
     return GD_ERR_INVALID_ARG;

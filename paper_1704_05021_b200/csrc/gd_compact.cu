@@ -95,6 +95,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   load_tables(T, LK, &s_tab, &scopes, &tile0);
   const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS || T.value_mode == GD_VALUES_COLUMN_MEANS;   // sums are kept
   const bool packed = T.value_mode != GD_VALUES_FP32;
+  const bool feedback = (T.flags & GD_FLAG_QUANT_ERROR_FEEDBACK) != 0;   // kept slots keep v for feedback_kernel
   const uint32_t ltm = lanemask_lt();
   uint4* desc = reinterpret_cast<uint4*>(T.desc_cand);
   // The lists' capacities are a multiple of what they hold.  With few scopes only the tiles that hold
@@ -214,7 +215,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
           const uint64_t idx = ib[j];
           if (pos < d.k && idx < T.n) {
             const uint32_t b = vb[j];
-            T.residual[idx] = 0.0f;
+            if (!feedback) T.residual[idx] = 0.0f;
             if (packed) {
               const uint32_t sgn = b >> 31;
               T.out_idx[d.out_base + pos] = (uint32_t)idx | (sgn << 31);
@@ -301,6 +302,7 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
   load_tables(T, L_DCOMP, &s_tab, &scopes, &tile0);
   const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS || T.value_mode == GD_VALUES_COLUMN_MEANS;   // sums are kept
   const bool packed = T.value_mode != GD_VALUES_FP32;
+  const bool feedback = (T.flags & GD_FLAG_QUANT_ERROR_FEEDBACK) != 0;   // kept slots keep v for feedback_kernel
   const uint32_t ltm = lanemask_lt();
   uint4* desc = reinterpret_cast<uint4*>(T.desc_dcomp);
 
@@ -416,7 +418,7 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
             const uint64_t idx = d.lo + i;
             if (pos < d.k && idx < T.n) {
               const uint32_t b = __float_as_uint(vals[i]);   // read again: only survivors get here
-              T.residual[idx] = 0.0f;
+              if (!feedback) T.residual[idx] = 0.0f;
               if (packed) {
                 const uint32_t sgn = b >> 31;
                 T.out_idx[d.out_base + pos] = (uint32_t)idx | (sgn << 31);
@@ -554,6 +556,19 @@ __global__ void __launch_bounds__(kThreads) means_kernel(const __grid_constant__
   }
 }
 
+// GD_FLAG_QUANT_ERROR_FEEDBACK: the compaction left v in the residual slots of the survivors; once the
+// decode table (out_means) is final, every such slot becomes v minus the value its survivor decodes to.
+__global__ void __launch_bounds__(kThreads) feedback_kernel(const __grid_constant__ DevTables T) {
+  const uint64_t stride = (uint64_t)gridDim.x * kThreads;
+  for (uint64_t j = (uint64_t)blockIdx.x * kThreads + threadIdx.x; j < T.k_total; j += stride) {
+    const uint32_t w = T.out_idx[j];
+    const uint64_t idx = w & kAbsMask;
+    if (idx >= T.n) continue;
+    const uint64_t pr = pair_of(T.layer_off, T.pair_off, T.layer_cols, T.n_layers, idx);
+    T.residual[idx] = __fsub_rn(T.residual[idx], T.out_means[2 * pr + (w >> 31)]);
+  }
+}
+
 // Self-test kernel of the bounded waits: tile 1 waits on tile 0, which nothing publishes; tile 2
 // then meets the aborted tile 1.
 __global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(Ctl* ctl, uint4* desc, uint32_t spin_limit) {
@@ -589,6 +604,17 @@ cudaError_t launch_means(const DevTables& T, cudaStream_t stream) {
   const uint64_t cap = (uint64_t)sm_count() * 8;
   if (blocks > cap) blocks = cap;
   means_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(T);
+  GD_LAUNCH_CHECK();
+  return cudaSuccess;
+}
+
+cudaError_t launch_feedback(const DevTables& T, cudaStream_t stream) {
+  if (!T.k_total) return cudaSuccess;
+  ProfileScope prof(stream, PT_FEEDBACK);
+  uint64_t blocks = (T.k_total + kThreads - 1) / kThreads;
+  const uint64_t cap = (uint64_t)sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  feedback_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(T);
   GD_LAUNCH_CHECK();
   return cudaSuccess;
 }

@@ -210,6 +210,7 @@ cudaError_t launch_dense_select(const DevTables& T, const uint32_t* tiles, cudaS
 cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, bool finalize, cudaStream_t stream);
 cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream);
 cudaError_t launch_means(const DevTables& T, cudaStream_t stream);
+cudaError_t launch_feedback(const DevTables& T, cudaStream_t stream);
 cudaError_t launch_pack_sampled(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream);
 int sm_count();   // multiprocessors of the current device (0 on error)
@@ -218,7 +219,7 @@ int sm_count();   // multiprocessors of the current device (0 on error)
 void note_launches(uint32_t count);
 // Kernel tags of the measurement hooks, in the order a step launches them.
 enum ProfileTag : uint32_t { PT_SETUP = 0, PT_PACK_SAMPLED = 9, PT_MEANS = 10, PT_SAMPLE_SELECT = 1, PT_ADD_EMIT = 2, PT_DENSE_SELECT = 3, PT_DENSE_COMPACT = 4,
-                             PT_CAND_SELECT = 5, PT_CAND_COMPACT = 6, PT_FINALIZE = 7, PT_APPLY = 8 };
+                             PT_CAND_SELECT = 5, PT_CAND_COMPACT = 6, PT_FINALIZE = 7, PT_APPLY = 8, PT_FEEDBACK = 11 };
 void profile_mark(cudaStream_t stream, bool begin, uint32_t tag);
 struct ProfileScope {   // records an event pair around the launches made during its lifetime
   cudaStream_t stream;

@@ -76,7 +76,8 @@ def run_steps(w, device, steps, flags=0, method="sort", grads=None, alpha=1.0, w
         g = grads[step].to(device) if grads is not None else W.make_gradient(w, step, device)
         g_host = g.cpu().numpy()
         exp = orc.compress(g_host, r_host, w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
-                           method=method, layer_cols=layer_cols)
+                           method=method, layer_cols=layer_cols,
+                           error_feedback=bool(flags & B.GD_FLAG_QUANT_ERROR_FEEDBACK))
         g_before = g.clone()
         sess.compress(g)
         tag = f"{w.name} step {step} flags {flags}"
@@ -560,6 +561,40 @@ def test_column_means_on_the_nmt_shapes(cuda_device):
     assert sess.n_pairs == sum(w.layer_cols) == 500 + 500 + 85000 + 1 + 8 * 1000
 
 
+# ---------------------------------------------------------------- quantisation error fed back into the residual
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
+@pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
+@pytest.mark.parametrize("value_mode", [B.GD_VALUES_TWO_MEANS, B.GD_VALUES_THRESHOLD, B.GD_VALUES_COLUMN_MEANS])
+def test_quantisation_error_feedback(cuda_device, flags, scope_mode, value_mode):
+    """Kept slots hold v - decoded instead of +0.  The kept magnitudes of a layer span far less than 2^18, so
+    the fp64 sums behind the means are exact in any order and the residual is compared bit for bit, over
+    three steps with the residual carried (a difference in step 1 would change the selection of step 2)."""
+    shapes = [(600, 50), (4097,), (128, 1000), (3,), (5000, 8)]
+    sizes = [int(np.prod(s_)) for s_ in shapes]
+    cols = [s_[-1] if len(s_) > 1 else 1 for s_ in shapes] if value_mode == B.GD_VALUES_COLUMN_MEANS else None
+    rng = np.random.default_rng(4242)
+    w = W.small_layered(len(sizes), sizes, 980_000, scope_mode, value_mode, 3)
+    grads = [torch.from_numpy(rng.laplace(0, 1e-3, w.n).astype(np.float32)) for _ in range(3)]
+    sess = run_steps(w, cuda_device, 3, flags=flags | B.GD_FLAG_QUANT_ERROR_FEEDBACK, grads=grads, layer_cols=cols,
+                     alpha=0.5)
+    # the fed-back error is not zero: some kept slot holds a non-zero residual
+    kept = _np_u32(sess.out_idx)[:sess.k_total] & np.uint32(0x7FFFFFFF)
+    assert np.count_nonzero(sess.residual.cpu().numpy()[kept.astype(np.int64)]) > 0
+
+
+def test_quantisation_error_feedback_on_the_nmt_shapes(cuda_device):
+    w = W.workload(4)
+    run_steps(w, cuda_device, 2, flags=B.GD_FLAG_QUANT_ERROR_FEEDBACK, method="select")
+
+
+def test_quantisation_error_feedback_needs_a_one_bit_mode(cuda_device):
+    w = W.small_layered(1, [100_000], 990_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 1)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
+                           B.GD_FLAG_QUANT_ERROR_FEEDBACK, cuda_device)
+    with pytest.raises(B.GdError):
+        sess.compress(torch.zeros(w.n, device=cuda_device))
+
+
 # ---------------------------------------------------------------- randomised layouts
 @pytest.mark.parametrize("seed", range(12))
 def test_random_layouts_and_modes(cuda_device, seed):
@@ -598,8 +633,10 @@ def test_random_layouts_and_modes(cuda_device, seed):
         else:
             g = rng.choice(np.array([0.0, 0.25, -0.25, 0.5, 1.0, -2.0]), w.n)           # few distinct values
         grads.append(torch.from_numpy(g.astype(np.float32)))
-    run_steps(w, cuda_device, 3, flags=flags, grads=grads, layer_cols=cols,
-              alpha=float(rng.choice([1.0, 0.5, -1.25])))
+    alpha = float(rng.choice([1.0, 0.5, -1.25]))
+    if value_mode == B.GD_VALUES_THRESHOLD and rng.random() < 0.5:
+        flags |= B.GD_FLAG_QUANT_ERROR_FEEDBACK      # the +-tau table is exact, so the fed-back residual is too
+    run_steps(w, cuda_device, 3, flags=flags, grads=grads, layer_cols=cols, alpha=alpha)
 
 
 def test_config5_full_scale_against_the_oracle(cuda_device):

@@ -393,6 +393,45 @@ def test_threshold_quantisation_values():
 
 
 # ---------------------------------------------------------------- parameter pulls as dropped deltas
+def test_quantisation_error_feedback_by_hand_and_conservation():
+    # kept: 4, -3, 2 (k = 3 of 10): mu+ = 3, mu- = -3; each kept slot keeps v - decoded, dropped slots keep v
+    v = np.array([4.0, 0.5, -3.0, 0.25, 2.0, -0.5, 1.0, -1.0, 0.0, 0.125], dtype=np.float32)
+    base = run_flat(v, 700_000, value_mode=orc.VALUES_TWO_MEANS)
+    out = run_flat(v, 700_000, value_mode=orc.VALUES_TWO_MEANS, error_feedback=True)
+    assert out["idx"].tolist() == base["idx"].tolist() == [0, 2 | (1 << 31), 4]
+    assert out["means"].tolist() == [[3.0, -3.0]]
+    assert out["residual"].tolist() == [1.0, 0.5, 0.0, 0.25, -1.0, -0.5, 1.0, -1.0, 0.0, 0.125]
+    # without the option the same slots hold +0 (Algorithm 1 as printed)
+    assert base["residual"].tolist() == [0.0, 0.5, 0.0, 0.25, 0.0, -0.5, 1.0, -1.0, 0.0, 0.125]
+    # threshold quantiser: decoded = +-2, so 4 -> 2, -3 -> -1, and the entry at the threshold leaves +0
+    thr = run_flat(v, 700_000, value_mode=orc.VALUES_THRESHOLD, error_feedback=True)
+    assert thr["residual"].tolist() == [2.0, 0.5, -1.0, 0.25, 0.0, -0.5, 1.0, -1.0, 0.0, 0.125]
+    # conservation: what the receiver decodes plus what stays is v (exact here: small dyadic numbers), per
+    # layer and per column, over several steps with the residual carried
+    rng = np.random.default_rng(11)
+    layer_off, cols = [0, 64, 64 + 96], [8, 1]
+    n = layer_off[-1]
+    for mode in (orc.VALUES_TWO_MEANS, orc.VALUES_THRESHOLD, orc.VALUES_COLUMN_MEANS):
+        r = np.zeros(n, dtype=np.float32)
+        total = np.zeros(n, dtype=np.float64)
+        received = np.zeros(n, dtype=np.float64)
+        for _ in range(4):
+            g = (rng.integers(-64, 65, size=n) * 0.25).astype(np.float32)
+            total += g
+            o = orc.compress(g, r, layer_off, [0, n], 750_000, orc.SCOPE_PER_LAYER, mode, layer_cols=cols,
+                             error_feedback=True)
+            pos, dec = orc.decode_push(o["idx"], None, mode, o["means"], layer_off, cols)
+            # dyadic inputs, but a mean of them need not be: compare against the fp32 subtraction by hand
+            manual = o["v"].copy()
+            manual[pos] = o["v"][pos] - dec
+            assert np.array_equal(manual.view(np.uint32), o["residual"].view(np.uint32))
+            received[pos] += dec
+            r = o["residual"]
+            assert np.allclose(received + r, total, rtol=0, atol=1e-4)
+    with pytest.raises(ValueError):
+        run_flat(v, 700_000, error_feedback=True)
+
+
 def test_delta_pull_by_hand_and_invariants():
     # by hand: delta = p - last = [0.5, -4, 0.25, 3, 0, -1]; keep 2 of 6 (drop 2/3): -4 and 3
     p = np.array([1.5, -3.0, 0.25, 5.0, 2.0, 0.0], dtype=np.float32)
