@@ -167,6 +167,49 @@ def test_signed_zero_and_subnormals(cuda_device):
     run_steps(w, cuda_device, 3, grads=[torch.from_numpy(g), torch.from_numpy(-g), torch.from_numpy(g)])
 
 
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
+def test_infinities_are_the_largest_magnitudes(cuda_device, flags):
+    """+-inf order above every finite value by bit pattern and add deterministically, so parity stays bit-exact
+    (the infinities leave the residual when they are sent, so no inf - inf arises)."""
+    n = (1 << 22) + 77
+    rng = np.random.default_rng(21)
+    g = rng.laplace(0, 1e-3, n).astype(np.float32)
+    pos = rng.choice(n, size=300, replace=False)
+    g[pos[:150]] = np.inf
+    g[pos[150:]] = -np.inf
+    g[-1] = np.float32(3.4028235e38)                                     # the largest finite value
+    w = W.small_layered(1, [n], 999_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 2)
+    run_steps(w, cuda_device, 2, flags=flags, grads=[torch.from_numpy(g), torch.from_numpy(g)], with_apply=False)
+
+
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
+def test_nan_inputs_are_sent_not_stuck(cuda_device, flags):
+    """NaNs are outside the bit-exact contract (the payload of NaN + x differs between processors), but they
+    must behave: every NaN has a larger key than any number, so all of them are sent (there are fewer than k),
+    the numbers that fill the rest of the quota are the oracle's, and the call ends with status ok."""
+    n = (1 << 22) + 5
+    rng = np.random.default_rng(22)
+    g = rng.laplace(0, 1e-3, n).astype(np.float32)
+    nan_pos = np.sort(rng.choice(n, size=200, replace=False))
+    g[nan_pos] = np.nan
+    w = W.small_layered(1, [n], 999_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 2)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, flags, cuda_device)
+    sess.compress(torch.from_numpy(g).to(cuda_device))
+    assert sess.status() == B.GD_OK
+    exp = orc.compress(g, orc.residual_reset(n), w.layer_off, w.shard_off, w.drop_ppm)
+    k = sess.k_total
+    got_idx = _np_u32(sess.out_idx)[:k]
+    got_val = sess.out_val.cpu().numpy()[:k]
+    assert np.array_equal(got_idx, exp["idx"])                           # same positions: NaNs first in rank, then numbers
+    assert np.array_equal(np.flatnonzero(np.isnan(got_val)), np.flatnonzero(np.isin(got_idx, nan_pos)))
+    finite = ~np.isnan(got_val)
+    assert np.array_equal(got_val[finite].view(np.uint32), exp["val"][finite].view(np.uint32))
+    res = sess.residual.cpu().numpy()
+    assert not np.isnan(res).any()
+    assert np.array_equal(res.view(np.uint32), exp["residual"].view(np.uint32))
+    assert int(_np_u32(sess.out_tau)[0]) == int(exp["tau"][0])
+
+
 def test_integer_gradients_conserve_mass(cuda_device):
     """Error feedback loses nothing: sent mass + residual == sum of the gradients, exactly."""
     n, steps = 1 << 18, 8
