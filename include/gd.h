@@ -153,7 +153,11 @@ int gd_means_pairs(uint32_t n_layers, const uint32_t* layer_cols, int value_mode
  * whose fp64 partial sums are combined in an unspecified order.  Non-finite inputs are ordered by
  * their bit pattern (NaN above Inf above finite); NaN payloads follow the device's fp32 add.
  * grad, residual, the outputs and the workspace must not overlap.  Calls that share a workspace
- * must be ordered (same stream, or otherwise serialised).
+ * must be ordered (same stream, or otherwise serialised).  Host threads may call concurrently with
+ * workspaces of their own, but calls on ONE device should be ordered with respect to each other
+ * (one stream, or events): the selection kernels are cooperative launches sized to fill the device,
+ * so two calls that overlap on a GPU gain nothing and may end with GD_ERR_DEVICE_TIMEOUT when neither
+ * grid becomes fully resident (every device-side wait is bounded; nothing hangs).
  */
 typedef struct gd_compress_args {
   const float* grad;          /* device, n fp32, 16-byte aligned, read-only */

@@ -1,5 +1,6 @@
 // Host side of libgd.so: argument checks, the per-call plan (scopes, tile tables, workspace
 // layout) and the C entry points declared in include/gd.h.
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -237,11 +238,11 @@ cudaEvent_t g_ev_begin[kProfilePairs], g_ev_end[kProfilePairs];
 uint32_t g_ev_tag[kProfilePairs];
 uint32_t g_ev_created = 0, g_ev_used = 0;
 bool g_pair_open = false;
-uint64_t g_launches = 0;
+std::atomic<uint64_t> g_launches{0};   // calls may come from several host threads
 
 }  // namespace
 
-void note_launches(uint32_t count) { g_launches += count; }
+void note_launches(uint32_t count) { g_launches.fetch_add(count, std::memory_order_relaxed); }
 
 cudaError_t launch_setup(void* tables_dst, const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes,
                          cudaStream_t stream) {
@@ -265,14 +266,14 @@ cudaError_t launch_setup(void* tables_dst, const void* tables_src, size_t tables
 }
 
 int sm_count() {
-  static int cached = 0;
-  if (cached > 0) return cached;
+  static std::atomic<int> cached{0};
+  if (cached.load(std::memory_order_relaxed) > 0) return cached.load(std::memory_order_relaxed);
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return 148;   // B200; only sizes grids
-  cached = sms;
-  return cached;
+  cached.store(sms, std::memory_order_relaxed);
+  return sms;
 }
 
 void profile_mark(cudaStream_t stream, bool begin, uint32_t tag) {
@@ -594,7 +595,7 @@ int gd_selftest_bounded_wait(void* workspace, size_t workspace_bytes, uint32_t s
 
 int gd_launch_count(uint64_t* count_out) {
   if (!count_out) return GD_ERR_INVALID_ARG;
-  *count_out = g_launches;
+  *count_out = g_launches.load(std::memory_order_relaxed);
   return GD_OK;
 }
 
