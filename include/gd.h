@@ -61,7 +61,8 @@ const char* gd_status_string(int status);
 /*
  * Entries kept in one threshold scope of n_scope elements when drop_ppm parts per million are
  * dropped: k = n_scope - floor(n_scope * drop_ppm / 1e6), in 64-bit integers.
- * Algorithm 1, "Select threshold: R% of |grad| is smaller"; R is passed as an integer so that
+ * Algorithm 1, the threshold-selection step (a fraction R of the magnitudes lies below the threshold);
+ * R is passed as an integer so that
  * every party computes the same count.  drop_ppm must be <= 1000000.
  */
 int gd_kept_count(uint64_t n_scope, uint32_t drop_ppm, uint64_t* k_out);
@@ -69,7 +70,7 @@ int gd_kept_count(uint64_t n_scope, uint32_t drop_ppm, uint64_t* k_out);
 /*
  * Total survivors of one gd_compress call, so that outputs can be sized before the launch.
  * layer_off: HOST, n_layers + 1 ascending offsets (first 0, last n).  Section 4, last paragraph:
- * the threshold is chosen "locally to each matrix" (GD_SCOPE_PER_LAYER: one scope per layer) or
+ * the threshold is chosen for every parameter matrix on its own (GD_SCOPE_PER_LAYER: one scope per layer) or
  * globally (GD_SCOPE_GLOBAL: one scope [0, n)).
  */
 int gd_total_kept(const uint64_t* layer_off, uint32_t n_layers, int scope_mode, uint32_t drop_ppm,
@@ -108,25 +109,25 @@ int gd_means_pairs(uint32_t n_layers, const uint32_t* layer_cols, int value_mode
  *   residual  = v where dropped, +0.0f where kept      (Algorithm 1: residuals <- grad - dropped)
  *   out_shard_cnt_off[j] = number of survivors with index < shard_off[j]   (Section 3: the
  *              gradient is split into N pieces, one per server)
- *   two-means mode (Section 5.4, quantisation by "the averages of values being quantized"): per
+ *   two-means mode (Section 5.4, the 1-bit quantisation whose two centres are the means of the values they replace): per
  *              layer, mu+ = mean of kept v with sign bit 0 and mu- = mean of kept v with sign bit 1
  *              (fp64 accumulation, rounded to fp32, +0.0f for an empty group); out_idx[t] carries
  *              index | signbit << 31 and out_val is not written.  The residual is unchanged by the
  *              value mode: it holds the dropped mass only.
- *   column-means mode (Section 5.4: the averages are taken "at the column level, rather than choosing
- *              centers globally"): layer l is a row-major matrix with layer_cols[l] columns (its size must
+ *   column-means mode (Section 5.4: the centres are chosen per column of a matrix instead of one pair
+ *              per tensor): layer l is a row-major matrix with layer_cols[l] columns (its size must
  *              be a multiple of layer_cols[l]; 1 = one pair for the whole layer, as in two-means mode), and
  *              every column c gets its own pair: pair index = sum of layer_cols of the earlier layers + c,
  *              out_means[2 * pair] = mu+, out_means[2 * pair + 1] = mu-.  Packing as in two-means mode.
- *   threshold mode (Section 5.4, the quantisation that maps "all surviving values to the dropping
- *              threshold, effectively the minimum surviving absolute value"): same packing as two-means
+ *   threshold mode (Section 5.4, the quantisation in which every survivor stands for the dropping
+ *              threshold, i.e. the smallest magnitude that survived): same packing as two-means
  *              mode; out_means[l] = (+t, -t) with t the float whose bit pattern is the tau of the scope
  *              that holds layer l (+0, -0 if that scope keeps nothing), so that a push decodes exactly
  *              like a two-means push.
  *
  *   delta mode (delta_base != NULL; Section 4, third paragraph: the same function is applied to
- *              parameter pulls "encoded as deltas from the last version pulled by the client", the
- *              server keeping that last version): grad holds the server's current parameters,
+ *              parameter pulls, sent as differences from the version the client pulled last, of which
+ *              the server keeps a copy): grad holds the server's current parameters,
  *              delta_base the copy the client is known to hold, and
  *                  v[i] = grad[i] - delta_base[i]          (one fp32 subtraction)
  *              takes the place of grad + residual; the residual's old contents are not read.  After the
@@ -136,8 +137,8 @@ int gd_means_pairs(uint32_t n_layers, const uint32_t* layer_cols, int value_mode
  *              residual buffer is used as scratch and returns v where dropped, +0 where kept.  Delta
  *              mode needs GD_VALUES_FP32.
  *
- *   sampled-threshold mode (GD_FLAG_SAMPLED_THRESHOLD; Section 4, fourth paragraph: "We sample 0.1% of
- *              the gradient and obtain the threshold by running selection on the samples"): per scope,
+ *   sampled-threshold mode (GD_FLAG_SAMPLED_THRESHOLD; Section 4, fourth paragraph: the threshold is
+ *              selected on a 0.1 % sample of the gradient instead of on all of it): per scope,
  *              m = n_s if n_s <= 4096, else max(4096, ceil(n_s / 1000)) positions are sampled, one in each
  *              of m strata (with w = floor(n_s / m) and rem = n_s mod m, stratum i starts at
  *              a = i w + min(i, rem) and has w + 1 elements if i < rem, else w; sample i of scope s is at

@@ -10,11 +10,11 @@ the paper prints); no function here is "parity unpinned".
 What the path computes (Algorithm 1, in its order):
 
   1. grad += residuals                      (fp32 add, round to nearest even)
-  2. select threshold: R% of |grad| smaller  (single threshold on |value|, Section 4 par. 1)
+  2. choose the threshold below which a fraction R of the |grad| values lies  (one threshold on |value|, Section 4 par. 1)
   3. kept[i] = grad[i] where |grad[i]| is above the threshold, else 0
   4. residuals = grad - kept                 (the dropped mass stays local)
   5. return sparse(kept)                     (index + value pairs, 8 bytes per survivor;
-                                              the "50x less data at 99%" of Section 5.1)
+                                              the factor 50 at 99 % in Section 5.1)
 
 Readings taken where the paper is silent:
   * exactly k = n - floor(n * drop_ppm / 1e6) entries are kept per threshold scope; the
@@ -22,14 +22,14 @@ Readings taken where the paper is silent:
     the lower index; the reported threshold tau is the smallest kept |v| bit pattern
     (0xFFFFFFFF when nothing is kept);
   * a scope is either the whole gradient ("global") or each parameter tensor on its own
-    ("locally to each matrix", Section 4 last paragraph);
-  * two-value quantisation (Section 5.4, "averages of values being quantized"): one pair
+    (the per-matrix thresholds of Section 4, last paragraph);
+  * two-value quantisation (Section 5.4, centres = the means of the values they replace): one pair
     (mean of kept entries with sign bit 0, mean of kept entries with sign bit 1) per layer,
     survivors packed as index | signbit << 31; the residual still holds only the dropped mass;
-  * column-wise averages (Section 5.4: centres chosen "at the column level" rather than per tensor):
+  * column-wise averages (Section 5.4: centres chosen per column rather than per tensor):
     a layer is a row-major matrix with layer_cols[l] columns and every column has its own pair;
   * threshold quantisation (Section 5.4: every surviving value is mapped to the dropping
-    threshold, "effectively the minimum surviving absolute value"): same packing; the pair of a
+    threshold, i.e. the smallest magnitude that survived): same packing; the pair of a
     layer is (+t, -t) with t the float whose bit pattern is the tau of the scope holding the layer;
   * the server applies a push as p[idx - shard_start] += alpha * value (Section 3: a server
     owns 1/N of the parameters); this oracle evaluates that sum in fp64.
@@ -112,7 +112,7 @@ def _mix32(x: np.ndarray) -> np.ndarray:
 
 
 def sampled_positions(lo: int, hi: int, scope_index: int) -> np.ndarray:
-    """Positions read by the sampled-threshold mode in scope [lo, hi) (Section 4: "We sample 0.1% of the gradient").
+    """Positions read by the sampled-threshold mode in scope [lo, hi) (Section 4, fourth paragraph: a 0.1 % sample).
 
     m = n_s if n_s <= 4096 else max(4096, ceil(n_s / 1000)); the scope is cut into m strata, the first
     (n_s mod m) of floor(n_s / m) + 1 elements and the rest of floor(n_s / m), and stratum i contributes

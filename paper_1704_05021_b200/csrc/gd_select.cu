@@ -1,4 +1,4 @@
-// Threshold selection of gd_compress (Algorithm 1, "Select threshold: R% of |grad| is smaller"):
+// Threshold selection of gd_compress (Algorithm 1, the threshold-selection step):
 // an exact radix select on the bit pattern of |v|, run over three kinds of lists -
 //   the sample   -> tau_lo, the predicted lower bound used by the fused pass,
 //   the candidate list the fused pass emitted -> tau and the tie quota (the usual case),
