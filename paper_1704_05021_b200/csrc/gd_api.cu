@@ -15,8 +15,16 @@ namespace {
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-// Sample size per scope: kSampleFactor expected samples above the threshold, within [min, max].
-constexpr double kSampleFactor = 256.0, kSampleMin = 16384.0, kSampleMax = 262144.0;
+// Sample size per scope: the sample is sized for a number of expected samples above the threshold
+// ("hits") that grows with the scope's k.  A sample costs scattered reads in proportion to its size; a
+// small one costs a wider safety margin, i.e. extra candidates in proportion to k / sqrt(hits).  The sum
+// is smallest near hits ~ k^(2/3) (the measured costs per sample and per candidate are about equal;
+// factors of 0.12, 0.25 and 0.5 were timed on layered models of 12 to 387 tensors), so:
+// hits = kHitsFactor * k^(2/3) within [kHitsMin, kHitsMax], and never more than kSampleMax samples or a
+// sixteenth of the scope.
+constexpr double kHitsFactor = 0.25, kHitsMin = 32.0, kHitsMax = 256.0, kSampleMax = 262144.0;
+constexpr uint64_t kSampleAllMax = 8192;         // scopes up to this length are sampled completely
+constexpr uint64_t kClusterMaxStride = 1024;      // strata up to this many elements wide are sampled in groups of 8
 constexpr uint64_t kAutoDenseMax = 1ull << 21;   // vectors up to this length skip the prediction (measured crossover: 2^22)
 
 inline uint64_t kept_count(uint64_t n, uint32_t drop_ppm) {
@@ -29,18 +37,29 @@ inline uint64_t kept_count(uint64_t n, uint32_t drop_ppm) {
 // above the prediction is at least k with a margin of six standard deviations plus 12.5 %.  Small
 // scopes are sampled completely, which makes the prediction the exact threshold.  None of this
 // affects results: a scope whose prediction fails is selected densely.
-void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint64_t* cap) {
+void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint64_t* cap, uint32_t* cluster) {
+  *cluster = 1;
   if (k == 0 || ns == 0) { *m = 0; *rank = 0; *cap = 0; return; }
-  double target = kSampleFactor * (double)ns / (double)k;
-  if (target < kSampleMin) target = kSampleMin;
+  double hits = kHitsFactor * std::cbrt((double)k * (double)k);
+  if (hits < kHitsMin) hits = kHitsMin;
+  if (hits > kHitsMax) hits = kHitsMax;
+  double target = hits * (double)ns / (double)k;
   if (target > kSampleMax) target = kSampleMax;
-  const uint64_t mt = (uint64_t)target;
-  if (mt * 2 >= ns) {
+  if (target > (double)ns / 16.0) target = (double)ns / 16.0;
+  uint64_t mt = (uint64_t)target;
+  if (ns <= kSampleAllMax || mt < 64) {
     *m = ns;
     *rank = k;
     uint64_t c = 3 * k + 1024;
     *cap = c < ns ? c : ns;
     return;
+  }
+  // Narrow strata (a sample every few sectors): sample whole groups of 8 consecutive elements instead, so that
+  // the sample costs an eighth of the scattered sector reads.  Wide strata keep single elements, which
+  // spread the sample over more rows of a matrix.
+  if (ns / mt <= kClusterMaxStride) {
+    mt &= ~7ull;
+    *cluster = 8;
   }
   *m = mt;
   const double x = (double)k * (double)mt / (double)ns;
@@ -149,12 +168,13 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
     d.out_base = out_base;
     out_base += d.k;
     uint64_t m = 0, rank = 0, cap = 0;
+    uint32_t cluster = 1;
     if (sampled) {
       m = sampled_m(ns);
       rank = kept_count(m, drop_ppm);
       cap = sampled_cap(ns, d.k);
     } else if (predict) {
-      plan_prediction(ns, d.k, &m, &rank, &cap);
+      plan_prediction(ns, d.k, &m, &rank, &cap, &cluster);
     }
     d.cand_base = cand_base;
     d.cand_cap = cap;
@@ -162,8 +182,16 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
     d.samp_base = samp_base;
     d.samp_m = m;
     d.samp_rank = rank;
-    d.samp_w = m ? ns / m : 0;
-    d.samp_rem = m ? ns % m : 0;
+    d.samp_cluster = cluster;
+    if (cluster == 8) {   // strata of groups of 8 elements, from the first multiple of 8 at or after lo
+      const uint64_t first = (d.lo + 7) & ~7ull;
+      const uint64_t groups = (d.hi - first) / 8, strata = m / 8;
+      d.samp_w = groups / strata;
+      d.samp_rem = (uint32_t)(groups % strata);
+    } else {
+      d.samp_w = m ? ns / m : 0;
+      d.samp_rem = m ? (uint32_t)(ns % m) : 0;
+    }
     samp_base += m;
     for (int l = 0; l < L_COUNT; ++l) P->tile0[l][s] = (uint32_t)tiles[l];
     P->samp_off[s] = d.samp_base;

@@ -100,19 +100,17 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   uint4* desc = reinterpret_cast<uint4*>(T.desc_cand);
   // The lists' capacities are a multiple of what they hold.  With few scopes only the tiles that hold
   // candidates are numbered (in list order), so that no ticket is spent on an empty tile.
-  __shared__ uint32_t s_vt0[kSmemScopes + 1];
-  const bool compacted = T.n_scopes <= kSmemScopes;
+  __shared__ uint32_t s_vt0[kVtScopes + 1];
+  const bool compacted = T.n_scopes <= kVtScopes;
   if (compacted) {
     __syncthreads();                       // the table copy is complete
-    if (tid < T.n_scopes) {                 // one thread per scope reads its count, then a short serial prefix
-      const ScopeState* sx = T.state + tid;
-      s_vt0[tid + 1] = predicted_ok(T, scopes[tid], *sx) ? (uint32_t)((sx->cand_count + kTile - 1) / kTile) : 0u;
+    for (uint32_t x = tid; x < T.n_scopes; x += kThreads) {
+      const ScopeState* sx = T.state + x;
+      s_vt0[x + 1] = predicted_ok(T, scopes[x], *sx) ? (uint32_t)((sx->cand_count + kTile - 1) / kTile) : 0u;
     }
     if (tid == 0) s_vt0[0] = 0;
     __syncthreads();
-    if (tid == 0)
-      for (uint32_t x = 0; x < T.n_scopes; ++x) s_vt0[x + 1] += s_vt0[x];
-    __syncthreads();
+    block_inclusive_scan(s_vt0 + 1, T.n_scopes);
     total_tiles = s_vt0[T.n_scopes];
   }
 
@@ -124,8 +122,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
     if (t >= total_tiles) break;
     uint32_t s, first;
     if (compacted) {
-      s = 0;
-      while (t >= s_vt0[s + 1]) ++s;
+      s = scope_of_tile(s_vt0, T.n_scopes, t);   // a binary search in shared memory
       first = s_vt0[s];
     } else {
       s = scope_of_tile(tile0, T.n_scopes, t);

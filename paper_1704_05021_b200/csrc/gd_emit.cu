@@ -18,7 +18,10 @@ namespace gd {
 
 namespace {
 
-constexpr uint32_t kStash = 128;   // candidate slots per warp and chunk in shared memory
+#ifndef GD_EMIT_STASH
+#define GD_EMIT_STASH 256
+#endif
+constexpr uint32_t kStash = GD_EMIT_STASH;   // candidate slots per warp and chunk in shared memory
 #ifndef GD_EMIT_WARPS
 #define GD_EMIT_WARPS 8
 #endif

@@ -47,7 +47,10 @@ struct ScopeDesc {       // built on the host for every call, read-only on the d
   uint64_t samp_m;       // samples drawn from the scope
   uint64_t samp_rank;    // the prediction is the samp_rank-th largest sample key
   uint64_t samp_w;       // floor(n_s / samp_m): width of a stratum (the first samp_rem strata are one wider)
-  uint64_t samp_rem;     // n_s mod samp_m
+  uint32_t samp_rem;     // n_s mod samp_m
+  uint32_t samp_cluster; // 1: strata of elements, one sample each.  8: the prediction samples whole groups of 8
+                         // consecutive elements (one 32-byte sector of each input); the strata (samp_w, samp_rem)
+                         // then count groups, starting at the first multiple of 8 at or after lo
 };
 
 struct SelState {        // running state of one radix selection
@@ -143,6 +146,37 @@ struct SmemTables {
   ScopeDesc scopes[kSmemScopes];
   uint32_t tile0[kSmemScopes + 1];
 };
+
+// Most scopes for which the kernels over the candidate lists number only the tiles that hold
+// candidates (a table of this many counters in shared memory).
+constexpr uint32_t kVtScopes = 2048;
+
+// In-place inclusive prefix sum of a[0 .. n) in shared memory, by a whole CTA of kThreads threads.
+// The caller synchronises between filling a[] and the call; the result is visible to all on return.
+__device__ __forceinline__ void block_inclusive_scan(uint32_t* a, uint32_t n) {
+  __shared__ uint32_t s_scan_warp[kThreads / 32];
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const uint32_t per = (n + kThreads - 1) / kThreads;
+  const uint32_t b = tid * per < n ? tid * per : n;
+  const uint32_t e = b + per < n ? b + per : n;
+  uint32_t sum = 0;
+  for (uint32_t i = b; i < e; ++i) sum += a[i];
+  uint32_t inc = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+    if ((int)lane >= o) inc += y;
+  }
+  if (lane == 31u) s_scan_warp[warp] = inc;
+  __syncthreads();
+  uint32_t run = inc - sum;
+  for (uint32_t w = 0; w < warp; ++w) run += s_scan_warp[w];
+  for (uint32_t i = b; i < e; ++i) {
+    run += a[i];
+    a[i] = run;
+  }
+  __syncthreads();
+}
 
 // Called by all threads of a CTA; the caller synchronises before using the result.  Returns the
 // tables to use: the shared copy when the scopes fit, else the global ones.

@@ -8,6 +8,8 @@
 // 31-bit magnitude key (11 + 10 + 10 bits) over its share of the tiles, the grid meets at a
 // barrier, and every CTA works out the next digit of the scopes it touches from the finished
 // histogram.  The barrier is a counter in the workspace; its wait is bounded like every other wait.
+#include <atomic>
+
 #include "gd_internal.cuh"
 
 namespace gd {
@@ -52,11 +54,16 @@ __device__ bool grid_barrier(uint32_t* counter, uint32_t& phase, Ctl* ctl) {
 // The value of sample li of scope s: the scope is cut into m strata and one position inside stratum li
 // is read.  The sample only steers the prediction; any sample gives the same final result.
 __device__ __forceinline__ float sample_value(const DevTables& T, const ScopeDesc& d, uint32_t s, uint64_t li) {
-  // m strata: the first (n_s mod m) have floor(n_s / m) + 1 elements, the others floor(n_s / m)
-  const uint64_t a = li * d.samp_w + (li < d.samp_rem ? li : d.samp_rem);
-  const uint32_t width = (uint32_t)d.samp_w + (li < d.samp_rem ? 1u : 0u);
-  uint64_t pos = d.lo + a;
-  if (width > 1) pos += mix32((uint32_t)li * 0x9E3779B9u + s) % width;
+  // m strata: the first (n_s mod m) have floor(n_s / m) + 1 elements, the others floor(n_s / m).
+  // Where the strata are narrow, a sample per stratum would touch nearly every 32-byte sector of the
+  // scope; there the strata are made of groups of 8 elements and a whole group is sampled (samples
+  // 8c .. 8c+7 are group c), which reads an eighth of the sectors for the same number of samples.
+  const uint64_t u = d.samp_cluster == 8u ? li >> 3 : li;      // stratum
+  const uint64_t a = u * d.samp_w + (u < d.samp_rem ? u : d.samp_rem);
+  const uint32_t width = (uint32_t)d.samp_w + (u < d.samp_rem ? 1u : 0u);
+  uint64_t unit = a;
+  if (width > 1) unit += mix32((uint32_t)u * 0x9E3779B9u + s) % width;
+  const uint64_t pos = d.samp_cluster == 8u ? ((d.lo + 7u) & ~7ull) + unit * 8u + (li & 7u) : d.lo + unit;
   return T.delta_base ? __fsub_rn(__ldg(T.grad + pos), T.delta_base[pos]) : __fadd_rn(__ldg(T.grad + pos), T.residual[pos]);
 }
 
@@ -82,10 +89,14 @@ __device__ __forceinline__ unsigned long long* hist_of(const DevTables& T, uint3
   return base + (view == V_SAMPLE ? 0u : 4096u) + off;
 }
 
-// Run by a whole CTA after the grid barrier that completes histogram `gh`: walks it from the top
-// bin down and fixes the next digit.  Every CTA that needs the digit computes it for itself, so no
-// second barrier is needed to hand it around.
-__device__ SelRun next_digit(const unsigned long long* gh, int bits, SelRun in, Ctl* ctl) {
+__device__ __forceinline__ unsigned long long load_bin(const unsigned long long* p) { return __ldcg(p); }
+__device__ __forceinline__ unsigned long long load_bin(const uint32_t* p) { return *p; }
+
+// Run by a whole CTA on a finished histogram `gh` (a global one after the grid barrier that completes
+// it, or the CTA's own in shared memory): walks it from the top bin down and fixes the next digit.
+// Every CTA that needs the digit computes it for itself, so no second barrier is needed to hand it around.
+template <typename Bin>
+__device__ SelRun next_digit(const Bin* gh, int bits, SelRun in, Ctl* ctl) {
   __shared__ unsigned long long s_warp[kWarps];
   __shared__ unsigned long long s_acc;
   __shared__ uint32_t s_digit;
@@ -97,7 +108,7 @@ __device__ SelRun next_digit(const unsigned long long* gh, int bits, SelRun in, 
   unsigned long long cs = 0;
 #pragma unroll
   for (uint32_t j = 0; j < 8; ++j) {
-    bin[j] = j < C ? __ldcg(gh + top - j) : 0ull;
+    bin[j] = j < C ? load_bin(gh + top - j) : 0ull;
     cs += bin[j];
   }
   unsigned long long inc = cs;
@@ -148,20 +159,111 @@ __device__ SelRun state_before(const DevTables& T, const ScopeDesc& d, uint32_t 
   return r;
 }
 
+// One key into the CTA's shared histogram.  A warp whose 32 keys share one bin (all zeros in a
+// row-sparse layer, or nothing to count) issues one add; otherwise plain shared-memory adds.  Measured
+// on skewed keys, this beats grouping equal digits with match.any, whose cost is paid on every round.
+__device__ __forceinline__ void count_digit(uint32_t* sh, uint32_t digit, uint32_t lane) {
+  constexpr uint32_t NONE = 0xFFFFFFFFu;
+  const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, digit, 0);
+  if (__all_sync(0xFFFFFFFFu, digit == d0)) {
+    if (lane == 0 && d0 != NONE) atomicAdd(&sh[d0], 32u);
+  } else if (digit != NONE) {
+    atomicAdd(&sh[digit], 1u);
+  }
+}
+
+// Number of entries of the ascending table base[0 .. count) that are <= t, counted by the whole CTA
+// in one round of loads (a binary search would be a chain of dependent global loads).
+__device__ uint32_t block_count_le(const uint32_t* base, uint32_t count, uint32_t t) {
+  __shared__ uint32_t s_cnt;
+  if (threadIdx.x == 0) s_cnt = 0;
+  __syncthreads();
+  uint32_t c = 0;
+  for (uint32_t i = threadIdx.x; i < count; i += kThreads) c += base[i] <= t ? 1u : 0u;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+  if ((threadIdx.x & 31u) == 0 && c) atomicAdd(&s_cnt, c);
+  __syncthreads();
+  const uint32_t r = s_cnt;
+  __syncthreads();
+  return r;
+}
+
+// The whole selection of a list of at most kTile entries, by one CTA in its shared histogram `sh`
+// (all zero on entry and on return): no global histogram, no grid barrier.  The entries are read again
+// in every pass (they sit in L2) so that the caller's registers stay free.
 template <int VIEW>
-__global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
+__device__ __noinline__ SelRun local_select(const DevTables& T, const ScopeDesc& d, uint32_t s, uint32_t len,
+                                            const float* vals, int passes, uint32_t* sh) {
+  constexpr uint32_t NONE = 0xFFFFFFFFu;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
+  SelRun run;
+  run.prefix = 0;
+  run.rank = VIEW == V_SAMPLE ? d.samp_rank : d.k;
+  run.gt = 0;
+  for (int p = 0; p < passes; ++p) {
+    const int shift = p == 0 ? kShift0 : (p == 1 ? kShift1 : kShift2);
+    const int bits = p == 0 ? kRadixBits0 : 10;
+    const int pshift = p == 1 ? kShift0 : kShift1;
+    uint32_t keys[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const uint32_t i = (uint32_t)j * kThreads + tid;
+      float x = 0.f;
+      if (i < len) x = (VIEW == V_SAMPLE && p == 0) ? sample_value(T, d, s, i) : vals[i];
+      keys[j] = __float_as_uint(x);
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const uint32_t i = (uint32_t)j * kThreads + tid;
+      uint32_t digit = NONE;
+      if (i < len) {
+        if (VIEW == V_SAMPLE && p == 0) T.samp_val[d.samp_base + i] = __uint_as_float(keys[j]);   // read back by this thread
+        const uint32_t key = keys[j] & kAbsMask;
+        if (p == 0 || (key >> pshift) == run.prefix) digit = (key >> shift) & ((1u << bits) - 1u);
+      }
+      count_digit(sh, digit, lane);
+    }
+    __syncthreads();
+    run = next_digit(sh, bits, run, T.ctl);
+    for (uint32_t b = tid; b < (1u << bits); b += kThreads) sh[b] = 0;
+    __syncthreads();
+  }
+  return run;
+}
+
+// MANY = false: at most kSmemScopes scopes, all tables in shared memory, every list goes through the
+// global histograms (with few scopes a CTA rarely holds tiles of more than one, and the per-scope
+// steps run side by side in different CTAs).  MANY = true (models with hundreds of tensors): a CTA's
+// run of tiles crosses several scopes, so it keeps a window of the tables from its first scope on, and
+// selects every list of a single tile by itself in shared memory.
+template <int VIEW, bool MANY>
+__global__ void __launch_bounds__(kThreads, MANY ? (VIEW == V_DENSE ? 4 : 2) : 1) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
   constexpr int LK = VIEW == V_SAMPLE ? L_SAMP : (VIEW == V_CAND ? L_CAND : L_DSEL);
   const uint32_t TILE = VIEW == V_DENSE ? T.dense_sel_tile : kTile;
   const int PASSES = VIEW == V_SAMPLE ? (int)T.sample_passes : 3;   // the prediction needs 21 bits only
   constexpr uint32_t NONE = 0xFFFFFFFFu;
   __shared__ uint32_t sh[kRadixBins0];
-  __shared__ SmemTables s_tab;
+  __shared__ SmemTables s_tab;                          // the scopes [w0, w0 + kSmemScopes) this CTA starts in
+  __shared__ uint32_t s_vt0[VIEW == V_CAND ? (MANY ? kVtScopes : kSmemScopes) + 1 : 1];
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   if (T.ctl->status != GD_OK) return;   // set only by an earlier kernel of this call: uniform over the grid
   if (VIEW == V_DENSE && !(T.flags & GD_FLAG_NO_PREDICTION) && T.ctl->dense_needed == 0u) return;
-  const ScopeDesc* scopes;
-  const uint32_t* tile0;
-  load_tables(T, LK, &s_tab, &scopes, &tile0);
+  // Several candidate lists: their capacities are a multiple of what they hold, so only the tiles that
+  // hold candidates are numbered (in list order); every CTA works the numbering out for itself.
+  const bool compacted = VIEW == V_CAND && T.n_scopes > 1u && T.n_scopes <= (MANY ? kVtScopes : kSmemScopes);
+  const uint32_t* base = T.tile0[LK];                   // base[s] = tiles before scope s
+  if (compacted) {
+    for (uint32_t x = tid; x < T.n_scopes; x += kThreads) {
+      const ScopeState* sx = T.state + x;
+      s_vt0[x + 1] = predicted_ok(T, T.scopes[x], *sx) ? (uint32_t)((sx->cand_count + kTile - 1) / kTile) : 0u;
+    }
+    if (tid == 0) s_vt0[0] = 0;
+    __syncthreads();
+    block_inclusive_scan(s_vt0 + 1, T.n_scopes);
+    total_tiles = s_vt0[T.n_scopes];
+    base = s_vt0;
+  }
   // Each CTA takes a contiguous run of tiles (one flush of its histogram, and one pass over the finished
   // histograms, per scope it touches), except for a single list: its tiles beyond its length (the capacity
   // is a multiple of what it holds) are empty, and dealing the tiles out round-robin spreads the real ones
@@ -172,27 +274,23 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
   const uint32_t t_beg = round_robin ? blockIdx.x : blockIdx.x * per;
   const uint32_t t_end = round_robin ? total_tiles : ((t_beg + per < total_tiles) ? t_beg + per : total_tiles);
   const uint32_t t_step = round_robin ? gridDim.x : 1u;
-  // Several candidate lists: their capacities are a multiple of what they hold, so only the tiles that
-  // hold candidates are numbered (in list order) and split evenly, a contiguous run per CTA.
-  __shared__ uint32_t s_vt0[kSmemScopes + 1];
-  const bool compacted = VIEW == V_CAND && T.n_scopes > 1u && T.n_scopes <= kSmemScopes;
-  uint32_t v_beg = 0, v_end = 0;
-  if (compacted) {
-    __syncthreads();                                    // the table copy is complete
-    if (tid < T.n_scopes) {                 // one thread per scope reads its count, then a short serial prefix
-      const ScopeState* sx = T.state + tid;
-      s_vt0[tid + 1] = predicted_ok(T, scopes[tid], *sx) ? (uint32_t)((sx->cand_count + kTile - 1) / kTile) : 0u;
-    }
-    if (tid == 0) s_vt0[0] = 0;
+  // The scope the run starts in, and a copy of the tables of the scopes from there on: with few
+  // scopes per CTA (the usual case) every later lookup is a shared-memory read.
+  uint32_t w0 = 0;
+  if (MANY && t_beg < t_end) w0 = block_count_le(base, T.n_scopes, t_beg) - 1u;   // else all scopes fit
+  {
+    const uint32_t cnt = T.n_scopes - w0 < kSmemScopes ? T.n_scopes - w0 : kSmemScopes;
+    const uint32_t words = cnt * (uint32_t)(sizeof(ScopeDesc) / 8);
+    const uint64_t* src = reinterpret_cast<const uint64_t*>(T.scopes + w0);
+    uint64_t* dst = reinterpret_cast<uint64_t*>(s_tab.scopes);
+    for (uint32_t i = tid; i < words; i += kThreads) dst[i] = src[i];
+    for (uint32_t i = tid; i <= cnt; i += kThreads) s_tab.tile0[i] = base[w0 + i];
     __syncthreads();
-    if (tid == 0)
-      for (uint32_t x = 0; x < T.n_scopes; ++x) s_vt0[x + 1] += s_vt0[x];
-    __syncthreads();
-    const uint32_t valid = s_vt0[T.n_scopes];
-    const uint32_t per_v = (valid + gridDim.x - 1) / gridDim.x;
-    v_beg = blockIdx.x * per_v;
-    v_end = (v_beg + per_v < valid) ? v_beg + per_v : valid;
   }
+  auto desc_of = [&](uint32_t s) -> const ScopeDesc& {
+    return (!MANY || s - w0 < kSmemScopes) ? s_tab.scopes[s - w0] : T.scopes[s];
+  };
+  auto base_of = [&](uint32_t s) -> uint32_t { return (!MANY || s - w0 <= kSmemScopes) ? s_tab.tile0[s - w0] : base[s]; };
   uint32_t phase = 0;
 
   for (int pass = 0; pass <= PASSES; ++pass) {
@@ -205,21 +303,26 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
     __syncthreads();
     uint32_t cur = NONE;                                // scope the shared histogram belongs to
     uint32_t seen = NONE;                               // scope whose values are cached below
-    bool active = false, have_run = false, zero_case = false;
+    uint32_t s = w0;
+    bool active = false, have_run = false, zero_case = false, local = false;
     uint64_t len = 0;
     uint32_t prefix = 0;
     const float* vals = nullptr;
-    for (uint32_t t = compacted ? v_beg : t_beg; t < (compacted ? v_end : t_end); t += (compacted ? 1u : t_step)) {
-      uint32_t s, lt;
-      if (compacted) {                                  // t numbers the tiles that hold candidates
-        s = seen != NONE ? seen : 0u;
-        while (t >= s_vt0[s + 1]) ++s;
-        lt = t - s_vt0[s];
-      } else {
-        s = (seen != NONE && t < tile0[seen + 1]) ? seen : scope_of_tile(tile0, T.n_scopes, t);
-        lt = t - tile0[s];
+    auto flush = [&]() {                                // adds the shared histogram to scope cur's global one
+      __syncthreads();
+      unsigned long long* gh = hist_of(T, cur, VIEW, pass);
+      for (uint32_t b = tid; b < nbins; b += kThreads) {
+        const uint32_t c = sh[b];
+        if (c) atomicAdd(gh + b, (unsigned long long)c);
+        sh[b] = 0;
       }
-      const ScopeDesc& d = scopes[s];
+      __syncthreads();
+      cur = NONE;
+    };
+    for (uint32_t t = t_beg; t < t_end; t += t_step) {
+      while (t >= base_of(s + 1)) ++s;                  // base[n_scopes] = total_tiles > t
+      const uint32_t lt = t - base_of(s);
+      const ScopeDesc& d = desc_of(s);
       if (s != seen) {                                  // per-scope values, worked out once per scope
         seen = s;
         ScopeState* st = T.state + s;
@@ -232,12 +335,30 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
         // every non-zero entry is kept and the tie quota is the rest.  No histogram is needed.
         zero_case = VIEW == V_DENSE && active && !(T.flags & GD_FLAG_NO_PREDICTION) && d.k != 0 &&
                     st->tau_lo == 0u && st->cand_count < d.k;
+        // A list of one tile is selected by this CTA alone, in shared memory, during the first pass.
+        local = MANY && len <= kTile;
       }
       if (!active) continue;
       if (zero_case) {
         if (pass == PASSES && lt == 0 && tid == 0) {
           ScopeState* st = T.state + s;
           st->tau = 0u; st->gt = st->cand_count; st->q = d.k - st->cand_count; st->used_dense = 1u;
+        }
+        continue;
+      }
+      if (local) {
+        if (pass != 0 || lt != 0) continue;
+        if (cur != NONE) flush();                       // the shared histogram must be free (and is zero)
+        const SelRun run = local_select<VIEW>(T, d, s, (uint32_t)len, vals, PASSES, sh);
+        if (tid == 0) {
+          ScopeState* st = T.state + s;
+          if (VIEW == V_SAMPLE) {
+            st->tau_lo = PASSES == 3 ? run.prefix : run.prefix << kShift1;
+            if (PASSES == 3) st->tau = run.prefix;
+          } else {
+            st->tau = run.prefix; st->q = run.rank; st->gt = run.gt;
+            if (VIEW == V_DENSE) st->used_dense = 1u;
+          }
         }
         continue;
       }
@@ -261,16 +382,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
       }
       if (pass == PASSES) continue;
       if (s != cur) {
-        if (cur != NONE) {
-          __syncthreads();
-          unsigned long long* gh = hist_of(T, cur, VIEW, pass);
-          for (uint32_t b = tid; b < nbins; b += kThreads) {
-            const uint32_t c = sh[b];
-            if (c) atomicAdd(gh + b, (unsigned long long)c);
-            sh[b] = 0;
-          }
-          __syncthreads();
-        }
+        if (cur != NONE) flush();
         cur = s;
       }
       const uint64_t end = (beg + TILE < len) ? beg + TILE : len;
@@ -296,51 +408,44 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
             const uint32_t key = keys[j] & kAbsMask;
             if (pass == 0 || (key >> pshift) == prefix) digit = (key >> shift) & (nbins - 1u);
           }
-          // A warp whose 32 keys share one bin (all zeros in a row-sparse layer, or nothing to count)
-          // issues one add; otherwise plain shared-memory adds.  Measured on skewed keys, this beats
-          // grouping equal digits with match.any, whose cost is paid on every round.
-          const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, digit, 0);
-          if (__all_sync(0xFFFFFFFFu, digit == d0)) {
-            if (lane == 0 && d0 != NONE) atomicAdd(&sh[d0], 32u);
-          } else if (digit != NONE) {
-            atomicAdd(&sh[digit], 1u);
-          }
+          count_digit(sh, digit, lane);
         }
       }
     }
     if (pass == PASSES) break;
-    __syncthreads();
-    if (cur != NONE) {
-      unsigned long long* gh = hist_of(T, cur, VIEW, pass);
-      for (uint32_t b = tid; b < nbins; b += kThreads) {
-        const uint32_t c = sh[b];
-        if (c) atomicAdd(gh + b, (unsigned long long)c);
-      }
-    }
+    if (cur != NONE) flush();
     if (!grid_barrier(&T.ctl->barrier[VIEW], phase, T.ctl)) return;
   }
 }
 
-template <int VIEW>
-cudaError_t launch_select(const DevTables& T, uint32_t total_tiles, uint32_t ctas_per_sm, cudaStream_t stream) {
+template <int VIEW, bool MANY>
+cudaError_t launch_select_impl(const DevTables& T, uint32_t total_tiles, uint32_t ctas_per_sm, cudaStream_t stream) {
   if (!total_tiles) return cudaSuccess;
   ProfileScope prof(stream, VIEW == V_SAMPLE ? PT_SAMPLE_SELECT : (VIEW == V_CAND ? PT_CAND_SELECT : PT_DENSE_SELECT));
-  static int resident = 0;                                 // co-resident CTAs per SM of this kernel
+  static std::atomic<int> cached{0};                       // co-resident CTAs per SM of this kernel
+  int resident = cached.load(std::memory_order_relaxed);
   if (resident == 0) {
     int r = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, select_kernel<VIEW>, kThreads, 0) != cudaSuccess || r <= 0)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, select_kernel<VIEW, MANY>, kThreads, 0) != cudaSuccess || r <= 0)
       return cudaErrorLaunchFailure;
     resident = r;
+    cached.store(r, std::memory_order_relaxed);
   }
   const uint32_t per_sm = ctas_per_sm < (uint32_t)resident ? ctas_per_sm : (uint32_t)resident;
   uint32_t grid = (uint32_t)sm_count() * per_sm;
   if (grid > total_tiles) grid = total_tiles;
   DevTables Tc = T;
   void* args[] = {(void*)&Tc, (void*)&total_tiles};
-  cudaError_t e = cudaLaunchCooperativeKernel((const void*)select_kernel<VIEW>, dim3(grid), dim3(kThreads), args, 0, stream);
+  cudaError_t e = cudaLaunchCooperativeKernel((const void*)select_kernel<VIEW, MANY>, dim3(grid), dim3(kThreads), args, 0, stream);
   if (e != cudaSuccess) return e;
   note_launches(1);
   return cudaSuccess;
+}
+
+template <int VIEW>
+cudaError_t launch_select(const DevTables& T, uint32_t total_tiles, uint32_t ctas_per_sm, cudaStream_t stream) {
+  return T.n_scopes > kSmemScopes ? launch_select_impl<VIEW, true>(T, total_tiles, ctas_per_sm, stream)
+                                  : launch_select_impl<VIEW, false>(T, total_tiles, ctas_per_sm, stream);
 }
 
 }  // namespace

@@ -358,6 +358,29 @@ def test_many_layers_and_shards(cuda_device, value_mode):
         run_steps(w, cuda_device, 2, grads=grads)
 
 
+@pytest.mark.parametrize("value_mode", [B.GD_VALUES_FP32, B.GD_VALUES_TWO_MEANS])
+@pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
+def test_many_layers_on_the_predicted_path(cuda_device, scope_mode, value_mode):
+    """A model with a hundred and twenty tensors, long enough (about 12 M elements) to take the predicted path:
+    more scopes than the kernels keep in shared memory, tables too large for a kernel argument, layers that are
+    empty, tiny, unaligned, all zero, or sampled completely."""
+    rng = np.random.default_rng(1234)
+    sizes = [int(x) for x in rng.integers(1, 200_000, size=120)]
+    sizes[3], sizes[4], sizes[50], sizes[77], sizes[119] = 0, 1, 7, 1_000_003, 33
+    w = W.small_layered(len(sizes), sizes, 990_000, scope_mode, value_mode, 5)
+    assert w.n > (1 << 21)
+    grads = []
+    for _ in range(2):
+        g = rng.laplace(0, 1e-3, w.n).astype(np.float32)
+        g[w.layer_off[10]:w.layer_off[11]] = 0.0                          # an all-zero layer: every entry ties
+        lo, hi = w.layer_off[20], w.layer_off[21]
+        g[lo:hi] = np.where(rng.random(hi - lo) < 0.002, g[lo:hi], 0.0)    # fewer non-zeros than k
+        grads.append(torch.from_numpy(g))
+    sess = run_steps(w, cuda_device, 2, grads=grads)
+    st = sess.stats()
+    assert st["n_scopes_predicted"] >= 1
+
+
 # ---------------------------------------------------------------- other drop ratios (Section 5.1: 90 %, 99 %, 99.9 %)
 @pytest.mark.parametrize("drop_ppm", [900_000, 999_000])
 @pytest.mark.parametrize("config", [2, 3])
@@ -680,6 +703,39 @@ def test_random_layouts_and_modes(cuda_device, seed):
     if value_mode == B.GD_VALUES_THRESHOLD and rng.random() < 0.5:
         flags |= B.GD_FLAG_QUANT_ERROR_FEEDBACK      # the +-tau table is exact, so the fed-back residual is too
     run_steps(w, cuda_device, 3, flags=flags, grads=grads, layer_cols=cols, alpha=alpha)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_models_of_many_tensors(cuda_device, seed):
+    """Models of 40 to 400 tensors with log-uniform sizes (1 to 300 k elements, a few of 2 M), long enough for the
+    predicted path: CTAs of the selection kernels cross many scopes, single-tile lists are selected locally,
+    the candidate tiles are renumbered over hundreds of scopes."""
+    rng = np.random.default_rng(7000 + seed)
+    n_layers = int(rng.integers(40, 401))
+    sizes = [int(np.exp(rng.uniform(0, np.log(300_000)))) for _ in range(n_layers)]
+    for _ in range(3):
+        sizes[int(rng.integers(0, n_layers))] = int(rng.integers(1_000_000, 2_000_000))
+    sizes[int(rng.integers(0, n_layers))] = 0
+    ppm = int(rng.choice([900_000, 990_000, 990_000, 999_000]))
+    scope_mode = int(rng.choice([B.GD_SCOPE_PER_LAYER, B.GD_SCOPE_PER_LAYER, B.GD_SCOPE_GLOBAL]))
+    value_mode = int(rng.choice([B.GD_VALUES_FP32, B.GD_VALUES_FP32, B.GD_VALUES_TWO_MEANS, B.GD_VALUES_THRESHOLD]))
+    w = W.small_layered(n_layers, sizes, ppm, scope_mode, value_mode, int(rng.integers(1, 9)))
+    assert w.n > (1 << 21)
+    grads = []
+    for _ in range(2):
+        g = rng.laplace(0, 1e-3, w.n).astype(np.float32)
+        for _ in range(4):                                      # some layers all zero, some nearly so, some tied
+            l = int(rng.integers(0, n_layers))
+            lo, hi = w.layer_off[l], w.layer_off[l + 1]
+            kind = int(rng.integers(0, 3))
+            if kind == 0:
+                g[lo:hi] = 0.0
+            elif kind == 1:
+                g[lo:hi] = np.where(rng.random(hi - lo) < 0.003, g[lo:hi], 0.0)
+            else:
+                g[lo:hi] = rng.choice(np.array([0.0, 0.5, -0.5, 1.0], dtype=np.float32), hi - lo)
+        grads.append(torch.from_numpy(g))
+    run_steps(w, cuda_device, 2, grads=grads, alpha=0.5)
 
 
 def test_config5_full_scale_against_the_oracle(cuda_device):
