@@ -48,12 +48,17 @@ enum {
                                  whole dense vector (same results, more memory traffic) */
   GD_FLAG_SAMPLED_THRESHOLD = 2u, /* the approximation of Section 4: the threshold is selected on a 0.1 %
                                  sample and every entry at or above it is kept (see gd_compress) */
-  GD_FLAG_QUANT_ERROR_FEEDBACK = 4u /* 1-bit value modes only (Section 5.4).  The paper does not say whether
+  GD_FLAG_QUANT_ERROR_FEEDBACK = 4u, /* 1-bit value modes only (Section 5.4).  The paper does not say whether
                                  the error of the 1-bit quantisation is kept; Algorithm 1 keeps only the
                                  dropped mass, which is the default here.  With this flag the residual of a
                                  KEPT entry is v minus the fp32 value the receiver will decode for it (one
                                  fp32 subtraction), as in the error feedback of 1-bit SGD that Section 2
                                  describes, instead of +0; dropped entries are unchanged. */
+  GD_FLAG_NO_EARLY_ZERO = 8u /* an implementation switch with no effect on results (for tests and timing):
+                                 by default the fused pass already writes +0 into the residual slots
+                                 of the entries the sample predicts to be kept, and the compaction
+                                 only settles the few for which the prediction was wrong; with this
+                                 flag the compaction clears every kept slot itself. */
 };
 
 const char* gd_status_string(int status);

@@ -31,6 +31,7 @@ GD_VALUES_COLUMN_MEANS = 3
 GD_FLAG_NO_PREDICTION = 1
 GD_FLAG_SAMPLED_THRESHOLD = 2
 GD_FLAG_QUANT_ERROR_FEEDBACK = 4
+GD_FLAG_NO_EARLY_ZERO = 8
 GD_ERR_OVERFLOW = -7
 
 EXPORTS = [

@@ -428,7 +428,8 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     if (n_sh != n || a->n != n) return GD_ERR_INVALID_ARG;
     if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_COLUMN_MEANS) return GD_ERR_INVALID_ARG;
     if (a->value_mode != GD_VALUES_FP32 && n > (1ull << 31)) return GD_ERR_TOO_LARGE;
-    if (a->flags & ~(uint32_t)(GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD | GD_FLAG_QUANT_ERROR_FEEDBACK))
+    if (a->flags & ~(uint32_t)(GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD | GD_FLAG_QUANT_ERROR_FEEDBACK |
+                               GD_FLAG_NO_EARLY_ZERO))
       return GD_ERR_INVALID_ARG;
     if ((a->flags & GD_FLAG_QUANT_ERROR_FEEDBACK) && a->value_mode == GD_VALUES_FP32) return GD_ERR_INVALID_ARG;
     const bool sampled = (a->flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;

@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
   const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS || T.value_mode == GD_VALUES_COLUMN_MEANS;   // sums are kept
   const bool packed = T.value_mode != GD_VALUES_FP32;
   const bool feedback = (T.flags & GD_FLAG_QUANT_ERROR_FEEDBACK) != 0;   // kept slots keep v for feedback_kernel
+  const bool early = early_zero_enabled(T);
   const uint32_t ltm = lanemask_lt();
   uint4* desc = reinterpret_cast<uint4*>(T.desc_cand);
   // The lists' capacities are a multiple of what they hold.  With few scopes only the tiles that hold
@@ -139,6 +140,11 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
     const float* vals = T.cand_val + d.cand_base;
     const uint32_t tau = st->tau;
     const uint64_t q = st->q;
+    // Entries with key > zthr had +0 written over their residual slot by the fused pass.  Kept ones
+    // need no store then (unless some entry of the scope could not be treated so: early_bad); the few
+    // that are not kept after all get v back.
+    const uint32_t zthr = early ? st->tau_hi : 0xFFFFFFFFu;
+    const bool skip_cleared = early && st->early_bad == 0u;
 
     if (two_means && tid == 0) {
       const uint64_t i_first = T.cand_idx[d.cand_base + beg];
@@ -205,14 +211,16 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
     for (int j = 0; j < ROUNDS; ++j) {
       const bool isgt = (gtm >> j) & 1u, iseq = (eqm >> j) & 1u;
       const uint32_t mg = __ballot_sync(0xFFFFFFFFu, isgt), me = __ballot_sync(0xFFFFFFFFu, iseq);
+      bool kept = false;
       if (isgt || iseq) {
         const uint64_t gb = rg + __popc(mg & ltm), eb = re + __popc(me & ltm);
         if (isgt || eb < q) {
+          kept = true;
           const uint64_t pos = gb + (eb < q ? eb : q);
           const uint64_t idx = ib[j];
           if (pos < d.k && idx < T.n) {
             const uint32_t b = vb[j];
-            if (!feedback) T.residual[idx] = 0.0f;
+            if (!feedback && !(skip_cleared && (b & kAbsMask) > zthr)) T.residual[idx] = 0.0f;
             if (packed) {
               const uint32_t sgn = b >> 31;
               T.out_idx[d.out_base + pos] = (uint32_t)idx | (sgn << 31);
@@ -236,6 +244,9 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
           }
         }
       }
+      // cleared early but not kept after all (the estimate was below tau, or a tie beyond the quota)
+      if (!kept && (vb[j] & kAbsMask) > zthr && wbeg + (uint64_t)j * 32u < end && ib[j] < T.n)
+        T.residual[ib[j]] = __uint_as_float(vb[j]);
       rg += __popc(mg);
       re += __popc(me);
     }

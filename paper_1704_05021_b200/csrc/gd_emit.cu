@@ -72,6 +72,11 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
   uint32_t tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || d.k == 0) ? 0xFFFFFFFFu : T.state[s].tau_lo;
   const bool sampled = (T.flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;   // tau_lo is the threshold itself: keep key >= tau_lo
   if (tau_lo == 0u && !sampled) tau_lo = 1u;
+  // Entries with key > zthr (the sample's estimate of the threshold itself) are almost surely kept:
+  // their residual slot gets +0 right here, in the streaming store, instead of a scattered store later.
+  // Each of them is a candidate, so its value is in the list, from which the compaction puts it back
+  // should it not be kept after all.  Only entries that reached the stash are treated so.
+  const uint32_t zthr = (early_zero_enabled(T) && tau_lo != 0xFFFFFFFFu) ? T.state[s].tau_hi : 0xFFFFFFFFu;
   const uint64_t toff = (uint64_t)warp * 512u + lane * 4u;   // this thread's first element inside a tile
   const uint32_t ltm = lanemask_lt();
   StashEntry* stash = s_stash[warp];
@@ -98,7 +103,6 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
         x[1] = delta ? __fsub_rn(g4[j].y, r4[j].y) : __fadd_rn(g4[j].y, r4[j].y);
         x[2] = delta ? __fsub_rn(g4[j].z, r4[j].z) : __fadd_rn(g4[j].z, r4[j].z);
         x[3] = delta ? __fsub_rn(g4[j].w, r4[j].w) : __fadd_rn(g4[j].w, r4[j].w);
-        *reinterpret_cast<float4*>(T.residual + e0 + j * 128) = make_float4(x[0], x[1], x[2], x[3]);
         uint32_t f = 0;
 #pragma unroll
         for (int c = 0; c < 4; ++c) f |= ((__float_as_uint(x[c]) & kAbsMask) >= tau_lo ? 1u : 0u) << c;
@@ -110,25 +114,30 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
               if (f & (1u << c)) {
-                if (p < kStash) { stash[p].idx = (uint32_t)(e0 + j * 128 + c); stash[p].val = x[c]; }
+                if (p < kStash) {
+                  stash[p].idx = (uint32_t)(e0 + j * 128 + c);
+                  stash[p].val = x[c];
+                  if ((__float_as_uint(x[c]) & kAbsMask) > zthr) x[c] = 0.0f;
+                }
                 ++p;
               }
             }
           }
           wc += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
         }
+        *reinterpret_cast<float4*>(T.residual + e0 + j * 128) = make_float4(x[0], x[1], x[2], x[3]);
       }
     } else if (base < hi && base + kEmitTile > lo) {   // tile cut by the scope (or by the end of the vector)
 #pragma unroll 1
       for (int j = 0; j < 4; ++j) {
         float x[4] = {0.f, 0.f, 0.f, 0.f};
-        uint32_t f = 0;
+        uint32_t f = 0, in = 0;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           const uint64_t e = base + toff + j * 128 + c;
           if (e >= lo && e < hi) {
             x[c] = delta ? __fsub_rn(__ldg(T.grad + e), second[e]) : __fadd_rn(__ldg(T.grad + e), second[e]);
-            T.residual[e] = x[c];
+            in |= 1u << c;
             f |= ((__float_as_uint(x[c]) & kAbsMask) >= tau_lo ? 1u : 0u) << c;
           }
         }
@@ -140,13 +149,20 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
               if (f & (1u << c)) {
-                if (p < kStash) { stash[p].idx = (uint32_t)(base + toff + j * 128 + c); stash[p].val = x[c]; }
+                if (p < kStash) {
+                  stash[p].idx = (uint32_t)(base + toff + j * 128 + c);
+                  stash[p].val = x[c];
+                  if ((__float_as_uint(x[c]) & kAbsMask) > zthr) x[c] = 0.0f;
+                }
                 ++p;
               }
             }
           }
           wc += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
         }
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (in & (1u << c)) T.residual[base + toff + j * 128 + c] = x[c];
       }
     }
     fill += wc;
@@ -198,12 +214,26 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
         const uint64_t dst = excl + s_off[i * kEmitWarps + warp];
         for (uint32_t e = lane; e < c; e += 32) {
           const uint64_t pos = dst + e;
-          if (pos < cap) { cidx[pos] = stash[a + e].idx; cval[pos] = stash[a + e].val; }
+          if (pos < cap) {
+            cidx[pos] = stash[a + e].idx;
+            cval[pos] = stash[a + e].val;
+          } else if ((__float_as_uint(stash[a + e].val) & kAbsMask) > zthr) {
+            // the list is full (the scope will be selected densely): the slot must hold v again
+            T.residual[stash[a + e].idx] = stash[a + e].val;
+            T.state[s].early_bad = 1u;
+          }
         }
         a += c;
       }
     } else {
-      // more candidates than the stash holds: read this warp's elements back (they are v now)
+      // more candidates than the stash holds: read this warp's elements back.  They are v, once the
+      // slots that were cleared early (all of them are in the stash) hold v again; every entry above zthr
+      // is cleared (again) as it goes to the list.
+      if (zthr != 0xFFFFFFFFu) {
+        for (uint32_t e = lane; e < kStash; e += 32)
+          if ((__float_as_uint(stash[e].val) & kAbsMask) > zthr) T.residual[stash[e].idx] = stash[e].val;
+        __syncwarp();
+      }
 #pragma unroll 1
       for (int i = 0; i < CT; ++i) {
         if (s_cnt[i * kEmitWarps + warp] == 0u) continue;
@@ -217,7 +247,7 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
           for (int c = 0; c < 4; ++c) {
             const uint64_t e = base + toff + j * 128 + c;
             if (e >= lo && e < hi) {
-              x[c] = T.residual[e];
+              x[c] = __ldcg(T.residual + e);   // from L2: other lanes may just have put v back
               f |= ((__float_as_uint(x[c]) & kAbsMask) >= tau_lo ? 1u : 0u) << c;
             }
           }
@@ -228,7 +258,11 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
               if (f & (1u << c)) {
-                if (pos < cap) { cidx[pos] = (uint32_t)(base + toff + j * 128 + c); cval[pos] = x[c]; }
+                if (pos < cap) {
+                  cidx[pos] = (uint32_t)(base + toff + j * 128 + c);
+                  cval[pos] = x[c];
+                  if ((__float_as_uint(x[c]) & kAbsMask) > zthr) T.residual[base + toff + j * 128 + c] = 0.0f;
+                }
                 ++pos;
               }
             }

@@ -53,22 +53,19 @@ struct ScopeDesc {       // built on the host for every call, read-only on the d
                          // then count groups, starting at the first multiple of 8 at or after lo
 };
 
-struct SelState {        // running state of one radix selection
-  uint32_t prefix;       // digits fixed so far
-  uint32_t pad;
-  uint64_t rank;         // rank still to find inside the prefix bucket
-  uint64_t gt;           // elements strictly above the prefix bucket so far
-};
-
 struct ScopeState {      // zeroed at the start of every call
   uint64_t cand_count;   // candidates the fused pass counted (may exceed cand_cap)
   uint32_t tau_lo;       // predicted lower bound of the threshold key
   uint32_t tau;          // threshold key: smallest kept |v| bit pattern
   uint64_t q;            // ties at tau that are kept (the lowest indices)
   uint64_t gt;           // entries with key > tau
-  SelState sel[3];       // one per view
-  uint32_t done[3][3];   // finished tiles per view and pass
+  uint32_t tau_hi;       // the sample's estimate of tau itself: the fused pass writes +0 instead of v into the
+                         // residual where key > tau_hi (these entries are almost surely kept; the compaction
+                         // settles the few for which that is wrong, from the candidate list)
+  uint32_t early_bad;    // set when some such entry could not be recorded (a full stash, a full list): the
+                         // compaction then clears every kept slot itself
   uint32_t used_dense;   // 1 if the dense path produced this scope's result
+  uint32_t pad;
 };
 
 struct Ctl {             // zeroed at the start of every call
@@ -232,6 +229,14 @@ __device__ __forceinline__ bool predicted_ok(const DevTables& T, const ScopeDesc
   if (T.flags & GD_FLAG_NO_PREDICTION) return false;
   uint64_t m = st.cand_count;
   return m >= d.k && m <= d.cand_cap;
+}
+
+// True when the fused pass writes +0 over the entries it expects to be kept (ScopeState::tau_hi).  Not
+// with quantisation-error feedback (the kept slots must hold v until the decode table exists), not in
+// sampled-threshold mode (its pack kernel clears the slots), not without a prediction.
+__device__ __forceinline__ bool early_zero_enabled(const DevTables& T) {
+  return (T.flags & (GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD | GD_FLAG_QUANT_ERROR_FEEDBACK |
+                     GD_FLAG_NO_EARLY_ZERO)) == 0u;
 }
 
 // Host-side launchers of the kernel groups (one per .cu file); `tiles` is indexed by Launch.

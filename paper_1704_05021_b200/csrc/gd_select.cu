@@ -95,11 +95,12 @@ __device__ __forceinline__ unsigned long long load_bin(const uint32_t* p) { retu
 // Run by a whole CTA on a finished histogram `gh` (a global one after the grid barrier that completes
 // it, or the CTA's own in shared memory): walks it from the top bin down and fixes the next digit.
 // Every CTA that needs the digit computes it for itself, so no second barrier is needed to hand it around.
+// The same for two ranks at once (one pass over the bins): io[0] and io[1] are replaced by their successors.
 template <typename Bin>
-__device__ SelRun next_digit(const Bin* gh, int bits, SelRun in, Ctl* ctl) {
+__device__ void next_digit_pair(const Bin* gh, int bits, SelRun* io, int count, Ctl* ctl) {
   __shared__ unsigned long long s_warp[kWarps];
-  __shared__ unsigned long long s_acc;
-  __shared__ uint32_t s_digit;
+  __shared__ unsigned long long s_acc[2];
+  __shared__ uint32_t s_digit[2];
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const uint32_t nbins = 1u << bits;
   const uint32_t C = nbins / kThreads;                 // 8 or 4 bins per thread: [top - C + 1, top]
@@ -122,30 +123,41 @@ __device__ SelRun next_digit(const Bin* gh, int bits, SelRun in, Ctl* ctl) {
   __syncthreads();
   unsigned long long above = inc - cs;
   for (uint32_t w = 0; w < warp; ++w) above += s_warp[w];
-  if (tid == kThreads - 1 && above + cs < in.rank) atomicCAS(&ctl->status, (int)GD_OK, (int)GD_ERR_INTERNAL);
-  const bool owner = in.rank == 0 ? (tid == 0) : (above < in.rank && in.rank <= above + cs);
-  if (owner) {
-    uint32_t digit = nbins - 1u;
-    unsigned long long acc = 0;
-    if (in.rank != 0) {
-      acc = above;
+  for (int r = 0; r < count; ++r) {
+    const SelRun in = io[r];
+    if (tid == kThreads - 1 && above + cs < in.rank) atomicCAS(&ctl->status, (int)GD_OK, (int)GD_ERR_INTERNAL);
+    const bool owner = in.rank == 0 ? (tid == 0) : (above < in.rank && in.rank <= above + cs);
+    if (owner) {
+      uint32_t digit = nbins - 1u;
+      unsigned long long acc = 0;
+      if (in.rank != 0) {
+        acc = above;
 #pragma unroll
-      for (uint32_t j = 0; j < 8; ++j) {
-        if (j < C) {
-          if (acc + bin[j] >= in.rank) { digit = top - j; break; }
-          acc += bin[j];
+        for (uint32_t j = 0; j < 8; ++j) {
+          if (j < C) {
+            if (acc + bin[j] >= in.rank) { digit = top - j; break; }
+            acc += bin[j];
+          }
         }
       }
+      s_digit[r] = digit;
+      s_acc[r] = acc;
     }
-    s_digit = digit;
-    s_acc = acc;
   }
   __syncthreads();
-  SelRun out;
-  out.prefix = (in.prefix << bits) | s_digit;
-  out.rank = in.rank - s_acc;
-  out.gt = in.gt + s_acc;
-  return out;
+  for (int r = 0; r < count; ++r) {
+    SelRun out;
+    out.prefix = (io[r].prefix << bits) | s_digit[r];
+    out.rank = io[r].rank - s_acc[r];
+    out.gt = io[r].gt + s_acc[r];
+    io[r] = out;
+  }
+}
+
+template <typename Bin>
+__device__ SelRun next_digit(const Bin* gh, int bits, SelRun in, Ctl* ctl) {
+  next_digit_pair(gh, bits, &in, 1, ctl);
+  return in;
 }
 
 // State of scope s before pass `pass`, recomputed from the finished histograms of the earlier passes.
@@ -156,6 +168,16 @@ __device__ SelRun state_before(const DevTables& T, const ScopeDesc& d, uint32_t 
   r.rank = VIEW == V_SAMPLE ? d.samp_rank : d.k;
   r.gt = 0;
   for (int p = 0; p < pass; ++p) r = next_digit(hist_of(T, s, VIEW, p), p == 0 ? kRadixBits0 : 10, r, T.ctl);
+  return r;
+}
+
+// Rank, in a scope's sample, of the best estimate of the threshold itself: the expected number of
+// samples above it (the prediction tau_lo uses a larger rank, i.e. a lower key, for its margin).
+__device__ __forceinline__ uint64_t rank_hi_of(const ScopeDesc& d) {
+  const uint64_t ns = d.hi - d.lo;
+  uint64_t r = ns ? (d.k * d.samp_m + ns / 2) / ns : 0;     // k <= 2^32, samp_m <= 2^22: no overflow
+  if (r < 1) r = 1;
+  if (r > d.samp_m) r = d.samp_m;
   return r;
 }
 
@@ -194,12 +216,12 @@ __device__ uint32_t block_count_le(const uint32_t* base, uint32_t count, uint32_
 // in every pass (they sit in L2) so that the caller's registers stay free.
 template <int VIEW>
 __device__ __noinline__ SelRun local_select(const DevTables& T, const ScopeDesc& d, uint32_t s, uint32_t len,
-                                            const float* vals, int passes, uint32_t* sh) {
+                                            const float* vals, int passes, uint32_t* sh, uint64_t rank, bool gather) {
   constexpr uint32_t NONE = 0xFFFFFFFFu;
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   SelRun run;
   run.prefix = 0;
-  run.rank = VIEW == V_SAMPLE ? d.samp_rank : d.k;
+  run.rank = rank;
   run.gt = 0;
   for (int p = 0; p < passes; ++p) {
     const int shift = p == 0 ? kShift0 : (p == 1 ? kShift1 : kShift2);
@@ -210,7 +232,7 @@ __device__ __noinline__ SelRun local_select(const DevTables& T, const ScopeDesc&
     for (int j = 0; j < 16; ++j) {
       const uint32_t i = (uint32_t)j * kThreads + tid;
       float x = 0.f;
-      if (i < len) x = (VIEW == V_SAMPLE && p == 0) ? sample_value(T, d, s, i) : vals[i];
+      if (i < len) x = (VIEW == V_SAMPLE && p == 0 && gather) ? sample_value(T, d, s, i) : vals[i];
       keys[j] = __float_as_uint(x);
     }
 #pragma unroll
@@ -218,7 +240,7 @@ __device__ __noinline__ SelRun local_select(const DevTables& T, const ScopeDesc&
       const uint32_t i = (uint32_t)j * kThreads + tid;
       uint32_t digit = NONE;
       if (i < len) {
-        if (VIEW == V_SAMPLE && p == 0) T.samp_val[d.samp_base + i] = __uint_as_float(keys[j]);   // read back by this thread
+        if (VIEW == V_SAMPLE && p == 0 && gather) T.samp_val[d.samp_base + i] = __uint_as_float(keys[j]);   // read back by this thread
         const uint32_t key = keys[j] & kAbsMask;
         if (p == 0 || (key >> pshift) == run.prefix) digit = (key >> shift) & ((1u << bits) - 1u);
       }
@@ -238,7 +260,7 @@ __device__ __noinline__ SelRun local_select(const DevTables& T, const ScopeDesc&
 // run of tiles crosses several scopes, so it keeps a window of the tables from its first scope on, and
 // selects every list of a single tile by itself in shared memory.
 template <int VIEW, bool MANY>
-__global__ void __launch_bounds__(kThreads, MANY ? (VIEW == V_DENSE ? 4 : 2) : 1) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
+__global__ void __launch_bounds__(kThreads, (MANY && VIEW != V_DENSE) ? 2 : 4) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
   constexpr int LK = VIEW == V_SAMPLE ? L_SAMP : (VIEW == V_CAND ? L_CAND : L_DSEL);
   const uint32_t TILE = VIEW == V_DENSE ? T.dense_sel_tile : kTile;
   const int PASSES = VIEW == V_SAMPLE ? (int)T.sample_passes : 3;   // the prediction needs 21 bits only
@@ -293,6 +315,25 @@ __global__ void __launch_bounds__(kThreads, MANY ? (VIEW == V_DENSE ? 4 : 2) : 1
   auto base_of = [&](uint32_t s) -> uint32_t { return (!MANY || s - w0 <= kSmemScopes) ? s_tab.tile0[s - w0] : base[s]; };
   uint32_t phase = 0;
 
+  if (VIEW == V_DENSE && early_zero_enabled(T)) {
+    // Scopes that fall back to the dense range: the fused pass wrote +0 over the entries it expected
+    // to be kept; all of them are in the scope's candidate list, from which v is put back before
+    // anything reads the range.  (Entries that did not fit the list were put back by the fused pass.)
+    const uint64_t gtid = (uint64_t)blockIdx.x * kThreads + tid, gsize = (uint64_t)gridDim.x * kThreads;
+    for (uint32_t x = 0; x < T.n_scopes; ++x) {
+      const ScopeDesc& dx = T.scopes[x];
+      const ScopeState* sx = T.state + x;
+      if (dx.samp_m == 0 || predicted_ok(T, dx, *sx)) continue;
+      const uint64_t mm = sx->cand_count < dx.cand_cap ? sx->cand_count : dx.cand_cap;
+      const uint32_t zthr = sx->tau_hi;
+      for (uint64_t i = gtid; i < mm; i += gsize) {
+        const float v = T.cand_val[dx.cand_base + i];
+        if ((__float_as_uint(v) & kAbsMask) > zthr) T.residual[T.cand_idx[dx.cand_base + i]] = v;
+      }
+    }
+    if (!grid_barrier(&T.ctl->barrier[VIEW], phase, T.ctl)) return;
+  }
+
   for (int pass = 0; pass <= PASSES; ++pass) {
     const int shift = pass == 0 ? kShift0 : (pass == 1 ? kShift1 : kShift2);
     const int bits = pass == 0 ? kRadixBits0 : 10;
@@ -306,12 +347,15 @@ __global__ void __launch_bounds__(kThreads, MANY ? (VIEW == V_DENSE ? 4 : 2) : 1
     uint32_t s = w0;
     bool active = false, have_run = false, zero_case = false, local = false;
     uint64_t len = 0;
-    uint32_t prefix = 0;
+    uint32_t prefix = 0, prefix_b = NONE;               // prefix_b: first digit of the second rank (sample view)
     const float* vals = nullptr;
+    // In the second pass over a sample the upper half of the shared histogram counts the keys under the
+    // second rank's first digit; the two halves go to the second and third histogram slots, which are adjacent.
+    const uint32_t flush_bins = (VIEW == V_SAMPLE && PASSES == 2 && pass == 1) ? 2048u : nbins;
     auto flush = [&]() {                                // adds the shared histogram to scope cur's global one
       __syncthreads();
       unsigned long long* gh = hist_of(T, cur, VIEW, pass);
-      for (uint32_t b = tid; b < nbins; b += kThreads) {
+      for (uint32_t b = tid; b < flush_bins; b += kThreads) {
         const uint32_t c = sh[b];
         if (c) atomicAdd(gh + b, (unsigned long long)c);
         sh[b] = 0;
@@ -349,12 +393,16 @@ __global__ void __launch_bounds__(kThreads, MANY ? (VIEW == V_DENSE ? 4 : 2) : 1
       if (local) {
         if (pass != 0 || lt != 0) continue;
         if (cur != NONE) flush();                       // the shared histogram must be free (and is zero)
-        const SelRun run = local_select<VIEW>(T, d, s, (uint32_t)len, vals, PASSES, sh);
+        const SelRun run = local_select<VIEW>(T, d, s, (uint32_t)len, vals, PASSES, sh,
+                                              VIEW == V_SAMPLE ? d.samp_rank : d.k, true);
+        uint32_t tau_hi = 0;
+        if (VIEW == V_SAMPLE && PASSES == 2)
+          tau_hi = local_select<VIEW>(T, d, s, (uint32_t)len, vals, PASSES, sh, rank_hi_of(d), false).prefix << kShift1;
         if (tid == 0) {
           ScopeState* st = T.state + s;
           if (VIEW == V_SAMPLE) {
             st->tau_lo = PASSES == 3 ? run.prefix : run.prefix << kShift1;
-            if (PASSES == 3) st->tau = run.prefix;
+            if (PASSES == 3) st->tau = run.prefix; else st->tau_hi = tau_hi;
           } else {
             st->tau = run.prefix; st->q = run.rank; st->gt = run.gt;
             if (VIEW == V_DENSE) st->used_dense = 1u;
@@ -365,7 +413,30 @@ __global__ void __launch_bounds__(kThreads, MANY ? (VIEW == V_DENSE ? 4 : 2) : 1
       const uint64_t beg = (uint64_t)lt * TILE;
       if (pass == PASSES ? lt != 0 : beg >= len) continue;
       if (pass > 0 && !have_run) {                      // digits fixed by the earlier passes
-        const SelRun run = state_before<VIEW>(T, d, s, pass);
+        SelRun run;
+        uint32_t tau_hi = 0;
+        if (VIEW == V_SAMPLE && PASSES == 2) {
+          // Two ranks walk the histograms together: the prediction's, and the rank of the estimate of
+          // tau itself.  Their first digits may differ; the second rank's second-pass histogram is then
+          // the one kept in the third slot.
+          SelRun two[2];
+          two[0].prefix = 0; two[0].rank = d.samp_rank; two[0].gt = 0;
+          two[1].prefix = 0; two[1].rank = rank_hi_of(d); two[1].gt = 0;
+          next_digit_pair(hist_of(T, s, VIEW, 0), kRadixBits0, two, 2, T.ctl);
+          prefix_b = two[1].prefix;
+          if (pass == PASSES) {
+            if (two[1].prefix == two[0].prefix) {
+              next_digit_pair(hist_of(T, s, VIEW, 1), 10, two, 2, T.ctl);
+            } else {
+              two[0] = next_digit(hist_of(T, s, VIEW, 1), 10, two[0], T.ctl);
+              two[1] = next_digit(hist_of(T, s, VIEW, 2), 10, two[1], T.ctl);
+            }
+            tau_hi = two[1].prefix << kShift1;
+          }
+          run = two[0];
+        } else {
+          run = state_before<VIEW>(T, d, s, pass);
+        }
         have_run = true;
         prefix = run.prefix;
         if (pass == PASSES && tid == 0) {               // the CTA with the scope's first tile records the result
@@ -373,7 +444,7 @@ __global__ void __launch_bounds__(kThreads, MANY ? (VIEW == V_DENSE ? 4 : 2) : 1
           if (VIEW == V_SAMPLE) {
             // prediction: lower edge of the 21-bit bucket; sampled-threshold mode: the full key, which is the result
             st->tau_lo = PASSES == 3 ? run.prefix : run.prefix << kShift1;
-            if (PASSES == 3) st->tau = run.prefix;
+            if (PASSES == 3) st->tau = run.prefix; else st->tau_hi = tau_hi;
           } else {
             st->tau = run.prefix; st->q = run.rank; st->gt = run.gt;
             if (VIEW == V_DENSE) st->used_dense = 1u;
@@ -407,8 +478,15 @@ __global__ void __launch_bounds__(kThreads, MANY ? (VIEW == V_DENSE ? 4 : 2) : 1
             if (VIEW == V_SAMPLE && pass == 0) T.samp_val[d.samp_base + i] = __uint_as_float(keys[j]);
             const uint32_t key = keys[j] & kAbsMask;
             if (pass == 0 || (key >> pshift) == prefix) digit = (key >> shift) & (nbins - 1u);
+            else if (VIEW == V_SAMPLE && pass == 1 && (key >> pshift) == prefix_b) digit = 1024u + ((key >> shift) & 1023u);
           }
-          count_digit(sh, digit, lane);
+          // (written out here rather than through count_digit(): the adds must be seen to hit shared memory)
+          const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, digit, 0);
+          if (__all_sync(0xFFFFFFFFu, digit == d0)) {
+            if (lane == 0 && d0 != NONE) atomicAdd(&sh[d0], 32u);
+          } else if (digit != NONE) {
+            atomicAdd(&sh[digit], 1u);
+          }
         }
       }
     }

@@ -101,10 +101,11 @@ def test_config1_five_steps(cuda_device, flags):
     run_steps(W.workload(1), cuda_device, 5, flags=flags, expect_dense=True)     # short vectors are selected densely
 
 
-@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION, B.GD_FLAG_NO_EARLY_ZERO])
 def test_config1_shape_at_2_23(cuda_device, flags):
     """The same distribution just above the length where the prediction is switched on."""
-    run_steps(W.workload(1, scale_log2=23), cuda_device, 3, flags=flags, method="select", expect_dense=bool(flags))
+    run_steps(W.workload(1, scale_log2=23), cuda_device, 3, flags=flags, method="select",
+              expect_dense=bool(flags & B.GD_FLAG_NO_PREDICTION))
 
 
 # ---------------------------------------------------------------- edge sizes and drop ratios
@@ -155,6 +156,33 @@ def test_heavy_ties(cuda_device, flags):
             w = W.small_layered(3, [100_000, 7, n - 100_007], 990_000, scope_mode, B.GD_VALUES_FP32, 2)
             w.name = name
             run_steps(w, cuda_device, 2, flags=flags, grads=[torch.from_numpy(g), torch.from_numpy(g)])
+
+
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_EARLY_ZERO])
+def test_ties_and_dense_runs_on_the_predicted_path(cuda_device, flags):
+    """Vectors long enough for the prediction (above 2^21 elements), shaped to reach every branch behind it:
+    lists that overflow (the scope is then selected densely, after the slots cleared early got v back), warps
+    whose stash overflows (runs of candidates), estimates of tau above and below the real one, ties at the cut."""
+    rng = np.random.default_rng(17)
+    n = (1 << 22) + 12_345
+    one_up = np.frombuffer(np.uint32(0x3F800001).tobytes(), dtype=np.float32)[0]       # just above a bucket edge
+    base = (rng.laplace(0, 1e-3, n)).astype(np.float32)
+    cases = {}
+    g = base.copy(); g[rng.random(n) < 0.4] = one_up; cases["many_ties_above_a_bucket_edge"] = g
+    g = base.copy(); g[1_000_000:1_005_000] = 0.5; g[3_000_000:3_002_000] = -0.75; cases["runs_of_kept_entries"] = g
+    g = base.copy(); g[500_000:540_000] = np.float32(6.5e-3) * rng.choice([-1, 1], 40_000).astype(np.float32)
+    cases["run_of_ties_around_the_cut"] = g                      # about k entries share one magnitude near tau
+    g = np.where(rng.random(n) < 0.012, rng.standard_normal(n), 0.0).astype(np.float32)
+    cases["mostly_zero_just_above_k_nonzeros"] = g
+    g = np.where(rng.random(n) < 0.008, rng.standard_normal(n), 0.0).astype(np.float32)
+    cases["mostly_zero_fewer_nonzeros_than_k"] = g
+    cases["all_equal"] = np.full(n, -2.5, np.float32)
+    g = base.copy(); g[::3] *= 40.0; cases["a_third_forty_times_larger"] = g
+    for name, g in cases.items():
+        for scope_mode in (B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER):
+            w = W.small_layered(3, [1_500_000, 7, n - 1_500_007], 990_000, scope_mode, B.GD_VALUES_FP32, 2)
+            w.name = name
+            run_steps(w, cuda_device, 2, flags=flags, grads=[torch.from_numpy(g), torch.from_numpy(-g)])
 
 
 def test_signed_zero_and_subnormals(cuda_device):
@@ -700,6 +728,8 @@ def test_random_layouts_and_modes(cuda_device, seed):
             g = rng.choice(np.array([0.0, 0.25, -0.25, 0.5, 1.0, -2.0]), w.n)           # few distinct values
         grads.append(torch.from_numpy(g.astype(np.float32)))
     alpha = float(rng.choice([1.0, 0.5, -1.25]))
+    if flags == 0 and rng.random() < 0.3:
+        flags = B.GD_FLAG_NO_EARLY_ZERO
     if value_mode == B.GD_VALUES_THRESHOLD and rng.random() < 0.5:
         flags |= B.GD_FLAG_QUANT_ERROR_FEEDBACK      # the +-tau table is exact, so the fed-back residual is too
     run_steps(w, cuda_device, 3, flags=flags, grads=grads, layer_cols=cols, alpha=alpha)
@@ -735,7 +765,7 @@ def test_random_models_of_many_tensors(cuda_device, seed):
             else:
                 g[lo:hi] = rng.choice(np.array([0.0, 0.5, -0.5, 1.0], dtype=np.float32), hi - lo)
         grads.append(torch.from_numpy(g))
-    run_steps(w, cuda_device, 2, grads=grads, alpha=0.5)
+    run_steps(w, cuda_device, 2, grads=grads, alpha=0.5, flags=int(rng.choice([0, 0, B.GD_FLAG_NO_EARLY_ZERO])))
 
 
 def test_config5_full_scale_against_the_oracle(cuda_device):
