@@ -487,8 +487,9 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
 }
 
 // Sampled-threshold mode: the candidate lists ARE the survivors.  Copies every scope's list to its
-// place in the output (scopes concatenated in index order), clears the survivors' residual slots,
-// and lets the last CTA finish the call with the survivor count found here.
+// place in the output (scopes concatenated in index order), clears the survivors' residual slots
+// unless the fused pass has done so already, and lets the last CTA finish the call with the survivor
+// count found here.
 __global__ void __launch_bounds__(kThreads) pack_sampled_kernel(const __grid_constant__ DevTables T) {
   __shared__ unsigned long long s_part[kWarps];
   __shared__ unsigned long long s_off;
@@ -522,6 +523,7 @@ __global__ void __launch_bounds__(kThreads) pack_sampled_kernel(const __grid_con
     __syncthreads();
     return s_off;
   };
+  const bool cleared = !(T.flags & GD_FLAG_NO_EARLY_ZERO);   // the fused pass wrote +0 over every listed survivor's slot
   const unsigned long long m_all = T.state[s].cand_count;
   const uint64_t m = m_all < d.cand_cap ? m_all : d.cand_cap;
   const uint64_t beg = (uint64_t)(t - tile0[s]) * kTile;
@@ -541,7 +543,7 @@ __global__ void __launch_bounds__(kThreads) pack_sampled_kernel(const __grid_con
       if (i < end && ib[j] < T.n && out_off + i < T.k_total) {
         T.out_idx[out_off + i] = ib[j];
         T.out_val[out_off + i] = __uint_as_float(vb[j]);
-        T.residual[ib[j]] = 0.0f;
+        if (!cleared) T.residual[ib[j]] = 0.0f;
         if (T.delta_base) T.delta_base[ib[j]] = __fadd_rn(T.delta_base[ib[j]], __uint_as_float(vb[j]));
       }
     }

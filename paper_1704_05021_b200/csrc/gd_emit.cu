@@ -72,11 +72,16 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
   uint32_t tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || d.k == 0) ? 0xFFFFFFFFu : T.state[s].tau_lo;
   const bool sampled = (T.flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;   // tau_lo is the threshold itself: keep key >= tau_lo
   if (tau_lo == 0u && !sampled) tau_lo = 1u;
-  // Entries with key > zthr (the sample's estimate of the threshold itself) are almost surely kept:
+  // Entries with key >= zmin (above tau_hi, the sample's estimate of the threshold itself) are almost surely kept:
   // their residual slot gets +0 right here, in the streaming store, instead of a scattered store later.
   // Each of them is a candidate, so its value is in the list, from which the compaction puts it back
   // should it not be kept after all.  Only entries that reached the stash are treated so.
-  const uint32_t zthr = (early_zero_enabled(T) && tau_lo != 0xFFFFFFFFu) ? T.state[s].tau_hi : 0xFFFFFFFFu;
+  // In sampled-threshold mode every candidate is kept, so every candidate is treated so.
+  uint32_t zmin = 0xFFFFFFFFu;               // smallest key cleared early (keys are at most 0x7FFFFFFF: none)
+  if (tau_lo != 0xFFFFFFFFu) {
+    if (sampled) { if (!(T.flags & GD_FLAG_NO_EARLY_ZERO)) zmin = tau_lo; }
+    else if (early_zero_enabled(T)) zmin = T.state[s].tau_hi + 1u;
+  }
   const uint64_t toff = (uint64_t)warp * 512u + lane * 4u;   // this thread's first element inside a tile
   const uint32_t ltm = lanemask_lt();
   StashEntry* stash = s_stash[warp];
@@ -117,7 +122,7 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
                 if (p < kStash) {
                   stash[p].idx = (uint32_t)(e0 + j * 128 + c);
                   stash[p].val = x[c];
-                  if ((__float_as_uint(x[c]) & kAbsMask) > zthr) x[c] = 0.0f;
+                  if ((__float_as_uint(x[c]) & kAbsMask) >= zmin) x[c] = 0.0f;
                 }
                 ++p;
               }
@@ -152,7 +157,7 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
                 if (p < kStash) {
                   stash[p].idx = (uint32_t)(base + toff + j * 128 + c);
                   stash[p].val = x[c];
-                  if ((__float_as_uint(x[c]) & kAbsMask) > zthr) x[c] = 0.0f;
+                  if ((__float_as_uint(x[c]) & kAbsMask) >= zmin) x[c] = 0.0f;
                 }
                 ++p;
               }
@@ -217,7 +222,7 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
           if (pos < cap) {
             cidx[pos] = stash[a + e].idx;
             cval[pos] = stash[a + e].val;
-          } else if ((__float_as_uint(stash[a + e].val) & kAbsMask) > zthr) {
+          } else if ((__float_as_uint(stash[a + e].val) & kAbsMask) >= zmin) {
             // the list is full (the scope will be selected densely): the slot must hold v again
             T.residual[stash[a + e].idx] = stash[a + e].val;
             T.state[s].early_bad = 1u;
@@ -227,11 +232,11 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
       }
     } else {
       // more candidates than the stash holds: read this warp's elements back.  They are v, once the
-      // slots that were cleared early (all of them are in the stash) hold v again; every entry above zthr
+      // slots that were cleared early (all of them are in the stash) hold v again; every entry at or above zmin
       // is cleared (again) as it goes to the list.
-      if (zthr != 0xFFFFFFFFu) {
+      if (zmin != 0xFFFFFFFFu) {
         for (uint32_t e = lane; e < kStash; e += 32)
-          if ((__float_as_uint(stash[e].val) & kAbsMask) > zthr) T.residual[stash[e].idx] = stash[e].val;
+          if ((__float_as_uint(stash[e].val) & kAbsMask) >= zmin) T.residual[stash[e].idx] = stash[e].val;
         __syncwarp();
       }
 #pragma unroll 1
@@ -261,7 +266,7 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
                 if (pos < cap) {
                   cidx[pos] = (uint32_t)(base + toff + j * 128 + c);
                   cval[pos] = x[c];
-                  if ((__float_as_uint(x[c]) & kAbsMask) > zthr) T.residual[base + toff + j * 128 + c] = 0.0f;
+                  if ((__float_as_uint(x[c]) & kAbsMask) >= zmin) T.residual[base + toff + j * 128 + c] = 0.0f;
                 }
                 ++pos;
               }

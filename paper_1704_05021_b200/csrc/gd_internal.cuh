@@ -232,8 +232,8 @@ __device__ __forceinline__ bool predicted_ok(const DevTables& T, const ScopeDesc
 }
 
 // True when the fused pass writes +0 over the entries it expects to be kept (ScopeState::tau_hi).  Not
-// with quantisation-error feedback (the kept slots must hold v until the decode table exists), not in
-// sampled-threshold mode (its pack kernel clears the slots), not without a prediction.
+// with quantisation-error feedback (the kept slots must hold v until the decode table exists), not
+// without a prediction.  (Sampled-threshold mode has its own, simpler form: every candidate is kept.)
 __device__ __forceinline__ bool early_zero_enabled(const DevTables& T) {
   return (T.flags & (GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD | GD_FLAG_QUANT_ERROR_FEEDBACK |
                      GD_FLAG_NO_EARLY_ZERO)) == 0u;

@@ -530,14 +530,15 @@ def compare_sampled(sess, exp, tag):
     assert np.array_equal(_np_u32(sess.out_shard_cnt_off), exp["shard_cnt_off"]), f"{tag}: shard offsets"
 
 
+@pytest.mark.parametrize("extra_flags", [0, B.GD_FLAG_NO_EARLY_ZERO])
 @pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
-def test_sampled_threshold_matches_oracle(cuda_device, scope_mode):
+def test_sampled_threshold_matches_oracle(cuda_device, scope_mode, extra_flags):
     rng = np.random.default_rng(61)
     sizes = [3000, 0, 4096, 4097, 10, 700_001, 64_000]           # whole-scope samples, 4096-sample scopes, a 0.1 % scope
     for ppm in (990_000, 900_000, 1_000_000):
         w = W.small_layered(len(sizes), sizes, ppm, scope_mode, B.GD_VALUES_FP32, 3)
         sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
-                               B.GD_FLAG_SAMPLED_THRESHOLD, cuda_device)
+                               B.GD_FLAG_SAMPLED_THRESHOLD | extra_flags, cuda_device)
         params = torch.zeros(w.n, dtype=torch.float32, device=cuda_device)
         views = sess.shard_views(params)
         r_host = orc.residual_reset(w.n)
