@@ -59,7 +59,10 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
   load_tables(T, L_EMIT, &s_tab, &scopes, &tile0);
   __syncthreads();
   const uint32_t t = s_chunk;
-  const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
+  // With more scopes than the shared tables hold, the chunk's scope is found by one CTA-wide count
+  // over the global table (a binary search there would be a chain of dependent loads).
+  const uint32_t s = T.n_scopes <= kSmemScopes ? scope_of_tile(tile0, T.n_scopes, t)
+                                                : block_count_le(tile0, T.n_scopes, t) - 1u;
   const ScopeDesc& d = scopes[s];
   const uint64_t lo = d.lo, hi = d.hi;
   const uint32_t first = tile0[s], nchunks = tile0[s + 1] - first;

@@ -175,6 +175,23 @@ __device__ __forceinline__ void block_inclusive_scan(uint32_t* a, uint32_t n) {
   __syncthreads();
 }
 
+// Number of entries of the ascending table base[0 .. count) that are <= t, counted by the whole CTA
+// in one round of loads (a binary search would be a chain of dependent global loads).
+__device__ __forceinline__ uint32_t block_count_le(const uint32_t* base, uint32_t count, uint32_t t) {
+  __shared__ uint32_t s_cnt;
+  if (threadIdx.x == 0) s_cnt = 0;
+  __syncthreads();
+  uint32_t c = 0;
+  for (uint32_t i = threadIdx.x; i < count; i += blockDim.x) c += base[i] <= t ? 1u : 0u;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+  if ((threadIdx.x & 31u) == 0 && c) atomicAdd(&s_cnt, c);
+  __syncthreads();
+  const uint32_t r = s_cnt;
+  __syncthreads();
+  return r;
+}
+
 // Called by all threads of a CTA; the caller synchronises before using the result.  Returns the
 // tables to use: the shared copy when the scopes fit, else the global ones.
 __device__ __forceinline__ void load_tables(const DevTables& T, int launch_kind, SmemTables* sm,

@@ -194,23 +194,6 @@ __device__ __forceinline__ void count_digit(uint32_t* sh, uint32_t digit, uint32
   }
 }
 
-// Number of entries of the ascending table base[0 .. count) that are <= t, counted by the whole CTA
-// in one round of loads (a binary search would be a chain of dependent global loads).
-__device__ uint32_t block_count_le(const uint32_t* base, uint32_t count, uint32_t t) {
-  __shared__ uint32_t s_cnt;
-  if (threadIdx.x == 0) s_cnt = 0;
-  __syncthreads();
-  uint32_t c = 0;
-  for (uint32_t i = threadIdx.x; i < count; i += kThreads) c += base[i] <= t ? 1u : 0u;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
-  if ((threadIdx.x & 31u) == 0 && c) atomicAdd(&s_cnt, c);
-  __syncthreads();
-  const uint32_t r = s_cnt;
-  __syncthreads();
-  return r;
-}
-
 // The whole selection of a list of at most kTile entries, by one CTA in its shared histogram `sh`
 // (all zero on entry and on return): no global histogram, no grid barrier.  The entries are read again
 // in every pass (they sit in L2) so that the caller's registers stay free.
