@@ -102,3 +102,45 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(gd_build, "LIB_PATH", str(tmp_path / "libgd.so"))
     with pytest.raises(RuntimeError):
         B.load_library()
+
+
+def test_header_is_plain_c_and_links_from_c(lib, tmp_path):
+    """include/gd.h compiles as C99 without CUDA headers, and a C program links against libgd.so and calls the
+    host-only entry points (sizes, counts, status strings: nothing that needs a GPU)."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler here")
+    src = tmp_path / "use_gd.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include "gd.h"
+int main(void) {
+  uint64_t k = 0, total = 0, cap = 0, pairs = 0;
+  size_t ws = 0, aws = 0;
+  const uint64_t layer_off[3] = {0, 1000000, 1048576};
+  const uint32_t cols[2] = {1000, 1};
+  gd_compress_args a;
+  gd_apply_args b;
+  gd_push p;
+  (void)a; (void)b; (void)p;
+  if (gd_kept_count(1048576, 990000, &k) != GD_OK || k != 10486) return 1;
+  if (gd_total_kept(layer_off, 2, GD_SCOPE_PER_LAYER, 990000, &total) != GD_OK || total != 10000 + 486) return 2;
+  if (gd_sampled_capacity(layer_off, 2, GD_SCOPE_GLOBAL, 990000, &cap) != GD_OK || cap < k) return 3;
+  if (gd_means_pairs(2, cols, GD_VALUES_COLUMN_MEANS, &pairs) != GD_OK || pairs != 1001) return 4;
+  if (gd_workspace_bytes(layer_off, 2, cols, 4, GD_SCOPE_PER_LAYER, 990000, &ws) != GD_OK || ws == 0) return 5;
+  if (gd_apply_workspace_bytes(4, 2, &aws) != GD_OK || aws == 0) return 6;
+  if (gd_compress(NULL, NULL) != GD_ERR_INVALID_ARG) return 7;
+  printf("%s|%llu|%llu\n", gd_status_string(GD_ERR_WORKSPACE), (unsigned long long)k, (unsigned long long)total);
+  return 0;
+}
+''')
+    exe = tmp_path / "use_gd"
+    libdir = os.path.dirname(gd_build.LIB_PATH)
+    cmd = ["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"), str(src),
+           "-L", libdir, "-l:libgd.so", "-Wl,-rpath," + libdir, "-o", str(exe)]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    assert res.returncode == 0, res.stderr
+    out = subprocess.run([str(exe)], capture_output=True, text=True, timeout=120)
+    assert out.returncode == 0, (out.returncode, out.stderr)
+    assert out.stdout.strip() == "workspace missing or too small|10486|10486"
