@@ -736,6 +736,20 @@ def test_random_layouts_and_modes(cuda_device, seed):
     run_steps(w, cuda_device, 3, flags=flags, grads=grads, layer_cols=cols, alpha=alpha)
 
 
+@pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
+def test_more_scopes_than_the_tile_table_holds(cuda_device, scope_mode):
+    """2600 tensors: more scopes than the shared-memory table of candidate tiles covers (2048), so the kernels over the
+    candidate lists fall back to the numbering by capacity and to the tables in global memory."""
+    rng = np.random.default_rng(2600)
+    sizes = [int(x) for x in rng.integers(1, 2000, size=2600)]
+    sizes[100], sizes[1500], sizes[2599] = 700_000, 300_000, 5
+    w = W.small_layered(len(sizes), sizes, 990_000, scope_mode, B.GD_VALUES_FP32, 3)
+    assert w.n > (1 << 21)
+    grads = [torch.from_numpy(rng.laplace(0, 1e-3, w.n).astype(np.float32)) for _ in range(2)]
+    sess = run_steps(w, cuda_device, 2, grads=grads)
+    assert sess.stats()["n_scopes_predicted"] >= 1
+
+
 @pytest.mark.parametrize("seed", range(6))
 def test_random_models_of_many_tensors(cuda_device, seed):
     """Models of 40 to 400 tensors with log-uniform sizes (1 to 300 k elements, a few of 2 M), long enough for the
