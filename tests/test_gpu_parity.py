@@ -490,13 +490,19 @@ def test_three_workers_push_into_each_server(cuda_device, value_mode):
 
 # ---------------------------------------------------------------- parameter pulls as dropped deltas
 @pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
-def test_delta_pull_matches_oracle_and_client_copy(cuda_device, flags):
+@pytest.mark.parametrize("layout", ["short", "long_global", "long_per_layer", "long_many"])
+def test_delta_pull_matches_oracle_and_client_copy(cuda_device, flags, layout):
     """Section 4, third paragraph: the server sends GradDrop(params - last pulled copy).  The library's
     delta mode must equal the oracle bit for bit, and the server's record of the client's copy must stay
     identical to what the client holds after applying the pull with alpha = 1."""
     rng = np.random.default_rng(23)
-    sizes = [70_000, 9, 4096, 130_003]
-    w = W.small_layered(len(sizes), sizes, 980_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 2)
+    # short vectors are selected densely; the long ones take the predicted path (fused subtraction, candidates,
+    # slots cleared in the stream), the last one with more scopes than the kernels keep in shared memory
+    sizes = {"short": [70_000, 9, 4096, 130_003], "long_global": [1_500_000, 9, 4096, 900_003],
+             "long_per_layer": [1_500_000, 9, 4096, 900_003],
+             "long_many": [1_200_000] + [int(x) for x in rng.integers(1, 6000, size=50)] + [1_000_000]}[layout]
+    scope = B.GD_SCOPE_GLOBAL if layout in ("short", "long_global") else B.GD_SCOPE_PER_LAYER
+    w = W.small_layered(len(sizes), sizes, 980_000, scope, B.GD_VALUES_FP32, 2)
     sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, flags, cuda_device)
     p_host = (rng.standard_normal(w.n) * 0.1).astype(np.float32)
     last_host = np.zeros(w.n, dtype=np.float32)
@@ -554,6 +560,24 @@ def test_sampled_threshold_matches_oracle(cuda_device, scope_mode, extra_flags):
             r_host = exp["residual"]
         torch.cuda.synchronize()
         assert np.array_equal(_np_u32(params), sent.view(np.uint32))
+
+
+def test_sampled_threshold_with_many_scopes(cuda_device):
+    """Sixty tensors, each its own scope (the many-scope instantiation of the selection kernel, where lists of a
+    single tile are selected inside one CTA), in sampled-threshold mode with its three radix passes."""
+    rng = np.random.default_rng(62)
+    sizes = [int(x) for x in rng.integers(1, 9000, size=56)] + [0, 4096, 250_000, 1_200_000]
+    w = W.small_layered(len(sizes), sizes, 990_000, B.GD_SCOPE_PER_LAYER, B.GD_VALUES_FP32, 4)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
+                           B.GD_FLAG_SAMPLED_THRESHOLD, cuda_device)
+    r_host = orc.residual_reset(w.n)
+    for step in range(3):
+        g = rng.laplace(0, 1e-3, w.n).astype(np.float32)
+        g[rng.random(w.n) < 0.1] = 0.0
+        exp = orc.compress_sampled(g, r_host, w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode)
+        sess.compress(torch.from_numpy(g).to(cuda_device))
+        compare_sampled(sess, exp, f"sampled, 60 scopes, step {step}")
+        r_host = exp["residual"]
 
 
 def test_sampled_threshold_on_workload_shapes(cuda_device):
@@ -664,7 +688,7 @@ def test_quantisation_error_feedback(cuda_device, flags, scope_mode, value_mode)
     """Kept slots hold v - decoded instead of +0.  The kept magnitudes of a layer span far less than 2^18, so
     the fp64 sums behind the means are exact in any order and the residual is compared bit for bit, over
     three steps with the residual carried (a difference in step 1 would change the selection of step 2)."""
-    shapes = [(600, 50), (4097,), (128, 1000), (3,), (5000, 8)]
+    shapes = [(600, 50), (4097,), (128, 1000), (3,), (5000, 8), (2300, 1000)]   # 2.5 M elements: the predicted path
     sizes = [int(np.prod(s_)) for s_ in shapes]
     cols = [s_[-1] if len(s_) > 1 else 1 for s_ in shapes] if value_mode == B.GD_VALUES_COLUMN_MEANS else None
     rng = np.random.default_rng(4242)
