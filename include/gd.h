@@ -15,7 +15,9 @@
  *   - Every function returns a gd_status_t.  Argument errors are detected on the host before
  *     anything is enqueued.  Conditions detected on the device (a bounded wait that ran out,
  *     an inconsistent count) are written to a status word in the workspace and are returned
- *     by gd_status(); device code never traps, asserts or spins without a limit.
+ *     by gd_status(); device code never traps, asserts or spins without a limit.  After such a
+ *     status the outputs AND the residual of that call are undefined (the call updates the
+ *     residual in place); a caller that wants to retry keeps its own copy of the residual.
  *   - No CUDA headers are needed to include this file.
  */
 #ifndef GD_H
