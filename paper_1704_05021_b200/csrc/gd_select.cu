@@ -443,22 +443,34 @@ __global__ void __launch_bounds__(kThreads, (MANY && VIEW != V_DENSE) ? 2 : 4) s
       // batches of 16 elements per thread: all loads of a batch are in flight before the first is used
       for (uint64_t b0 = beg; b0 < end; b0 += kTile) {
         uint32_t keys[16];
+        const bool gather = VIEW == V_SAMPLE && pass == 0;
+        // a whole batch inside the list (the usual case): no bounds checks, one address computation
+        const bool whole = b0 + kTile <= end;
+        const uint32_t valid = whole ? kTile : (uint32_t)(end - b0);   // elements of this batch
+        if (gather) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const uint64_t i = b0 + (uint64_t)j * kThreads + tid;
-          float x = 0.f;
-          if (i < end) {
-            if (VIEW == V_SAMPLE && pass == 0) x = sample_value(T, d, s, i);
-            else x = vals[i];
+          for (int j = 0; j < 16; ++j) {
+            const uint32_t o = (uint32_t)j * kThreads + tid;
+            keys[j] = o < valid ? __float_as_uint(sample_value(T, d, s, b0 + o)) : 0u;
           }
-          keys[j] = __float_as_uint(x);
+        } else if (whole) {
+          const float* src = vals + b0 + tid;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) keys[j] = __float_as_uint(src[j * kThreads]);
+        } else {
+          const float* src = vals + b0;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const uint32_t o = (uint32_t)j * kThreads + tid;
+            keys[j] = o < valid ? __float_as_uint(src[o]) : 0u;
+          }
         }
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const uint64_t i = b0 + (uint64_t)j * kThreads + tid;
+          const uint32_t o = (uint32_t)j * kThreads + tid;
           uint32_t digit = NONE;                                           // "does not count"
-          if (i < end) {
-            if (VIEW == V_SAMPLE && pass == 0) T.samp_val[d.samp_base + i] = __uint_as_float(keys[j]);
+          if (whole || o < valid) {
+            if (gather) T.samp_val[d.samp_base + b0 + o] = __uint_as_float(keys[j]);
             const uint32_t key = keys[j] & kAbsMask;
             if (pass == 0 || (key >> pshift) == prefix) digit = (key >> shift) & (nbins - 1u);
             else if (VIEW == V_SAMPLE && pass == 1 && (key >> pshift) == prefix_b) digit = 1024u + ((key >> shift) & 1023u);
