@@ -155,27 +155,36 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
       s_single = (l0 == l1 && T.layer_cols[l0] == 1u) ? 1 : 0;
     }
 
-    // phase 1: load, classify, count
-    const uint64_t wbeg = beg + (uint64_t)warp * (32u * ROUNDS) + lane;
+    // phase 1: load, classify, count.  Offsets inside the tile are 32-bit; a whole tile skips the bounds checks.
+    const uint32_t wofs = warp * (32u * ROUNDS) + lane;          // this thread's first element inside the tile
+    const uint32_t valid = (uint32_t)(end - beg);                // elements of this tile
+    const bool whole = valid == kTile;
+    const uint32_t* tile_idx = T.cand_idx + d.cand_base + beg;
+    const float* tile_val = vals + beg;
     uint32_t vb[ROUNDS], ib[ROUNDS];
     uint32_t gtm = 0, eqm = 0, wg = 0, we = 0;
 #pragma unroll
     for (int j = 0; j < ROUNDS; ++j) {   // the candidates' indices travel with their values: loaded up front
-      const uint64_t i = wbeg + (uint64_t)j * 32u;
-      ib[j] = i < end ? T.cand_idx[d.cand_base + i] : 0u;
+      const uint32_t o = wofs + (uint32_t)j * 32u;
+      ib[j] = (whole || o < valid) ? tile_idx[o] : 0u;
+    }
+#pragma unroll
+    for (int j = 0; j < ROUNDS; ++j) vb[j] = 0u;
+#pragma unroll
+    for (int j = 0; j < ROUNDS; ++j) {
+      const uint32_t o = wofs + (uint32_t)j * 32u;
+      if (whole || o < valid) vb[j] = __float_as_uint(tile_val[o]);
     }
 #pragma unroll
     for (int j = 0; j < ROUNDS; ++j) {
-      const uint64_t i = wbeg + (uint64_t)j * 32u;
-      uint32_t b = 0;
+      const uint32_t o = wofs + (uint32_t)j * 32u;
+      const uint32_t b = vb[j];
       bool isgt = false, iseq = false;
-      if (i < end) {
-        b = __float_as_uint(vals[i]);
+      if (whole || o < valid) {
         const uint32_t key = b & kAbsMask;
         isgt = key > tau;
         iseq = key == tau;
       }
-      vb[j] = b;
       gtm |= (isgt ? 1u : 0u) << j;
       eqm |= (iseq ? 1u : 0u) << j;
       wg += __popc(__ballot_sync(0xFFFFFFFFu, isgt));
@@ -245,7 +254,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
         }
       }
       // cleared early but not kept after all (the estimate was below tau, or a tie beyond the quota)
-      if (!kept && (vb[j] & kAbsMask) > zthr && wbeg + (uint64_t)j * 32u < end && ib[j] < T.n)
+      if (!kept && (vb[j] & kAbsMask) > zthr && (whole || wofs + (uint32_t)j * 32u < valid) && ib[j] < T.n)
         T.residual[ib[j]] = __uint_as_float(vb[j]);
       rg += __popc(mg);
       re += __popc(me);
