@@ -160,17 +160,6 @@ __device__ SelRun next_digit(const Bin* gh, int bits, SelRun in, Ctl* ctl) {
   return in;
 }
 
-// State of scope s before pass `pass`, recomputed from the finished histograms of the earlier passes.
-template <int VIEW>
-__device__ SelRun state_before(const DevTables& T, const ScopeDesc& d, uint32_t s, int pass) {
-  SelRun r;
-  r.prefix = 0;
-  r.rank = VIEW == V_SAMPLE ? d.samp_rank : d.k;
-  r.gt = 0;
-  for (int p = 0; p < pass; ++p) r = next_digit(hist_of(T, s, VIEW, p), p == 0 ? kRadixBits0 : 10, r, T.ctl);
-  return r;
-}
-
 // Rank, in a scope's sample, of the best estimate of the threshold itself: the expected number of
 // samples above it (the prediction tau_lo uses a larger rank, i.e. a lower key, for its margin).
 __device__ __forceinline__ uint64_t rank_hi_of(const ScopeDesc& d) {
@@ -250,6 +239,8 @@ __global__ void __launch_bounds__(kThreads, (MANY && VIEW != V_DENSE) ? 2 : 4) s
   constexpr uint32_t NONE = 0xFFFFFFFFu;
   __shared__ uint32_t sh[kRadixBins0];
   __shared__ SmemTables s_tab;                          // the scopes [w0, w0 + kSmemScopes) this CTA starts in
+  __shared__ SelRun s_runs[kSmemScopes][2];             // where the walks of those scopes stand ...
+  __shared__ int s_level[kSmemScopes];                  // ... and after how many histograms (0: not started)
   __shared__ uint32_t s_vt0[VIEW == V_CAND ? (MANY ? kVtScopes : kSmemScopes) + 1 : 1];
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   if (T.ctl->status != GD_OK) return;   // set only by an earlier kernel of this call: uniform over the grid
@@ -290,6 +281,7 @@ __global__ void __launch_bounds__(kThreads, (MANY && VIEW != V_DENSE) ? 2 : 4) s
     uint64_t* dst = reinterpret_cast<uint64_t*>(s_tab.scopes);
     for (uint32_t i = tid; i < words; i += kThreads) dst[i] = src[i];
     for (uint32_t i = tid; i <= cnt; i += kThreads) s_tab.tile0[i] = base[w0 + i];
+    for (uint32_t i = tid; i < kSmemScopes; i += kThreads) s_level[i] = 0;
     __syncthreads();
   }
   auto desc_of = [&](uint32_t s) -> const ScopeDesc& {
@@ -396,29 +388,43 @@ __global__ void __launch_bounds__(kThreads, (MANY && VIEW != V_DENSE) ? 2 : 4) s
       const uint64_t beg = (uint64_t)lt * TILE;
       if (pass == PASSES ? lt != 0 : beg >= len) continue;
       if (pass > 0 && !have_run) {                      // digits fixed by the earlier passes
-        SelRun run;
-        uint32_t tau_hi = 0;
-        if (VIEW == V_SAMPLE && PASSES == 2) {
-          // Two ranks walk the histograms together: the prediction's, and the rank of the estimate of
-          // tau itself.  Their first digits may differ; the second rank's second-pass histogram is then
-          // the one kept in the third slot.
-          SelRun two[2];
-          two[0].prefix = 0; two[0].rank = d.samp_rank; two[0].gt = 0;
-          two[1].prefix = 0; two[1].rank = rank_hi_of(d); two[1].gt = 0;
-          next_digit_pair(hist_of(T, s, VIEW, 0), kRadixBits0, two, 2, T.ctl);
-          prefix_b = two[1].prefix;
-          if (pass == PASSES) {
-            if (two[1].prefix == two[0].prefix) {
-              next_digit_pair(hist_of(T, s, VIEW, 1), 10, two, 2, T.ctl);
-            } else {
-              two[0] = next_digit(hist_of(T, s, VIEW, 1), 10, two[0], T.ctl);
-              two[1] = next_digit(hist_of(T, s, VIEW, 2), 10, two[1], T.ctl);
-            }
-            tau_hi = two[1].prefix << kShift1;
-          }
-          run = two[0];
+        // The walk down the finished histograms resumes from where this CTA left it in the previous pass
+        // (kept in shared memory for the scopes of its window), else starts from the top.  In the sample
+        // view two ranks walk together: the prediction's, and the rank of the estimate of tau itself; their
+        // first digits may differ, and the second rank's second-pass histogram is then the one in the third slot.
+        const bool pair = VIEW == V_SAMPLE && PASSES == 2;
+        const uint32_t c = s - w0;
+        SelRun two[2];
+        int level = 0;
+        if (c < kSmemScopes && s_level[c] > 0) {
+          two[0] = s_runs[c][0];
+          two[1] = s_runs[c][1];
+          level = s_level[c];
         } else {
-          run = state_before<VIEW>(T, d, s, pass);
+          two[0].prefix = 0; two[0].rank = VIEW == V_SAMPLE ? d.samp_rank : d.k; two[0].gt = 0;
+          two[1].prefix = 0; two[1].rank = pair ? rank_hi_of(d) : 0; two[1].gt = 0;
+        }
+        for (; level < pass; ++level) {
+          const int lbits = level == 0 ? kRadixBits0 : 10;
+          if (!pair) {
+            two[0] = next_digit(hist_of(T, s, VIEW, level), lbits, two[0], T.ctl);
+          } else if (level == 0 || two[1].prefix == two[0].prefix) {
+            next_digit_pair(hist_of(T, s, VIEW, level), lbits, two, 2, T.ctl);
+          } else {
+            two[0] = next_digit(hist_of(T, s, VIEW, 1), 10, two[0], T.ctl);
+            two[1] = next_digit(hist_of(T, s, VIEW, 2), 10, two[1], T.ctl);
+          }
+        }
+        if (c < kSmemScopes && tid == 0) {              // read again after the next grid barrier
+          s_runs[c][0] = two[0];
+          s_runs[c][1] = two[1];
+          s_level[c] = pass;
+        }
+        const SelRun run = two[0];
+        uint32_t tau_hi = 0;
+        if (pair) {
+          if (pass == 1) prefix_b = two[1].prefix;
+          else tau_hi = two[1].prefix << kShift1;
         }
         have_run = true;
         prefix = run.prefix;
