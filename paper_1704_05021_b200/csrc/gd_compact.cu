@@ -1,6 +1,8 @@
 // Survivor compaction of gd_compress (Algorithm 1, steps 3-5: mask, residual rewrite, sparse
 // output), the two-means sums of Section 5.4, and the kernel that finishes a call (thresholds,
 // shard offsets of Section 3, the means).
+#include <atomic>
+
 #include "gd_scan.cuh"
 
 namespace gd {
@@ -31,6 +33,8 @@ __device__ void finalize_call(const DevTables& T, uint64_t k_total) {
   for (uint32_t j = warp; j <= T.n_shards; j += kWarps) {
     const uint64_t bound = T.shard_off[j];
     uint64_t lo = 0, hi = k_total;                   // answer in [lo, hi]
+    if (bound == 0) hi = 0;                           // nothing lies below the first boundary ...
+    if (bound >= T.n) lo = k_total;                   // ... and everything below the last: no search
     while (hi - lo > 32) {
       const uint64_t span = hi - lo;
       const uint64_t p = lo + span * (lane + 1) / 33;   // lo < p < hi, ascending in lane
@@ -209,8 +213,19 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
     __syncthreads();
     if (!s_ok) continue;
 
-    // phase 2: place the survivors
-    uint64_t rg = s_exg + woff_g, re = s_exe + woff_e;   // running counts before this warp's round
+    // phase 2: place the survivors.  Slot of an entry = (#above before it) + min(#ties before it, q); with
+    // EXG / EXE the counts before this tile that is
+    //   out_base + EXG + min(EXE, q)  +  (above before it in the tile) + min(ties before it in the tile, q - EXE),
+    // one 64-bit base per tile and 32-bit arithmetic per entry.
+    const uint64_t exg = s_exg, exe = s_exe;
+    const uint64_t tie_base = exe < q ? exe : q;
+    const uint64_t q_left64 = q - tie_base;               // ties of this tile that are still kept
+    const uint32_t q_left = q_left64 < 0xFFFFu ? (uint32_t)q_left64 : 0xFFFFu;   // a tile has at most 4096 entries
+    const uint64_t slot0 = exg + tie_base;                // slot, inside the scope, of the tile's first survivor
+    const uint64_t room = d.k > slot0 ? d.k - slot0 : 0;  // slots left in the scope from there
+    uint32_t* const oi = T.out_idx + d.out_base + slot0;
+    float* const ov = T.out_val ? T.out_val + d.out_base + slot0 : nullptr;
+    uint32_t rg = woff_g, re = woff_e;                    // counts inside the tile before this warp's round
     const bool single = two_means && s_single;
     const uint32_t tile_layer = two_means ? s_layer : 0u;
     double sum_p = 0.0, sum_n = 0.0;
@@ -222,17 +237,17 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
       const uint32_t mg = __ballot_sync(0xFFFFFFFFu, isgt), me = __ballot_sync(0xFFFFFFFFu, iseq);
       bool kept = false;
       if (isgt || iseq) {
-        const uint64_t gb = rg + __popc(mg & ltm), eb = re + __popc(me & ltm);
-        if (isgt || eb < q) {
+        const uint32_t gb = rg + __popc(mg & ltm), eb = re + __popc(me & ltm);
+        if (isgt || eb < q_left) {
           kept = true;
-          const uint64_t pos = gb + (eb < q ? eb : q);
+          const uint32_t pos = gb + (eb < q_left ? eb : q_left);
           const uint64_t idx = ib[j];
-          if (pos < d.k && idx < T.n) {
+          if (pos < room && idx < T.n) {
             const uint32_t b = vb[j];
             if (!feedback && !(skip_cleared && (b & kAbsMask) > zthr)) T.residual[idx] = 0.0f;
             if (packed) {
               const uint32_t sgn = b >> 31;
-              T.out_idx[d.out_base + pos] = (uint32_t)idx | (sgn << 31);
+              oi[pos] = (uint32_t)idx | (sgn << 31);
               const double x = (double)__uint_as_float(b);
               if (!two_means) {
                 // threshold mode: the value is implied by the scope's tau
@@ -244,8 +259,8 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant
                 atomicAdd(T.cnts + 2 * pr + sgn, 1ull);
               }
             } else {
-              T.out_idx[d.out_base + pos] = (uint32_t)idx;
-              T.out_val[d.out_base + pos] = __uint_as_float(b);
+              oi[pos] = (uint32_t)idx;
+              ov[pos] = __uint_as_float(b);
               if (T.delta_base) T.delta_base[idx] = __fadd_rn(T.delta_base[idx], __uint_as_float(b));
             }
           } else {
@@ -650,7 +665,17 @@ cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense
   const uint32_t total = tiles[dense ? L_DCOMP : L_CAND];
   if (!total) return finalize ? launch_finalize(T, stream) : cudaSuccess;
   ProfileScope prof(stream, dense ? PT_DENSE_COMPACT : PT_CAND_COMPACT);
-  const uint32_t cap = (uint32_t)sm_count() * (dense ? 3u : 8u);
+  // The kernels take tiles from a ticket until none is left: no more CTAs than are resident at once,
+  // or the later ones would only start, find nothing and leave.
+  static std::atomic<int> resident[2] = {{0}, {0}};
+  int r = resident[dense ? 1 : 0].load(std::memory_order_relaxed);
+  if (r == 0) {
+    cudaError_t e = dense ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, compact_dense_kernel, kThreads, 0)
+                          : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, compact_kernel, kThreads, 0);
+    if (e != cudaSuccess || r <= 0) return cudaErrorLaunchFailure;
+    resident[dense ? 1 : 0].store(r, std::memory_order_relaxed);
+  }
+  const uint32_t cap = (uint32_t)sm_count() * (uint32_t)r;
   const uint32_t grid = total < cap ? total : cap;
   if (dense)
     compact_dense_kernel<<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
