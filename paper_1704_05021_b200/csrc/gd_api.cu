@@ -92,6 +92,7 @@ struct Plan {
   uint32_t n_scopes = 0;
   bool predict = true;
   uint32_t emit_chunk_tiles = 1, dense_sel_tile = kDenseSelTileMax, dense_chunk_tiles = kDenseChunkTilesMax;
+  uint32_t samp_tile = kTile;
   // workspace layout (byte offsets)
   size_t off_ctl = 0, off_state = 0, off_hist = 0, off_sums = 0, off_cnts = 0, off_desc_emit = 0,
          off_desc_cand = 0, off_desc_dcomp = 0, zero_bytes = 0;
@@ -207,6 +208,19 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
     if (tiles[l] > 0x7FFFFFFFull) return GD_ERR_TOO_LARGE;
     P->tile0[l][ns_count] = (uint32_t)tiles[l];
     P->tiles[l] = (uint32_t)tiles[l];
+  }
+  // The sample is gathered with scattered reads, of which one SM keeps only so many in flight: a short
+  // sample is cut into tiles of 1024 so that its gather spreads over all SMs.
+  P->samp_tile = kTile;
+  while (P->samp_tile > 1024u && samp_base / P->samp_tile < 2u * 148u) P->samp_tile >>= 2;
+  if (P->samp_tile != kTile) {
+    uint64_t t = 0;
+    for (uint32_t s = 0; s < ns_count; ++s) {
+      P->tile0[L_SAMP][s] = (uint32_t)t;
+      t += (P->scopes[s].samp_m + P->samp_tile - 1) / P->samp_tile;
+    }
+    P->tile0[L_SAMP][ns_count] = (uint32_t)t;
+    P->tiles[L_SAMP] = (uint32_t)t;
   }
   P->samp_off[ns_count] = samp_base;
   P->samp_total = samp_base;
@@ -473,6 +487,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     T.k_total = P.k_total;
     T.emit_chunk_tiles = P.emit_chunk_tiles;
     T.sample_passes = sampled ? 3u : 2u;
+    T.samp_tile = P.samp_tile;
     T.dense_sel_tile = P.dense_sel_tile;
     T.dense_chunk_tiles = P.dense_chunk_tiles;
     if (sampled) T.k_total = P.cand_total;   // capacity of the outputs; the count is found on the device

@@ -234,7 +234,7 @@ __device__ __noinline__ SelRun local_select(const DevTables& T, const ScopeDesc&
 template <int VIEW, bool MANY>
 __global__ void __launch_bounds__(kThreads, (MANY && VIEW != V_DENSE) ? 2 : 4) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
   constexpr int LK = VIEW == V_SAMPLE ? L_SAMP : (VIEW == V_CAND ? L_CAND : L_DSEL);
-  const uint32_t TILE = VIEW == V_DENSE ? T.dense_sel_tile : kTile;
+  const uint32_t TILE = VIEW == V_DENSE ? T.dense_sel_tile : (VIEW == V_SAMPLE ? T.samp_tile : kTile);
   const int PASSES = VIEW == V_SAMPLE ? (int)T.sample_passes : 3;   // the prediction needs 21 bits only
   constexpr uint32_t NONE = 0xFFFFFFFFu;
   __shared__ uint32_t sh[kRadixBins0];
