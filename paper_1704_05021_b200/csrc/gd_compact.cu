@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constan
 // above tau and keys equal to tau.  An element above tau goes to slot  (#above before it) +
 // min(#ties before it, q); a tie is kept iff fewer than q ties precede it.  CTAs take tiles from an
 // atomic ticket until none is left; the last CTA to leave finishes the call.
-__global__ void __launch_bounds__(kThreads) compact_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles,
+__global__ void __launch_bounds__(kThreads, 3) compact_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles,
                                                            int do_finalize) {
   constexpr int LK = L_CAND;
   constexpr int ROUNDS = kTile / kThreads;   // 16 elements per thread
