@@ -150,7 +150,9 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
   // vectors, which otherwise would not fill the GPU.
   uint32_t sel_tile = kDenseSelTileMax, dchunk = kDenseChunkTilesMax;
   while (sel_tile > kTile && n / sel_tile < 592u) sel_tile >>= 1;
-  while (dchunk > 1 && n / ((uint64_t)dchunk * kTile) < 888u) dchunk >>= 1;
+  // (chunks of the dense compaction: about 48 per resident CTA, so that scopes whose survivors crowd at one
+  // end - a sparse layer whose kept zeros are its first ones - still spread over the GPU)
+  while (dchunk > 1 && n / ((uint64_t)dchunk * kTile) < 7104u) dchunk >>= 1;
   P->dense_sel_tile = sel_tile;
   P->dense_chunk_tiles = dchunk;
   const uint32_t ns_count = scope_mode == GD_SCOPE_GLOBAL ? 1u : n_layers;
