@@ -139,11 +139,12 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
     P->pair_off[l + 1] = P->pair_off[l] + cols;
   }
   P->n_pairs = P->pair_off[n_layers];
-  // The fused pass gives each CTA a chunk of 1, 2, 4 or 8 tiles: as large as still leaves about
-  // four waves of CTAs (4 per SM on 148 SMs) for the whole vector.
+  // The fused pass gives each CTA a chunk of 1, 2, 4 or 8 tiles: as large as still leaves a wave and a
+  // half of CTAs (4 per SM on 148 SMs) for the whole vector.  (Measured on 2^21 .. 2^26 elements: four
+  // waves, the first rule, cost 20-30 % more time at 2^23 .. 2^25; one wave loses to the tail.)
   const uint64_t dense_tiles = (n + kTile - 1) / kTile;
   uint32_t chunk_tiles = 8;
-  while (chunk_tiles > 1 && dense_tiles < (uint64_t)chunk_tiles * 2368u) chunk_tiles >>= 1;
+  while (chunk_tiles > 1 && dense_tiles < (uint64_t)chunk_tiles * 888u) chunk_tiles >>= 1;
   P->emit_chunk_tiles = chunk_tiles;
   const uint64_t CH = (uint64_t)chunk_tiles * kTile;
   // The dense kernels (used when a prediction fails) take large tiles on long vectors, where the
