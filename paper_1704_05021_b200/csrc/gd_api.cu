@@ -532,11 +532,13 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     const bool predict = P.predict;
     if (predict && launch_sample_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
     if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
-    // The dense kernels are always enqueued: they return at once unless a prediction failed.  The
-    // compaction that runs last also finishes the call (thresholds, shard offsets, means).
-    if (launch_dense_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
-    if (launch_compact(T, tiles, true, !predict, stream) != cudaSuccess) return GD_ERR_CUDA;
-    if (predict) {
+    // Without a prediction: the selection and compaction over the dense range.  With one: the two kernels over
+    // the candidate lists, which first do the dense work of the scopes whose prediction failed (usually none).
+    // The compaction that runs last also finishes the call (thresholds, shard offsets, means).
+    if (!predict) {
+      if (launch_dense_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+      if (launch_compact(T, tiles, true, true, stream) != cudaSuccess) return GD_ERR_CUDA;
+    } else {
       if (launch_candidate_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
       if (launch_compact(T, tiles, false, true, stream) != cudaSuccess) return GD_ERR_CUDA;
     }

@@ -80,8 +80,7 @@ __global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constan
 // above tau and keys equal to tau.  An element above tau goes to slot  (#above before it) +
 // min(#ties before it, q); a tie is kept iff fewer than q ties precede it.  CTAs take tiles from an
 // atomic ticket until none is left; the last CTA to leave finishes the call.
-__global__ void __launch_bounds__(kThreads, 3) compact_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles,
-                                                           int do_finalize) {
+__device__ __forceinline__ void compact_cand_body(const DevTables& T, uint32_t total_tiles, int do_finalize) {
   constexpr int LK = L_CAND;
   constexpr int ROUNDS = kTile / kThreads;   // 16 elements per thread
   __shared__ uint32_t s_tile;
@@ -312,8 +311,7 @@ __global__ void __launch_bounds__(kThreads, 3) compact_kernel(const __grid_const
 // one look-back: at 4 bytes per element the chain of look-backs would otherwise have to advance about a
 // hundred tiles per microsecond, which the L2 round trips between CTAs cannot sustain.
 // The classification masks stay in registers; the values of the (few) survivors are read again.
-__global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid_constant__ DevTables T,
-                                                                    uint32_t total_chunks, int do_finalize) {
+__device__ __forceinline__ void compact_dense_body(const DevTables& T, uint32_t total_chunks, int do_finalize) {
   constexpr int CD = (int)kDenseChunkTilesMax;   // shared arrays are sized for the largest chunk
   const int cd = (int)T.dense_chunk_tiles;        // tiles per chunk in this call
   constexpr int ROUNDS = kTile / kThreads;   // 16 elements per thread and tile
@@ -510,6 +508,24 @@ __global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid
   finalize_call(T, T.k_total);
 }
 
+// (kept out of line so that the rare path does not weigh on the registers of the usual one)
+__device__ __noinline__ void compact_dense_outlined(const DevTables& T, uint32_t dense_chunks) {
+  compact_dense_body(T, dense_chunks, 0);
+}
+
+__global__ void __launch_bounds__(kThreads, 3) compact_dense_kernel(const __grid_constant__ DevTables T,
+                                                                    uint32_t total_chunks, int do_finalize) {
+  compact_dense_body(T, total_chunks, do_finalize);
+}
+
+// The compaction over the candidate lists also takes over, first, the compaction over the dense range of the
+// scopes whose prediction failed (dense_chunks != 0; rare), so that no launch is spent on looking at a flag.
+__global__ void __launch_bounds__(kThreads, 3) compact_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles,
+                                                              int do_finalize, uint32_t dense_chunks) {
+  if (dense_chunks != 0u && T.ctl->dense_needed != 0u) compact_dense_outlined(T, dense_chunks);
+  compact_cand_body(T, total_tiles, do_finalize);
+}
+
 // Sampled-threshold mode: the candidate lists ARE the survivors.  Copies every scope's list to its
 // place in the output (scopes concatenated in index order), clears the survivors' residual slots
 // unless the fused pass has done so already, and lets the last CTA finish the call with the survivor
@@ -661,6 +677,8 @@ cudaError_t launch_pack_sampled(const DevTables& T, const uint32_t* tiles, cudaS
   return cudaSuccess;
 }
 
+// dense = true: the dense compaction alone (no prediction in this call).  dense = false: the compaction over the
+// candidate lists, which also runs the dense one for scopes whose prediction failed.
 cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, bool finalize, cudaStream_t stream) {
   const uint32_t total = tiles[dense ? L_DCOMP : L_CAND];
   if (!total) return finalize ? launch_finalize(T, stream) : cudaSuccess;
@@ -680,7 +698,7 @@ cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense
   if (dense)
     compact_dense_kernel<<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
   else
-    compact_kernel<<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
+    compact_kernel<<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0, tiles[L_DCOMP]);
   GD_LAUNCH_CHECK();
   return cudaSuccess;
 }

@@ -13,7 +13,7 @@ constexpr int kThreads = 256;           // threads per CTA in every tiled kernel
 constexpr int kWarps = kThreads / 32;
 constexpr uint32_t kTile = 4096;        // elements per tile of the streaming kernels
 constexpr uint32_t kDenseSelTileMax = 32768;  // most elements per tile in the dense histogram passes
-constexpr uint32_t kDenseChunkTilesMax = 32;  // most tiles per ticket (and per look-back) in the dense compaction
+constexpr uint32_t kDenseChunkTilesMax = 16;  // most tiles per ticket (and per look-back) in the dense compaction
 constexpr int kRadixBits0 = 11;         // 31-bit magnitude key = 11 + 10 + 10 bits
 constexpr int kRadixBins0 = 1 << kRadixBits0;
 constexpr int kShift0 = 20, kShift1 = 10, kShift2 = 0;

@@ -232,7 +232,7 @@ __device__ __noinline__ SelRun local_select(const DevTables& T, const ScopeDesc&
 // run of tiles crosses several scopes, so it keeps a window of the tables from its first scope on, and
 // selects every list of a single tile by itself in shared memory.
 template <int VIEW, bool MANY>
-__global__ void __launch_bounds__(kThreads, (MANY && VIEW != V_DENSE) ? 2 : 4) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles) {
+__device__ __forceinline__ void select_body(const DevTables& T, uint32_t total_tiles) {
   constexpr int LK = VIEW == V_SAMPLE ? L_SAMP : (VIEW == V_CAND ? L_CAND : L_DSEL);
   const uint32_t TILE = VIEW == V_DENSE ? T.dense_sel_tile : (VIEW == V_SAMPLE ? T.samp_tile : kTile);
   const int PASSES = VIEW == V_SAMPLE ? (int)T.sample_passes : 3;   // the prediction needs 21 bits only
@@ -507,8 +507,27 @@ __global__ void __launch_bounds__(kThreads, (MANY && VIEW != V_DENSE) ? 2 : 4) s
   }
 }
 
+// (kept out of line so that the rare path does not weigh on the registers of the usual one)
+template <bool MANY>
+__device__ __noinline__ void select_dense_outlined(const DevTables& T, uint32_t dense_tiles) {
+  select_body<V_DENSE, MANY>(T, dense_tiles);
+}
+
+// One cooperative launch = one selection.  The selection over the candidate lists also takes over, first, the
+// selection over the dense range of the scopes whose prediction failed (dense_tiles != 0): such scopes are rare,
+// and two launches that start, look at a flag and leave cost every call about six microseconds.
 template <int VIEW, bool MANY>
-cudaError_t launch_select_impl(const DevTables& T, uint32_t total_tiles, uint32_t ctas_per_sm, cudaStream_t stream) {
+__global__ void __launch_bounds__(kThreads, (MANY && VIEW != V_DENSE) ? 2 : 4) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles,
+                                                                                             uint32_t dense_tiles) {
+  if (VIEW == V_CAND) {
+    if (dense_tiles != 0u && T.ctl->dense_needed != 0u) select_dense_outlined<MANY>(T, dense_tiles);
+  }
+  select_body<VIEW, MANY>(T, total_tiles);
+}
+
+template <int VIEW, bool MANY>
+cudaError_t launch_select_impl(const DevTables& T, uint32_t total_tiles, uint32_t dense_tiles, uint32_t ctas_per_sm,
+                               cudaStream_t stream) {
   if (!total_tiles) return cudaSuccess;
   ProfileScope prof(stream, VIEW == V_SAMPLE ? PT_SAMPLE_SELECT : (VIEW == V_CAND ? PT_CAND_SELECT : PT_DENSE_SELECT));
   static std::atomic<int> cached{0};                       // co-resident CTAs per SM of this kernel
@@ -524,7 +543,7 @@ cudaError_t launch_select_impl(const DevTables& T, uint32_t total_tiles, uint32_
   uint32_t grid = (uint32_t)sm_count() * per_sm;
   if (grid > total_tiles) grid = total_tiles;
   DevTables Tc = T;
-  void* args[] = {(void*)&Tc, (void*)&total_tiles};
+  void* args[] = {(void*)&Tc, (void*)&total_tiles, (void*)&dense_tiles};
   cudaError_t e = cudaLaunchCooperativeKernel((const void*)select_kernel<VIEW, MANY>, dim3(grid), dim3(kThreads), args, 0, stream);
   if (e != cudaSuccess) return e;
   note_launches(1);
@@ -532,23 +551,24 @@ cudaError_t launch_select_impl(const DevTables& T, uint32_t total_tiles, uint32_
 }
 
 template <int VIEW>
-cudaError_t launch_select(const DevTables& T, uint32_t total_tiles, uint32_t ctas_per_sm, cudaStream_t stream) {
-  return T.n_scopes > kSmemScopes ? launch_select_impl<VIEW, true>(T, total_tiles, ctas_per_sm, stream)
-                                  : launch_select_impl<VIEW, false>(T, total_tiles, ctas_per_sm, stream);
+cudaError_t launch_select(const DevTables& T, uint32_t total_tiles, uint32_t dense_tiles, uint32_t ctas_per_sm,
+                          cudaStream_t stream) {
+  return T.n_scopes > kSmemScopes ? launch_select_impl<VIEW, true>(T, total_tiles, dense_tiles, ctas_per_sm, stream)
+                                  : launch_select_impl<VIEW, false>(T, total_tiles, dense_tiles, ctas_per_sm, stream);
 }
 
 }  // namespace
 
 cudaError_t launch_sample_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
-  return launch_select<V_SAMPLE>(T, tiles[L_SAMP], 2, stream);
+  return launch_select<V_SAMPLE>(T, tiles[L_SAMP], 0u, 2, stream);
 }
 
 cudaError_t launch_candidate_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
-  return launch_select<V_CAND>(T, tiles[L_CAND], 2, stream);
+  return launch_select<V_CAND>(T, tiles[L_CAND], tiles[L_DSEL], 2, stream);   // and the dense selection, if needed
 }
 
 cudaError_t launch_dense_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
-  return launch_select<V_DENSE>(T, tiles[L_DSEL], 8, stream);
+  return launch_select<V_DENSE>(T, tiles[L_DSEL], 0u, 8, stream);
 }
 
 }  // namespace gd
