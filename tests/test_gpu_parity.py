@@ -760,6 +760,48 @@ def test_random_layouts_and_modes(cuda_device, seed):
     run_steps(w, cuda_device, 3, flags=flags, grads=grads, layer_cols=cols, alpha=alpha)
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_random_models_of_few_large_tensors(cuda_device, seed):
+    """One to nine tensors of 0.3 to 2.5 M elements (the predicted path with all tables in shared memory), random drop
+    ratio, scope, value mode (column-wise means and fed-back threshold quantisation included), flags and value
+    distribution (Laplace, mixed scales, mostly zero, heavy-tailed Student t, a run of tied values)."""
+    rng = np.random.default_rng(90000 + seed)
+    n_layers = int(rng.integers(1, 9))
+    sizes = [int(rng.integers(300_000, 2_500_000)) for _ in range(n_layers)]
+    if rng.random() < 0.5:
+        sizes.append(int(rng.integers(0, 5000)))
+    ppm = int(rng.choice([900_000, 984_000, 990_000, 990_000, 999_000, 999_900]))
+    scope_mode = int(rng.integers(0, 2))
+    value_mode = int(rng.choice([0, 0, 1, 2, 3]))
+    flags = int(rng.choice([0, 0, 0, B.GD_FLAG_NO_EARLY_ZERO, B.GD_FLAG_NO_PREDICTION]))
+    if value_mode == B.GD_VALUES_THRESHOLD and rng.random() < 0.5:
+        flags |= B.GD_FLAG_QUANT_ERROR_FEEDBACK
+    cols = None
+    if value_mode == B.GD_VALUES_COLUMN_MEANS:
+        cols = []
+        for s_ in sizes:
+            divs = [c for c in (1, 2, 4, 5, 8, 10, 16, 100, 1000) if s_ % c == 0] or [1]
+            cols.append(int(rng.choice(divs)))
+    w = W.small_layered(len(sizes), sizes, ppm, scope_mode, value_mode, int(rng.integers(1, 9)))
+    dist = int(rng.integers(0, 5))
+    grads = []
+    for _ in range(2):
+        if dist == 0:
+            g = rng.laplace(0, 1e-3, w.n)
+        elif dist == 1:
+            g = rng.standard_normal(w.n) * 10.0 ** rng.integers(-4, 1, w.n)
+        elif dist == 2:
+            g = np.where(rng.random(w.n) < 0.03, rng.standard_normal(w.n), 0.0)
+        elif dist == 3:
+            g = rng.standard_t(2.0, w.n) * 1e-3
+        else:
+            g = rng.laplace(0, 1e-3, w.n)
+            a = int(rng.integers(0, w.n - 20000))
+            g[a:a + 20000] = rng.choice([0.5, -0.5, 1.0], 20000)
+        grads.append(torch.from_numpy(g.astype(np.float32)))
+    run_steps(w, cuda_device, 2, flags=flags, grads=grads, layer_cols=cols, alpha=float(rng.choice([1.0, 0.5])))
+
+
 @pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
 def test_more_scopes_than_the_tile_table_holds(cuda_device, scope_mode):
     """2600 tensors: more scopes than the shared-memory table of candidate tiles covers (2048), so the kernels over the
