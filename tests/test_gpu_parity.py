@@ -409,6 +409,85 @@ def test_many_layers_on_the_predicted_path(cuda_device, scope_mode, value_mode):
     assert st["n_scopes_predicted"] >= 1
 
 
+# ---------------------------------------------------------------- guard words around every buffer
+@pytest.mark.parametrize("case", ["predicted_fp32", "predicted_two_means", "dense_fp32", "sampled", "many_scopes"])
+def test_nothing_is_written_outside_the_buffers(cuda_device, case):
+    """Every buffer the library writes (residual, outputs, workspace, parameters) sits between guard words; the guards
+    must be intact after compress + apply and the outputs must equal the oracle's.  Buffers have exactly the sizes the
+    sizing calls return."""
+    rng = np.random.default_rng(5150)
+    G = 1024                                                       # guard elements on either side
+    value_mode, flags, scope = B.GD_VALUES_FP32, 0, B.GD_SCOPE_PER_LAYER
+    sizes = [1_300_000, 9, 4097, 1_000_003]
+    if case == "predicted_two_means":
+        value_mode = B.GD_VALUES_TWO_MEANS
+    elif case == "dense_fp32":
+        sizes = [200_001, 9, 4097]
+    elif case == "sampled":
+        flags = B.GD_FLAG_SAMPLED_THRESHOLD
+    elif case == "many_scopes":
+        sizes = [1_200_000] + [int(x) for x in rng.integers(1, 5000, size=45)] + [900_001]
+    w = W.small_layered(len(sizes), sizes, 990_000, scope, value_mode, 3)
+    n = w.n
+    sampled = bool(flags & B.GD_FLAG_SAMPLED_THRESHOLD)
+    k_cap = (B.gd_sampled_capacity(w.layer_off, scope, w.drop_ppm) if sampled
+             else B.gd_total_kept(w.layer_off, scope, w.drop_ppm))
+    n_scopes = len(sizes)
+    ws_bytes = B.gd_workspace_bytes(w.layer_off, w.n_shards, scope, w.drop_ppm, None)
+    aws_bytes = B.gd_apply_workspace_bytes(w.n_shards, len(sizes))
+
+    def padded(count, dtype, fill):
+        t = torch.full((count + 2 * G,), fill, dtype=dtype, device=cuda_device)
+        return t, t[G:G + count]
+
+    def intact(t, count, fill):
+        ref = torch.full((G,), fill, dtype=t.dtype, device=t.device)
+        return torch.equal(t[:G], ref) and torch.equal(t[G + count:], ref)
+
+    res_t, res = padded(n, torch.float32, 7.0)
+    res.zero_()
+    par_t, par = padded(n, torch.float32, 7.0)
+    par.zero_()
+    idx_t, idx = padded(max(k_cap, 1), torch.int32, 0x5A5A5A5A)
+    val_t, val = padded(max(k_cap, 1), torch.float32, 7.0)
+    off_t, off = padded(w.n_shards + 1, torch.int32, 0x5A5A5A5A)
+    tau_t, tau = padded(n_scopes, torch.int32, 0x5A5A5A5A)
+    mean_t, mean = padded(2 * len(sizes), torch.float32, 7.0)
+    ws_t, ws = padded(ws_bytes, torch.uint8, 0x5A)
+    aws_t, aws = padded(aws_bytes, torch.uint8, 0x5A)
+    g_host = rng.laplace(0, 1e-3, n).astype(np.float32)
+    grad = torch.from_numpy(g_host).to(cuda_device)
+    call = B.CompressCall(grad, res, w.layer_off, w.shard_off, w.drop_ppm, scope, value_mode, idx, val, off, tau,
+                          mean.view(-1, 2), ws, flags=flags)
+    B.gd_compress(call)
+    assert B.gd_status(ws) == B.GD_OK
+    views = [par[w.shard_off[j]:w.shard_off[j + 1]] for j in range(w.n_shards)]
+    push = {"idx": idx, "val": None if value_mode != B.GD_VALUES_FP32 else val, "shard_cnt_off": off,
+            "means": mean.view(-1, 2) if value_mode != B.GD_VALUES_FP32 else None}
+    acall = B.ApplyCall(views, w.shard_off, [push], value_mode, 1.0, aws, layer_off=w.layer_off)
+    B.gd_decompress_apply(acall)
+    torch.cuda.synchronize()
+    for name, t, count, fill in (("residual", res_t, n, 7.0), ("params", par_t, n, 7.0),
+                                 ("out_idx", idx_t, max(k_cap, 1), 0x5A5A5A5A), ("out_val", val_t, max(k_cap, 1), 7.0),
+                                 ("out_shard_cnt_off", off_t, w.n_shards + 1, 0x5A5A5A5A),
+                                 ("out_tau", tau_t, n_scopes, 0x5A5A5A5A), ("out_means", mean_t, 2 * len(sizes), 7.0),
+                                 ("workspace", ws_t, ws_bytes, 0x5A), ("apply workspace", aws_t, aws_bytes, 0x5A)):
+        assert intact(t, count, fill), f"{case}: guard words around {name} were overwritten"
+    r0 = orc.residual_reset(n)
+    if sampled:
+        exp = orc.compress_sampled(g_host, r0, w.layer_off, w.shard_off, w.drop_ppm, scope)
+    else:
+        exp = orc.compress(g_host, r0, w.layer_off, w.shard_off, w.drop_ppm, scope, value_mode)
+    K = exp["idx"].shape[0]
+    assert np.array_equal(_np_u32(idx)[:K], exp["idx"])
+    assert np.array_equal(_np_u32(res), exp["residual"].view(np.uint32))
+    assert np.array_equal(_np_u32(tau), exp["tau"])
+    if value_mode == B.GD_VALUES_FP32:
+        sent = np.zeros(n, np.float32)
+        sent[exp["idx"]] = exp["val"]
+        assert np.array_equal(_np_u32(par), sent.view(np.uint32))
+
+
 # ---------------------------------------------------------------- other drop ratios (Section 5.1: 90 %, 99 %, 99.9 %)
 @pytest.mark.parametrize("drop_ppm", [900_000, 999_000])
 @pytest.mark.parametrize("config", [2, 3])
