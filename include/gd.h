@@ -18,6 +18,8 @@
  *     by gd_status(); device code never traps, asserts or spins without a limit.  After such a
  *     status the outputs AND the residual of that call are undefined (the call updates the
  *     residual in place); a caller that wants to retry keeps its own copy of the residual.
+ *   - gd_compress and gd_decompress_apply open an NVTX range of their own name, for profilers that
+ *     show them; without such a tool attached the ranges cost nothing to speak of.
  *   - No CUDA headers are needed to include this file.
  */
 #ifndef GD_H

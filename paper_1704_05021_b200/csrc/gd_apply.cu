@@ -5,6 +5,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "gd_internal.cuh"
 
 namespace gd {
@@ -96,6 +98,8 @@ int gd_apply_workspace_bytes(uint32_t n_shards, uint32_t n_layers, size_t* bytes
 }
 
 int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
+  nvtxRangePushA("gd_decompress_apply");
+  struct Pop { ~Pop() { nvtxRangePop(); } } pop_on_return;
   if (!a || !a->params || !a->shard_off || a->n_shards == 0) return GD_ERR_INVALID_ARG;
   if (a->n_pushes && !a->pushes) return GD_ERR_INVALID_ARG;
   if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_COLUMN_MEANS) return GD_ERR_INVALID_ARG;
