@@ -694,7 +694,8 @@ cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense
     resident[dense ? 1 : 0].store(r, std::memory_order_relaxed);
   }
   const uint32_t cap = (uint32_t)sm_count() * (uint32_t)r;
-  const uint32_t grid = total < cap ? total : cap;
+  const uint32_t most = (!dense && tiles[L_DCOMP] > total) ? tiles[L_DCOMP] : total;   // it may take over the dense chunks
+  const uint32_t grid = most < cap ? most : cap;
   if (dense)
     compact_dense_kernel<<<grid, kThreads, 0, stream>>>(T, total, finalize ? 1 : 0);
   else

@@ -541,7 +541,10 @@ cudaError_t launch_select_impl(const DevTables& T, uint32_t total_tiles, uint32_
   }
   const uint32_t per_sm = ctas_per_sm < (uint32_t)resident ? ctas_per_sm : (uint32_t)resident;
   uint32_t grid = (uint32_t)sm_count() * per_sm;
-  if (grid > total_tiles) grid = total_tiles;
+  // no more CTAs than tiles - counting the dense tiles this launch may have to take over, so that the
+  // rare dense selection is not left to the few CTAs a short candidate list would get
+  const uint32_t most_tiles = total_tiles > dense_tiles ? total_tiles : dense_tiles;
+  if (grid > most_tiles) grid = most_tiles;
   DevTables Tc = T;
   void* args[] = {(void*)&Tc, (void*)&total_tiles, (void*)&dense_tiles};
   cudaError_t e = cudaLaunchCooperativeKernel((const void*)select_kernel<VIEW, MANY>, dim3(grid), dim3(kThreads), args, 0, stream);
