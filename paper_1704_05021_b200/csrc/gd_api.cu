@@ -57,12 +57,16 @@ void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint6
     *cap = c < ns ? c : ns;
     return;
   }
-  // Narrow strata (a sample every few sectors): sample whole groups of 8 consecutive elements instead, so that
-  // the sample costs an eighth of the scattered sector reads.  Wide strata keep single elements, which
-  // spread the sample over more rows of a matrix.
+  // The sample is bound by the rate of scattered DRAM reads (about 22 G/s, two per sample).  Narrow strata (a
+  // sample every few sectors): whole groups of 8 consecutive elements are sampled, an eighth of the reads.  Wide
+  // strata: pairs of neighbours, half the reads; larger groups there would leave too few distinct places (rows
+  // of a matrix) in the sample - a pair at most doubles the variance the rank's margin of six sigma is sized for.
   if (ns / mt <= kClusterMaxStride) {
     mt &= ~7ull;
     *cluster = 8;
+  } else {
+    mt &= ~1ull;
+    *cluster = 2;
   }
   *m = mt;
   const double x = (double)k * (double)mt / (double)ns;
@@ -190,9 +194,9 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
     d.samp_m = m;
     d.samp_rank = rank;
     d.samp_cluster = cluster;
-    if (cluster == 8) {   // strata of groups of 8 elements, from the first multiple of 8 at or after lo
-      const uint64_t first = (d.lo + 7) & ~7ull;
-      const uint64_t groups = (d.hi - first) / 8, strata = m / 8;
+    if (cluster > 1) {   // strata of groups of 8 (or 2) elements, from the first multiple of that at or after lo
+      const uint64_t first = (d.lo + cluster - 1) & ~(uint64_t)(cluster - 1);
+      const uint64_t groups = (d.hi - first) / cluster, strata = m / cluster;
       d.samp_w = groups / strata;
       d.samp_rem = (uint32_t)(groups % strata);
     } else {

@@ -48,9 +48,9 @@ struct ScopeDesc {       // built on the host for every call, read-only on the d
   uint64_t samp_rank;    // the prediction is the samp_rank-th largest sample key
   uint64_t samp_w;       // floor(n_s / samp_m): width of a stratum (the first samp_rem strata are one wider)
   uint32_t samp_rem;     // n_s mod samp_m
-  uint32_t samp_cluster; // 1: strata of elements, one sample each.  8: the prediction samples whole groups of 8
-                         // consecutive elements (one 32-byte sector of each input); the strata (samp_w, samp_rem)
-                         // then count groups, starting at the first multiple of 8 at or after lo
+  uint32_t samp_cluster; // 1: strata of elements, one sample each.  8 (narrow strata) or 2 (wide ones): the prediction
+                         // samples whole groups of that many consecutive elements (one 32-byte sector of each input);
+                         // the strata (samp_w, samp_rem) then count groups, from the first multiple of it at or after lo
 };
 
 struct ScopeState {      // zeroed at the start of every call

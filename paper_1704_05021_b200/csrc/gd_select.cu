@@ -58,12 +58,16 @@ __device__ __forceinline__ float sample_value(const DevTables& T, const ScopeDes
   // Where the strata are narrow, a sample per stratum would touch nearly every 32-byte sector of the
   // scope; there the strata are made of groups of 8 elements and a whole group is sampled (samples
   // 8c .. 8c+7 are group c), which reads an eighth of the sectors for the same number of samples.
-  const uint64_t u = d.samp_cluster == 8u ? li >> 3 : li;      // stratum
+  // Wide strata are sampled in pairs of neighbours (samp_cluster = 2): half the scattered reads, and the
+  // sample still spreads over as many rows of a matrix as a pair allows.
+  const uint32_t cl = d.samp_cluster;                          // 1, 2 or 8 elements per group
+  const uint32_t sh = cl == 8u ? 3u : (cl == 2u ? 1u : 0u);
+  const uint64_t u = li >> sh;                                 // stratum
   const uint64_t a = u * d.samp_w + (u < d.samp_rem ? u : d.samp_rem);
   const uint32_t width = (uint32_t)d.samp_w + (u < d.samp_rem ? 1u : 0u);
   uint64_t unit = a;
   if (width > 1) unit += mix32((uint32_t)u * 0x9E3779B9u + s) % width;
-  const uint64_t pos = d.samp_cluster == 8u ? ((d.lo + 7u) & ~7ull) + unit * 8u + (li & 7u) : d.lo + unit;
+  const uint64_t pos = ((d.lo + cl - 1u) & ~(uint64_t)(cl - 1u)) + (unit << sh) + (li & (cl - 1u));
   return T.delta_base ? __fsub_rn(__ldg(T.grad + pos), T.delta_base[pos]) : __fadd_rn(__ldg(T.grad + pos), T.residual[pos]);
 }
 
