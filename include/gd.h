@@ -147,11 +147,13 @@ int gd_means_pairs(uint32_t n_layers, const uint32_t* layer_cols, int value_mode
  *              mode needs GD_VALUES_FP32.
  *
  *   sampled-threshold mode (GD_FLAG_SAMPLED_THRESHOLD; Section 4, fourth paragraph: the threshold is
- *              selected on a 0.1 % sample of the gradient instead of on all of it): per scope,
- *              m = n_s if n_s <= 4096, else max(4096, ceil(n_s / 1000)) positions are sampled, one in each
- *              of m strata (with w = floor(n_s / m) and rem = n_s mod m, stratum i starts at
- *              a = i w + min(i, rem) and has w + 1 elements if i < rem, else w; sample i of scope s is at
- *              a + (h mod width), h = mix(i * 0x9E3779B9 + s) in 32-bit arithmetic with
+ *              selected on a 0.1 % sample of the gradient instead of on all of it): a scope of up to 4096
+ *              elements is sampled completely; a longer one in m = max(4096, ceil(n_s / 1000)) (rounded up
+ *              to even) positions, taken as m / 2 pairs of neighbours (first + 2 j, first + 2 j + 1), first =
+ *              the smallest even index >= the scope's start, j < P = floor((end - first) / 2).  The P pairs
+ *              are cut into m / 2 strata (with w = floor(P / (m/2)) and rem = P mod (m/2), stratum i starts
+ *              at pair a = i w + min(i, rem) and has w + 1 pairs if i < rem, else w); stratum i of scope s
+ *              contributes pair a + (h mod width), h = mix(i * 0x9E3779B9 + s) in 32-bit arithmetic with
  *              mix(x): x ^= x >> 16; x *= 0x7FEB352D; x ^= x >> 15; x *= 0x846CA68B; x ^= x >> 16);
  *              the threshold key t is the (m - floor(m * drop_ppm / 1e6))-th largest sample key and EVERY
  *              entry of the scope with key >= t is kept, so the number of survivors varies: out_idx and

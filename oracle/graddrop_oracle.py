@@ -114,23 +114,30 @@ def _mix32(x: np.ndarray) -> np.ndarray:
 def sampled_positions(lo: int, hi: int, scope_index: int) -> np.ndarray:
     """Positions read by the sampled-threshold mode in scope [lo, hi) (Section 4, fourth paragraph: a 0.1 % sample).
 
-    m = n_s if n_s <= 4096 else max(4096, ceil(n_s / 1000)); the scope is cut into m strata, the first
-    (n_s mod m) of floor(n_s / m) + 1 elements and the rest of floor(n_s / m), and stratum i contributes
-    the position  start_i + (mix32(i * 0x9E3779B9 + scope_index) mod width_i).  The rule is part of this
-    mode's definition, which is why the CUDA library restates it; nothing else is shared.
+    Scopes of up to 4096 elements are sampled completely.  Longer ones are sampled in pairs of neighbours
+    (both reads of a pair fall into one 32-byte sector of memory): m = max(4096, ceil(n_s / 1000)) rounded up
+    to an even number; the pairs are (first + 2 j, first + 2 j + 1) with first = the smallest even index
+    >= lo and j < P = floor((hi - first) / 2); the P pairs are cut into m / 2 strata, the first (P mod m/2)
+    of floor(P / (m/2)) + 1 pairs and the rest of floor(P / (m/2)), and stratum i contributes the pair
+    start_i + (mix32(i * 0x9E3779B9 + scope_index) mod width_i).  The rule is part of this mode's
+    definition, which is why the CUDA library restates it; nothing else is shared.
     """
     ns = hi - lo
-    m = ns if ns <= 4096 else max(4096, -(-ns // 1000))
-    if m == 0:
-        return np.empty(0, dtype=np.int64)
-    w, rem = ns // m, ns % m
-    i = np.arange(m, dtype=np.uint64)
+    if ns <= 4096:
+        return np.arange(lo, hi, dtype=np.int64)
+    m = max(4096, -(-ns // 1000))
+    m += m & 1
+    first = lo + (lo & 1)
+    pairs, strata = (hi - first) // 2, m // 2
+    w, rem = pairs // strata, pairs % strata
+    i = np.arange(strata, dtype=np.uint64)
     a = i * np.uint64(w) + np.minimum(i, np.uint64(rem))
     width = np.uint64(w) + (i < np.uint64(rem)).astype(np.uint64)
     with np.errstate(over="ignore"):
         h = _mix32((i.astype(np.uint32) * np.uint32(0x9E3779B9) + np.uint32(scope_index)).astype(np.uint32))
     off = np.where(width > 1, h.astype(np.uint64) % np.maximum(width, np.uint64(1)), np.uint64(0))
-    return (np.uint64(lo) + a + off).astype(np.int64)
+    even = np.uint64(first) + np.uint64(2) * (a + off)
+    return np.stack([even, even + np.uint64(1)], axis=1).reshape(-1).astype(np.int64)
 
 
 def compress_sampled(grad, residual, layer_off, shard_off, drop_ppm, scope_mode=SCOPE_GLOBAL):

@@ -81,9 +81,10 @@ void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint6
 
 // Sampled-threshold mode (Section 4): sample size and output capacity of one scope.
 inline uint64_t sampled_m(uint64_t ns) {
-  if (ns <= 4096) return ns;
-  const uint64_t m = (ns + 999) / 1000;
-  return m < 4096 ? 4096 : m;
+  if (ns <= 4096) return ns;            // sampled completely, element by element
+  uint64_t m = (ns + 999) / 1000;
+  if (m < 4096) m = 4096;
+  return m + (m & 1);                   // longer scopes: pairs of neighbours
 }
 inline uint64_t sampled_cap(uint64_t ns, uint64_t k) {
   const uint64_t c = 4 * k + 8192;
@@ -182,6 +183,7 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
     uint32_t cluster = 1;
     if (sampled) {
       m = sampled_m(ns);
+      cluster = ns <= 4096 ? 1u : 2u;
       rank = kept_count(m, drop_ppm);
       cap = sampled_cap(ns, d.k);
     } else if (predict) {

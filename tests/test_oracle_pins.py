@@ -475,23 +475,31 @@ def _mix32_py(x):
     return x
 
 
-def test_sampled_positions_are_one_per_stratum():
-    for lo, hi, si in ((0, 10, 0), (5, 4101, 3), (100, 100 + 4097, 1), (0, 5_000_000, 7), (17, 17 + 123_457, 2)):
+def test_sampled_positions_are_one_pair_per_stratum():
+    for lo, hi, si in ((0, 10, 0), (5, 4101, 3), (100, 100 + 4097, 1), (101, 101 + 4097, 1), (0, 5_000_000, 7),
+                       (17, 17 + 123_457, 2), (0, 4_097_001, 4)):
         ns = hi - lo
         pos = orc.sampled_positions(lo, hi, si)
-        m = ns if ns <= 4096 else max(4096, -(-ns // 1000))
+        if ns <= 4096:
+            assert pos.tolist() == list(range(lo, hi))           # small scopes: everything
+            continue
+        m = max(4096, -(-ns // 1000))
+        m += m % 2
         assert pos.shape[0] == m
-        w_, rem = ns // m, ns % m
+        first = lo + lo % 2
+        pairs, strata = (hi - first) // 2, m // 2
+        w_, rem = pairs // strata, pairs % strata
         starts = [0]
-        for i in range(m):                                      # strata laid end to end: rem wide ones, then the rest
+        for i in range(strata):                                 # strata of pairs laid end to end: rem wide ones first
             starts.append(starts[-1] + w_ + (1 if i < rem else 0))
-        assert starts[-1] == ns
-        for i in (0, 1, m // 2, m - 1):                         # pure-Python restatement on a few strata
+        assert starts[-1] == pairs
+        for i in (0, 1, strata // 2, strata - 1):               # pure-Python restatement on a few strata
             width = starts[i + 1] - starts[i]
-            want = lo + starts[i] + (_mix32_py(i * 0x9E3779B9 + si) % width if width > 1 else 0)
-            assert int(pos[i]) == want
+            pair = starts[i] + (_mix32_py(i * 0x9E3779B9 + si) % width if width > 1 else 0)
+            assert int(pos[2 * i]) == first + 2 * pair and int(pos[2 * i + 1]) == first + 2 * pair + 1
+        assert np.all(pos[0::2] % 2 == 0)                       # both reads of a pair share an aligned 8 bytes
         assert np.all(np.diff(pos) > 0) and pos[0] >= lo and pos[-1] < hi      # distinct, ordered, in range
-    assert orc.sampled_positions(3, 3 + 4096, 0).tolist() == list(range(3, 3 + 4096))   # small scopes: everything
+    assert orc.sampled_positions(3, 3 + 4096, 0).tolist() == list(range(3, 3 + 4096))
 
 
 def test_sampled_threshold_small_scope_is_exact_selection_with_all_ties():
@@ -519,7 +527,7 @@ def test_sampled_threshold_keeps_about_the_requested_fraction():
     g = rng.laplace(0, 1e-3, n).astype(np.float32)
     r = np.zeros(n, np.float32)
     out = orc.compress_sampled(g, r, [0, n], [0, n], 990_000)
-    m = 4096                                                   # ceil(n / 1000) = 4000 < 4096
+    m = 4096                                                   # ceil(n / 1000) = 4000 < 4096 (and already even)
     pos = orc.sampled_positions(0, n, 0)
     assert pos.shape[0] == m
     k_m = m - (m * 990_000) // 1_000_000
