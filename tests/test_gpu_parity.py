@@ -686,16 +686,19 @@ def test_sampled_threshold_overflow_is_reported(cuda_device):
 
 
 # ---------------------------------------------------------------- beyond 2^31 elements (64-bit offsets, full uint32 indices)
-def test_more_than_2_31_elements(cuda_device):
-    """n = 2^31 + 2^20 + 5: byte offsets pass 2^33 and indices pass 2^31.  The oracle's sort does not fit here, so
-    the result is pinned by what defines it: tau is the k-th largest key iff #{key > tau} < k <= #{key >= tau};
-    the kept set is every key above tau plus the lowest-index ties; values and residual reassemble v."""
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION], ids=["predicted", "dense"])
+@pytest.mark.parametrize("n", [(1 << 31) + (1 << 20) + 5, 1 << 32], ids=["2^31+2^20+5", "2^32"])
+def test_more_than_2_31_elements(cuda_device, n, flags):
+    """n = 2^31 + 2^20 + 5: byte offsets pass 2^33 and indices pass 2^31; n = 2^32: the largest gradient the library
+    takes, whose last index is 0xFFFFFFFF.  The oracle's sort does not fit here, so the result is pinned by what
+    defines it: tau is the k-th largest key iff #{key > tau} < k <= #{key >= tau}; the kept set is every key above
+    tau plus the lowest-index ties; values and residual reassemble v; the push lands on exactly the kept slots."""
     free, _ = torch.cuda.mem_get_info()
-    if free < 60 * (1 << 30):
-        pytest.skip("needs 60 GiB of free device memory")
-    n = (1 << 31) + (1 << 20) + 5
+    need = (16 * n + (12 << 30))
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of free device memory")
     w = W.small_layered(1, [n], 999_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 3)
-    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, flags, cuda_device)
     gen = torch.Generator(device=cuda_device).manual_seed(2031)
     g = torch.empty(n, dtype=torch.float32, device=cuda_device)
     chunk = 1 << 26
@@ -710,7 +713,7 @@ def test_more_than_2_31_elements(cuda_device):
         r_before = sess.residual.clone()
         sess.compress(g)
         assert sess.status() == B.GD_OK
-        assert sess.stats()["n_scopes_dense"] == 0
+        assert sess.stats()["n_scopes_dense"] == (1 if flags else 0)
         tau = int(_np_u32(sess.out_tau)[0])
         idx = sess.out_idx[:k].to(torch.int64) & 0xFFFFFFFF
         assert bool((idx[1:] > idx[:-1]).all()) and int(idx[-1]) == n - 1
@@ -737,6 +740,15 @@ def test_more_than_2_31_elements(cuda_device):
         bounds = torch.tensor(w.shard_off, device=cuda_device)
         assert torch.equal(torch.searchsorted(idx, bounds).to(torch.int32), sess.out_shard_cnt_off)
         del r_before
+    # the server side at these indices: p <- 0 + 1 * value on the kept slots of the three shards, nothing else touched
+    params = torch.zeros(n, dtype=torch.float32, device=cuda_device)
+    sess.apply(sess.shard_views(params))
+    assert sess.status() == B.GD_OK
+    assert torch.equal(params[idx], sess.out_val[:k])
+    touched = 0
+    for lo in range(0, n, chunk):
+        touched += int(torch.count_nonzero(params[lo:min(lo + chunk, n)]))
+    assert touched == int(torch.count_nonzero(sess.out_val[:k]))
 
 
 # ---------------------------------------------------------------- column-wise averages (Section 5.4)
