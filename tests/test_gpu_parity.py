@@ -751,6 +751,59 @@ def test_more_than_2_31_elements(cuda_device, n, flags):
     assert touched == int(torch.count_nonzero(sess.out_val[:k]))
 
 
+def test_two_means_at_the_packing_limit(cuda_device):
+    """n = 2^31, the most a packed word (31 index bits + the sign, Section 5.4's 1-bit values) can address: the last
+    element is negative and kept, so its word is 0xFFFFFFFF.  Checked against the definitions: threshold by rank
+    counts, sign bits against v, centres against an fp64 mean of the kept values, the push against the centres."""
+    n = 1 << 31
+    free, _ = torch.cuda.mem_get_info()
+    if free < 16 * n + (8 << 30):
+        pytest.skip("needs 40 GiB of free device memory")
+    w = W.small_layered(1, [n], 999_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_TWO_MEANS, 2)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
+    gen = torch.Generator(device=cuda_device).manual_seed(2131)
+    g = torch.empty(n, dtype=torch.float32, device=cuda_device)
+    chunk = 1 << 26
+    for lo in range(0, n, chunk):
+        g[lo:lo + chunk] = torch.randn(chunk, generator=gen, device=cuda_device) * 1e-3
+    g[n - 1] = -4.0
+    g[0] = 3.0
+    k = sess.k_total
+    sess.compress(g)                                                       # residual is zero: v = g
+    assert sess.status() == B.GD_OK
+    tau = int(_np_u32(sess.out_tau)[0])
+    word = sess.out_idx[:k].to(torch.int64) & 0xFFFFFFFF
+    idx, sign = word & 0x7FFFFFFF, word >> 31
+    assert int(word[-1]) == 0xFFFFFFFF and int(word[0]) == 0
+    assert bool((idx[1:] > idx[:-1]).all())
+    v_kept = g[idx]
+    assert torch.equal(sign, (v_kept.view(torch.int32) >> 31) & 1)
+    n_gt = n_eq = 0
+    for lo in range(0, n, chunk):
+        keys = g[lo:lo + chunk].view(torch.int32) & 0x7FFFFFFF
+        n_gt += int((keys > tau).sum())
+        n_eq += int((keys == tau).sum())
+    assert n_gt < k <= n_gt + n_eq
+    assert int(((v_kept.view(torch.int32) & 0x7FFFFFFF) >= tau).sum()) == k
+    assert int(torch.count_nonzero(sess.residual[idx])) == 0
+    want_res = g.clone()
+    want_res[idx] = 0.0
+    assert torch.equal(sess.residual.view(torch.int32), want_res.view(torch.int32))
+    del want_res
+    means = sess.out_means[0].double().cpu().numpy()
+    for sgn in (0, 1):
+        ref = float(v_kept[sign == sgn].double().mean())
+        assert abs(means[sgn] - ref) <= REL_TOL * abs(ref), (sgn, means[sgn], ref)
+    params = torch.zeros(n, dtype=torch.float32, device=cuda_device)
+    sess.apply(sess.shard_views(params))
+    assert sess.status() == B.GD_OK
+    assert torch.equal(params[idx], sess.out_means[0][sign])               # 0 + 1 * centre, exactly
+    touched = 0
+    for lo in range(0, n, chunk):
+        touched += int(torch.count_nonzero(params[lo:lo + chunk]))
+    assert touched == k
+
+
 # ---------------------------------------------------------------- column-wise averages (Section 5.4)
 @pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
 @pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
