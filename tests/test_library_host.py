@@ -91,6 +91,14 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert lib.gd_compress(C.byref(a), None) == B.GD_ERR_WORKSPACE
     a.n = 99
     assert lib.gd_compress(C.byref(a), None) == B.GD_ERR_INVALID_ARG    # n disagrees with the offsets
+    # the packed 1-bit value modes address 31 index bits; full 32-bit indices are for fp32 values only
+    big = (1 << 31) + 16
+    lo_big = (C.c_uint64 * 2)(0, big)
+    a.layer_off, a.shard_off, a.n, a.out_means = lo_big, lo_big, big, 0x6000
+    a.value_mode = B.GD_VALUES_TWO_MEANS
+    assert lib.gd_compress(C.byref(a), None) == B.GD_ERR_TOO_LARGE
+    a.value_mode = B.GD_VALUES_FP32
+    assert lib.gd_compress(C.byref(a), None) == B.GD_ERR_WORKSPACE      # accepted as far as the (missing) workspace
     ap = B._ApplyArgs()
     assert lib.gd_decompress_apply(C.byref(ap), None) == B.GD_ERR_INVALID_ARG
     assert lib.gd_residual_reset(None, 5, None) == B.GD_ERR_INVALID_ARG
