@@ -3,6 +3,7 @@
 Bit-exact: thresholds, survivor indices, survivor values, residuals, shard offsets.
 Within 1e-6 relative: the two means (fp64 reference sums) and the scatter-added parameters.
 """
+import gc
 import numpy as np
 import pytest
 import torch
@@ -693,6 +694,8 @@ def test_more_than_2_31_elements(cuda_device, n, flags):
     takes, whose last index is 0xFFFFFFFF.  The oracle's sort does not fit here, so the result is pinned by what
     defines it: tau is the k-th largest key iff #{key > tau} < k <= #{key >= tau}; the kept set is every key above
     tau plus the lowest-index ties; values and residual reassemble v; the push lands on exactly the kept slots."""
+    gc.collect()
+    torch.cuda.empty_cache()                                              # what earlier tests left in the caching allocator
     free, _ = torch.cuda.mem_get_info()
     need = (16 * n + (12 << 30))
     if free < need:
@@ -756,6 +759,8 @@ def test_two_means_at_the_packing_limit(cuda_device):
     element is negative and kept, so its word is 0xFFFFFFFF.  Checked against the definitions: threshold by rank
     counts, sign bits against v, centres against an fp64 mean of the kept values, the push against the centres."""
     n = 1 << 31
+    gc.collect()
+    torch.cuda.empty_cache()                                              # what earlier tests left in the caching allocator
     free, _ = torch.cuda.mem_get_info()
     if free < 16 * n + (8 << 30):
         pytest.skip("needs 40 GiB of free device memory")
@@ -997,6 +1002,8 @@ def test_config5_full_scale_against_the_oracle(cuda_device):
     """One step of workload 5 at its full 2^30 elements, compared with the oracle itself (selection on the
     composite keys: tens of GB of host memory, about a minute of host time)."""
     import psutil
+    gc.collect()
+    torch.cuda.empty_cache()                                              # what earlier tests left in the caching allocator
     free, _ = torch.cuda.mem_get_info()
     if free < 40 * (1 << 30) or psutil.virtual_memory().available < 90 * (1 << 30):
         pytest.skip("needs 40 GiB of device memory and 90 GiB of host memory")
