@@ -754,6 +754,49 @@ def test_more_than_2_31_elements(cuda_device, n, flags):
     assert touched == int(torch.count_nonzero(sess.out_val[:k]))
 
 
+def test_sampled_threshold_on_the_largest_gradient(cuda_device):
+    """Section 4, fourth paragraph, at n = 2^32: the sample positions (from the oracle's statement of the rule, here
+    4.3 M of them, up to index 2^32 - 1) fix the threshold; the survivors are then every entry at or above it."""
+    n = 1 << 32
+    gc.collect()
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 12 * n + (12 << 30):
+        pytest.skip("needs 60 GiB of free device memory")
+    w = W.small_layered(1, [n], 999_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 3)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode,
+                           B.GD_FLAG_SAMPLED_THRESHOLD, cuda_device)
+    gen = torch.Generator(device=cuda_device).manual_seed(2032)
+    g = torch.empty(n, dtype=torch.float32, device=cuda_device)
+    chunk = 1 << 26
+    for lo in range(0, n, chunk):
+        g[lo:lo + chunk] = torch.randn(chunk, generator=gen, device=cuda_device) * 1e-3
+    g[n - 1] = 7.0
+    sess.compress(g)                                                       # residual is zero: v = g
+    assert sess.status() == B.GD_OK
+    pos = orc.sampled_positions(0, n, 0)
+    m = pos.shape[0]
+    assert m == ((n + 999) // 1000 + 1) // 2 * 2 and int(pos.max()) < n and int(pos.max()) > n - 4000
+    sample = g[torch.from_numpy(pos.astype(np.int64)).to(cuda_device)].cpu().numpy()
+    k_m = orc.kept_count(m, w.drop_ppm)
+    t = int(np.sort(orc.magnitude_keys(sample))[m - k_m])
+    assert int(_np_u32(sess.out_tau)[0]) == t
+    kept = sess.kept()
+    count = 0
+    for lo in range(0, n, chunk):
+        count += int(((g[lo:lo + chunk].view(torch.int32) & 0x7FFFFFFF) >= t).sum())
+    assert kept == count and abs(kept / (n / 1000) - 1.0) < 0.05
+    idx = sess.out_idx[:kept].to(torch.int64) & 0xFFFFFFFF
+    assert bool((idx[1:] > idx[:-1]).all()) and int(idx[-1]) == n - 1
+    assert torch.equal(sess.out_val[:kept].view(torch.int32), g[idx].view(torch.int32))
+    assert int(((g[idx].view(torch.int32) & 0x7FFFFFFF) >= t).sum()) == kept
+    assert int(torch.count_nonzero(sess.residual[idx])) == 0
+    g[idx] = 0.0                                                           # what the residual must be now
+    assert torch.equal(sess.residual.view(torch.int32), g.view(torch.int32))
+    bounds = torch.tensor(w.shard_off, device=cuda_device)
+    assert torch.equal(torch.searchsorted(idx, bounds).to(torch.int32), sess.out_shard_cnt_off)
+
+
 def test_two_means_at_the_packing_limit(cuda_device):
     """n = 2^31, the most a packed word (31 index bits + the sign, Section 5.4's 1-bit values) can address: the last
     element is negative and kept, so its word is 0xFFFFFFFF.  Checked against the definitions: threshold by rank
