@@ -797,6 +797,63 @@ def test_sampled_threshold_on_the_largest_gradient(cuda_device):
     assert torch.equal(torch.searchsorted(idx, bounds).to(torch.int32), sess.out_shard_cnt_off)
 
 
+def test_delta_pull_beyond_2_31_elements(cuda_device):
+    """Section 4, third paragraph, with indices on both sides of 2^31: the dropped delta v = params - last pulled copy,
+    pinned by the rank counts that define the threshold; the server's copy advances by exactly what was sent and the
+    client's copy, which applies the pull, stays identical to it."""
+    n = (1 << 31) + (1 << 20) + 5
+    gc.collect()
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 20 * n + (8 << 30):
+        pytest.skip("needs 50 GiB of free device memory")
+    w = W.small_layered(1, [n], 999_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 3)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
+    gen = torch.Generator(device=cuda_device).manual_seed(2033)
+    chunk = 1 << 26
+    params = torch.empty(n, dtype=torch.float32, device=cuda_device)
+    for lo in range(0, n, chunk):
+        hi = min(lo + chunk, n)
+        params[lo:hi] = torch.randn(hi - lo, generator=gen, device=cuda_device) * 0.1
+    last = torch.zeros(n, dtype=torch.float32, device=cuda_device)
+    client = torch.zeros(n, dtype=torch.float32, device=cuda_device)
+    client_views = sess.shard_views(client)
+    k = sess.k_total
+    for step in range(2):
+        for lo in range(0, n, chunk):                                      # the parameters move on between pulls
+            hi = min(lo + chunk, n)
+            params[lo:hi] += torch.randn(hi - lo, generator=gen, device=cuda_device) * 1e-2
+        params[n - 1] += 9.0
+        params[1 << 31] -= 8.0
+        last_before = last.clone()
+        sess.compress_delta(params, last)
+        assert sess.status() == B.GD_OK
+        tau = int(_np_u32(sess.out_tau)[0])
+        idx = sess.out_idx[:k].to(torch.int64) & 0xFFFFFFFF
+        assert bool((idx[1:] > idx[:-1]).all()) and int(idx[-1]) == n - 1 and bool((idx == (1 << 31)).any())
+        n_gt = n_eq = n_kept = 0
+        for lo in range(0, n, chunk):
+            hi = min(lo + chunk, n)
+            v = params[lo:hi] - last_before[lo:hi]
+            keys = v.view(torch.int32) & 0x7FFFFFFF
+            n_gt += int((keys > tau).sum())
+            n_eq += int((keys == tau).sum())
+            kept = torch.zeros(hi - lo, dtype=torch.bool, device=cuda_device)
+            kept[idx[(idx >= lo) & (idx < hi)] - lo] = True
+            n_kept += int(kept.sum())
+            assert bool((keys[kept] >= tau).all()) and bool((keys[~kept] <= tau).all())
+            assert torch.equal(sess.residual[lo:hi].view(torch.int32),
+                               torch.where(kept, torch.zeros_like(v), v).view(torch.int32))
+            assert torch.equal(last[lo:hi].view(torch.int32),
+                               torch.where(kept, last_before[lo:hi] + v, last_before[lo:hi]).view(torch.int32))
+        assert n_gt < k <= n_gt + n_eq and n_kept == k
+        assert torch.equal(sess.out_val[:k].view(torch.int32), (params[idx] - last_before[idx]).view(torch.int32))
+        del last_before
+        sess.apply(client_views, 1.0)
+        assert sess.status() == B.GD_OK
+        assert torch.equal(client.view(torch.int32), last.view(torch.int32))
+
+
 def test_two_means_at_the_packing_limit(cuda_device):
     """n = 2^31, the most a packed word (31 index bits + the sign, Section 5.4's 1-bit values) can address: the last
     element is negative and kept, so its word is 0xFFFFFFFF.  Checked against the definitions: threshold by rank
