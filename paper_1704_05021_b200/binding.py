@@ -282,6 +282,13 @@ def gd_step_host(call: CompressCall, apply: Optional[ApplyCall], grad_host: torc
 
 PROFILE_TAGS = ["setup", "sample_select", "add_emit", "dense_select", "dense_compact", "cand_select", "cand_compact",
                 "finalize", "apply", "pack_sampled", "means", "feedback"]
+# Kernels one gd_compress launches, in order, by the path the call takes (each is one launch and, with
+# gd_profile_enable(2), one tagged event pair); gd_decompress_apply adds one "apply" per push.
+STEP_KERNELS = {
+    "predicted": ["setup", "sample_select", "add_emit", "cand_select", "cand_compact"],
+    "dense": ["setup", "add_emit", "dense_select", "dense_compact"],
+    "sampled": ["setup", "sample_select", "add_emit", "pack_sampled"],
+}
 
 
 def gd_profile_enable(mode) -> None:

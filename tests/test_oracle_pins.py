@@ -502,6 +502,72 @@ def test_sampled_positions_are_one_pair_per_stratum():
     assert orc.sampled_positions(3, 3 + 4096, 0).tolist() == list(range(3, 3 + 4096))
 
 
+def test_sampled_positions_equal_the_stored_literals():
+    """The position rule is frozen: tests/golden/sampled_positions.txt holds literal positions (sample size,
+    first / middle / last eight) for five scopes, and the oracle must still produce exactly those."""
+    seen = 0
+    for line in open(os.path.join(GOLDEN, "sampled_positions.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        head, first, middle, last = [part.split() for part in line.split("|")]
+        lo, hi, scope, m = (int(x) for x in head)
+        pos = orc.sampled_positions(lo, hi, scope)
+        assert pos.shape[0] == m
+        mid = m // 2 - 4
+        assert pos[:8].tolist() == [int(x) for x in first]
+        assert pos[mid:mid + 8].tolist() == [int(x) for x in middle]
+        assert pos[-8:].tolist() == [int(x) for x in last]
+        seen += 1
+    assert seen == 5
+
+
+def test_sampled_positions_worked_by_hand():
+    """8200 elements from index 1, scope 0: m = 4096 samples = 2048 pairs out of the 4099 pairs that start at
+    even indices 2, 4, ..., 8198; 4099 = 2 * 2048 + 3, so strata 0..2 hold three pairs and the others two.
+    The mix of 0 is 0 (every step of it maps 0 to 0), so stratum 0 of scope 0 contributes its first pair,
+    (2, 3).  Stratum 2047, the last, holds the pairs starting at 8196 and 8198."""
+    pos = orc.sampled_positions(1, 8201, 0)
+    assert pos.shape[0] == 4096
+    assert pos[:2].tolist() == [2, 3]
+    assert pos[-2:].tolist() in ([8196, 8197], [8198, 8199])
+    # stratum i >= 3 starts at pair 2 i + 3: its sample is one of two pairs
+    for i in (3, 100, 2046):
+        assert int(pos[2 * i]) in (2 + 2 * (2 * i + 3), 2 + 2 * (2 * i + 4))
+    # every pair position is even and the index 1 (before the first even index) is never read
+    assert int(pos.min()) == 2 and int(pos.max()) <= 8199
+
+
+@pytest.mark.parametrize("config", [1, 2, 3, 5])
+def test_sampled_threshold_kept_count_error_on_the_workloads(config):
+    """Section 4 presents the sampled threshold as an approximation; this checks it as one, without the position
+    formula: on the workloads' own shapes the number kept per scope stays within the sampling error of the exact
+    count k.  A threshold from k_m tail samples has a relative error of about 1 / sqrt(k_m) in rank; samples are
+    taken in pairs of neighbours, which in the worst case (neighbours always equal) halves the effective
+    sample, so the band is 5 sqrt(2 / k_m).  Scopes sampled completely keep at least k (k plus ties)."""
+    from paper_1704_05021_b200 import workloads as W
+    if config == 5:
+        w = W.workload(5, scale_log2=24)                     # the flat stress shape, cut to what the CPU suite can afford
+    elif config == 2:
+        w = W.workload(2, scope_mode=orc.SCOPE_PER_LAYER)    # six scopes from 10 to 16.8 M elements
+    else:
+        w = W.workload(config)
+    g = W.make_gradient(w, 0, "cpu").numpy()
+    r = np.zeros(w.n, np.float32)
+    out = orc.compress_sampled(g, r, w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode)
+    idx = out["idx"].astype(np.int64)
+    for lo, hi in orc.scopes_of(w.layer_off, w.scope_mode):
+        ns = hi - lo
+        k = orc.kept_count(ns, w.drop_ppm)
+        kept = int(np.searchsorted(idx, hi) - np.searchsorted(idx, lo))
+        m = orc.sampled_positions(lo, hi, 0).shape[0]
+        k_m = orc.kept_count(m, w.drop_ppm)
+        if ns <= 4096:
+            assert kept >= k
+            continue
+        band = 5.0 * math.sqrt(2.0 / k_m)
+        assert abs(kept / k - 1.0) <= band, (config, lo, hi, kept, k, band)
+
+
 def test_sampled_threshold_small_scope_is_exact_selection_with_all_ties():
     rng = np.random.default_rng(41)
     n = 3000                                                   # <= 4096: the sample is the whole scope
