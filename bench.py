@@ -36,7 +36,44 @@ def _metric_name():
 
 METRIC = _metric_name()
 UNIT = "GB/s"
-ADD_EMIT_DRAM_BYTES_PER_ELEMENT = 11.72   # ncu, see profiles/add_emit_kernel_flat_2p27.md
+
+
+def dram_traffic_per_element(w):
+    """DRAM bytes per element of the fused pass as ncu measured them (dram__bytes_read.sum + dram__bytes_write.sum
+    of one launch, divided by the elements of that launch), for the family of workloads `w` belongs to, or None.
+
+    The figures live in profiles/add_emit_dram_traffic.json, which is rewritten whenever the capture is refreshed;
+    a workload the captures do not cover reports no traffic."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "add_emit_dram_traffic.json")) as fh:
+            table = json.load(fh)
+    except Exception:
+        return None
+    family = "flat" if len(w.layer_off) == 2 else ("nmt" if w.config in (3, 4) else None)
+    entry = table.get(family) if family else None
+    if not entry:
+        return None
+    return {"bytes_per_element": float(entry["bytes_per_element"]), "captured_n": int(entry["n"]),
+            "captured": entry.get("captured"), "workload": entry.get("workload")}
+
+
+class L2Flush:
+    """Empties L2 of the step's data between timed steps: writes a 512 MiB buffer (four times the 126 MB L2), then
+    reads another one, so that the dirty lines of that very write are written back before the step's clock starts
+    (otherwise the step is charged up to 126 MB of somebody else's write-back)."""
+
+    def __init__(self, dev):
+        import torch
+        self.w = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+        self.r = torch.zeros(512 << 20, dtype=torch.uint8, device=dev)
+        self.sink = torch.zeros(1, dtype=torch.int64, device=dev)
+
+    def __call__(self, it):
+        self.w.fill_(it & 0xFF)
+        self.sink += self.r.view(-1, 1 << 20).sum()
+
+    TEXT = ("L2 flushed between timed steps (512 MiB written, then 512 MiB read so that the flush's own dirty lines "
+            "are written back), steps timed one by one")
 
 
 def read_peaks():
@@ -202,11 +239,13 @@ def run_reference(args):
     w = W.workload(args.config)
     steps, warmup = max(1, args.steps), max(0, args.warmup)
     gbs, ms, sample = time_oracle_step(w, steps, warmup)
+    sw, _, _ = oracle_sample(w)
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": workload_config(w, {"timed_steps": steps, "timed_warmup": warmup}),
+        # `n` is what one timed step processed: the bounded sample of the workload, `workload_n` the workload itself
+        "config": workload_config(w, {"n": sw.n, "workload_n": w.n, "timed_steps": steps, "timed_warmup": warmup}),
         "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -231,46 +270,89 @@ def aggregate_gbs(n_elements: int, steps: int, world: int, total_ms: float) -> f
     return world * 4.0 * n_elements * steps / (total_ms * 1e-3) / 1e9
 
 
-def quick_measure(config: int, dev, steps: int = 5, warmup: int = 3):
+def quick_measure(config: int, dev, steps: int = 5, warmup: int = 3, flags: int = 0, drop_ppm=None, scope_mode=None,
+                  flush=None):
     """Step time of another workload (same timing rules), for the `also` entries of the JSON line."""
+    import dataclasses
     import torch
     from paper_1704_05021_b200 import binding as B
     from paper_1704_05021_b200 import workloads as W
     from paper_1704_05021_b200.session import GradDropSession
-    w = W.workload(config)
-    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, dev)
+    w = W.workload(config) if scope_mode is None else W.workload(config, scope_mode=scope_mode)
+    if drop_ppm is not None:
+        w = dataclasses.replace(w, drop_ppm=drop_ppm)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, flags, dev)
     params = W.make_params(w, dev)
     views = sess.shard_views(params)
     pool = steps + warmup
     grads = [W.make_gradient(w, s, dev) for s in range(pool)]
-    flush = 8 * w.n < 4 * 126_000_000
-    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if flush else None
+    do_flush = 8 * w.n < 4 * 126_000_000
+    if do_flush and flush is None:
+        flush = L2Flush(dev)
     for it in range(warmup):
         sess.compress(grads[it])
         sess.apply(views)
     torch.cuda.synchronize()
+    if sess.status() != B.GD_OK:
+        return {"workload": workload_config(w)["workload"], "error": f"device status {sess.status()}"}
     beg = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
     end = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    kept = []
     for it in range(steps):
-        if flush:
-            flush_buf.fill_(it & 0xFF)
+        if do_flush:
+            flush(it)
         beg[it].record()
         sess.compress(grads[warmup + it])
         sess.apply(views)
         end[it].record()
+        if sess.sampled:
+            kept.append(sess.kept())                 # (synchronises; after the step's end event)
     torch.cuda.synchronize()
-    if sess.status() != B.GD_OK:
-        raise RuntimeError(f"device status {sess.status()} on workload {config}")
+    stats = sess.stats()
+    if stats["status"] != B.GD_OK:
+        return {"workload": workload_config(w)["workload"], "error": f"device status {stats['status']}"}
     ms = [b.elapsed_time(e) for b, e in zip(beg, end)]
-    total = sum(ms) if flush else beg[0].elapsed_time(end[-1])
+    total = sum(ms) if (do_flush or sess.sampled) else beg[0].elapsed_time(end[-1])
     ms_per_step = total / steps
     per_surv = 16.0 if w.value_mode != B.GD_VALUES_FP32 else 24.0
-    alg = (12.0 + per_surv * sess.k_total / max(w.n, 1)) * w.n
+    k_exact = B.gd_total_kept(w.layer_off, w.scope_mode, w.drop_ppm)
+    k_used = (sum(kept) / len(kept)) if kept else k_exact
+    alg = (12.0 + per_surv * k_used / max(w.n, 1)) * w.n
     peak, _ = read_peaks()
-    return {"workload": workload_config(w)["workload"], "steps": steps, "ms_per_step": ms_per_step,
-            "value": 4.0 * w.n / (ms_per_step * 1e-3) / 1e9, "unit": UNIT,
-            "frac_of_peak": alg / (ms_per_step * 1e-3) / 1e9 / peak,
-            "l2": "flushed between steps" if flush else "inputs larger than L2"}
+    # the fused pass alone, from the library's event pair around it (three more steps, not part of the time above)
+    B.gd_profile_enable(1)
+    B.gd_profile_collect()
+    for it in range(3):
+        if do_flush:
+            flush(it)
+        sess.compress(grads[it])
+        sess.apply(views)
+    torch.cuda.synchronize()
+    fused = B.gd_profile_collect()
+    B.gd_profile_enable(0)
+    out = {"workload": workload_config(w)["workload"], "steps": steps, "ms_per_step": ms_per_step,
+           "value": 4.0 * w.n / (ms_per_step * 1e-3) / 1e9, "unit": UNIT,
+           "frac_of_peak": alg / (ms_per_step * 1e-3) / 1e9 / peak,
+           "add_emit_ms": (sum(fused) / len(fused)) if fused else None,
+           "scopes_predicted": stats["n_scopes_predicted"], "scopes_dense": stats["n_scopes_dense"],
+           "candidates": stats["n_candidates"], "kept": stats["n_kept"],
+           "l2": "flushed between steps" if do_flush else "inputs larger than L2"}
+    if sess.sampled:
+        # Section 4's approximation: survivors per scope against the exact count k, on the last step
+        n_kept = sess.kept()
+        idx = (sess.out_idx[:n_kept].to(torch.int64) & 0xFFFFFFFF)
+        lay = w.layer_off if w.scope_mode == B.GD_SCOPE_PER_LAYER else [0, w.n]
+        cnt = torch.searchsorted(idx, torch.tensor(lay, device=dev)).diff().tolist()
+        ratios = []
+        for i, c in enumerate(cnt):
+            k = B.gd_kept_count(lay[i + 1] - lay[i], w.drop_ppm)
+            if k:
+                ratios.append(c / k)
+        out["sampled_kept_over_exact"] = {"whole_call_mean": k_used / max(k_exact, 1), "per_scope_min": min(ratios),
+                                          "per_scope_max": max(ratios), "scopes": len(ratios)}
+    del grads, params, views, sess
+    torch.cuda.empty_cache()
+    return out
 
 
 # ---------------------------------------------------------------- the CUDA arm
@@ -330,13 +412,13 @@ def run_cuda(args):
     # with a write of a 512 MiB buffer (4x the 126 MB L2) between the steps; the large ones stream
     # far more than L2 holds per step and are timed back to back.
     flush = 8 * w.n < 4 * 126_000_000
-    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if flush else None
+    flusher = L2Flush(dev) if flush else None
     ev_beg = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ev_end = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     barrier()
     for it in range(args.steps):
         if flush:
-            flush_buf.fill_(it & 0xFF)
+            flusher(it)
         ev_beg[it].record()
         sess.compress(grads[(args.warmup + it) % pool])
         sess.apply(views)
@@ -360,7 +442,7 @@ def run_cuda(args):
     ev3 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(split_steps)]
     for it in range(split_steps):
         if flush:
-            flush_buf.fill_(it & 0xFF)
+            flusher(it)
         ev3[it][0].record()
         sess.compress(grads[it % pool])
         ev3[it][1].record()
@@ -417,11 +499,14 @@ def run_cuda(args):
         roofline["achieved"] = fused_bytes / (fused_avg_ms * 1e-3) / 1e9
         roofline["frac"] = roofline["achieved"] / peak
         roofline["avg_launch_ms"] = fused_avg_ms
-    # DRAM traffic of the fused pass from the ncu capture of the 2^27-element case of the same kernel
-    # (profiles/add_emit_kernel_flat_2p27.md): every element is read twice and written once, so the
-    # figure scales with n.
-    roofline["traffic"] = ADD_EMIT_DRAM_BYTES_PER_ELEMENT * w.n
-    roofline["traffic_source"] = "ncu dram__bytes_read.sum + dram__bytes_write.sum at n = 2^27, scaled by n"
+    # DRAM traffic of the fused pass: ncu's figure for a smaller launch of the same kernel on the same kind of input,
+    # scaled by the elements of this launch (every element is read twice and written once, so it grows with n)
+    traffic = dram_traffic_per_element(w)
+    if traffic and not args.no_prediction and not args.sampled:
+        roofline["traffic"] = traffic["bytes_per_element"] * w.n
+        roofline["traffic_source"] = (f"ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch at n = "
+                                      f"{traffic['captured_n']} ({traffic['workload']}, captured {traffic['captured']}), "
+                                      f"scaled by n")
     k_frac = (stats["n_kept"] if args.sampled else sess.k_total) / max(w.n, 1)
     per_surv = 16.0 if w.value_mode == B.GD_VALUES_TWO_MEANS else 24.0
     alg_step_bytes = (12.0 + per_surv * k_frac) * w.n
@@ -436,18 +521,36 @@ def run_cuda(args):
                             "kind": "oracle restated with OpenMP passes and a parallel sort, same sample"}
 
     also = None
-    if args.config == 5 and not args.scale_log2 and not args.no_also and not args.sampled and not args.no_prediction:
-        # the drop ratio the metric's name quotes (99 %): the MNIST- and NMT-shaped workloads, same rules, fewer steps
+    sampled_report = None
+    if args.sampled:
         del grads, params, views, sess
         torch.cuda.empty_cache()
-        also = [quick_measure(2, dev), quick_measure(3, dev)]
+        sampled_report = quick_measure(args.config, dev, flags=B.GD_FLAG_SAMPLED_THRESHOLD)["sampled_kept_over_exact"]
+    elif args.config == 5 and not args.scale_log2 and not args.no_also and not args.no_prediction:
+        # The other four workloads (the drop ratio the metric's name quotes, 99 %, on the MNIST- and NMT-shaped
+        # gradients), the paper's other drop ratios on those shapes, and Section 4's sampled threshold on all five:
+        # same timing rules, fewer steps.
+        del grads, params, views, sess
+        torch.cuda.empty_cache()
+        fl = L2Flush(dev)
+        also = {
+            "workloads": [quick_measure(1, dev, flush=fl), quick_measure(2, dev, flush=fl),
+                          quick_measure(2, dev, scope_mode=B.GD_SCOPE_PER_LAYER, flush=fl),
+                          quick_measure(3, dev), quick_measure(4, dev)],
+            "drop_ratio_sweep": [quick_measure(c, dev, steps=3, drop_ppm=ppm, scope_mode=B.GD_SCOPE_PER_LAYER, flush=fl)
+                                 for c in (2, 3) for ppm in (900_000, 999_000)],
+            "sampled_threshold": [quick_measure(c, dev, steps=3, flags=B.GD_FLAG_SAMPLED_THRESHOLD, flush=fl,
+                                                scope_mode=B.GD_SCOPE_PER_LAYER if c == 2 else None)
+                                  for c in (1, 2, 3, 5)],
+        }
+        del fl
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": workload_config(w, {
-            "l2": "L2 flushed between timed steps (512 MiB write), steps timed one by one" if flush
+            "l2": L2Flush.TEXT if flush
                   else "inputs larger than L2 (gradient + residual stream 8 bytes per element per step)",
             "gradient_pool": pool, "prediction": not args.no_prediction,
             "threshold": "sampled (0.1 % sample, approximate)" if args.sampled else "exact"}),
@@ -457,6 +560,8 @@ def run_cuda(args):
         "split": split, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
         "clocks": clocks, "stats": stats, "also": also,
     }
+    if sampled_report is not None:
+        line["sampled_kept_over_exact"] = sampled_report
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

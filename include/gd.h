@@ -58,11 +58,15 @@ enum {
                                  KEPT entry is v minus the fp32 value the receiver will decode for it (one
                                  fp32 subtraction), as in the error feedback of 1-bit SGD that Section 2
                                  describes, instead of +0; dropped entries are unchanged. */
-  GD_FLAG_NO_EARLY_ZERO = 8u /* an implementation switch with no effect on results (for tests and timing):
+  GD_FLAG_NO_EARLY_ZERO = 8u, /* an implementation switch with no effect on results (for tests and timing):
                                  by default the fused pass already writes +0 into the residual slots
                                  of the entries the sample predicts to be kept, and the compaction
                                  only settles the few for which the prediction was wrong; with this
                                  flag the compaction clears every kept slot itself. */
+  GD_FLAG_PLAIN_RADIX = 16u   /* another switch with no effect on results: the selection among the candidates
+                                 normally starts from a histogram the fused pass has prepared and needs one
+                                 more pass; with this flag it always runs its three plain radix passes, as it
+                                 does by itself when a threshold lies far above its prediction. */
 };
 
 const char* gd_status_string(int status);
@@ -318,7 +322,8 @@ int gd_compress_static(const gd_compress_args* args, void* stream, const void** 
  * durations in milliseconds (oldest first, at most `capacity`) and, if tags_out is not NULL, which
  * kernel each belongs to (0 setup, 1 sample selection, 2 fused pass, 3 dense selection, 4 dense
  * compaction, 5 candidate selection, 6 candidate compaction, 7 finalize, 8 apply, 9 sampled-mode pack,
- * 10 means division, 11 quantisation-error feedback), then forgets them.
+ * 10 means division, 11 quantisation-error feedback, 12 candidate selection and compaction in one launch,
+ * 13 setup and prediction in one launch), then forgets them.
  * At most 4096 pairs are held between two collects; later launches are not recorded.  Not thread-safe.
  */
 int gd_profile_enable(int mode);

@@ -32,6 +32,7 @@ GD_FLAG_NO_PREDICTION = 1
 GD_FLAG_SAMPLED_THRESHOLD = 2
 GD_FLAG_QUANT_ERROR_FEEDBACK = 4
 GD_FLAG_NO_EARLY_ZERO = 8
+GD_FLAG_PLAIN_RADIX = 16
 GD_ERR_OVERFLOW = -7
 
 EXPORTS = [
@@ -281,11 +282,13 @@ def gd_step_host(call: CompressCall, apply: Optional[ApplyCall], grad_host: torc
 
 
 PROFILE_TAGS = ["setup", "sample_select", "add_emit", "dense_select", "dense_compact", "cand_select", "cand_compact",
-                "finalize", "apply", "pack_sampled", "means", "feedback"]
+                "finalize", "apply", "pack_sampled", "means", "feedback", "cand_select_compact", "setup_predict"]
 # Kernels one gd_compress launches, in order, by the path the call takes (each is one launch and, with
 # gd_profile_enable(2), one tagged event pair); gd_decompress_apply adds one "apply" per push.
 STEP_KERNELS = {
-    "predicted": ["setup", "sample_select", "add_emit", "cand_select", "cand_compact"],
+    "predicted": ["setup_predict", "add_emit", "cand_select_compact"],
+    "predicted_large_sample": ["setup", "sample_select", "add_emit", "cand_select_compact"],
+    "predicted_many_scopes": ["setup", "sample_select", "add_emit", "cand_select", "cand_compact"],
     "dense": ["setup", "add_emit", "dense_select", "dense_compact"],
     "sampled": ["setup", "sample_select", "add_emit", "pack_sampled"],
 }
@@ -327,6 +330,13 @@ def gd_compress_static(call: CompressCall, stream=None) -> int:
 def gd_status_at(workspace_address: int, stream=None) -> int:
     """gd_status for a workspace known by its device address (e.g. the one gd_compress_static returns)."""
     return load_library().gd_status(C.c_void_p(workspace_address), _stream_handle(stream))
+
+
+def gd_get_stats_at(workspace_address: int, stream=None) -> dict:
+    """gd_get_stats for a workspace known by its device address (e.g. the one gd_compress_static returns)."""
+    st = _Stats()
+    _check(load_library().gd_get_stats(C.c_void_p(workspace_address), _stream_handle(stream), C.byref(st)), "gd_get_stats")
+    return {name: getattr(st, name) for name, _ in _Stats._fields_}
 
 
 def gd_selftest_bounded_wait(workspace: torch.Tensor, spin_limit: int = 2000, stream=None) -> None:

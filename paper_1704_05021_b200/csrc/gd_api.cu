@@ -99,6 +99,7 @@ struct Plan {
   uint64_t samp_total = 0, cand_total = 0, k_total = 0;
   uint32_t n_scopes = 0;
   bool predict = true;
+  bool local_predict = false;   // the prediction shares a launch with the start of the call (gd_predict.cu)
   uint32_t emit_chunk_tiles = 1, dense_sel_tile = kDenseSelTileMax, dense_chunk_tiles = kDenseChunkTilesMax;
   uint32_t samp_tile = kTile;
   // workspace layout (byte offsets)
@@ -110,7 +111,7 @@ struct Plan {
   std::vector<uint64_t> pair_off;
   std::vector<uint32_t> layer_cols;
   uint64_t n_pairs = 0;
-  size_t off_samp = 0, off_cand_idx = 0, off_cand_val = 0, total_bytes = 0;
+  size_t off_agg = 0, off_flags = 0, off_samp = 0, off_cand_idx = 0, off_cand_val = 0, total_bytes = 0;
 };
 
 int check_offsets(const uint64_t* off, uint32_t count, uint64_t* n_out) {
@@ -262,6 +263,26 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
   t = align_up(t);
   P->tables_bytes = t;
   off += t;
+  // Samples of at most local_sample_max() values per scope are gathered in tiles of 256 by the kernel that also starts
+  // the call; it marks every finished tile in an array of flags.
+  P->local_predict = predict && !sampled && P->tables_bytes <= kSetupBlobBytes;
+  for (uint32_t s = 0; P->local_predict && s < ns_count; ++s)
+    if (P->scopes[s].samp_m > local_sample_max()) P->local_predict = false;
+  if (P->local_predict) {
+    // tiles of 256 samples spread a short sample over many SMs; larger tiles keep all CTAs resident at once
+    for (P->samp_tile = 256;; P->samp_tile *= 2) {
+      uint64_t tt = 0;
+      for (uint32_t s = 0; s < ns_count; ++s) {
+        P->tile0[L_SAMP][s] = (uint32_t)tt;
+        tt += (P->scopes[s].samp_m + P->samp_tile - 1) / P->samp_tile;
+      }
+      P->tile0[L_SAMP][ns_count] = (uint32_t)tt;
+      P->tiles[L_SAMP] = (uint32_t)tt;
+      if (tt <= 2u * 148u || P->samp_tile == 1024u) break;
+    }
+  }
+  P->off_flags = off;        off = align_up(off + sizeof(uint32_t) * (size_t)P->tiles[L_SAMP]);   // not cleared
+  P->off_agg = off;          off = align_up(off + 32 * (size_t)select_compact_max_grid());   // per-CTA records, not cleared
   P->off_samp = off;         off = align_up(off + sizeof(float) * P->samp_total);
   P->off_cand_idx = off;     off = align_up(off + sizeof(uint32_t) * P->cand_total);
   P->off_cand_val = off;     off = align_up(off + sizeof(float) * P->cand_total);
@@ -271,10 +292,6 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
 
 // Start of a call in one launch: clears the control region of the workspace and writes the small
 // host-built tables, which travel as a kernel argument, behind it.
-constexpr size_t kSetupBlobBytes = 3584;
-struct SetupBlob {
-  unsigned char bytes[kSetupBlobBytes];
-};
 
 __global__ void __launch_bounds__(kThreads) setup_kernel(const __grid_constant__ SetupBlob blob, uint4* tables_dst,
                                                          uint32_t tables_vec, uint4* zero_dst, uint64_t zero_vec) {
@@ -462,7 +479,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_COLUMN_MEANS) return GD_ERR_INVALID_ARG;
     if (a->value_mode != GD_VALUES_FP32 && n > (1ull << 31)) return GD_ERR_TOO_LARGE;
     if (a->flags & ~(uint32_t)(GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD | GD_FLAG_QUANT_ERROR_FEEDBACK |
-                               GD_FLAG_NO_EARLY_ZERO))
+                               GD_FLAG_NO_EARLY_ZERO | GD_FLAG_PLAIN_RADIX))
       return GD_ERR_INVALID_ARG;
     if ((a->flags & GD_FLAG_QUANT_ERROR_FEEDBACK) && a->value_mode == GD_VALUES_FP32) return GD_ERR_INVALID_ARG;
     const bool sampled = (a->flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
@@ -489,9 +506,6 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     std::memcpy(blob.data() + P.t_layer_cols, P.layer_cols.data(), sizeof(uint32_t) * (size_t)a->n_layers);
 
     unsigned char* ws = (unsigned char*)a->workspace;
-    if (launch_setup(ws + P.off_tables, blob.data(), P.tables_bytes, ws, P.zero_bytes, stream) != cudaSuccess)
-      return GD_ERR_CUDA;
-
     DevTables T;
     std::memset(&T, 0, sizeof(T));
     T.grad = a->grad;
@@ -527,6 +541,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     T.pair_off = (const uint64_t*)(tb + P.t_pair_off);
     T.layer_cols = (const uint32_t*)(tb + P.t_layer_cols);
     T.n_pairs = P.n_pairs;
+    T.cta_agg = ws + P.off_agg;
     T.samp_val = (float*)(ws + P.off_samp);
     T.cand_idx = (uint32_t*)(ws + P.off_cand_idx);
     T.cand_val = (float*)(ws + P.off_cand_val);
@@ -538,6 +553,16 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
 
     uint32_t tiles[L_COUNT];
     for (int l = 0; l < L_COUNT; ++l) tiles[l] = P.tiles[l];
+    // The start of the call (clearing the control region, writing the tables) shares a launch with the prediction
+    // when every scope's sample is small enough for one CTA; otherwise it is a launch of its own.
+    const bool local_predict = P.local_predict;
+    if (local_predict) {
+      if (launch_setup_predict(T, tiles[L_SAMP], P.samp_tile, (uint32_t*)(ws + P.off_flags), ws + P.off_tables, blob.data(), P.tables_bytes, ws, P.zero_bytes, P.off_state,
+                               P.t_scopes, P.t_tile0[L_SAMP], stream) != cudaSuccess)
+        return GD_ERR_CUDA;
+    } else if (launch_setup(ws + P.off_tables, blob.data(), P.tables_bytes, ws, P.zero_bytes, stream) != cudaSuccess) {
+      return GD_ERR_CUDA;
+    }
     if (sampled) {
       if (launch_sample_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
       if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
@@ -545,7 +570,7 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
       return GD_OK;
     }
     const bool predict = P.predict;
-    if (predict && launch_sample_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+    if (predict && !local_predict && launch_sample_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
     if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
     // Without a prediction: the selection and compaction over the dense range.  With one: the two kernels over
     // the candidate lists, which first do the dense work of the scopes whose prediction failed (usually none).
@@ -553,6 +578,9 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     if (!predict) {
       if (launch_dense_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
       if (launch_compact(T, tiles, true, true, stream) != cudaSuccess) return GD_ERR_CUDA;
+    } else if (P.n_scopes <= kSmemScopes) {
+      // selection among the candidates and compaction in one cooperative launch
+      if (launch_select_compact(T, tiles, P.cand_total, stream) != cudaSuccess) return GD_ERR_CUDA;
     } else {
       if (launch_candidate_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
       if (launch_compact(T, tiles, false, true, stream) != cudaSuccess) return GD_ERR_CUDA;

@@ -41,9 +41,9 @@ struct ApplyInline {
   uint32_t layer_cols[kInlineLayers];
 };
 
-// Segmented scatter-add: the entries [cnt_off[0], cnt_off[n_shards]) of one push, one thread per
-// entry in a grid-stride loop.  Indices inside one push are unique, so a plain read-modify-write is
-// enough; pushes are separate launches in stream order.
+// Segmented scatter-add: the entries [cnt_off[0], cnt_off[n_shards]) of one push, in a grid-stride
+// loop.  Indices inside one push are unique, so a plain read-modify-write is enough; pushes are
+// separate launches in stream order.
 template <bool INLINE>
 __global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__ ApplyDev A,
                                                          const __grid_constant__ ApplyInline I) {
@@ -54,28 +54,43 @@ __global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__
   const uint32_t* layer_cols = INLINE ? I.layer_cols : A.layer_cols;
   const uint64_t begin = A.cnt_off[0], end = A.cnt_off[A.n_shards];
   const uint64_t lo_all = shard_off[0], hi_all = shard_off[A.n_shards];
+  // Each thread takes kBatch entries at a time, a grid-stride apart, and has all their loads in flight before the
+  // first add: the scattered reads of the parameters are bound by memory latency, not by bandwidth.  Indices
+  // inside a push are unique, so the entries of a batch never touch the same parameter.
+  constexpr int kBatch = 4;
   const uint64_t stride = (uint64_t)gridDim.x * kThreads;
-  for (uint64_t p = begin + (uint64_t)blockIdx.x * kThreads + threadIdx.x; p < end; p += stride) {
-    const uint32_t w = __ldcs(A.idx + p);
-    uint64_t pos = w;
-    float x;
-    if (A.value_mode != GD_VALUES_FP32) {
-      pos = w & kAbsMask;
-      const uint64_t pr = pair_of(layer_off, pair_off, layer_cols, A.n_layers, pos);
-      x = __ldg(A.means + 2 * pr + (w >> 31));
-    } else {
-      x = __ldcs(A.val + p);
+  for (uint64_t p0 = begin + (uint64_t)blockIdx.x * kThreads + threadIdx.x; p0 < end; p0 += stride * kBatch) {
+    uint32_t w[kBatch];
+    float x[kBatch], old[kBatch];
+    float* dst[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const uint64_t p = p0 + (uint64_t)u * stride;
+      w[u] = p < end ? __ldcs(A.idx + p) : 0xFFFFFFFFu;
+      x[u] = (p < end && A.value_mode == GD_VALUES_FP32) ? __ldcs(A.val + p) : 0.0f;
     }
-    if (pos < lo_all || pos >= hi_all) continue;
-    const uint32_t j = range_of(shard_off, A.n_shards, pos);
-    float* dst = params[j] + (pos - shard_off[j]);
-    // One scattered 4-byte read-modify-write per survivor, bound by the rate of random DRAM accesses
-    // (about 20 G/s measured for this pattern, whatever the cache operator).  Asking L2 to fetch 64
-    // bytes around the miss instead of its default measured 12 % faster; red.global.add.f32 is as fast
-    // but flushes subnormals, which would break bit-exactness.
-    float old;
-    asm volatile("ld.global.cg.L2::64B.f32 %0, [%1];" : "=f"(old) : "l"(dst) : "memory");
-    __stcg(dst, __fmaf_rn(A.alpha, x, old));
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const uint64_t p = p0 + (uint64_t)u * stride;
+      dst[u] = nullptr;
+      if (p >= end) continue;
+      uint64_t pos = w[u];
+      if (A.value_mode != GD_VALUES_FP32) {
+        pos = w[u] & kAbsMask;
+        const uint64_t pr = pair_of(layer_off, pair_off, layer_cols, A.n_layers, pos);
+        x[u] = __ldg(A.means + 2 * pr + (w[u] >> 31));
+      }
+      if (pos < lo_all || pos >= hi_all) continue;
+      const uint32_t j = range_of(shard_off, A.n_shards, pos);
+      dst[u] = params[j] + (pos - shard_off[j]);
+      // One scattered 4-byte read-modify-write per survivor, bound by the rate of random DRAM accesses.  Asking
+      // L2 to fetch 64 bytes around the miss instead of its default measured 12 % faster; red.global.add.f32
+      // is as fast but flushes subnormals, which would break bit-exactness.
+      asm volatile("ld.global.cg.L2::64B.f32 %0, [%1];" : "=f"(old[u]) : "l"(dst[u]) : "memory");
+    }
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u)
+      if (dst[u]) __stcg(dst[u], __fmaf_rn(A.alpha, x[u], old[u]));
   }
 }
 

@@ -18,8 +18,16 @@ constexpr int kRadixBits0 = 11;         // 31-bit magnitude key = 11 + 10 + 10 b
 constexpr int kRadixBins0 = 1 << kRadixBits0;
 constexpr int kShift0 = 20, kShift1 = 10, kShift2 = 0;
 constexpr uint32_t kHistBinsPerScope = 2 * (2048 + 1024 + 1024);   // three passes over the sample, three over the list
+// The selection among the candidates of the fused pass first counts them in a histogram of D = key - base (base: the
+// smallest key a candidate can have): 2047 bins of 2^kFineShift keys each, and a last bin for everything further up.
+// The threshold is usually a few per cent above the base, i.e. inside the fine bins, and one more 11-bit pass finds it.
+constexpr int kFineShift = 11;
+constexpr uint32_t kFineBins = 2048, kFineTop = kFineBins - 1u;
 constexpr uint32_t kAbsMask = 0x7FFFFFFFu;
-constexpr uint32_t kLookbackSpinLimit = 1u << 21;  // polls before a look-back wait gives up
+constexpr uint32_t kLookbackSpinLimit = 1u << 21;  // a device-side wait gives up after this many polls ...
+constexpr uint64_t kWaitBudgetNs = 2000000000ull;  // ... AND this much time (whichever comes later): on a GPU that is
+                                                   // shared by time slices a poll count alone can run out while the
+                                                   // CTA waited on is merely descheduled
 constexpr uint64_t kInlineMeansPairs = 2048;       // up to this many pairs the finishing CTA divides the sums itself
 
 // Kinds of tiled launches; each has its own tile -> scope table.
@@ -67,6 +75,7 @@ struct ScopeState {      // zeroed at the start of every call
   uint32_t used_dense;   // 1 if the dense path produced this scope's result
   uint32_t pad;
 };
+static_assert(sizeof(ScopeState) == 48, "ScopeState is cleared and addressed in 16-byte units");
 
 struct Ctl {             // zeroed at the start of every call
   int32_t status;
@@ -77,9 +86,11 @@ struct Ctl {             // zeroed at the start of every call
   uint32_t dense_needed;   // scopes whose prediction failed (set by the fused pass)
   uint32_t barrier[3];     // grid barriers of the three selection kernels
   uint32_t compact_done[2];// CTAs of each compaction kernel that have finished
-  uint32_t pad;
+  uint32_t barrier_mid;    // grid barrier between a dense selection and a dense compaction run by one kernel
   uint64_t n_candidates;
   uint64_t n_kept;
+  uint32_t generic_needed; // some scope's threshold lies beyond the fine bins of the candidates' first histogram
+  uint32_t pad;
 };
 
 struct DevTables {       // passed by value to every kernel
@@ -115,6 +126,7 @@ struct DevTables {       // passed by value to every kernel
   const uint32_t* layer_cols;        // [n_layers] columns per layer (1 unless column-means mode)
   uint64_t n_pairs;                  // pairs in total
   // buffers
+  void* cta_agg;                     // [grid] per-CTA survivor counts of the kernel that selects and compacts in one launch
   float* samp_val;
   uint32_t* cand_idx;
   float* cand_val;
@@ -134,6 +146,15 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
   return m;
 }
 __device__ __forceinline__ uint64_t pack_desc(uint64_t flag, uint64_t value) { return (value << 2) | flag; }
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// True when a wait that began at t0 (global_timer_ns) and has polled `spins` times should give up.
+__device__ __forceinline__ bool wait_expired(uint32_t spins, uint32_t spin_limit, uint64_t t0, uint64_t budget_ns) {
+  return spins > spin_limit && (budget_ns == 0 || global_timer_ns() - t0 > budget_ns);
+}
 
 // Copy of the small per-call tables in shared memory: scope descriptors and the tile -> scope table
 // of one launch kind.  With few scopes (the usual case) every later lookup is a shared-memory read
@@ -248,6 +269,14 @@ __device__ __forceinline__ bool predicted_ok(const DevTables& T, const ScopeDesc
   return m >= d.k && m <= d.cand_cap;
 }
 
+// Smallest key a candidate of the fused pass can have: the predicted lower bound, but never 0 (zeros are never
+// candidates).  The candidates' first histogram counts D = key - this.
+__device__ __forceinline__ uint32_t candidate_base_key(uint32_t tau_lo) { return tau_lo == 0u ? 1u : tau_lo; }
+__device__ __forceinline__ uint32_t fine_bin(uint32_t key, uint32_t base) {
+  const uint32_t b = (key - base) >> kFineShift;
+  return b < kFineTop ? b : kFineTop;
+}
+
 // True when the fused pass writes +0 over the entries it expects to be kept (ScopeState::tau_hi).  Not
 // with quantisation-error feedback (the kept slots must hold v until the decode table exists), not
 // without a prediction.  (Sampled-threshold mode has its own, simpler form: every candidate is kept.)
@@ -256,9 +285,19 @@ __device__ __forceinline__ bool early_zero_enabled(const DevTables& T) {
                      GD_FLAG_NO_EARLY_ZERO)) == 0u;
 }
 
+// The small host-built tables of a call travel to the device as a kernel argument of this size at most.
+constexpr size_t kSetupBlobBytes = 3584;
+struct SetupBlob {
+  unsigned char bytes[kSetupBlobBytes];
+};
+
 // Host-side launchers of the kernel groups (one per .cu file); `tiles` is indexed by Launch.
 cudaError_t launch_setup(void* tables_dst, const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes,
                          cudaStream_t stream);
+cudaError_t launch_setup_predict(const DevTables& T, uint32_t gather_ctas, uint32_t gather_tile, uint32_t* flags, void* tables_dst, const void* tables_src,
+                                 size_t tables_bytes, void* zero_dst, size_t zero_bytes, size_t state_off, size_t scopes_off,
+                                 size_t tile0_off, cudaStream_t stream);
+uint32_t local_sample_max();   // most samples of one scope that launch_setup_predict handles
 cudaError_t launch_sample_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_candidate_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
@@ -268,6 +307,8 @@ cudaError_t launch_finalize(const DevTables& T, cudaStream_t stream);
 cudaError_t launch_means(const DevTables& T, cudaStream_t stream);
 cudaError_t launch_feedback(const DevTables& T, cudaStream_t stream);
 cudaError_t launch_pack_sampled(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
+cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uint64_t cand_total, cudaStream_t stream);
+uint32_t select_compact_max_grid();   // most CTAs of that launch (sizes DevTables::cta_agg)
 cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream);
 int sm_count();   // multiprocessors of the current device (0 on error)
 
@@ -275,7 +316,8 @@ int sm_count();   // multiprocessors of the current device (0 on error)
 void note_launches(uint32_t count);
 // Kernel tags of the measurement hooks, in the order a step launches them.
 enum ProfileTag : uint32_t { PT_SETUP = 0, PT_PACK_SAMPLED = 9, PT_MEANS = 10, PT_SAMPLE_SELECT = 1, PT_ADD_EMIT = 2, PT_DENSE_SELECT = 3, PT_DENSE_COMPACT = 4,
-                             PT_CAND_SELECT = 5, PT_CAND_COMPACT = 6, PT_FINALIZE = 7, PT_APPLY = 8, PT_FEEDBACK = 11 };
+                             PT_CAND_SELECT = 5, PT_CAND_COMPACT = 6, PT_FINALIZE = 7, PT_APPLY = 8, PT_FEEDBACK = 11,
+                             PT_CAND_SELECT_COMPACT = 12, PT_SETUP_PREDICT = 13 };
 void profile_mark(cudaStream_t stream, bool begin, uint32_t tag);
 struct ProfileScope {   // records an event pair around the launches made during its lifetime
   cudaStream_t stream;

@@ -25,12 +25,13 @@ __device__ __forceinline__ uint64_t warp_sum(uint64_t x) {
 
 // Run by one full warp.  Publishes this tile's totals, waits (bounded) for the tiles [first, t) of
 // the same scope and returns their sums.  Tile ids come from an atomic ticket, so every tile waited
-// on has already started.  A wait that runs out marks the tile aborted, records
+// on has already started.  A wait gives up after spin_limit polls and budget_ns of time (whichever
+// comes later; budget_ns = 0: the polls alone).  A wait that runs out marks the tile aborted, records
 // GD_ERR_DEVICE_TIMEOUT and returns false; a tile that meets an aborted predecessor aborts too, so
 // nothing waits on a tile that gave up.
 __device__ __forceinline__ bool tile_lookback(uint4* desc, uint32_t t, uint32_t first, uint64_t tot_a, uint64_t tot_b,
                                               uint64_t& ex_a, uint64_t& ex_b, Ctl* ctl,
-                                              uint32_t spin_limit = kLookbackSpinLimit) {
+                                              uint32_t spin_limit = kLookbackSpinLimit, uint64_t budget_ns = kWaitBudgetNs) {
   const uint32_t lane = lane_id();
   ex_a = 0;
   ex_b = 0;
@@ -46,6 +47,7 @@ __device__ __forceinline__ bool tile_lookback(uint4* desc, uint32_t t, uint32_t 
     const bool real = my >= (int64_t)first;      // lanes before the scope's first tile act as a zero prefix
     uint64_t lo = pack_desc(F_PREFIX, 0), hi = 0;
     uint32_t nearest = 32, flag = F_PREFIX, spins = 0;
+    uint64_t t0 = 0;                               // read when the wait starts to sleep
     for (;;) {
       if (real) ld_desc(desc + my, lo, hi);
       flag = (uint32_t)(lo & 3u);
@@ -54,7 +56,9 @@ __device__ __forceinline__ bool tile_lookback(uint4* desc, uint32_t t, uint32_t 
       nearest = stop ? (uint32_t)__ffs((int)stop) - 1u : 32u;
       const uint32_t need = nearest >= 32u ? 0xFFFFFFFFu : ((1u << nearest) - 1u);
       if ((inv & need) == 0u) break;
-      if (++spins > spin_limit) { ok = false; break; }
+      ++spins;
+      if (spins == 8) t0 = global_timer_ns();
+      if (__any_sync(0xFFFFFFFFu, wait_expired(spins, spin_limit, t0, budget_ns))) { ok = false; break; }
       if (spins > 8) __nanosleep(64);
     }
     if (!ok) break;

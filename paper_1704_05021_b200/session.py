@@ -47,6 +47,7 @@ class GradDropSession:
         self.apply_workspace = torch.empty(aws, dtype=torch.uint8, device=dev)
         self._compress_call: Optional[B.CompressCall] = None
         self._apply_call: Optional[B.ApplyCall] = None
+        self._apply_params = None                     # the list the cached argument block was built from
         self.reset()
 
     def reset(self, stream=None) -> None:
@@ -90,8 +91,10 @@ class GradDropSession:
                            self.layer_cols)
 
     def apply(self, params: List[torch.Tensor], alpha: float = 1.0, stream=None) -> None:
-        if self._apply_call is None or self._apply_call._keep[0] is not params:
+        if self._apply_call is None or self._apply_params is not params:
             self._apply_call = self.apply_call(params, alpha)
+            self._apply_params = params
+        self._apply_call.args.alpha = float(alpha)       # (the cached argument block may carry another call's alpha)
         B.gd_decompress_apply(self._apply_call, stream)
 
     def shard_views(self, flat_params: torch.Tensor) -> List[torch.Tensor]:

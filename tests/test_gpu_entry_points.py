@@ -140,3 +140,27 @@ def test_profile_enable_rejects_unknown_modes(cuda_device):
         B.gd_profile_enable(3)
     with pytest.raises(B.GdError):
         B.gd_profile_enable(-1)
+
+
+def test_apply_with_two_alphas_in_one_session(cuda_device):
+    """Section 3's server update with two step sizes in a row on one session: each call uses its own alpha."""
+    w = _layout(B.GD_VALUES_FP32)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
+    g = torch.randn(w.n, device=cuda_device) * 1e-3
+    sess.compress(g)
+    exp = orc.compress(g.cpu().numpy(), orc.residual_reset(w.n), w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode)
+    params = torch.zeros(w.n, device=cuda_device)
+    views = sess.shard_views(params)
+    sess.apply(views)                 # alpha = 1
+    sess.apply(views, 0.5)
+    sess.apply(views, -2.0)
+    torch.cuda.synchronize()
+    push = {"idx": exp["idx"], "val": exp["val"]}
+    got = params.cpu().numpy().astype(np.float64)
+    ref, bound = np.zeros(w.n), np.zeros(w.n)
+    for alpha in (1.0, 0.5, -2.0):                       # the oracle's fp64 sum, one push per step size
+        r, b = orc.apply_pushes(np.zeros(w.n, np.float32), 0, [push], alpha=alpha)
+        ref += r
+        bound += b
+    assert np.all(np.abs(got - ref) <= REL_TOL * bound + 1e-45)
+    assert np.count_nonzero(got) == np.count_nonzero(ref)

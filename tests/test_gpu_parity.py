@@ -102,7 +102,7 @@ def test_config1_five_steps(cuda_device, flags):
     run_steps(W.workload(1), cuda_device, 5, flags=flags, expect_dense=True)     # short vectors are selected densely
 
 
-@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION, B.GD_FLAG_NO_EARLY_ZERO])
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION, B.GD_FLAG_NO_EARLY_ZERO, B.GD_FLAG_PLAIN_RADIX])
 def test_config1_shape_at_2_23(cuda_device, flags):
     """The same distribution just above the length where the prediction is switched on."""
     run_steps(W.workload(1, scale_log2=23), cuda_device, 3, flags=flags, method="select",
@@ -159,7 +159,7 @@ def test_heavy_ties(cuda_device, flags):
             run_steps(w, cuda_device, 2, flags=flags, grads=[torch.from_numpy(g), torch.from_numpy(g)])
 
 
-@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_EARLY_ZERO])
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_EARLY_ZERO, B.GD_FLAG_PLAIN_RADIX])
 def test_ties_and_dense_runs_on_the_predicted_path(cuda_device, flags):
     """Vectors long enough for the prediction (above 2^21 elements), shaped to reach every branch behind it:
     lists that overflow (the scope is then selected densely, after the slots cleared early got v back), warps
@@ -1131,6 +1131,8 @@ def test_random_models_of_few_large_tensors(cuda_device, seed):
     flags = int(rng.choice([0, 0, 0, B.GD_FLAG_NO_EARLY_ZERO, B.GD_FLAG_NO_PREDICTION]))
     if value_mode == B.GD_VALUES_THRESHOLD and rng.random() < 0.5:
         flags |= B.GD_FLAG_QUANT_ERROR_FEEDBACK
+    if seed % 2 == 1 and not flags & B.GD_FLAG_NO_PREDICTION:
+        flags |= B.GD_FLAG_PLAIN_RADIX                # the selection's three plain radix passes instead of its short cut
     cols = None
     if value_mode == B.GD_VALUES_COLUMN_MEANS:
         cols = []
@@ -1155,6 +1157,26 @@ def test_random_models_of_few_large_tensors(cuda_device, seed):
             g[a:a + 20000] = rng.choice([0.5, -0.5, 1.0], 20000)
         grads.append(torch.from_numpy(g.astype(np.float32)))
     run_steps(w, cuda_device, 2, flags=flags, grads=grads, layer_cols=cols, alpha=float(rng.choice([1.0, 0.5])))
+
+
+@pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
+def test_threshold_far_above_the_prediction(cuda_device, scope_mode):
+    """Magnitudes spread evenly over 120 binades: the prediction's safety margin (a multiple of the expected rank for
+    the small sample of a short tensor) then lies binades below the real threshold, beyond the range in which the
+    selection among the candidates can start from the fused pass's histogram, so it runs its plain radix passes
+    by itself.  Mixed with ordinary tensors in one call; three steps, residual carried."""
+    rng = np.random.default_rng(314)
+    sizes = [2_000_000, 20_000, 40_000, 1_000_000, 9_000]
+    w = W.small_layered(len(sizes), sizes, 990_000, scope_mode, B.GD_VALUES_FP32, 3)
+    grads = []
+    for _ in range(3):
+        g = rng.laplace(0, 1e-3, w.n).astype(np.float32)
+        for l in (1, 2, 4):
+            lo, hi = w.layer_off[l], w.layer_off[l + 1]
+            mag = np.exp2(rng.uniform(-126.0, -6.0, hi - lo))
+            g[lo:hi] = (mag * rng.choice([-1.0, 1.0], hi - lo)).astype(np.float32)
+        grads.append(torch.from_numpy(g))
+    run_steps(w, cuda_device, 3, grads=grads)
 
 
 @pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])

@@ -52,6 +52,34 @@ def test_static_scratch_matches_caller_workspace(cuda_device, value_mode):
             assert bool(((a - b).abs() <= 1e-6 * b.abs()).all()), f"call {call_no}: means"
 
 
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_SAMPLED_THRESHOLD], ids=["exact", "sampled_threshold"])
+def test_static_scratch_on_the_predicted_path(cuda_device, flags):
+    """A gradient long enough for the path that predicts the threshold from a sample (so that the sample, the
+    candidate lists and the kernels that work on them all run on the built-in scratch), and one call with the
+    threshold taken on a sample; two calls in a row each, same bytes as with a caller-owned workspace."""
+    w = W.workload(5, scale_log2=23)               # 2^23 elements, 99.9 %, 8 shards: about 3 MiB of scratch
+    assert B.gd_workspace_bytes(w.layer_off, w.n_shards, w.scope_mode, w.drop_ppm) <= B.GD_STATIC_WORKSPACE_BYTES
+    ref = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, flags, cuda_device)
+    sta = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, flags, cuda_device)
+    for call_no in range(2):
+        g = W.make_gradient(w, call_no, cuda_device)
+        ref.compress(g)
+        call = sta.compress_call(g)
+        call.args.workspace = None
+        call.args.workspace_bytes = 0
+        scratch = B.gd_compress_static(call)
+        st = B.gd_get_stats_at(scratch)
+        assert st["status"] == B.GD_OK and ref.status() == B.GD_OK
+        assert st["n_scopes_predicted"] == 1 and st["n_scopes_dense"] == 0, st
+        k = ref.kept()
+        assert int(sta.out_shard_cnt_off[-1]) == k if flags else True
+        assert torch.equal(_bits(sta.out_idx[:k]), _bits(ref.out_idx[:k])), f"call {call_no}: indices"
+        assert torch.equal(_bits(sta.out_val[:k]), _bits(ref.out_val[:k])), f"call {call_no}: values"
+        assert torch.equal(_bits(sta.residual), _bits(ref.residual)), f"call {call_no}: residual"
+        assert torch.equal(sta.out_tau, ref.out_tau), f"call {call_no}: thresholds"
+        assert torch.equal(sta.out_shard_cnt_off, ref.out_shard_cnt_off), f"call {call_no}: shard offsets"
+
+
 def test_static_scratch_refuses_oversized_calls(cuda_device):
     w = W.workload(5)    # 2^30 elements: needs about twice the scratch the built-in area holds
     assert B.gd_workspace_bytes(w.layer_off, w.n_shards, w.scope_mode, w.drop_ppm) > B.GD_STATIC_WORKSPACE_BYTES
