@@ -323,7 +323,7 @@ int gd_compress_static(const gd_compress_args* args, void* stream, const void** 
  * kernel each belongs to (0 setup, 1 sample selection, 2 fused pass, 3 dense selection, 4 dense
  * compaction, 5 candidate selection, 6 candidate compaction, 7 finalize, 8 apply, 9 sampled-mode pack,
  * 10 means division, 11 quantisation-error feedback, 12 candidate selection and compaction in one launch,
- * 13 setup and prediction in one launch), then forgets them.
+ * 13 setup and prediction in one launch, 14 dense histogram pass, 15 walk of the dense histogram), then forgets them.
  * At most 4096 pairs are held between two collects; later launches are not recorded.  Not thread-safe.
  */
 int gd_profile_enable(int mode);

@@ -100,6 +100,7 @@ struct Plan {
   uint32_t n_scopes = 0;
   bool predict = true;
   bool local_predict = false;   // the prediction shares a launch with the start of the call (gd_predict.cu)
+  bool dense_bound = false;     // no sample: the lower bounds come from a histogram pass over the dense vector (gd_dense.cu)
   uint32_t emit_chunk_tiles = 1, dense_sel_tile = kDenseSelTileMax, dense_chunk_tiles = kDenseChunkTilesMax;
   uint32_t samp_tile = kTile;
   // workspace layout (byte offsets)
@@ -137,6 +138,12 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
   // run out of L2 and cost less than sampling, predicting and selecting among candidates.
   const bool predict = !(flags & GD_FLAG_NO_PREDICTION) && (sampled || n > kAutoDenseMax);
   P->predict = predict;
+  // Without a sample, long vectors still go through the candidate lists: one histogram pass over the dense vector
+  // gives every scope an exact lower bound of its threshold (gd_dense.cu).  Short vectors, whose passes run out
+  // of L2, and calls with more scopes than the kernels over the lists keep in shared memory take the plain dense
+  // selection and compaction.
+  const uint32_t ns_planned = scope_mode == GD_SCOPE_GLOBAL ? 1u : n_layers;
+  P->dense_bound = !predict && !sampled && n > kAutoDenseMax && ns_planned <= kSmemScopes;
   P->pair_off.assign((size_t)n_layers + 1, 0);
   P->layer_cols.assign(n_layers, 1);
   for (uint32_t l = 0; l < n_layers; ++l) {
@@ -189,6 +196,10 @@ int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* laye
       cap = sampled_cap(ns, d.k);
     } else if (predict) {
       plan_prediction(ns, d.k, &m, &rank, &cap, &cluster);
+    } else if (P->dense_bound) {
+      // the candidates are the keys above the bin of the k-th largest key (fewer than k) and that bin itself
+      const uint64_t c = 3 * d.k + 4096;
+      cap = c < ns ? c : ns;
     }
     d.cand_base = cand_base;
     d.cand_cap = cap;
@@ -449,12 +460,14 @@ int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, const uint3
                        int scope_mode, uint32_t drop_ppm, size_t* bytes_out) {
   if (!bytes_out) return GD_ERR_INVALID_ARG;
   try {
-    Plan P, Q;
-    int rc = make_plan(layer_off, n_layers, layer_cols, n_shards, scope_mode, drop_ppm, 0u, &P);
-    if (rc != GD_OK) return rc;
-    rc = make_plan(layer_off, n_layers, layer_cols, n_shards, scope_mode, drop_ppm, GD_FLAG_SAMPLED_THRESHOLD, &Q);
-    if (rc != GD_OK) return rc;
-    *bytes_out = P.total_bytes > Q.total_bytes ? P.total_bytes : Q.total_bytes;   // whichever mode is used
+    size_t most = 0;                                       // whichever mode is used
+    for (uint32_t flags : {0u, (uint32_t)GD_FLAG_SAMPLED_THRESHOLD, (uint32_t)GD_FLAG_NO_PREDICTION}) {
+      Plan P;
+      int rc = make_plan(layer_off, n_layers, layer_cols, n_shards, scope_mode, drop_ppm, flags, &P);
+      if (rc != GD_OK) return rc;
+      if (P.total_bytes > most) most = P.total_bytes;
+    }
+    *bytes_out = most;
     return GD_OK;
   } catch (const std::bad_alloc&) {
     return GD_ERR_INVALID_ARG;
@@ -571,11 +584,19 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     }
     const bool predict = P.predict;
     if (predict && !local_predict && launch_sample_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
-    if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+    if (predict && launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
     // Without a prediction: the selection and compaction over the dense range.  With one: the two kernels over
     // the candidate lists, which first do the dense work of the scopes whose prediction failed (usually none).
     // The compaction that runs last also finishes the call (thresholds, shard offsets, means).
-    if (!predict) {
+    if (P.dense_bound) {
+      // histogram pass over grad + residual -> exact lower bounds -> the usual fused pass and the kernel over the lists
+      if (launch_dense_bound(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+      DevTables U = T;
+      U.flags = (T.flags & ~(uint32_t)GD_FLAG_NO_PREDICTION) | GD_FLAG_NO_EARLY_ZERO | kFlagDenseBound;
+      if (launch_add_emit(U, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+      if (launch_select_compact(U, tiles, P.cand_total, stream) != cudaSuccess) return GD_ERR_CUDA;
+    } else if (!predict) {
+      if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
       if (launch_dense_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
       if (launch_compact(T, tiles, true, true, stream) != cudaSuccess) return GD_ERR_CUDA;
     } else if (P.n_scopes <= kSmemScopes) {

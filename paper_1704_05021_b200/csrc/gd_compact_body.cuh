@@ -23,7 +23,7 @@ __device__ void finalize_call(const DevTables& T, uint64_t k_total) {
     const ScopeDesc& d = T.scopes[s];
     const ScopeState* st = T.state + s;
     if (T.out_tau) T.out_tau[s] = d.k == 0 ? 0xFFFFFFFFu : __ldcg(&st->tau);
-    if (__ldcg(&st->used_dense)) ++n_dense; else ++n_pred;
+    if (__ldcg(&st->used_dense) || (T.flags & kFlagDenseBound)) ++n_dense; else ++n_pred;
     n_cand += __ldcg(reinterpret_cast<const unsigned long long*>(&st->cand_count));
   }
   if (n_pred) atomicAdd(&T.ctl->n_scopes_predicted, n_pred);

@@ -73,7 +73,7 @@ struct ScopeState {      // zeroed at the start of every call
   uint32_t early_bad;    // set when some such entry could not be recorded (a full stash, a full list): the
                          // compaction then clears every kept slot itself
   uint32_t used_dense;   // 1 if the dense path produced this scope's result
-  uint32_t pad;
+  uint32_t top_bin_max;  // dense histogram pass: largest first digit (key >> 20) seen in the scope so far
 };
 static_assert(sizeof(ScopeState) == 48, "ScopeState is cleared and addressed in 16-byte units");
 
@@ -90,7 +90,7 @@ struct Ctl {             // zeroed at the start of every call
   uint64_t n_candidates;
   uint64_t n_kept;
   uint32_t generic_needed; // some scope's threshold lies beyond the fine bins of the candidates' first histogram
-  uint32_t pad;
+  uint32_t hist_redo;      // dense histogram pass: some scope's k-th largest key lay below the window that was counted
 };
 
 struct DevTables {       // passed by value to every kernel
@@ -261,6 +261,10 @@ __device__ __forceinline__ uint64_t pair_of(const uint64_t* __restrict__ layer_o
   return pair_off[l] + (cols > 1 ? (idx - layer_off[l]) % cols : 0ull);
 }
 
+// Internal bit of DevTables::flags (never passed by a caller): the lower bounds of this call come from a histogram
+// over the dense vector (gd_dense.cu), not from a sample; its scopes count as selected densely in the statistics.
+constexpr uint32_t kFlagDenseBound = 1u << 31;
+
 // True when the scope's result comes from the candidate list the fused pass emitted: the
 // prediction was a valid lower bound (at least k candidates) and the list did not overflow.
 __device__ __forceinline__ bool predicted_ok(const DevTables& T, const ScopeDesc& d, const ScopeState& st) {
@@ -308,6 +312,7 @@ cudaError_t launch_means(const DevTables& T, cudaStream_t stream);
 cudaError_t launch_feedback(const DevTables& T, cudaStream_t stream);
 cudaError_t launch_pack_sampled(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uint64_t cand_total, cudaStream_t stream);
+cudaError_t launch_dense_bound(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 uint32_t select_compact_max_grid();   // most CTAs of that launch (sizes DevTables::cta_agg)
 cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream);
 int sm_count();   // multiprocessors of the current device (0 on error)
@@ -317,7 +322,8 @@ void note_launches(uint32_t count);
 // Kernel tags of the measurement hooks, in the order a step launches them.
 enum ProfileTag : uint32_t { PT_SETUP = 0, PT_PACK_SAMPLED = 9, PT_MEANS = 10, PT_SAMPLE_SELECT = 1, PT_ADD_EMIT = 2, PT_DENSE_SELECT = 3, PT_DENSE_COMPACT = 4,
                              PT_CAND_SELECT = 5, PT_CAND_COMPACT = 6, PT_FINALIZE = 7, PT_APPLY = 8, PT_FEEDBACK = 11,
-                             PT_CAND_SELECT_COMPACT = 12, PT_SETUP_PREDICT = 13 };
+                             PT_CAND_SELECT_COMPACT = 12, PT_SETUP_PREDICT = 13,
+                             PT_DENSE_HIST = 14, PT_DENSE_FIND = 15 };
 void profile_mark(cudaStream_t stream, bool begin, uint32_t tag);
 struct ProfileScope {   // records an event pair around the launches made during its lifetime
   cudaStream_t stream;

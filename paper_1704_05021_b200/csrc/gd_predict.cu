@@ -106,7 +106,7 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
   const uint32_t m = (uint32_t)d.samp_m;
   if (lt == 0 && tid == 0) {
     // everything but the prediction, which is written by the CTA that finishes the scope
-    st->cand_count = 0; st->tau = 0; st->q = 0; st->gt = 0; st->early_bad = 0; st->used_dense = 0; st->pad = 0;
+    st->cand_count = 0; st->tau = 0; st->q = 0; st->gt = 0; st->early_bad = 0; st->used_dense = 0; st->top_bin_max = 0;
   }
   if (tid < kGather) {
     const uint32_t li = lt * kGather + tid;
