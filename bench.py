@@ -355,6 +355,51 @@ def quick_measure(config: int, dev, steps: int = 5, warmup: int = 3, flags: int 
     return out
 
 
+def multi_push_measure(config: int, dev, drop_ppm: int, workers=(2, 4, 8), reps: int = 3, flush=None):
+    """Section 3's server receiving a piece from every worker: W pushes (W different gradients of the workload,
+    compressed by W sessions) applied to one set of parameter shards, one launch per push in order against one
+    launch with atomic updates (GD_APPLY_ATOMIC).  Time of the apply alone, L2 flushed before every repetition."""
+    import dataclasses
+    import torch
+    from paper_1704_05021_b200 import binding as B
+    from paper_1704_05021_b200 import workloads as W
+    from paper_1704_05021_b200.session import GradDropSession
+    w = dataclasses.replace(W.workload(config), drop_ppm=drop_ppm)
+    flush = flush or L2Flush(dev)
+    sessions = []
+    g = torch.empty(w.n, dtype=torch.float32, device=dev)
+    for i in range(max(workers)):
+        sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, dev)
+        W.make_gradient(w, i, dev, out=g)
+        sess.compress(g)
+        if sess.status() != B.GD_OK:
+            return {"workload": workload_config(w)["workload"], "error": f"device status {sess.status()}"}
+        sessions.append(sess)
+    params = W.make_params(w, dev)
+    views = sessions[0].shard_views(params)
+    out = {"workload": workload_config(w)["workload"], "survivors_per_push": sessions[0].k_total, "apply_ms": []}
+    for nw in workers:
+        pushes = [s_.push() for s_ in sessions[:nw]]
+        row = {"pushes": nw}
+        for name, fl in (("ordered", 0), ("atomic", B.GD_APPLY_ATOMIC)):
+            call = sessions[0].apply_call(views, 1.0, pushes, fl)
+            B.gd_decompress_apply(call)                       # warm-up
+            ms = []
+            for it in range(reps):
+                flush(it)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                B.gd_decompress_apply(call)
+                e1.record()
+                torch.cuda.synchronize()
+                ms.append(e0.elapsed_time(e1))
+            row[name] = sum(ms) / len(ms)
+        out["apply_ms"].append(row)
+    del sessions, params, views, g
+    torch.cuda.empty_cache()
+    return out
+
+
 # ---------------------------------------------------------------- the CUDA arm
 def run_cuda(args):
     import torch
@@ -542,6 +587,7 @@ def run_cuda(args):
             "sampled_threshold": [quick_measure(c, dev, steps=3, flags=B.GD_FLAG_SAMPLED_THRESHOLD, flush=fl,
                                                 scope_mode=B.GD_SCOPE_PER_LAYER if c == 2 else None)
                                   for c in (1, 2, 3, 5)],
+            "multi_push_apply": [multi_push_measure(3, dev, ppm, flush=fl) for ppm in (900_000, 990_000)],
         }
         del fl
 

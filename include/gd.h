@@ -221,10 +221,20 @@ typedef struct gd_push {
  * with value = val[t] (fp32 mode) or means[pair of the entry][sign] (the packed modes; the pair is the
  * entry's layer, or its layer and column in column-means mode).
  * One fused multiply-add in fp32 per entry; with alpha = 1 the result is fl32(p + value).
- * Pushes are applied one after another in stream order; indices inside one push are unique.
+ * Pushes are applied one after another in stream order (unless GD_APPLY_ATOMIC is set); indices inside one push are unique.
  * Entries whose index lies outside every shard are skipped.  The optimiser is not part of
  * this library.
  */
+/* gd_apply_args.flags */
+enum {
+  GD_APPLY_ATOMIC = 1u /* Section 3 has every server receive a piece from every worker.  By default the pushes of a
+                          call are applied one after another (one launch each, array order).  With this flag all of
+                          them are applied by one launch and entries of different pushes that meet in one parameter
+                          are combined with atomic read-modify-writes, in no defined order: every entry still lands
+                          exactly once as one fused multiply-add (subnormals kept), so the result differs from the
+                          ordered one by the rounding of a different summation order only. */
+};
+
 typedef struct gd_apply_args {
   float* const* params;        /* HOST array of n_shards device pointers */
   const uint64_t* shard_off;   /* HOST, n_shards + 1 ascending global offsets */
@@ -235,7 +245,7 @@ typedef struct gd_apply_args {
   float alpha;
   const uint64_t* layer_off;   /* HOST, n_layers + 1; packed modes only */
   uint32_t n_layers;
-  uint32_t reserved;
+  uint32_t flags;              /* GD_APPLY_* (0: pushes applied one after another) */
   void* workspace;             /* device, 256-byte aligned, >= gd_apply_workspace_bytes() */
   size_t workspace_bytes;
   const uint32_t* layer_cols;  /* HOST, n_layers column counts; GD_VALUES_COLUMN_MEANS only, else may be NULL */

@@ -34,6 +34,7 @@ GD_FLAG_QUANT_ERROR_FEEDBACK = 4
 GD_FLAG_NO_EARLY_ZERO = 8
 GD_FLAG_PLAIN_RADIX = 16
 GD_ERR_OVERFLOW = -7
+GD_APPLY_ATOMIC = 1
 
 EXPORTS = [
     "gd_status_string", "gd_kept_count", "gd_total_kept", "gd_workspace_bytes", "gd_apply_workspace_bytes",
@@ -72,7 +73,7 @@ class _ApplyArgs(C.Structure):
         ("params", C.POINTER(C.c_void_p)), ("shard_off", C.POINTER(C.c_uint64)),
         ("n_shards", C.c_uint32), ("n_pushes", C.c_uint32), ("pushes", C.POINTER(_Push)),
         ("value_mode", C.c_int32), ("alpha", C.c_float),
-        ("layer_off", C.POINTER(C.c_uint64)), ("n_layers", C.c_uint32), ("reserved", C.c_uint32),
+        ("layer_off", C.POINTER(C.c_uint64)), ("n_layers", C.c_uint32), ("flags", C.c_uint32),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("layer_cols", C.POINTER(C.c_uint32)),
     ]
 
@@ -223,7 +224,7 @@ class ApplyCall:
     """The marshalled argument block of one gd_decompress_apply call."""
 
     def __init__(self, params: Sequence[torch.Tensor], shard_off, pushes, value_mode, alpha, workspace,
-                 layer_off=None, layer_cols=None):
+                 layer_off=None, layer_cols=None, flags=0):
         self._keep = (list(params), pushes, workspace)
         n_shards = len(shard_off) - 1
         self._params = (C.c_void_p * n_shards)(*[p.data_ptr() if p.numel() else None for p in params])
@@ -238,7 +239,7 @@ class ApplyCall:
         a = _ApplyArgs()
         a.params, a.shard_off, a.n_shards = self._params, self._shard_off, n_shards
         a.n_pushes, a.pushes = len(pushes), self._pushes
-        a.value_mode, a.alpha = value_mode, float(alpha)
+        a.value_mode, a.alpha, a.flags = value_mode, float(alpha), int(flags)
         if self._layer_off is not None:
             a.layer_off, a.n_layers = self._layer_off, len(layer_off) - 1
         a.workspace = _ptr(workspace)

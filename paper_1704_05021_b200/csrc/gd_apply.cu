@@ -94,6 +94,56 @@ __global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__
   }
 }
 
+// Up to kPushSet pushes applied by ONE launch (blockIdx.y = push).  Entries of different pushes may hit the same
+// parameter, so every update is an atomic read-modify-write: a compare-and-swap loop around the same fused
+// multiply-add as above (atom.global.add.f32 would be shorter but flushes subnormals, and it would round alpha * x
+// before the add).  The order in which colliding pushes land is not defined; each lands exactly once.
+constexpr uint32_t kPushSet = 32;
+struct PushSet {
+  const uint32_t* idx[kPushSet];
+  const float* val[kPushSet];
+  const uint32_t* cnt_off[kPushSet];
+  const float* means[kPushSet];
+};
+
+template <bool INLINE>
+__global__ void __launch_bounds__(kThreads) apply_atomic_kernel(const __grid_constant__ ApplyDev A,
+                                                                const __grid_constant__ ApplyInline I,
+                                                                const __grid_constant__ PushSet P) {
+  float* const* params = INLINE ? I.params : A.params;
+  const uint64_t* shard_off = INLINE ? I.shard_off : A.shard_off;
+  const uint64_t* layer_off = INLINE ? I.layer_off : A.layer_off;
+  const uint64_t* pair_off = INLINE ? I.pair_off : A.pair_off;
+  const uint32_t* layer_cols = INLINE ? I.layer_cols : A.layer_cols;
+  const uint32_t w = blockIdx.y;
+  const uint32_t* idx = P.idx[w];
+  const float* val = P.val[w];
+  const float* means = P.means[w];
+  const uint64_t begin = P.cnt_off[w][0], end = P.cnt_off[w][A.n_shards];
+  const uint64_t lo_all = shard_off[0], hi_all = shard_off[A.n_shards];
+  const uint64_t stride = (uint64_t)gridDim.x * kThreads;
+  for (uint64_t p = begin + (uint64_t)blockIdx.x * kThreads + threadIdx.x; p < end; p += stride) {
+    const uint32_t word = __ldcs(idx + p);
+    uint64_t pos = word;
+    float x;
+    if (A.value_mode != GD_VALUES_FP32) {
+      pos = word & kAbsMask;
+      const uint64_t pr = pair_of(layer_off, pair_off, layer_cols, A.n_layers, pos);
+      x = __ldg(means + 2 * pr + (word >> 31));
+    } else {
+      x = __ldcs(val + p);
+    }
+    if (pos < lo_all || pos >= hi_all) continue;
+    const uint32_t j = range_of(shard_off, A.n_shards, pos);
+    unsigned int* dst = reinterpret_cast<unsigned int*>(params[j] + (pos - shard_off[j]));
+    unsigned int old = __ldcg(dst), assumed;
+    do {   // (a retry means that another push's entry landed in between: at most one per colliding push)
+      assumed = old;
+      old = atomicCAS(dst, assumed, __float_as_uint(__fmaf_rn(A.alpha, x, __uint_as_float(assumed))));
+    } while (old != assumed);
+  }
+}
+
 }  // namespace
 
 }  // namespace gd
@@ -119,6 +169,7 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
   if (a->n_pushes && !a->pushes) return GD_ERR_INVALID_ARG;
   if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_COLUMN_MEANS) return GD_ERR_INVALID_ARG;
   if (a->value_mode == GD_VALUES_COLUMN_MEANS && !a->layer_cols) return GD_ERR_INVALID_ARG;
+  if (a->flags & ~(uint32_t)GD_APPLY_ATOMIC) return GD_ERR_INVALID_ARG;
   const bool two_means = a->value_mode != GD_VALUES_FP32;   // the packed modes decode through the means table
   if (two_means && (!a->layer_off || a->n_layers == 0)) return GD_ERR_INVALID_ARG;
   for (uint32_t j = 0; j < a->n_shards; ++j) {
@@ -191,6 +242,27 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
     A.value_mode = a->value_mode;
     A.alpha = a->alpha;
     const unsigned grid = (unsigned)sm_count() * 8u;
+    if (a->flags & GD_APPLY_ATOMIC) {
+      // all pushes in one launch (sets of kPushSet, should there be more), colliding entries combined atomically
+      for (uint32_t w0 = 0; w0 < a->n_pushes; w0 += kPushSet) {
+        const uint32_t cnt = a->n_pushes - w0 < kPushSet ? a->n_pushes - w0 : kPushSet;
+        PushSet P;
+        std::memset(&P, 0, sizeof(P));
+        for (uint32_t w = 0; w < cnt; ++w) {
+          const gd_push& p = a->pushes[w0 + w];
+          P.idx[w] = p.idx; P.val[w] = p.val; P.cnt_off[w] = p.shard_cnt_off; P.means[w] = p.means;
+        }
+        const unsigned per_push = grid / cnt > 0 ? (grid + cnt - 1) / cnt : 1u;
+        ProfileScope prof(stream, PT_APPLY);
+        if (use_inline)
+          apply_atomic_kernel<true><<<dim3(per_push, cnt), kThreads, 0, stream>>>(A, I, P);
+        else
+          apply_atomic_kernel<false><<<dim3(per_push, cnt), kThreads, 0, stream>>>(A, I, P);
+        if (cudaPeekAtLastError() != cudaSuccess) return GD_ERR_CUDA;
+        note_launches(1);
+      }
+      return GD_OK;
+    }
     for (uint32_t w = 0; w < a->n_pushes; ++w) {
       const gd_push& p = a->pushes[w];
       A.idx = p.idx;

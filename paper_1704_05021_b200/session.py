@@ -84,11 +84,11 @@ class GradDropSession:
             p["val"] = self.out_val
         return p
 
-    def apply_call(self, params: List[torch.Tensor], alpha: float = 1.0, pushes=None) -> B.ApplyCall:
+    def apply_call(self, params: List[torch.Tensor], alpha: float = 1.0, pushes=None, flags: int = 0) -> B.ApplyCall:
         pushes = [self.push()] if pushes is None else pushes
         lo = self.layer_off if self.value_mode != B.GD_VALUES_FP32 else None
         return B.ApplyCall(params, self.shard_off, pushes, self.value_mode, alpha, self.apply_workspace, lo,
-                           self.layer_cols)
+                           self.layer_cols, flags)
 
     def apply(self, params: List[torch.Tensor], alpha: float = 1.0, stream=None) -> None:
         if self._apply_call is None or self._apply_params is not params:

@@ -556,11 +556,13 @@ def test_more_kept_than_nonzero(cuda_device):
 
 
 # ---------------------------------------------------------------- several workers pushing into one server shard
+@pytest.mark.parametrize("apply_flags", [0, B.GD_APPLY_ATOMIC], ids=["ordered", "atomic"])
 @pytest.mark.parametrize("value_mode", [B.GD_VALUES_FP32, B.GD_VALUES_TWO_MEANS])
-def test_three_workers_push_into_each_server(cuda_device, value_mode):
+def test_three_workers_push_into_each_server(cuda_device, value_mode, apply_flags):
     """Section 3: every server owns 1/N of the parameters and receives one piece from every worker.  Three
     workers compress their own gradients; each of the 4 servers applies the three pieces of its shard in
-    one call (pushes collide on many indices and are applied in order)."""
+    one call (pushes collide on many indices), either one after another or - GD_APPLY_ATOMIC - in one launch
+    with atomic updates; the fp64 reference admits any order."""
     rng = np.random.default_rng(17)
     sizes = [30_000, 11, 50_001]
     w = W.small_layered(3, sizes, 950_000, B.GD_SCOPE_PER_LAYER, value_mode, 4)
@@ -589,8 +591,10 @@ def test_three_workers_push_into_each_server(cuda_device, value_mode):
                 p["means"] = sess.out_means
             pushes.append(p)
         call = B.ApplyCall([params[lo:hi]], [lo, hi], pushes, value_mode, 0.25, aws,
-                           w.layer_off if value_mode != B.GD_VALUES_FP32 else None)
+                           w.layer_off if value_mode != B.GD_VALUES_FP32 else None, flags=apply_flags)
+        before = B.gd_launch_count()
         B.gd_decompress_apply(call)
+        assert B.gd_launch_count() - before == (1 if apply_flags else 3)
     torch.cuda.synchronize()
     got = params.cpu().numpy().astype(np.float64)
     collisions = 0
@@ -602,6 +606,44 @@ def test_three_workers_push_into_each_server(cuda_device, value_mode):
     for exp in expected:
         hits[(exp["idx"] & np.uint32(0x7FFFFFFF)).astype(np.int64)] += 1
     assert (hits >= 2).sum() > 100                                 # the pushes really collide
+
+
+def test_atomic_apply_of_many_colliding_pushes_keeps_subnormals(cuda_device):
+    """Forty workers (more than one launch's worth of pushes) push the same positions into one server at once.
+    With values that are small multiples of the smallest subnormal every partial sum is exact in fp32, so the
+    atomic apply must give the exact total whatever the order - which an add that flushed subnormals would not -
+    and a second set of ordinary values stays within the fp64 reference's tolerance."""
+    n, workers = 50_000, 40
+    w = W.small_layered(1, [n], 900_000, B.GD_SCOPE_GLOBAL, B.GD_VALUES_FP32, 1)
+    tiny = np.float32(1.401298464324817e-45)                      # 2^-149
+    rng = np.random.default_rng(5)
+    for scale, exact in ((tiny, True), (np.float32(1e-3), False)):
+        sessions, expected = [], []
+        for wk in range(workers):
+            mult = rng.integers(1, 8, n).astype(np.float32)
+            sign = rng.choice(np.array([-1.0, 1.0], np.float32), n)
+            g = (mult * sign * scale).astype(np.float32) if exact else (rng.laplace(0, 1, n).astype(np.float32) * scale)
+            g[rng.random(n) < 0.5] *= np.float32(0.125) if not exact else np.float32(1.0)
+            g[::7] = np.float32(64.0) * scale * sign[::7]         # every worker keeps these: they all collide
+            sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
+            sess.compress(torch.from_numpy(g).to(cuda_device))
+            assert sess.status() == B.GD_OK
+            expected.append(orc.compress(g, orc.residual_reset(n), w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode))
+            sessions.append(sess)
+        params = torch.zeros(n, device=cuda_device)
+        aws = torch.empty(B.gd_apply_workspace_bytes(1, 1), dtype=torch.uint8, device=cuda_device)
+        call = B.ApplyCall([params], [0, n], [s_.push() for s_ in sessions], B.GD_VALUES_FP32, 1.0, aws, flags=B.GD_APPLY_ATOMIC)
+        before = B.gd_launch_count()
+        B.gd_decompress_apply(call)
+        torch.cuda.synchronize()
+        assert B.gd_launch_count() - before == 2                   # forty pushes: a set of 32 and a set of 8
+        ref, bound = orc.apply_pushes(np.zeros(n, np.float32), 0, expected)
+        got = params.cpu().numpy()
+        if exact:
+            assert np.array_equal(got.astype(np.float64), ref)     # sums of small multiples of 2^-149: no rounding anywhere
+            assert np.count_nonzero(got) > 1000
+        else:
+            assert np.all(np.abs(got.astype(np.float64) - ref) <= REL_TOL * bound + 1e-45)
 
 
 # ---------------------------------------------------------------- parameter pulls as dropped deltas
