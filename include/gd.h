@@ -12,6 +12,12 @@
  *   - Unless stated otherwise a call only enqueues work on the stream and returns; it never
  *     synchronises and never allocates or frees device memory.  All device buffers, the
  *     residual and the workspace included, are owned by the caller.
+ *   - gd_compress keeps the plan it derives from a layout (offsets, drop ratio, scope mode) in a small
+ *     per-process cache, so that a training loop pays for it once.  For layouts whose tables do not fit
+ *     a kernel argument (roughly more than thirty tensors) the cached plan holds a page-locked HOST
+ *     image of the tables, allocated by the first call with that layout (make that call outside any
+ *     stream capture); without it, and always in gd_compress_static, such tables travel in pieces
+ *     as arguments of a few extra small launches.  Host memory is never copied from pageable buffers.
  *   - Every function returns a gd_status_t.  Argument errors are detected on the host before
  *     anything is enqueued.  Conditions detected on the device (a bounded wait that ran out,
  *     an inconsistent count) are written to a status word in the workspace and are returned

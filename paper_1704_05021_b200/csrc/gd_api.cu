@@ -3,303 +3,19 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
+#include <memory>
+#include <mutex>
 #include <new>
 #include <vector>
 
 #include <nvtx3/nvToolsExt.h>
 
 #include "gd_internal.cuh"
+#include "gd_plan.hpp"
 
 namespace gd {
 
 namespace {
-
-constexpr size_t kAlign = 256;
-inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
-
-// Sample size per scope: the sample is sized for a number of expected samples above the threshold
-// ("hits") that grows with the scope's k.  A sample costs scattered reads in proportion to its size; a
-// small one costs a wider safety margin, i.e. extra candidates in proportion to k / sqrt(hits).  The sum
-// is smallest near hits ~ k^(2/3) (the measured costs per sample and per candidate are about equal;
-// factors of 0.12, 0.25 and 0.5 were timed on layered models of 12 to 387 tensors), so:
-// hits = kHitsFactor * k^(2/3) within [kHitsMin, kHitsMax], and never more than kSampleMax samples or a
-// sixteenth of the scope.
-constexpr double kHitsFactor = 0.25, kHitsMin = 32.0, kHitsMax = 256.0, kSampleMax = 262144.0;
-constexpr uint64_t kSampleAllMax = 8192;         // scopes up to this length are sampled completely
-constexpr uint64_t kClusterMaxStride = 1024;      // strata up to this many elements wide are sampled in groups of 8
-constexpr uint64_t kAutoDenseMax = 3ull << 19;   // vectors up to this length skip the prediction (measured: dense 69 us
-                                                 // against 87 us at 2^20, 93 against 89 at 2^21)
-
-inline uint64_t kept_count(uint64_t n, uint32_t drop_ppm) {
-  return n - (n * (uint64_t)drop_ppm) / 1000000ull;   // n <= 2^32, drop_ppm <= 1e6: no overflow
-}
-
-// How one scope is sampled for the prediction and how many candidate slots it gets.  A scope of
-// ns elements keeping k: m stratified samples are read and the predicted lower bound is the rank-th
-// largest sample key.  rank is chosen so that, for independent samples, the number of entries at or
-// above the prediction is at least k with a margin of six standard deviations plus 12.5 %.  Small
-// scopes are sampled completely, which makes the prediction the exact threshold.  None of this
-// affects results: a scope whose prediction fails is selected densely.
-void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint64_t* cap, uint32_t* cluster) {
-  *cluster = 1;
-  if (k == 0 || ns == 0) { *m = 0; *rank = 0; *cap = 0; return; }
-  double hits = kHitsFactor * std::cbrt((double)k * (double)k);
-  if (hits < kHitsMin) hits = kHitsMin;
-  if (hits > kHitsMax) hits = kHitsMax;
-  double target = hits * (double)ns / (double)k;
-  if (target > kSampleMax) target = kSampleMax;
-  if (target > (double)ns / 16.0) target = (double)ns / 16.0;
-  uint64_t mt = (uint64_t)target;
-  if (ns <= kSampleAllMax || mt < 64) {
-    *m = ns;
-    *rank = k;
-    uint64_t c = 3 * k + 1024;
-    *cap = c < ns ? c : ns;
-    return;
-  }
-  // The sample is bound by the rate of scattered DRAM reads (about 22 G/s, two per sample).  Narrow strata (a
-  // sample every few sectors): whole groups of 8 consecutive elements are sampled, an eighth of the reads.  Wide
-  // strata: pairs of neighbours, half the reads; larger groups there would leave too few distinct places (rows
-  // of a matrix) in the sample - a pair at most doubles the variance the rank's margin of six sigma is sized for.
-  if (ns / mt <= kClusterMaxStride) {
-    mt &= ~7ull;
-    *cluster = 8;
-  } else {
-    mt &= ~1ull;
-    *cluster = 2;
-  }
-  *m = mt;
-  const double x = (double)k * (double)mt / (double)ns;
-  const double y = 3.0 + std::sqrt(9.0 + 1.125 * x + 1.0);
-  uint64_t r = (uint64_t)std::ceil(y * y);
-  if (r > mt) r = mt;
-  if (r < 1) r = 1;
-  *rank = r;
-  uint64_t c = 3 * k + 128 * (ns / mt) + 1024;
-  *cap = c < ns ? c : ns;
-}
-
-// Sampled-threshold mode (Section 4): sample size and output capacity of one scope.
-inline uint64_t sampled_m(uint64_t ns) {
-  if (ns <= 4096) return ns;            // sampled completely, element by element
-  uint64_t m = (ns + 999) / 1000;
-  if (m < 4096) m = 4096;
-  return m + (m & 1);                   // longer scopes: pairs of neighbours
-}
-inline uint64_t sampled_cap(uint64_t ns, uint64_t k) {
-  const uint64_t c = 4 * k + 8192;
-  return c < ns ? c : ns;
-}
-
-struct Plan {
-  std::vector<ScopeDesc> scopes;
-  std::vector<uint32_t> tile0[L_COUNT];
-  std::vector<uint64_t> samp_off;
-  uint32_t tiles[L_COUNT] = {0, 0, 0, 0, 0};
-  uint64_t samp_total = 0, cand_total = 0, k_total = 0;
-  uint32_t n_scopes = 0;
-  bool predict = true;
-  bool local_predict = false;   // the prediction shares a launch with the start of the call (gd_predict.cu)
-  bool dense_bound = false;     // no sample: the lower bounds come from a histogram pass over the dense vector (gd_dense.cu)
-  uint32_t emit_chunk_tiles = 1, dense_sel_tile = kDenseSelTileMax, dense_chunk_tiles = kDenseChunkTilesMax;
-  uint32_t samp_tile = kTile;
-  // workspace layout (byte offsets)
-  size_t off_ctl = 0, off_state = 0, off_hist = 0, off_sums = 0, off_cnts = 0, off_desc_emit = 0,
-         off_desc_cand = 0, off_desc_dcomp = 0, zero_bytes = 0;
-  size_t off_tables = 0, tables_bytes = 0;
-  size_t t_scopes = 0, t_tile0[L_COUNT] = {0, 0, 0, 0, 0}, t_samp_off = 0, t_layer_off = 0, t_shard_off = 0,
-         t_pair_off = 0, t_layer_cols = 0;
-  std::vector<uint64_t> pair_off;
-  std::vector<uint32_t> layer_cols;
-  uint64_t n_pairs = 0;
-  size_t off_agg = 0, off_flags = 0, off_samp = 0, off_cand_idx = 0, off_cand_val = 0, total_bytes = 0;
-};
-
-int check_offsets(const uint64_t* off, uint32_t count, uint64_t* n_out) {
-  if (!off || count == 0) return GD_ERR_INVALID_ARG;
-  if (off[0] != 0) return GD_ERR_INVALID_ARG;
-  for (uint32_t i = 0; i < count; ++i)
-    if (off[i + 1] < off[i]) return GD_ERR_INVALID_ARG;
-  *n_out = off[count];
-  return GD_OK;
-}
-
-// layer_cols == NULL: one (mu+, mu-) pair per layer.
-int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* layer_cols, uint32_t n_shards, int scope_mode,
-              uint32_t drop_ppm, uint32_t flags, Plan* P) {
-  uint64_t n = 0;
-  int rc = check_offsets(layer_off, n_layers, &n);
-  if (rc != GD_OK) return rc;
-  if (n_shards == 0 || drop_ppm > 1000000u) return GD_ERR_INVALID_ARG;
-  if (scope_mode != GD_SCOPE_GLOBAL && scope_mode != GD_SCOPE_PER_LAYER) return GD_ERR_INVALID_ARG;
-  if (n > (1ull << 32)) return GD_ERR_TOO_LARGE;
-  const bool sampled = (flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
-  // Short vectors are selected densely right away: below about 2^21 elements the three dense passes
-  // run out of L2 and cost less than sampling, predicting and selecting among candidates.
-  const bool predict = !(flags & GD_FLAG_NO_PREDICTION) && (sampled || n > kAutoDenseMax);
-  P->predict = predict;
-  // Without a sample, long vectors still go through the candidate lists: one histogram pass over the dense vector
-  // gives every scope an exact lower bound of its threshold (gd_dense.cu).  Short vectors, whose passes run out
-  // of L2, and calls with more scopes than the kernels over the lists keep in shared memory take the plain dense
-  // selection and compaction.
-  const uint32_t ns_planned = scope_mode == GD_SCOPE_GLOBAL ? 1u : n_layers;
-  P->dense_bound = !predict && !sampled && n > kAutoDenseMax && ns_planned <= kSmemScopes;
-  P->pair_off.assign((size_t)n_layers + 1, 0);
-  P->layer_cols.assign(n_layers, 1);
-  for (uint32_t l = 0; l < n_layers; ++l) {
-    const uint64_t size = layer_off[l + 1] - layer_off[l];
-    uint32_t cols = layer_cols ? layer_cols[l] : 1u;
-    if (cols == 0 || (size % cols) != 0) return GD_ERR_INVALID_ARG;   // a layer is rows x cols, row-major
-    P->layer_cols[l] = cols;
-    P->pair_off[l + 1] = P->pair_off[l] + cols;
-  }
-  P->n_pairs = P->pair_off[n_layers];
-  // The fused pass gives each CTA a chunk of 1, 2, 4 or 8 tiles: as large as still leaves a wave and a
-  // half of CTAs (4 per SM on 148 SMs) for the whole vector.  (Measured on 2^21 .. 2^26 elements: four
-  // waves, the first rule, cost 20-30 % more time at 2^23 .. 2^25; one wave loses to the tail.)
-  const uint64_t dense_tiles = (n + kTile - 1) / kTile;
-  uint32_t chunk_tiles = 8;
-  while (chunk_tiles > 1 && dense_tiles < (uint64_t)chunk_tiles * 888u) chunk_tiles >>= 1;
-  P->emit_chunk_tiles = chunk_tiles;
-  const uint64_t CH = (uint64_t)chunk_tiles * kTile;
-  // The dense kernels (used when a prediction fails) take large tiles on long vectors, where the
-  // chain of look-backs and the flushes of histograms must stay rare, and small ones on short
-  // vectors, which otherwise would not fill the GPU.
-  uint32_t sel_tile = kDenseSelTileMax, dchunk = kDenseChunkTilesMax;
-  while (sel_tile > kTile && n / sel_tile < 592u) sel_tile >>= 1;
-  // (chunks of the dense compaction: about 48 per resident CTA, so that scopes whose survivors crowd at one
-  // end - a sparse layer whose kept zeros are its first ones - still spread over the GPU)
-  while (dchunk > 1 && n / ((uint64_t)dchunk * kTile) < 7104u) dchunk >>= 1;
-  P->dense_sel_tile = sel_tile;
-  P->dense_chunk_tiles = dchunk;
-  const uint32_t ns_count = scope_mode == GD_SCOPE_GLOBAL ? 1u : n_layers;
-  P->n_scopes = ns_count;
-  P->scopes.resize(ns_count);
-  for (int l = 0; l < L_COUNT; ++l) P->tile0[l].assign(ns_count + 1, 0);
-  P->samp_off.assign(ns_count + 1, 0);
-  uint64_t tiles[L_COUNT] = {0, 0, 0, 0, 0};
-  uint64_t out_base = 0, cand_base = 0, samp_base = 0;
-  for (uint32_t s = 0; s < ns_count; ++s) {
-    ScopeDesc& d = P->scopes[s];
-    d.lo = scope_mode == GD_SCOPE_GLOBAL ? 0 : layer_off[s];
-    d.hi = scope_mode == GD_SCOPE_GLOBAL ? n : layer_off[s + 1];
-    const uint64_t ns = d.hi - d.lo;
-    d.k = kept_count(ns, drop_ppm);
-    d.out_base = out_base;
-    out_base += d.k;
-    uint64_t m = 0, rank = 0, cap = 0;
-    uint32_t cluster = 1;
-    if (sampled) {
-      m = sampled_m(ns);
-      cluster = ns <= 4096 ? 1u : 2u;
-      rank = kept_count(m, drop_ppm);
-      cap = sampled_cap(ns, d.k);
-    } else if (predict) {
-      plan_prediction(ns, d.k, &m, &rank, &cap, &cluster);
-    } else if (P->dense_bound) {
-      // the candidates are the keys above the bin of the k-th largest key (fewer than k) and that bin itself
-      const uint64_t c = 3 * d.k + 4096;
-      cap = c < ns ? c : ns;
-    }
-    d.cand_base = cand_base;
-    d.cand_cap = cap;
-    cand_base += (cap + 3) / 4 * 4;
-    d.samp_base = samp_base;
-    d.samp_m = m;
-    d.samp_rank = rank;
-    d.samp_cluster = cluster;
-    if (cluster > 1) {   // strata of groups of 8 (or 2) elements, from the first multiple of that at or after lo
-      const uint64_t first = (d.lo + cluster - 1) & ~(uint64_t)(cluster - 1);
-      const uint64_t groups = (d.hi - first) / cluster, strata = m / cluster;
-      d.samp_w = groups / strata;
-      d.samp_rem = (uint32_t)(groups % strata);
-    } else {
-      d.samp_w = m ? ns / m : 0;
-      d.samp_rem = m ? (uint32_t)(ns % m) : 0;
-    }
-    samp_base += m;
-    for (int l = 0; l < L_COUNT; ++l) P->tile0[l][s] = (uint32_t)tiles[l];
-    P->samp_off[s] = d.samp_base;
-    if (ns) {
-      tiles[L_EMIT] += (d.hi + CH - 1) / CH - d.lo / CH;
-      tiles[L_DSEL] += (ns + sel_tile - 1) / sel_tile;
-      tiles[L_DCOMP] += (ns + (uint64_t)dchunk * kTile - 1) / ((uint64_t)dchunk * kTile);
-    }
-    tiles[L_SAMP] += (m + kTile - 1) / kTile;
-    tiles[L_CAND] += (cap + kTile - 1) / kTile;
-  }
-  for (int l = 0; l < L_COUNT; ++l) {
-    if (tiles[l] > 0x7FFFFFFFull) return GD_ERR_TOO_LARGE;
-    P->tile0[l][ns_count] = (uint32_t)tiles[l];
-    P->tiles[l] = (uint32_t)tiles[l];
-  }
-  // The sample is gathered with scattered reads, of which one SM keeps only so many in flight: a short
-  // sample is cut into tiles of 1024 so that its gather spreads over all SMs.
-  P->samp_tile = kTile;
-  while (P->samp_tile > 1024u && samp_base / P->samp_tile < 2u * 148u) P->samp_tile >>= 2;
-  if (P->samp_tile != kTile) {
-    uint64_t t = 0;
-    for (uint32_t s = 0; s < ns_count; ++s) {
-      P->tile0[L_SAMP][s] = (uint32_t)t;
-      t += (P->scopes[s].samp_m + P->samp_tile - 1) / P->samp_tile;
-    }
-    P->tile0[L_SAMP][ns_count] = (uint32_t)t;
-    P->tiles[L_SAMP] = (uint32_t)t;
-  }
-  P->samp_off[ns_count] = samp_base;
-  P->samp_total = samp_base;
-  P->cand_total = cand_base;
-  P->k_total = out_base;
-
-  size_t off = 0;
-  P->off_ctl = off;          off = align_up(off + sizeof(Ctl));
-  P->off_state = off;        off = align_up(off + sizeof(ScopeState) * ns_count);
-  P->off_hist = off;         off = align_up(off + sizeof(unsigned long long) * kHistBinsPerScope * (size_t)ns_count);
-  P->off_sums = off;         off = align_up(off + sizeof(double) * 2 * (size_t)P->n_pairs);
-  P->off_cnts = off;         off = align_up(off + sizeof(unsigned long long) * 2 * (size_t)P->n_pairs);
-  P->off_desc_emit = off;    off = align_up(off + 16 * (size_t)P->tiles[L_EMIT]);
-  P->off_desc_cand = off;    off = align_up(off + 16 * (size_t)P->tiles[L_CAND]);
-  P->off_desc_dcomp = off;   off = align_up(off + 16 * (size_t)P->tiles[L_DCOMP]);
-  P->zero_bytes = off;
-  P->off_tables = off;
-  size_t t = 0;
-  auto sub = [](size_t x) { return (x + 15) / 16 * 16; };   // tables are packed at 16-byte steps
-  P->t_scopes = t;           t = sub(t + sizeof(ScopeDesc) * ns_count);
-  for (int l = 0; l < L_COUNT; ++l) { P->t_tile0[l] = t; t = sub(t + sizeof(uint32_t) * (ns_count + 1)); }
-  P->t_samp_off = t;         t = sub(t + sizeof(uint64_t) * (ns_count + 1));
-  P->t_layer_off = t;        t = sub(t + sizeof(uint64_t) * ((size_t)n_layers + 1));
-  P->t_shard_off = t;        t = sub(t + sizeof(uint64_t) * ((size_t)n_shards + 1));
-  P->t_pair_off = t;         t = sub(t + sizeof(uint64_t) * ((size_t)n_layers + 1));
-  P->t_layer_cols = t;       t = sub(t + sizeof(uint32_t) * (size_t)n_layers);
-  t = align_up(t);
-  P->tables_bytes = t;
-  off += t;
-  // Samples of at most local_sample_max() values per scope are gathered in tiles of 256 by the kernel that also starts
-  // the call; it marks every finished tile in an array of flags.
-  P->local_predict = predict && !sampled && P->tables_bytes <= kSetupBlobBytes;
-  for (uint32_t s = 0; P->local_predict && s < ns_count; ++s)
-    if (P->scopes[s].samp_m > local_sample_max()) P->local_predict = false;
-  if (P->local_predict) {
-    // tiles of 256 samples spread a short sample over many SMs; larger tiles keep all CTAs resident at once
-    for (P->samp_tile = 256;; P->samp_tile *= 2) {
-      uint64_t tt = 0;
-      for (uint32_t s = 0; s < ns_count; ++s) {
-        P->tile0[L_SAMP][s] = (uint32_t)tt;
-        tt += (P->scopes[s].samp_m + P->samp_tile - 1) / P->samp_tile;
-      }
-      P->tile0[L_SAMP][ns_count] = (uint32_t)tt;
-      P->tiles[L_SAMP] = (uint32_t)tt;
-      if (tt <= 2u * 148u || P->samp_tile == 1024u) break;
-    }
-  }
-  P->off_flags = off;        off = align_up(off + sizeof(uint32_t) * (size_t)P->tiles[L_SAMP]);   // not cleared
-  P->off_agg = off;          off = align_up(off + 32 * (size_t)select_compact_max_grid());   // per-CTA records, not cleared
-  P->off_samp = off;         off = align_up(off + sizeof(float) * P->samp_total);
-  P->off_cand_idx = off;     off = align_up(off + sizeof(uint32_t) * P->cand_total);
-  P->off_cand_val = off;     off = align_up(off + sizeof(float) * P->cand_total);
-  P->total_bytes = off;
-  return GD_OK;
-}
 
 // Start of a call in one launch: clears the control region of the workspace and writes the small
 // host-built tables, which travel as a kernel argument, behind it.
@@ -328,39 +44,136 @@ uint32_t g_ev_created = 0, g_ev_used = 0;
 bool g_pair_open = false;
 std::atomic<uint64_t> g_launches{0};   // calls may come from several host threads
 
+// Plans are pure functions of the layout arguments and are kept: a training loop calls with the same layout every
+// step, and should not pay for vectors, square roots and table images again.  Entries are immutable once stored and
+// never dropped (a full cache just stops caching), so a pointer to one stays valid.
+struct PlanEntry {
+  std::vector<uint64_t> layer_off, shard_off;
+  std::vector<uint32_t> layer_cols;
+  int scope_mode = 0;
+  uint32_t drop_ppm = 0, plan_flags = 0;
+  Plan P;
+  std::vector<unsigned char> blob;      // host image of the tables
+  unsigned char* pinned = nullptr;      // the same in page-locked memory, for tables too large for a kernel argument
+};
+constexpr size_t kPlanCacheEntries = 64;
+std::mutex g_plan_mutex;
+std::vector<std::unique_ptr<PlanEntry>> g_plans;
+
+bool same_layout(const PlanEntry& e, const gd_compress_args* a, const uint32_t* cols, uint32_t plan_flags) {
+  if (e.scope_mode != a->scope_mode || e.drop_ppm != a->drop_ppm || e.plan_flags != plan_flags) return false;
+  if (e.layer_off.size() != (size_t)a->n_layers + 1 || e.shard_off.size() != (size_t)a->n_shards + 1) return false;
+  if (e.layer_cols.empty() != (cols == nullptr)) return false;
+  if (std::memcmp(e.layer_off.data(), a->layer_off, sizeof(uint64_t) * e.layer_off.size()) != 0) return false;
+  if (std::memcmp(e.shard_off.data(), a->shard_off, sizeof(uint64_t) * e.shard_off.size()) != 0) return false;
+  return !cols || std::memcmp(e.layer_cols.data(), cols, sizeof(uint32_t) * e.layer_cols.size()) == 0;
+}
+
+// The plan and table image for these arguments: from the cache, or built now (and stored if there is room).
+// *owned receives the entry when it was not stored.  may_allocate: whether page-locked memory may be asked for.
+int plan_for(const gd_compress_args* a, bool may_allocate, const PlanEntry** out, std::unique_ptr<PlanEntry>* owned) {
+  if (!a->layer_off || !a->shard_off || a->n_layers == 0 || a->n_shards == 0) return GD_ERR_INVALID_ARG;
+  const uint32_t* cols = a->value_mode == GD_VALUES_COLUMN_MEANS ? a->layer_cols : nullptr;
+  const uint32_t plan_flags = a->flags & (GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD);
+  {
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    for (const auto& e : g_plans)
+      if (same_layout(*e, a, cols, plan_flags)) { *out = e.get(); return GD_OK; }
+  }
+  std::unique_ptr<PlanEntry> e(new PlanEntry);
+  int rc = make_plan(a->layer_off, a->n_layers, cols, a->n_shards, a->scope_mode, a->drop_ppm, a->flags, &e->P);
+  if (rc != GD_OK) return rc;
+  uint64_t n_sh = 0;
+  rc = check_offsets(a->shard_off, a->n_shards, &n_sh);
+  if (rc != GD_OK) return rc;
+  if (n_sh != a->layer_off[a->n_layers]) return GD_ERR_INVALID_ARG;
+  e->layer_off.assign(a->layer_off, a->layer_off + a->n_layers + 1);
+  e->shard_off.assign(a->shard_off, a->shard_off + a->n_shards + 1);
+  if (cols) e->layer_cols.assign(cols, cols + a->n_layers);
+  e->scope_mode = a->scope_mode;
+  e->drop_ppm = a->drop_ppm;
+  e->plan_flags = plan_flags;
+  const Plan& P = e->P;
+  e->blob.assign(P.tables_bytes, 0);
+  unsigned char* b = e->blob.data();
+  std::memcpy(b + P.t_scopes, P.scopes.data(), sizeof(ScopeDesc) * P.n_scopes);
+  for (int l = 0; l < L_COUNT; ++l) std::memcpy(b + P.t_tile0[l], P.tile0[l].data(), sizeof(uint32_t) * (P.n_scopes + 1));
+  std::memcpy(b + P.t_samp_off, P.samp_off.data(), sizeof(uint64_t) * (P.n_scopes + 1));
+  std::memcpy(b + P.t_layer_off, a->layer_off, sizeof(uint64_t) * ((size_t)a->n_layers + 1));
+  std::memcpy(b + P.t_shard_off, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
+  std::memcpy(b + P.t_pair_off, P.pair_off.data(), sizeof(uint64_t) * ((size_t)a->n_layers + 1));
+  std::memcpy(b + P.t_layer_cols, P.layer_cols.data(), sizeof(uint32_t) * (size_t)a->n_layers);
+  std::lock_guard<std::mutex> lock(g_plan_mutex);
+  for (const auto& other : g_plans)                        // (another thread may have stored the same layout meanwhile)
+    if (same_layout(*other, a, cols, plan_flags)) { *out = other.get(); return GD_OK; }
+  if (g_plans.size() < kPlanCacheEntries) {
+    if (may_allocate && P.tables_bytes > kSetupBlobBytes) {
+      void* p = nullptr;
+      if (cudaHostAlloc(&p, P.tables_bytes, cudaHostAllocDefault) == cudaSuccess && p) {
+        std::memcpy(p, b, P.tables_bytes);
+        e->pinned = (unsigned char*)p;
+      } else {
+        (void)cudaGetLastError();                          // no page-locked image: the tables go up in pieces
+      }
+    }
+    *out = e.get();
+    g_plans.push_back(std::move(e));
+  } else {
+    *out = e.get();
+    *owned = std::move(e);
+  }
+  return GD_OK;
+}
+
 }  // namespace
 
 void note_launches(uint32_t count) { g_launches.fetch_add(count, std::memory_order_relaxed); }
 
-cudaError_t launch_setup(void* tables_dst, const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes,
-                         cudaStream_t stream) {
-  if (tables_bytes > kSetupBlobBytes) {   // many layers: the tables do not fit a kernel argument
-    cudaError_t e = cudaMemsetAsync(zero_dst, 0, zero_bytes, stream);
-    if (e != cudaSuccess) return e;
-    return cudaMemcpyAsync(tables_dst, tables_src, tables_bytes, cudaMemcpyHostToDevice, stream);
-  }
-  ProfileScope prof(stream, PT_SETUP);
+// Writes `bytes` (a multiple of 16) of host data to device memory in pieces that travel as kernel arguments: no
+// staging buffer, nothing that blocks the host, and the host data may be freed when the call returns.
+cudaError_t upload_by_launches(void* dst, const void* src, size_t bytes, cudaStream_t stream) {
   SetupBlob blob;
-  std::memcpy(blob.bytes, tables_src, tables_bytes);
+  for (size_t off = 0; off < bytes; off += kSetupBlobBytes) {
+    const size_t len = bytes - off < kSetupBlobBytes ? bytes - off : kSetupBlobBytes;
+    std::memcpy(blob.bytes, (const unsigned char*)src + off, len);
+    setup_kernel<<<1, kThreads, 0, stream>>>(blob, (uint4*)((unsigned char*)dst + off), (uint32_t)(len / 16), nullptr, 0);
+    GD_LAUNCH_CHECK();
+  }
+  return cudaSuccess;
+}
+
+cudaError_t launch_setup(void* tables_dst, const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes,
+                         cudaStream_t stream, bool src_is_pinned) {
+  ProfileScope prof(stream, PT_SETUP);
   const uint64_t zero_vec = zero_bytes / 16;   // both regions are 256-byte aligned and padded
   uint64_t blocks = (zero_vec + kThreads * 8 - 1) / (kThreads * 8);
   const uint64_t cap = (uint64_t)sm_count() * 4;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  setup_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(blob, (uint4*)tables_dst, (uint32_t)(tables_bytes / 16),
-                                                         (uint4*)zero_dst, zero_vec);
+  // Tables of up to kSetupBlobBytes travel with the launch that clears the control region.  Larger ones (models
+  // with many tensors) are copied from the page-locked image kept with the cached plan - an asynchronous copy -
+  // or, where there is no such image, in pieces by further launches.  Never from pageable memory: that copy would
+  // block the host and could not be captured.
+  SetupBlob blob;
+  const size_t first = tables_bytes <= kSetupBlobBytes ? tables_bytes : (src_is_pinned ? 0 : kSetupBlobBytes);
+  std::memcpy(blob.bytes, tables_src, first);
+  setup_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(blob, (uint4*)tables_dst, (uint32_t)(first / 16), (uint4*)zero_dst,
+                                                         zero_vec);
   GD_LAUNCH_CHECK();
-  return cudaSuccess;
+  if (first == tables_bytes) return cudaSuccess;
+  if (src_is_pinned) return cudaMemcpyAsync(tables_dst, tables_src, tables_bytes, cudaMemcpyHostToDevice, stream);
+  return upload_by_launches((unsigned char*)tables_dst + first, (const unsigned char*)tables_src + first, tables_bytes - first,
+                            stream);
 }
 
 int sm_count() {
-  static std::atomic<int> cached{0};
-  if (cached.load(std::memory_order_relaxed) > 0) return cached.load(std::memory_order_relaxed);
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-    return 148;   // B200; only sizes grids
-  cached.store(sms, std::memory_order_relaxed);
+  static PerDeviceInt cached;
+  int dev = -1;
+  int sms = cached.get(&dev);
+  if (sms > 0) return sms;
+  if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;   // B200; only sizes grids
+  if (dev < kMaxDevices) cached.set(dev, sms);
   return sms;
 }
 
@@ -474,21 +287,21 @@ int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, const uint3
   }
 }
 
-int gd_compress(const gd_compress_args* a, void* stream_v) {
+namespace {
+
+int compress_impl(const gd_compress_args* a, void* stream_v, bool may_allocate) {
   NvtxRange range("gd_compress");
   if (!a) return GD_ERR_INVALID_ARG;
   cudaStream_t stream = (cudaStream_t)stream_v;
   try {
-    Plan P;
     if (a->value_mode == GD_VALUES_COLUMN_MEANS && !a->layer_cols) return GD_ERR_INVALID_ARG;
-    int rc = make_plan(a->layer_off, a->n_layers, a->value_mode == GD_VALUES_COLUMN_MEANS ? a->layer_cols : nullptr,
-                       a->n_shards, a->scope_mode, a->drop_ppm, a->flags, &P);
+    const PlanEntry* entry = nullptr;
+    std::unique_ptr<PlanEntry> owned;
+    int rc = plan_for(a, may_allocate, &entry, &owned);
     if (rc != GD_OK) return rc;
-    uint64_t n_sh = 0;
-    rc = check_offsets(a->shard_off, a->n_shards, &n_sh);
-    if (rc != GD_OK) return rc;
+    const Plan& P = entry->P;
     const uint64_t n = a->layer_off[a->n_layers];
-    if (n_sh != n || a->n != n) return GD_ERR_INVALID_ARG;
+    if (a->n != n) return GD_ERR_INVALID_ARG;
     if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_COLUMN_MEANS) return GD_ERR_INVALID_ARG;
     if (a->value_mode != GD_VALUES_FP32 && n > (1ull << 31)) return GD_ERR_TOO_LARGE;
     if (a->flags & ~(uint32_t)(GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD | GD_FLAG_QUANT_ERROR_FEEDBACK |
@@ -506,17 +319,8 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     if (a->value_mode != GD_VALUES_FP32 && !a->out_means) return GD_ERR_INVALID_ARG;
     if (!a->workspace || ((uintptr_t)a->workspace & (kAlign - 1))) return GD_ERR_WORKSPACE;
     if (a->workspace_bytes < P.total_bytes) return GD_ERR_WORKSPACE;
-
-    // host image of the tables
-    std::vector<unsigned char> blob(P.tables_bytes, 0);
-    std::memcpy(blob.data() + P.t_scopes, P.scopes.data(), sizeof(ScopeDesc) * P.n_scopes);
-    for (int l = 0; l < L_COUNT; ++l)
-      std::memcpy(blob.data() + P.t_tile0[l], P.tile0[l].data(), sizeof(uint32_t) * (P.n_scopes + 1));
-    std::memcpy(blob.data() + P.t_samp_off, P.samp_off.data(), sizeof(uint64_t) * (P.n_scopes + 1));
-    std::memcpy(blob.data() + P.t_layer_off, a->layer_off, sizeof(uint64_t) * ((size_t)a->n_layers + 1));
-    std::memcpy(blob.data() + P.t_shard_off, a->shard_off, sizeof(uint64_t) * ((size_t)a->n_shards + 1));
-    std::memcpy(blob.data() + P.t_pair_off, P.pair_off.data(), sizeof(uint64_t) * ((size_t)a->n_layers + 1));
-    std::memcpy(blob.data() + P.t_layer_cols, P.layer_cols.data(), sizeof(uint32_t) * (size_t)a->n_layers);
+    const unsigned char* tables_image = entry->pinned ? entry->pinned : entry->blob.data();
+    const bool image_is_pinned = entry->pinned != nullptr;
 
     unsigned char* ws = (unsigned char*)a->workspace;
     DevTables T;
@@ -570,10 +374,10 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
     // when every scope's sample is small enough for one CTA; otherwise it is a launch of its own.
     const bool local_predict = P.local_predict;
     if (local_predict) {
-      if (launch_setup_predict(T, tiles[L_SAMP], P.samp_tile, (uint32_t*)(ws + P.off_flags), ws + P.off_tables, blob.data(), P.tables_bytes, ws, P.zero_bytes, P.off_state,
+      if (launch_setup_predict(T, tiles[L_SAMP], P.samp_tile, (uint32_t*)(ws + P.off_flags), ws + P.off_tables, tables_image, P.tables_bytes, ws, P.zero_bytes, P.off_state,
                                P.t_scopes, P.t_tile0[L_SAMP], stream) != cudaSuccess)
         return GD_ERR_CUDA;
-    } else if (launch_setup(ws + P.off_tables, blob.data(), P.tables_bytes, ws, P.zero_bytes, stream) != cudaSuccess) {
+    } else if (launch_setup(ws + P.off_tables, tables_image, P.tables_bytes, ws, P.zero_bytes, stream, image_is_pinned) != cudaSuccess) {
       return GD_ERR_CUDA;
     }
     if (sampled) {
@@ -616,6 +420,10 @@ int gd_compress(const gd_compress_args* a, void* stream_v) {
   }
 }
 
+}  // namespace
+
+int gd_compress(const gd_compress_args* a, void* stream) { return compress_impl(a, stream, true); }
+
 int gd_residual_reset(float* residual, uint64_t n, void* stream) {
   if (n == 0) return GD_OK;
   if (!residual) return GD_ERR_INVALID_ARG;
@@ -648,27 +456,32 @@ static __device__ __align__(256) unsigned char g_static_workspace[GD_STATIC_WORK
 
 int gd_compress_static(const gd_compress_args* a, void* stream, const void** workspace_out) {
   if (!a) return GD_ERR_INVALID_ARG;
-  size_t need = 0;
-  int rc = gd_workspace_bytes(a->layer_off, a->n_layers, a->value_mode == GD_VALUES_COLUMN_MEANS ? a->layer_cols : nullptr,
-                              a->n_shards, a->scope_mode, a->drop_ppm, &need);
+  if (a->value_mode == GD_VALUES_COLUMN_MEANS && !a->layer_cols) return GD_ERR_INVALID_ARG;
+  const PlanEntry* entry = nullptr;
+  std::unique_ptr<PlanEntry> owned;
+  int rc;
+  try {
+    rc = plan_for(a, false, &entry, &owned);
+  } catch (const std::bad_alloc&) {
+    return GD_ERR_INVALID_ARG;
+  }
   if (rc != GD_OK) return rc;
-  if (need > (size_t)GD_STATIC_WORKSPACE_BYTES) return GD_ERR_TOO_LARGE;
+  if (entry->P.total_bytes > (size_t)GD_STATIC_WORKSPACE_BYTES) return GD_ERR_TOO_LARGE;   // what THIS call needs
   // In host code g_static_workspace is only a handle: its device address has to be asked for, once
   // per device, with that device current.
-  constexpr int kMaxDevices = 64;
-  static void* scratch_of_device[kMaxDevices] = {nullptr};
+  static std::atomic<void*> scratch_of_device[kMaxDevices];
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GD_ERR_CUDA;
-  if (!scratch_of_device[dev]) {
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return GD_ERR_CUDA;
-    scratch_of_device[dev] = p;
+  void* scratch = scratch_of_device[dev].load(std::memory_order_acquire);
+  if (!scratch) {
+    if (cudaGetSymbolAddress(&scratch, g_static_workspace) != cudaSuccess || !scratch) return GD_ERR_CUDA;
+    scratch_of_device[dev].store(scratch, std::memory_order_release);   // (two threads may both ask: same answer)
   }
   gd_compress_args b = *a;
-  b.workspace = scratch_of_device[dev];
+  b.workspace = scratch;
   b.workspace_bytes = (size_t)GD_STATIC_WORKSPACE_BYTES;
   if (workspace_out) *workspace_out = b.workspace;
-  return gd_compress(&b, stream);
+  return compress_impl(&b, stream, false);   // (nothing is allocated on this path, page-locked host memory included)
 }
 
 int gd_profile_enable(int mode) {

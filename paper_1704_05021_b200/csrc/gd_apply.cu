@@ -228,7 +228,9 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
         std::memcpy(blob.data() + o_pair, pair_off.data(), sizeof(uint64_t) * ((size_t)n_layers + 1));
         std::memcpy(blob.data() + o_cols, cols.data(), sizeof(uint32_t) * (size_t)n_layers);
       }
-      if (cudaMemcpyAsync(ws, blob.data(), need, cudaMemcpyHostToDevice, stream) != cudaSuccess) return GD_ERR_CUDA;
+      // (in pieces that travel as kernel arguments: a copy from this pageable vector would block the host)
+      blob.resize((need + 15) / 16 * 16, 0);
+      if (upload_by_launches(ws, blob.data(), blob.size(), stream) != cudaSuccess) return GD_ERR_CUDA;
     }
     ApplyDev A;
     std::memset(&A, 0, sizeof(A));

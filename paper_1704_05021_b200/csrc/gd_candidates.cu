@@ -44,11 +44,12 @@ constexpr int kCtasPerSm = GD_K2_CTAS;     // co-resident CTAs per SM the kernel
 constexpr int kRounds = kTile / kThreads;   // 16 entries per thread and block of kTile entries
 constexpr uint32_t kWinBins = kRadixBins0 - 2u;   // fine bins of the window; bin 0: below it, bin 2047: above it
 
-// Debug builds (-DGD_PHASE_STAMPS) leave time stamps of CTA 0 in the unused tail of the control block.
+// Debug builds (-DGD_PHASE_STAMPS) leave, in the unused tail of the control block, the time at which the last CTA
+// passed each phase boundary.
 #ifdef GD_PHASE_STAMPS
 #define GD_STAMP(i)                                                                                                      \
   do {                                                                                                                   \
-    if (blockIdx.x == 0 && threadIdx.x == 0) reinterpret_cast<unsigned long long*>(T.ctl)[12 + (i)] = global_timer_ns(); \
+    if (threadIdx.x == 0) atomicMax(reinterpret_cast<unsigned long long*>(T.ctl) + 12 + (i), global_timer_ns());         \
   } while (0)
 #else
 #define GD_STAMP(i) do { } while (0)
@@ -56,7 +57,7 @@ constexpr uint32_t kWinBins = kRadixBins0 - 2u;   // fine bins of the window; bi
 
 struct Shared {
   uint32_t stage[kStage];        // value bits of the share's first kStage entries
-  uint32_t idx[kTile];           // positions of the block being placed
+  uint32_t idx[kStage];          // their positions in the gradient
   uint32_t hist[kRadixBins0];    // digit histogram of the scope being counted
 };
 
@@ -203,48 +204,59 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
     return run;
   };
 
-  // ---- the share into shared memory; coarse histogram around the estimate
+  // ---- the share into shared memory (values and positions); coarse histogram around the estimate
   for (uint32_t b = tid; b < kRadixBins0; b += kThreads) sm.hist[b] = 0;
+  // Coalesced 128-bit loads, those of a block's values and positions all in flight before the first store.  Nothing
+  // is written past the block's end: that part of the stage belongs to the share's next segment.
   for_segments([&](const Segment& g) {
-    const float* vals = T.cand_val + s_scope[g.s].cand_base;
-    const uint32_t wlo = s_wlo[g.s];
-    uint32_t below = 0, above = 0;                           // this thread's entries outside the window
+    const uint32_t* vals = reinterpret_cast<const uint32_t*>(T.cand_val + s_scope[g.s].cand_base);
+    const uint32_t* idxs = T.cand_idx + s_scope[g.s].cand_base;
     for (uint64_t b0 = g.beg; b0 < g.end; b0 += kTile) {
       const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
       const uint32_t sp = g.sp0 + (uint32_t)(b0 - g.beg);
-      const bool stage_it = sp + kTile <= kStage;            // else: read from the list every time
-#pragma unroll 2
-      for (int r = 0; r < kRounds / 4; ++r) {                // coalesced 128-bit loads
-        const uint32_t e = 4u * ((uint32_t)r * kThreads + tid);
-        if (e >= valid) break;
-        uint32_t w[4] = {0u, 0u, 0u, 0u};
-        if (e + 4u <= valid) {
-          const uint4 v4 = __ldcg(reinterpret_cast<const uint4*>(vals + b0 + e));
-          w[0] = v4.x; w[1] = v4.y; w[2] = v4.z; w[3] = v4.w;
-          if (stage_it) *reinterpret_cast<uint4*>(sm.stage + sp + e) = v4;
-        } else {
-          // (nothing is written past the block's end: that part of the stage belongs to the share's next segment)
-          for (uint32_t c = 0; e + c < valid; ++c) {
-            w[c] = __float_as_uint(__ldcg(vals + b0 + e + c));
-            if (stage_it) sm.stage[sp + e + c] = w[c];
-          }
-        }
-        if (!plain) {
+      if (sp + kTile > kStage) break;                        // the rest of the share is read from the lists every time
+      uint4 v4[kRounds / 4], i4[kRounds / 4];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            if (e + c < valid) {
-              const uint32_t key = w[c] & kAbsMask;
-              if (key < wlo) ++below;
-              else {
-                const uint32_t bin = (key - wlo) >> kFineShift;
-                if (bin < kWinBins) atomicAdd(&sm.hist[1u + bin], 1u); else ++above;
-              }
-            }
+      for (int r = 0; r < kRounds / 4; ++r) {
+        const uint32_t e = 4u * ((uint32_t)r * kThreads + tid);
+        const bool whole = e + 4u <= valid;
+        v4[r] = whole ? __ldcg(reinterpret_cast<const uint4*>(vals + b0 + e)) : make_uint4(0u, 0u, 0u, 0u);
+        i4[r] = whole ? __ldcg(reinterpret_cast<const uint4*>(idxs + b0 + e)) : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int r = 0; r < kRounds / 4; ++r) {
+        const uint32_t e = 4u * ((uint32_t)r * kThreads + tid);
+        if (e + 4u <= valid) {
+          *reinterpret_cast<uint4*>(sm.stage + sp + e) = v4[r];
+          *reinterpret_cast<uint4*>(sm.idx + sp + e) = i4[r];
+        } else {
+          for (uint32_t c = 0; e + c < valid; ++c) {
+            sm.stage[sp + e + c] = __ldcg(vals + b0 + e + c);
+            sm.idx[sp + e + c] = __ldcg(idxs + b0 + e + c);
           }
         }
       }
     }
-    if (!plain) {
+  });
+  __syncthreads();
+  if (!plain) {
+    for_segments([&](const Segment& g) {
+      const float* vals = T.cand_val + s_scope[g.s].cand_base;
+      const uint32_t wlo = s_wlo[g.s];
+      uint32_t below = 0, above = 0;                         // this thread's entries outside the window
+      for (uint64_t b0 = g.beg; b0 < g.end; b0 += kTile) {
+        const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
+        const uint32_t* src = block_values(vals, b0, g.sp0 + (uint32_t)(b0 - g.beg));
+#pragma unroll 4
+        for (uint32_t o = tid; o < valid; o += kThreads) {
+          const uint32_t key = src[o] & kAbsMask;
+          if (key < wlo) ++below;
+          else {
+            const uint32_t bin = (key - wlo) >> kFineShift;
+            if (bin < kWinBins) atomicAdd(&sm.hist[1u + bin], 1u); else ++above;
+          }
+        }
+      }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
         below += __shfl_xor_sync(0xFFFFFFFFu, below, o);
@@ -253,8 +265,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       if (lane == 0 && below) atomicAdd(&sm.hist[0], below);
       if (lane == 0 && above) atomicAdd(&sm.hist[kRadixBins0 - 1u], above);
       flush_hist(hist_of(T, g.s, V_CAND, 0), kRadixBins0);
-    }
-  });
+    });
+  }
   GD_STAMP(2);
   if (!grid_barrier(&T.ctl->barrier[V_CAND], phase, T.ctl)) return;
   GD_STAMP(3);
@@ -421,16 +433,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
     for (uint64_t b0 = g.beg; b0 < g.end; b0 += kTile) {
       const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
       const uint32_t* tile_idx = T.cand_idx + d.cand_base + b0;
-      const uint32_t* src = block_values(vals, b0, g.sp0 + (uint32_t)(b0 - g.beg));
+      const uint32_t sp = g.sp0 + (uint32_t)(b0 - g.beg);
+      const uint32_t* src = block_values(vals, b0, sp);
+      const uint32_t* isrc = sp + kTile <= kStage ? sm.idx + sp : tile_idx;   // the block's positions
       __syncthreads();                                       // the previous block is done with the shared variables
-      if (g.first && b0 == g.beg) GD_STAMP(10);
-      // the block's positions: coalesced 128-bit loads into shared memory, in flight during the classification
-      uint4 i4[kRounds / 4];
-#pragma unroll
-      for (int r = 0; r < kRounds / 4; ++r) {
-        const uint32_t e = 4u * ((uint32_t)r * kThreads + tid);
-        i4[r] = e + 4u <= valid ? __ldcg(reinterpret_cast<const uint4*>(tile_idx + e)) : make_uint4(0u, 0u, 0u, 0u);
-      }
       if (two_means && tid == 0) {
         const uint32_t l0 = range_of(T.layer_off, T.n_layers, tile_idx[0]);
         const uint32_t l1 = range_of(T.layer_off, T.n_layers, tile_idx[valid - 1]);
@@ -453,18 +459,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
         we += __popc(__ballot_sync(0xFFFFFFFFu, iseq));
       }
       if (lane == 0) { s_wg[warp] = wg; s_we[warp] = we; }
-      if (g.first && b0 == g.beg) GD_STAMP(11);
-#pragma unroll
-      for (int r = 0; r < kRounds / 4; ++r) {
-        const uint32_t e = 4u * ((uint32_t)r * kThreads + tid);
-        if (e + 4u <= valid) {
-          *reinterpret_cast<uint4*>(sm.idx + e) = i4[r];
-        } else {
-          for (uint32_t c = 0; e + c < valid; ++c) sm.idx[e + c] = __ldcg(tile_idx + e + c);
-        }
-      }
       __syncthreads();
-      if (g.first && b0 == g.beg) GD_STAMP(12);
       uint32_t rg = 0, re = 0, tot_g = 0, tot_e = 0;          // counts inside the block before this warp / in all of it
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) {
@@ -492,15 +487,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       bool bad = false;
 #pragma unroll 1
       for (int j = 0; j < kRounds; ++j) {
-#ifdef GD_PHASE_STAMPS
-        if (g.first && b0 == g.beg && blockIdx.x == 0 && tid == 0) reinterpret_cast<unsigned long long*>(T.ctl)[40 + j] = global_timer_ns();
-#endif
         const bool isgt = (gm >> j) & 1u, iseq = (em >> j) & 1u, cleared = (zm >> j) & 1u;
         const uint32_t mg = __ballot_sync(0xFFFFFFFFu, isgt), me = __ballot_sync(0xFFFFFFFFu, iseq);
         if (isgt || iseq || cleared) {
           const uint32_t o = wofs + (uint32_t)j * 32u;
           const uint32_t eb = re + __popc(me & ltm);
-          const uint64_t idx = sm.idx[o];
+          const uint64_t idx = isrc[o];
           const uint32_t b = src[o];
           if (isgt || (iseq && eb < q_left)) {
             const uint32_t pos = rg + __popc(mg & ltm) + (eb < q_left ? eb : q_left);
@@ -535,7 +527,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
         rg += __popc(mg);
         re += __popc(me);
       }
-      if (g.first && b0 == g.beg) GD_STAMP(13);
       if (bad) atomicCAS(&T.ctl->status, (int)GD_OK, (int)GD_ERR_INTERNAL);
       if (single) {   // uniform over the CTA
 #pragma unroll
@@ -575,17 +566,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
 
 }  // namespace
 
-// Most CTAs the kernel is ever launched with (the per-CTA records in the workspace are sized for it).
-uint32_t select_compact_max_grid() { return 4096u; }
 
 cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uint64_t cand_total, cudaStream_t stream) {
   ProfileScope prof(stream, PT_CAND_SELECT_COMPACT);
-  constexpr int kMaxDevices = 64;
-  static std::atomic<int> resident_of[kMaxDevices];        // co-resident CTAs per SM, per device (0: not asked yet)
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  static PerDeviceInt resident_of;                         // co-resident CTAs per SM, per device (0: not asked yet)
+  int dev = -1;
   const size_t smem = sizeof(Shared);
-  int resident = resident_of[dev].load(std::memory_order_relaxed);
+  int resident = resident_of.get(&dev);
+  if (dev < 0) return cudaErrorInvalidDevice;              // (the shared-memory attribute below is per device)
   if (resident == 0) {
     cudaError_t e = cudaFuncSetAttribute(select_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -594,7 +582,7 @@ cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uin
     if (e != cudaSuccess) return e;
     if (r <= 0) return cudaErrorLaunchFailure;
     resident = r;
-    resident_of[dev].store(r, std::memory_order_relaxed);
+    resident_of.set(dev, r);
   }
   const uint32_t per_sm = resident < kCtasPerSm ? (uint32_t)resident : (uint32_t)kCtasPerSm;
   uint32_t grid = (uint32_t)sm_count() * per_sm;
@@ -603,7 +591,7 @@ cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uin
   if (units < tiles[L_DSEL]) units = tiles[L_DSEL];
   if (units < 1) units = 1;
   if (grid > units) grid = (uint32_t)units;
-  if (grid > select_compact_max_grid()) grid = select_compact_max_grid();
+  if (grid > kSelectCompactMaxGrid) grid = kSelectCompactMaxGrid;
   DevTables Tc = T;
   uint32_t dsel = tiles[L_DSEL], dchunks = tiles[L_DCOMP];
   void* args[] = {(void*)&Tc, (void*)&dsel, (void*)&dchunks};

@@ -185,13 +185,14 @@ cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense
   ProfileScope prof(stream, dense ? PT_DENSE_COMPACT : PT_CAND_COMPACT);
   // The kernels take tiles from a ticket until none is left: no more CTAs than are resident at once,
   // or the later ones would only start, find nothing and leave.
-  static std::atomic<int> resident[2] = {{0}, {0}};
-  int r = resident[dense ? 1 : 0].load(std::memory_order_relaxed);
+  static PerDeviceInt resident[2];                         // per kernel and device
+  int dev = -1;
+  int r = resident[dense ? 1 : 0].get(&dev);
   if (r == 0) {
     cudaError_t e = dense ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, compact_dense_kernel, kThreads, 0)
                           : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, compact_kernel, kThreads, 0);
     if (e != cudaSuccess || r <= 0) return cudaErrorLaunchFailure;
-    resident[dense ? 1 : 0].store(r, std::memory_order_relaxed);
+    resident[dense ? 1 : 0].set(dev, r);
   }
   const uint32_t cap = (uint32_t)sm_count() * (uint32_t)r;
   const uint32_t most = (!dense && tiles[L_DCOMP] > total) ? tiles[L_DCOMP] : total;   // it may take over the dense chunks

@@ -4,7 +4,7 @@
 // it become candidates) and an estimate tau_hi of the threshold itself (entries above it have their
 // residual slot cleared in the stream).  Both are order statistics of a small stratified sample of
 // v = grad + residual (Algorithm 1's threshold-selection step, run on a sample; the result of the call
-// never depends on it).  When every scope's sample is at most local_sample_max() values, the sample is
+// never depends on it).  When every scope's sample is at most kLocalSampleMax values, the sample is
 // gathered in tiles of 256 to 1024 by CTAs spread over the whole GPU (one SM keeps too few scattered reads in
 // flight), and the CTA that finishes a scope's gather last selects both ranks by itself, in a
 // shared-memory histogram, with two radix passes over the gathered values (11 + 10 bits: the
@@ -204,7 +204,7 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
 
 }  // namespace
 
-uint32_t local_sample_max() { return 32u * kPredictThreads; }   // what one CTA's registers hold: 32 keys per thread
+static_assert(kLocalSampleMax == 32u * kPredictThreads, "what one CTA's registers hold: 32 keys per thread");
 
 // gather_ctas: CTAs that gather the samples (the scopes' sample tiles of gather_tile values); flags: one word per such CTA; tables_src: the host image of the
 // tables (at most kSetupBlobBytes); scopes_off, tile0_off: where the scope descriptors and the first sample tile of

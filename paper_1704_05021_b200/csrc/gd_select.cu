@@ -39,14 +39,15 @@ cudaError_t launch_select_impl(const DevTables& T, uint32_t total_tiles, uint32_
                                cudaStream_t stream) {
   if (!total_tiles) return cudaSuccess;
   ProfileScope prof(stream, VIEW == V_SAMPLE ? PT_SAMPLE_SELECT : (VIEW == V_CAND ? PT_CAND_SELECT : PT_DENSE_SELECT));
-  static std::atomic<int> cached{0};                       // co-resident CTAs per SM of this kernel
-  int resident = cached.load(std::memory_order_relaxed);
+  static PerDeviceInt cached;                              // co-resident CTAs per SM of this kernel, per device
+  int dev = -1;
+  int resident = cached.get(&dev);
   if (resident == 0) {
     int r = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, select_kernel<VIEW, MANY>, kThreads, 0) != cudaSuccess || r <= 0)
       return cudaErrorLaunchFailure;
     resident = r;
-    cached.store(r, std::memory_order_relaxed);
+    cached.set(dev, r);
   }
   const uint32_t per_sm = ctas_per_sm < (uint32_t)resident ? ctas_per_sm : (uint32_t)resident;
   uint32_t grid = (uint32_t)sm_count() * per_sm;

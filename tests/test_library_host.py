@@ -152,3 +152,26 @@ int main(void) {
     out = subprocess.run([str(exe)], capture_output=True, text=True, timeout=120)
     assert out.returncode == 0, (out.returncode, out.stderr)
     assert out.stdout.strip() == "workspace missing or too small|10486|10486"
+
+
+def test_planner_under_address_and_undefined_behaviour_sanitizers(tmp_path):
+    """The host-side planner (scopes, sample sizes, capacities, tile tables, workspace layout: offset arithmetic
+    that runs on every call) built by itself with -fsanitize=address,undefined and driven over a few thousand
+    layouts; the driver checks the invariants the kernels rely on."""
+    import shutil
+    import subprocess
+    gxx = shutil.which("g++")
+    if gxx is None:
+        pytest.skip("no host compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    exe = str(tmp_path / "plan_sanitize")
+    build = subprocess.run([gxx, "-std=c++17", "-O1", "-g", "-fsanitize=address,undefined", "-fno-sanitize-recover=all",
+                            "-I", os.path.join(root, "include"), "-I", os.path.join(root, "paper_1704_05021_b200", "csrc"),
+                            os.path.join(root, "tests", "host", "plan_sanitize.cpp"), "-o", exe],
+                           capture_output=True, text=True)
+    if build.returncode != 0 and "sanitize" in build.stderr and "cannot find" in build.stderr:
+        pytest.skip("the sanitizer run-time libraries are not installed")
+    assert build.returncode == 0, build.stderr
+    run = subprocess.run([exe], capture_output=True, text=True, env=dict(os.environ, ASAN_OPTIONS="detect_leaks=1"))
+    assert run.returncode == 0, run.stdout + run.stderr
+    assert run.stdout.startswith("ok ") and int(run.stdout.split()[1]) > 2000
