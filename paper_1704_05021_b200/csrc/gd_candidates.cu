@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
   __shared__ uint32_t s_vt0[kSmemScopes + 1];      // units before each scope
   __shared__ SelRun s_run[kSmemScopes];            // where the walk down each scope's histograms stands ...
   __shared__ int s_level[kSmemScopes];             // ... and after how many of them
-  __shared__ uint32_t s_wg[kWarps], s_we[kWarps];
+  __shared__ uint32_t s_cnt[kRounds * kWarps], s_tot;    // placement: keys above | equal << 16 per (round, warp)
   __shared__ unsigned long long s_pre[2];
   __shared__ uint32_t s_layer;
   __shared__ int s_single, s_last;
@@ -206,8 +206,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
 
   // ---- the share into shared memory (values and positions); coarse histogram around the estimate
   for (uint32_t b = tid; b < kRadixBins0; b += kThreads) sm.hist[b] = 0;
-  // Coalesced 128-bit loads, those of a block's values and positions all in flight before the first store.  Nothing
-  // is written past the block's end: that part of the stage belongs to the share's next segment.
+  // Asynchronous 16-byte copies from the lists straight into shared memory (cp.async), all of the share's in flight
+  // at once and none of them through registers.  Nothing is written past a block's end: that part of the stage
+  // belongs to the share's next segment.
   for_segments([&](const Segment& g) {
     const uint32_t* vals = reinterpret_cast<const uint32_t*>(T.cand_val + s_scope[g.s].cand_base);
     const uint32_t* idxs = T.cand_idx + s_scope[g.s].cand_base;
@@ -215,20 +216,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
       const uint32_t sp = g.sp0 + (uint32_t)(b0 - g.beg);
       if (sp + kTile > kStage) break;                        // the rest of the share is read from the lists every time
-      uint4 v4[kRounds / 4], i4[kRounds / 4];
-#pragma unroll
-      for (int r = 0; r < kRounds / 4; ++r) {
-        const uint32_t e = 4u * ((uint32_t)r * kThreads + tid);
-        const bool whole = e + 4u <= valid;
-        v4[r] = whole ? __ldcg(reinterpret_cast<const uint4*>(vals + b0 + e)) : make_uint4(0u, 0u, 0u, 0u);
-        i4[r] = whole ? __ldcg(reinterpret_cast<const uint4*>(idxs + b0 + e)) : make_uint4(0u, 0u, 0u, 0u);
-      }
 #pragma unroll
       for (int r = 0; r < kRounds / 4; ++r) {
         const uint32_t e = 4u * ((uint32_t)r * kThreads + tid);
         if (e + 4u <= valid) {
-          *reinterpret_cast<uint4*>(sm.stage + sp + e) = v4[r];
-          *reinterpret_cast<uint4*>(sm.idx + sp + e) = i4[r];
+          const uint32_t dv = (uint32_t)__cvta_generic_to_shared(sm.stage + sp + e);
+          const uint32_t di = (uint32_t)__cvta_generic_to_shared(sm.idx + sp + e);
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dv), "l"(vals + b0 + e) : "memory");
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(di), "l"(idxs + b0 + e) : "memory");
         } else {
           for (uint32_t c = 0; e + c < valid; ++c) {
             sm.stage[sp + e + c] = __ldcg(vals + b0 + e + c);
@@ -238,6 +233,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       }
     }
   });
+  asm volatile("cp.async.wait_all;" ::: "memory");
   __syncthreads();
   if (!plain) {
     for_segments([&](const Segment& g) {
@@ -443,32 +439,48 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
         s_layer = (uint32_t)T.pair_off[l0];                  // the one pair of the block, if it has only one
         s_single = (l0 == l1 && T.layer_cols[l0] == 1u) ? 1 : 0;
       }
-      // classification: warp w owns entries [512 w, 512 w + 512), lane l its entries 512 w + 32 j + l
-      const uint32_t wofs = warp * (32u * kRounds) + lane;
-      uint32_t gm = 0, em = 0, zm = 0, wg = 0, we = 0;
+      // classification: round j covers entries [256 j, 256 j + 256), thread t its entry 256 j + t; only the rounds that
+      // hold entries run.  Keys above / equal to tau per (round, warp), packed (a block has at most 4096 entries).
+      const int rounds = (int)((valid + kThreads - 1) / kThreads);
+      uint32_t gm = 0, em = 0, zm = 0;
 #pragma unroll 4
-      for (int j = 0; j < kRounds; ++j) {
-        const uint32_t o = wofs + (uint32_t)j * 32u;
+      for (int j = 0; j < rounds; ++j) {
+        const uint32_t o = (uint32_t)j * kThreads + tid;
         const bool in = o < valid;
         const uint32_t key = in ? (src[o] & kAbsMask) : 0u;
         const bool isgt = in && key > tau, iseq = in && key == tau;
         gm |= (isgt ? 1u : 0u) << j;
         em |= (iseq ? 1u : 0u) << j;
         zm |= (in && key > zthr ? 1u : 0u) << j;
-        wg += __popc(__ballot_sync(0xFFFFFFFFu, isgt));
-        we += __popc(__ballot_sync(0xFFFFFFFFu, iseq));
+        const uint32_t cg = __popc(__ballot_sync(0xFFFFFFFFu, isgt)), ce = __popc(__ballot_sync(0xFFFFFFFFu, iseq));
+        if (lane == 0) s_cnt[j * kWarps + (int)warp] = cg | (ce << 16);
       }
-      if (lane == 0) { s_wg[warp] = wg; s_we[warp] = we; }
       __syncthreads();
-      uint32_t rg = 0, re = 0, tot_g = 0, tot_e = 0;          // counts inside the block before this warp / in all of it
+      if (warp == 0) {                                        // exclusive prefix over the (round, warp) counts, in that order
+        constexpr int kPerLane = kRounds * kWarps / 32;       // 4
+        uint32_t c[kPerLane], sum = 0;
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) {
-        const uint32_t cg = s_wg[w], ce = s_we[w];
-        rg += (w < (int)warp) ? cg : 0u;
-        re += (w < (int)warp) ? ce : 0u;
-        tot_g += cg;
-        tot_e += ce;
+        for (int u = 0; u < kPerLane; ++u) {
+          const int e = (int)lane * kPerLane + u;
+          c[u] = e < rounds * kWarps ? s_cnt[e] : 0u;
+          sum += c[u];
+        }
+        uint32_t inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+          if ((int)lane >= o) inc += y;
+        }
+        uint32_t run = inc - sum;
+#pragma unroll
+        for (int u = 0; u < kPerLane; ++u) {
+          s_cnt[(int)lane * kPerLane + u] = run;
+          run += c[u];
+        }
+        if (lane == 31) s_tot = inc;
       }
+      __syncthreads();
+      const uint32_t tot_g = s_tot & 0xFFFFu, tot_e = s_tot >> 16;
       // Slot of an entry = (#above before it) + min(#ties before it, q); with seg_g / seg_e the counts before this
       // block that is  out_base + seg_g + min(seg_e, q) + (above before it in the block) + min(ties before it in
       // the block, q - min(seg_e, q)): one 64-bit base per block and 32-bit arithmetic per entry.
@@ -486,11 +498,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       uint32_t cnt_p = 0, cnt_n = 0;
       bool bad = false;
 #pragma unroll 1
-      for (int j = 0; j < kRounds; ++j) {
+      for (int j = 0; j < rounds; ++j) {
         const bool isgt = (gm >> j) & 1u, iseq = (em >> j) & 1u, cleared = (zm >> j) & 1u;
         const uint32_t mg = __ballot_sync(0xFFFFFFFFu, isgt), me = __ballot_sync(0xFFFFFFFFu, iseq);
         if (isgt || iseq || cleared) {
-          const uint32_t o = wofs + (uint32_t)j * 32u;
+          const uint32_t o = (uint32_t)j * kThreads + tid;
+          const uint32_t before = s_cnt[j * kWarps + (int)warp];          // in the block, before this warp's round
+          const uint32_t rg = before & 0xFFFFu, re = before >> 16;
           const uint32_t eb = re + __popc(me & ltm);
           const uint64_t idx = isrc[o];
           const uint32_t b = src[o];
@@ -524,8 +538,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
             T.residual[idx] = __uint_as_float(b);
           }
         }
-        rg += __popc(mg);
-        re += __popc(me);
       }
       if (bad) atomicCAS(&T.ctl->status, (int)GD_OK, (int)GD_ERR_INTERNAL);
       if (single) {   // uniform over the CTA
