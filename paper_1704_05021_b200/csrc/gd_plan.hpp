@@ -23,8 +23,9 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 constexpr double kHitsFactor = 0.25, kHitsMin = 32.0, kHitsMax = 256.0, kSampleMax = 262144.0;
 constexpr uint64_t kSampleAllMax = 8192;         // scopes up to this length are sampled completely
 constexpr uint64_t kClusterMaxStride = 1024;      // strata up to this many elements wide are sampled in groups of 8
-constexpr uint64_t kAutoDenseMax = 3ull << 19;   // vectors up to this length skip the prediction (measured: dense 69 us
-                                                 // against 87 us at 2^20, 93 against 89 at 2^21)
+constexpr uint64_t kAutoDenseMax = 3ull << 18;   // vectors up to this length skip the prediction (measured, step time
+                                                 // with L2 flushed: dense 56 us against 58 us predicted at 2^19 elements,
+                                                 // 65 against 59 at 2^20, 83 against 63 at 2^21)
 
 inline uint64_t kept_count(uint64_t n, uint32_t drop_ppm) {
   return n - (n * (uint64_t)drop_ppm) / 1000000ull;   // n <= 2^32, drop_ppm <= 1e6: no overflow
@@ -130,7 +131,7 @@ inline int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_
   if (scope_mode != GD_SCOPE_GLOBAL && scope_mode != GD_SCOPE_PER_LAYER) return GD_ERR_INVALID_ARG;
   if (n > (1ull << 32)) return GD_ERR_TOO_LARGE;
   const bool sampled = (flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
-  // Short vectors are selected densely right away: below about 2^21 elements the three dense passes
+  // Short vectors are selected densely right away: below about 2^20 elements the three dense passes
   // run out of L2 and cost less than sampling, predicting and selecting among candidates.
   const bool predict = !(flags & GD_FLAG_NO_PREDICTION) && (sampled || n > kAutoDenseMax);
   P->predict = predict;

@@ -99,7 +99,13 @@ def run_steps(w, device, steps, flags=0, method="sort", grads=None, alpha=1.0, w
 # ---------------------------------------------------------------- workload 1: 2^20 flat, 5 steps
 @pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
 def test_config1_five_steps(cuda_device, flags):
-    run_steps(W.workload(1), cuda_device, 5, flags=flags, expect_dense=True)     # short vectors are selected densely
+    run_steps(W.workload(1), cuda_device, 5, flags=flags, expect_dense=bool(flags & B.GD_FLAG_NO_PREDICTION))
+
+
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
+def test_config1_shape_at_2_19(cuda_device, flags):
+    """Half the length of workload 1: short enough to be selected densely whatever the flags (three passes out of L2)."""
+    run_steps(W.workload(1, scale_log2=19), cuda_device, 3, flags=flags, expect_dense=True)
 
 
 @pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION, B.GD_FLAG_NO_EARLY_ZERO, B.GD_FLAG_PLAIN_RADIX])
