@@ -319,7 +319,7 @@ struct CompactDenseSmem {
 };
 
 // Compaction over the dense range itself, for scopes whose prediction failed.  Same placement rule
-// as above, but one ticket covers a chunk of up to 32 tiles (512 KiB of values on long vectors) and the chunk does
+// as above, but one ticket covers a chunk of up to 16 tiles (256 KiB of values on long vectors) and the chunk does
 // one look-back: at 4 bytes per element the chain of look-backs would otherwise have to advance about a
 // hundred tiles per microsecond, which the L2 round trips between CTAs cannot sustain.
 // The classification masks stay in registers; the values of the (few) survivors are read again.

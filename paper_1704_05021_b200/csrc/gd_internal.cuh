@@ -29,7 +29,7 @@ struct DevTables {       // passed by value to every kernel
   uint32_t emit_chunk_tiles;         // tiles of kTile elements one CTA of the fused pass streams (1, 2, 4 or 8)
   uint32_t sample_passes;            // radix passes over the sample: 2 (prediction, 21 bits) or 3 (sampled-threshold mode)
   uint32_t dense_sel_tile;           // elements per tile of the dense selection (4096 .. 32768, by vector length)
-  uint32_t dense_chunk_tiles;        // tiles per chunk of the dense compaction (1 .. 32, by vector length)
+  uint32_t dense_chunk_tiles;        // tiles per chunk of the dense compaction (1 .. 16, by vector length)
   uint32_t samp_tile;                // samples per tile of the sample selection (1024 for short samples, else 4096)
   uint64_t k_total;
   // zeroed region
