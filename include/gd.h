@@ -69,10 +69,13 @@ enum {
                                  of the entries the sample predicts to be kept, and the compaction
                                  only settles the few for which the prediction was wrong; with this
                                  flag the compaction clears every kept slot itself. */
-  GD_FLAG_PLAIN_RADIX = 16u   /* another switch with no effect on results: the selection among the candidates
+  GD_FLAG_PLAIN_RADIX = 16u,  /* another switch with no effect on results: the selection among the candidates
                                  normally starts from a histogram the fused pass has prepared and needs one
                                  more pass; with this flag it always runs its three plain radix passes, as it
                                  does by itself when a threshold lies far above its prediction. */
+  GD_FLAG_PREDICT_ALWAYS = 32u /* a third: predict the threshold from a sample however short the vector is (by
+                                 default short vectors are selected densely, which is faster there).  Not
+                                 together with GD_FLAG_NO_PREDICTION. */
 };
 
 const char* gd_status_string(int status);
@@ -333,13 +336,15 @@ int gd_compress_static(const gd_compress_args* args, void* stream, const void** 
 /*
  * Measurement hooks (no counterpart in the paper).  gd_profile_enable(1) makes every gd_compress
  * record a pair of CUDA events on its stream around the fused full pass (the kernel that streams
- * the dense gradient and residual once); gd_profile_enable(2) brackets every kernel the library
+ * the dense gradient and residual once: tag 2 below, or 16 where a short vector takes one launch for
+ * everything); gd_profile_enable(2) brackets every kernel the library
  * launches; 0 switches the hooks off.  gd_profile_collect waits for the recorded pairs, writes their
  * durations in milliseconds (oldest first, at most `capacity`) and, if tags_out is not NULL, which
  * kernel each belongs to (0 setup, 1 sample selection, 2 fused pass, 3 dense selection, 4 dense
  * compaction, 5 candidate selection, 6 candidate compaction, 7 finalize, 8 apply, 9 sampled-mode pack,
  * 10 means division, 11 quantisation-error feedback, 12 candidate selection and compaction in one launch,
- * 13 setup and prediction in one launch, 14 dense histogram pass, 15 walk of the dense histogram), then forgets them.
+ * 13 setup and prediction in one launch, 14 dense histogram pass, 15 walk of the dense histogram,
+ * 16 add, selection and compaction of a short vector in one launch), then forgets them.
  * At most 4096 pairs are held between two collects; later launches are not recorded.  Not thread-safe.
  */
 int gd_profile_enable(int mode);

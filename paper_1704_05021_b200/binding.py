@@ -33,6 +33,7 @@ GD_FLAG_SAMPLED_THRESHOLD = 2
 GD_FLAG_QUANT_ERROR_FEEDBACK = 4
 GD_FLAG_NO_EARLY_ZERO = 8
 GD_FLAG_PLAIN_RADIX = 16
+GD_FLAG_PREDICT_ALWAYS = 32
 GD_ERR_OVERFLOW = -7
 GD_APPLY_ATOMIC = 1
 
@@ -283,7 +284,7 @@ def gd_step_host(call: CompressCall, apply: Optional[ApplyCall], grad_host: torc
 
 
 PROFILE_TAGS = ["setup", "sample_select", "add_emit", "dense_select", "dense_compact", "cand_select", "cand_compact",
-                "finalize", "apply", "pack_sampled", "means", "feedback", "cand_select_compact", "setup_predict", "dense_hist", "dense_find"]
+                "finalize", "apply", "pack_sampled", "means", "feedback", "cand_select_compact", "setup_predict", "dense_hist", "dense_find", "dense_fused"]
 # Kernels one gd_compress launches, in order, by the path the call takes (each is one launch and, with
 # gd_profile_enable(2), one tagged event pair); gd_decompress_apply adds one "apply" per push.
 STEP_KERNELS = {
@@ -291,7 +292,8 @@ STEP_KERNELS = {
     "predicted_large_sample": ["setup", "sample_select", "add_emit", "cand_select_compact"],
     "predicted_many_scopes": ["setup", "sample_select", "add_emit", "cand_select", "cand_compact"],
     "dense": ["setup", "dense_hist", "dense_find", "dense_hist", "dense_find", "add_emit", "cand_select_compact"],
-    "dense_short_vector": ["setup", "add_emit", "dense_select", "dense_compact"],
+    "dense_short_vector": ["setup", "dense_fused"],
+    "dense_many_scopes": ["setup", "add_emit", "dense_select", "dense_compact"],
     "sampled": ["setup", "sample_select", "add_emit", "pack_sampled"],
 }
 

@@ -37,7 +37,7 @@ struct NvtxRange {
 
 // measurement hooks
 constexpr uint32_t kProfilePairs = 4096;
-int g_profile_mode = 0;   // 0 off, 1 the fused pass only, 2 every kernel
+int g_profile_mode = 0;   // 0 off, 1 the pass over the dense vector only, 2 every kernel
 cudaEvent_t g_ev_begin[kProfilePairs], g_ev_end[kProfilePairs];
 uint32_t g_ev_tag[kProfilePairs];
 uint32_t g_ev_created = 0, g_ev_used = 0;
@@ -52,6 +52,7 @@ struct PlanEntry {
   std::vector<uint32_t> layer_cols;
   int scope_mode = 0;
   uint32_t drop_ppm = 0, plan_flags = 0;
+  uint64_t fused_units = 0;             // what the device the plan was made for takes in one launch (part of the key)
   Plan P;
   std::vector<unsigned char> blob;      // host image of the tables
   unsigned char* pinned = nullptr;      // the same in page-locked memory, for tables too large for a kernel argument
@@ -60,8 +61,8 @@ constexpr size_t kPlanCacheEntries = 64;
 std::mutex g_plan_mutex;
 std::vector<std::unique_ptr<PlanEntry>> g_plans;
 
-bool same_layout(const PlanEntry& e, const gd_compress_args* a, const uint32_t* cols, uint32_t plan_flags) {
-  if (e.scope_mode != a->scope_mode || e.drop_ppm != a->drop_ppm || e.plan_flags != plan_flags) return false;
+bool same_layout(const PlanEntry& e, const gd_compress_args* a, const uint32_t* cols, uint32_t plan_flags, uint64_t fused_units) {
+  if (e.scope_mode != a->scope_mode || e.drop_ppm != a->drop_ppm || e.plan_flags != plan_flags || e.fused_units != fused_units) return false;
   if (e.layer_off.size() != (size_t)a->n_layers + 1 || e.shard_off.size() != (size_t)a->n_shards + 1) return false;
   if (e.layer_cols.empty() != (cols == nullptr)) return false;
   if (std::memcmp(e.layer_off.data(), a->layer_off, sizeof(uint64_t) * e.layer_off.size()) != 0) return false;
@@ -74,14 +75,15 @@ bool same_layout(const PlanEntry& e, const gd_compress_args* a, const uint32_t* 
 int plan_for(const gd_compress_args* a, bool may_allocate, const PlanEntry** out, std::unique_ptr<PlanEntry>* owned) {
   if (!a->layer_off || !a->shard_off || a->n_layers == 0 || a->n_shards == 0) return GD_ERR_INVALID_ARG;
   const uint32_t* cols = a->value_mode == GD_VALUES_COLUMN_MEANS ? a->layer_cols : nullptr;
-  const uint32_t plan_flags = a->flags & (GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD);
+  const uint32_t plan_flags = a->flags & (GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD | GD_FLAG_PREDICT_ALWAYS);
+  const uint64_t fused_units = dense_fused_capacity();     // (of the current device: plans differ between unlike devices)
   {
     std::lock_guard<std::mutex> lock(g_plan_mutex);
     for (const auto& e : g_plans)
-      if (same_layout(*e, a, cols, plan_flags)) { *out = e.get(); return GD_OK; }
+      if (same_layout(*e, a, cols, plan_flags, fused_units)) { *out = e.get(); return GD_OK; }
   }
   std::unique_ptr<PlanEntry> e(new PlanEntry);
-  int rc = make_plan(a->layer_off, a->n_layers, cols, a->n_shards, a->scope_mode, a->drop_ppm, a->flags, &e->P);
+  int rc = make_plan(a->layer_off, a->n_layers, cols, a->n_shards, a->scope_mode, a->drop_ppm, a->flags, &e->P, fused_units);
   if (rc != GD_OK) return rc;
   uint64_t n_sh = 0;
   rc = check_offsets(a->shard_off, a->n_shards, &n_sh);
@@ -93,6 +95,7 @@ int plan_for(const gd_compress_args* a, bool may_allocate, const PlanEntry** out
   e->scope_mode = a->scope_mode;
   e->drop_ppm = a->drop_ppm;
   e->plan_flags = plan_flags;
+  e->fused_units = fused_units;
   const Plan& P = e->P;
   e->blob.assign(P.tables_bytes, 0);
   unsigned char* b = e->blob.data();
@@ -105,7 +108,7 @@ int plan_for(const gd_compress_args* a, bool may_allocate, const PlanEntry** out
   std::memcpy(b + P.t_layer_cols, P.layer_cols.data(), sizeof(uint32_t) * (size_t)a->n_layers);
   std::lock_guard<std::mutex> lock(g_plan_mutex);
   for (const auto& other : g_plans)                        // (another thread may have stored the same layout meanwhile)
-    if (same_layout(*other, a, cols, plan_flags)) { *out = other.get(); return GD_OK; }
+    if (same_layout(*other, a, cols, plan_flags, fused_units)) { *out = other.get(); return GD_OK; }
   if (g_plans.size() < kPlanCacheEntries) {
     if (may_allocate && P.tables_bytes > kSetupBlobBytes) {
       void* p = nullptr;
@@ -178,7 +181,7 @@ int sm_count() {
 }
 
 void profile_mark(cudaStream_t stream, bool begin, uint32_t tag) {
-  if (g_profile_mode == 0 || (g_profile_mode == 1 && tag != PT_ADD_EMIT)) return;
+  if (g_profile_mode == 0 || (g_profile_mode == 1 && tag != PT_ADD_EMIT && tag != PT_DENSE_FUSED)) return;
   if (begin) {
     g_pair_open = false;
     if (g_ev_used >= kProfilePairs) return;
@@ -273,12 +276,14 @@ int gd_workspace_bytes(const uint64_t* layer_off, uint32_t n_layers, const uint3
                        int scope_mode, uint32_t drop_ppm, size_t* bytes_out) {
   if (!bytes_out) return GD_ERR_INVALID_ARG;
   try {
-    size_t most = 0;                                       // whichever mode is used
-    for (uint32_t flags : {0u, (uint32_t)GD_FLAG_SAMPLED_THRESHOLD, (uint32_t)GD_FLAG_NO_PREDICTION}) {
-      Plan P;
-      int rc = make_plan(layer_off, n_layers, layer_cols, n_shards, scope_mode, drop_ppm, flags, &P);
-      if (rc != GD_OK) return rc;
-      if (P.total_bytes > most) most = P.total_bytes;
+    size_t most = 0;                                       // whichever mode is used, on whichever device
+    for (uint32_t flags : {0u, (uint32_t)GD_FLAG_SAMPLED_THRESHOLD, (uint32_t)GD_FLAG_NO_PREDICTION, (uint32_t)GD_FLAG_PREDICT_ALWAYS}) {
+      for (uint64_t fused_units : {(uint64_t)0, ~(uint64_t)0}) {
+        Plan P;
+        int rc = make_plan(layer_off, n_layers, layer_cols, n_shards, scope_mode, drop_ppm, flags, &P, fused_units);
+        if (rc != GD_OK) return rc;
+        if (P.total_bytes > most) most = P.total_bytes;
+      }
     }
     *bytes_out = most;
     return GD_OK;
@@ -305,8 +310,9 @@ int compress_impl(const gd_compress_args* a, void* stream_v, bool may_allocate) 
     if (a->value_mode < GD_VALUES_FP32 || a->value_mode > GD_VALUES_COLUMN_MEANS) return GD_ERR_INVALID_ARG;
     if (a->value_mode != GD_VALUES_FP32 && n > (1ull << 31)) return GD_ERR_TOO_LARGE;
     if (a->flags & ~(uint32_t)(GD_FLAG_NO_PREDICTION | GD_FLAG_SAMPLED_THRESHOLD | GD_FLAG_QUANT_ERROR_FEEDBACK |
-                               GD_FLAG_NO_EARLY_ZERO | GD_FLAG_PLAIN_RADIX))
+                               GD_FLAG_NO_EARLY_ZERO | GD_FLAG_PLAIN_RADIX | GD_FLAG_PREDICT_ALWAYS))
       return GD_ERR_INVALID_ARG;
+    if ((a->flags & GD_FLAG_NO_PREDICTION) && (a->flags & GD_FLAG_PREDICT_ALWAYS)) return GD_ERR_INVALID_ARG;
     if ((a->flags & GD_FLAG_QUANT_ERROR_FEEDBACK) && a->value_mode == GD_VALUES_FP32) return GD_ERR_INVALID_ARG;
     const bool sampled = (a->flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
     if (sampled && ((a->flags & GD_FLAG_NO_PREDICTION) || a->value_mode != GD_VALUES_FP32)) return GD_ERR_INVALID_ARG;
@@ -400,9 +406,15 @@ int compress_impl(const gd_compress_args* a, void* stream_v, bool may_allocate) 
       if (launch_add_emit(U, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
       if (launch_select_compact(U, tiles, P.cand_total, stream) != cudaSuccess) return GD_ERR_CUDA;
     } else if (!predict) {
-      if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
-      if (launch_dense_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
-      if (launch_compact(T, tiles, true, true, stream) != cudaSuccess) return GD_ERR_CUDA;
+      // short vectors: add, select and compact over the dense range in one cooperative launch where the vector
+      // fits its CTAs' shared memory and the scopes its tables (the plan says); else the three separate kernels
+      if (P.dense_fused) {
+        if (launch_dense_fused(T, P.dense_units, stream) != cudaSuccess) return GD_ERR_CUDA;
+      } else {
+        if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+        if (launch_dense_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+        if (launch_compact(T, tiles, true, true, stream) != cudaSuccess) return GD_ERR_CUDA;
+      }
     } else if (P.n_scopes <= kSmemScopes) {
       // selection among the candidates and compaction in one cooperative launch
       if (launch_select_compact(T, tiles, P.cand_total, stream) != cudaSuccess) return GD_ERR_CUDA;

@@ -88,6 +88,11 @@ __device__ __noinline__ bool dense_takeover(const DevTables& T, uint32_t dense_s
 static_assert(sizeof(SelectSmem<V_DENSE, false>) <= sizeof(Shared) && sizeof(CompactDenseSmem) <= sizeof(Shared),
               "the dense selection and compaction borrow this kernel's shared memory");
 
+// DENSE_IN = false: the entries are the candidate lists the fused pass left.  DENSE_IN = true (short vectors, which
+// need no prediction): the "list" of a scope is its dense range itself - the kernel forms v = grad + residual as it
+// loads its share, selects with the three plain radix passes, and writes the whole new residual (v where dropped,
+// +0 where kept) as it places the survivors: add, select and compact of Algorithm 1 in one launch.
+template <bool DENSE_IN>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(const __grid_constant__ DevTables T,
                                                                       uint32_t dense_sel_tiles, uint32_t dense_chunks) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -109,7 +114,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
 
   GD_STAMP(0);
   if (T.ctl->status != GD_OK) return;               // set only by an earlier kernel of this call: uniform over the grid
-  if (dense_sel_tiles != 0u && T.ctl->dense_needed != 0u) {
+  if (!DENSE_IN && dense_sel_tiles != 0u && T.ctl->dense_needed != 0u) {
     if (!dense_takeover(T, dense_sel_tiles, dense_chunks, smem_raw)) return;
   }
 
@@ -123,7 +128,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
     __syncthreads();
     for (uint32_t x = tid; x < T.n_scopes; x += kThreads) {
       const ScopeState* sx = T.state + x;
-      const uint64_t m = predicted_ok(T, s_scope[x], *sx) ? sx->cand_count : 0ull;
+      const uint64_t m = DENSE_IN ? s_scope[x].hi - s_scope[x].lo : (predicted_ok(T, s_scope[x], *sx) ? sx->cand_count : 0ull);
       s_len[x] = m;
       // the window of fine bins is centred on the sample's estimate of the threshold, but starts no lower than
       // the smallest key a candidate can have
@@ -143,7 +148,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
   const uint32_t s_first = t_beg < t_end ? scope_of_tile(s_vt0, T.n_scopes, t_beg) : 0u;
   // The plain radix passes, should they be needed, use the scopes' sample histograms (the sample selection is
   // long finished): cleared here by the whole grid, used only after the second barrier.
-  {
+  // (With dense input the plain passes start at once, in the histograms the start of the call has cleared.)
+  constexpr int kPlainView = DENSE_IN ? V_CAND : V_SAMPLE;
+  if (!DENSE_IN) {
     const uint64_t per_scope = 2048 + 1024 + 1024;
     const uint64_t total = (uint64_t)T.n_scopes * per_scope;
     for (uint64_t i = (uint64_t)blockIdx.x * kThreads + tid; i < total; i += (uint64_t)gridDim.x * kThreads)
@@ -153,8 +160,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
   const bool two_means = T.value_mode == GD_VALUES_TWO_MEANS || T.value_mode == GD_VALUES_COLUMN_MEANS;
   const bool packed = T.value_mode != GD_VALUES_FP32;
   const bool feedback = (T.flags & GD_FLAG_QUANT_ERROR_FEEDBACK) != 0;   // kept slots keep v for feedback_kernel
-  const bool early = early_zero_enabled(T);
-  const bool plain = (T.flags & GD_FLAG_PLAIN_RADIX) != 0;
+  const bool early = !DENSE_IN && early_zero_enabled(T);
+  const bool plain = DENSE_IN || (T.flags & GD_FLAG_PLAIN_RADIX) != 0;
   uint4* agg = reinterpret_cast<uint4*>(T.cta_agg);   // two uint4 per CTA: {last scope, -, gt lo, gt hi}, {eq lo, eq hi, -, -}
   uint32_t phase = 0;
   GD_STAMP(1);
@@ -178,8 +185,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
   };
   // Where the value bits of the block that starts at entry b0 of a scope's list (position sp inside the share) are
   // read from: shared memory if the block was staged, else the list itself.
-  auto block_values = [&](const float* vals, uint64_t b0, uint32_t sp) -> const uint32_t* {
-    return sp + kTile <= kStage ? sm.stage + sp : reinterpret_cast<const uint32_t*>(vals + b0);
+  auto block_values = [&](const float* vals, uint64_t b0, uint32_t sp, uint32_t valid) -> const uint32_t* {
+    return sp + valid <= kStage ? sm.stage + sp : reinterpret_cast<const uint32_t*>(vals + b0);
   };
   // Flushes the CTA's digit histogram into a scope's global one and clears it.
   auto flush_hist = [&](unsigned long long* gh, uint32_t nbins) {
@@ -198,7 +205,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
     else { run.prefix = 0; run.rank = s_scope[s].k; run.gt = 0; }
     __syncthreads();
     for (; have < level; ++have)
-      run = next_digit(hist_of(T, s, V_SAMPLE, have), have == 0 ? kRadixBits0 : 10, run, T.ctl);
+      run = next_digit(hist_of(T, s, kPlainView, have), have == 0 ? kRadixBits0 : 10, run, T.ctl);
     if (tid == 0) { s_run[s] = run; s_level[s] = level; }
     __syncthreads();
     return run;
@@ -206,6 +213,33 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
 
   // ---- the share into shared memory (values and positions); coarse histogram around the estimate
   for (uint32_t b = tid; b < kRadixBins0; b += kThreads) sm.hist[b] = 0;
+  if (DENSE_IN) {
+    // v = grad + residual (or grad - base for a pull) of the share, formed on the way into shared memory: batches of
+    // 16 elements per thread, all loads of a batch in flight before the first add.  (The host gives this kernel only
+    // vectors whose shares fit the stage.)
+    const bool delta = T.delta_base != nullptr;
+    const float* second = delta ? T.delta_base : T.residual;
+    for_segments([&](const Segment& g) {
+      const uint64_t lo = s_scope[g.s].lo;
+      for (uint64_t b0 = g.beg; b0 < g.end; b0 += kTile) {
+        const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
+        const uint32_t sp = g.sp0 + (uint32_t)(b0 - g.beg);
+        if (sp + valid > kStage) break;
+        float gv[kRounds], rv[kRounds];
+#pragma unroll
+        for (int j = 0; j < kRounds; ++j) {
+          const uint32_t o = (uint32_t)j * kThreads + tid;
+          gv[j] = o < valid ? __ldcs(T.grad + lo + b0 + o) : 0.0f;
+          rv[j] = o < valid ? second[lo + b0 + o] : 0.0f;
+        }
+#pragma unroll
+        for (int j = 0; j < kRounds; ++j) {
+          const uint32_t o = (uint32_t)j * kThreads + tid;
+          if (o < valid) sm.stage[sp + o] = __float_as_uint(delta ? __fsub_rn(gv[j], rv[j]) : __fadd_rn(gv[j], rv[j]));
+        }
+      }
+    });
+  } else {
   // Asynchronous 16-byte copies from the lists straight into shared memory (cp.async), all of the share's in flight
   // at once and none of them through registers.  Nothing is written past a block's end: that part of the stage
   // belongs to the share's next segment.
@@ -215,7 +249,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
     for (uint64_t b0 = g.beg; b0 < g.end; b0 += kTile) {
       const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
       const uint32_t sp = g.sp0 + (uint32_t)(b0 - g.beg);
-      if (sp + kTile > kStage) break;                        // the rest of the share is read from the lists every time
+      if (sp + valid > kStage) break;                        // the rest of the share is read from the lists every time
 #pragma unroll
       for (int r = 0; r < kRounds / 4; ++r) {
         const uint32_t e = 4u * ((uint32_t)r * kThreads + tid);
@@ -234,6 +268,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
     }
   });
   asm volatile("cp.async.wait_all;" ::: "memory");
+  }
   __syncthreads();
   if (!plain) {
     for_segments([&](const Segment& g) {
@@ -242,7 +277,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       uint32_t below = 0, above = 0;                         // this thread's entries outside the window
       for (uint64_t b0 = g.beg; b0 < g.end; b0 += kTile) {
         const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
-        const uint32_t* src = block_values(vals, b0, g.sp0 + (uint32_t)(b0 - g.beg));
+        const uint32_t* src = block_values(vals, b0, g.sp0 + (uint32_t)(b0 - g.beg), valid);
 #pragma unroll 4
         for (uint32_t o = tid; o < valid; o += kThreads) {
           const uint32_t key = src[o] & kAbsMask;
@@ -264,7 +299,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
     });
   }
   GD_STAMP(2);
-  if (!grid_barrier(&T.ctl->barrier[V_CAND], phase, T.ctl)) return;
+  if (!DENSE_IN && !grid_barrier(&T.ctl->barrier[V_CAND], phase, T.ctl)) return;   // (dense input: nothing to wait for yet)
   GD_STAMP(3);
 
   // ---- the bin that holds each scope's threshold; refine: the low 11 bits among the entries of that bin
@@ -283,7 +318,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       const uint32_t lo = s_wlo[g.s] + ((bin - 1u) << kFineShift);            // keys [lo, lo + 2^11) are the bin
       for (uint64_t b0 = g.beg; b0 < g.end; b0 += kTile) {
         const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
-        const uint32_t* src = block_values(vals, b0, g.sp0 + (uint32_t)(b0 - g.beg));
+        const uint32_t* src = block_values(vals, b0, g.sp0 + (uint32_t)(b0 - g.beg), valid);
 #pragma unroll 4
         for (uint32_t o = tid; o < valid; o += kThreads) {
           const uint32_t dd = (src[o] & kAbsMask) - lo;                       // (wraps for keys below the bin)
@@ -295,10 +330,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
   }
   if (outside && tid == 0) atomicOr(&T.ctl->generic_needed, 1u);
   GD_STAMP(4);
-  if (!grid_barrier(&T.ctl->barrier[V_CAND], phase, T.ctl)) return;
+  if (!DENSE_IN && !grid_barrier(&T.ctl->barrier[V_CAND], phase, T.ctl)) return;
   GD_STAMP(5);
 
-  if (__ldcg(&T.ctl->generic_needed) == 0u) {
+  if (!DENSE_IN && __ldcg(&T.ctl->generic_needed) == 0u) {
     // the threshold key = lower edge of the bin + the digit found in the refined histogram
     for_segments([&](const Segment& g) {
       if (s_level[g.s] != 1) return;
@@ -325,14 +360,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
         const uint32_t prefix = plain_walk(g.s, pass).prefix;
         for (uint64_t b0 = g.beg; b0 < g.end; b0 += kTile) {
           const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
-          const uint32_t* src = block_values(vals, b0, g.sp0 + (uint32_t)(b0 - g.beg));
+          const uint32_t* src = block_values(vals, b0, g.sp0 + (uint32_t)(b0 - g.beg), valid);
 #pragma unroll 4
           for (uint32_t o = tid; o < valid; o += kThreads) {
             const uint32_t key = src[o] & kAbsMask;
             if (pass == 0 || (key >> pshift) == prefix) atomicAdd(&sm.hist[(key >> shift) & dmask], 1u);
           }
         }
-        flush_hist(hist_of(T, g.s, V_SAMPLE, pass), dmask + 1u);
+        flush_hist(hist_of(T, g.s, kPlainView, pass), dmask + 1u);
       });
       if (!grid_barrier(&T.ctl->barrier[V_CAND], phase, T.ctl)) return;
     }
@@ -349,6 +384,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       if (g.beg == 0 && tid == 0) {                          // the CTA that holds the scope's first entries
         ScopeState* st = T.state + g.s;
         st->tau = run.prefix; st->q = run.rank; st->gt = run.gt;
+        if (DENSE_IN) st->used_dense = 1u;                   // (statistics: selected over the dense range)
       }
       if (!g.last) return;
       const float* vals = T.cand_val + s_scope[g.s].cand_base;
@@ -356,7 +392,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       uint32_t cg = 0, ce = 0;
       for (uint64_t b0 = g.beg; b0 < g.end; b0 += kTile) {
         const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
-        const uint32_t* src = block_values(vals, b0, g.sp0 + (uint32_t)(b0 - g.beg));
+        const uint32_t* src = block_values(vals, b0, g.sp0 + (uint32_t)(b0 - g.beg), valid);
 #pragma unroll 4
         for (uint32_t o = tid; o < valid; o += kThreads) {
           const uint32_t key = src[o] & kAbsMask;
@@ -430,12 +466,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       const uint32_t valid = (uint32_t)min64(kTile, g.end - b0);
       const uint32_t* tile_idx = T.cand_idx + d.cand_base + b0;
       const uint32_t sp = g.sp0 + (uint32_t)(b0 - g.beg);
-      const uint32_t* src = block_values(vals, b0, sp);
-      const uint32_t* isrc = sp + kTile <= kStage ? sm.idx + sp : tile_idx;   // the block's positions
+      const uint32_t* src = block_values(vals, b0, sp, valid);
+      const uint32_t* isrc = sp + valid <= kStage ? sm.idx + sp : tile_idx;   // the block's positions (lists)
+      const uint64_t pos0 = d.lo + b0;                        // position of the block's first entry (dense input)
       __syncthreads();                                       // the previous block is done with the shared variables
       if (two_means && tid == 0) {
-        const uint32_t l0 = range_of(T.layer_off, T.n_layers, tile_idx[0]);
-        const uint32_t l1 = range_of(T.layer_off, T.n_layers, tile_idx[valid - 1]);
+        const uint32_t l0 = range_of(T.layer_off, T.n_layers, DENSE_IN ? pos0 : (uint64_t)tile_idx[0]);
+        const uint32_t l1 = range_of(T.layer_off, T.n_layers, DENSE_IN ? pos0 + valid - 1 : (uint64_t)tile_idx[valid - 1]);
         s_layer = (uint32_t)T.pair_off[l0];                  // the one pair of the block, if it has only one
         s_single = (l0 == l1 && T.layer_cols[l0] == 1u) ? 1 : 0;
       }
@@ -501,17 +538,21 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       for (int j = 0; j < rounds; ++j) {
         const bool isgt = (gm >> j) & 1u, iseq = (em >> j) & 1u, cleared = (zm >> j) & 1u;
         const uint32_t mg = __ballot_sync(0xFFFFFFFFu, isgt), me = __ballot_sync(0xFFFFFFFFu, iseq);
-        if (isgt || iseq || cleared) {
-          const uint32_t o = (uint32_t)j * kThreads + tid;
+        const uint32_t o = (uint32_t)j * kThreads + tid;
+        if (DENSE_IN ? o < valid : (isgt || iseq || cleared)) {
           const uint32_t before = s_cnt[j * kWarps + (int)warp];          // in the block, before this warp's round
           const uint32_t rg = before & 0xFFFFu, re = before >> 16;
           const uint32_t eb = re + __popc(me & ltm);
-          const uint64_t idx = isrc[o];
+          const uint64_t idx = DENSE_IN ? pos0 + o : (uint64_t)isrc[o];
           const uint32_t b = src[o];
-          if (isgt || (iseq && eb < q_left)) {
+          const bool keep = isgt || (iseq && eb < q_left);
+          // dense input: this is where the new residual is written, every element of it (v where dropped, +0 where
+          // kept, v for kept entries whose quantisation error is fed back later)
+          if (DENSE_IN && idx < T.n) T.residual[idx] = (keep && !feedback) ? 0.0f : __uint_as_float(b);
+          if (keep) {
             const uint32_t pos = rg + __popc(mg & ltm) + (eb < q_left ? eb : q_left);
             if (pos < room && idx < T.n) {
-              if (!feedback && !(skip_cleared && cleared)) T.residual[idx] = 0.0f;
+              if (!DENSE_IN && !feedback && !(skip_cleared && cleared)) T.residual[idx] = 0.0f;
               if (packed) {
                 const uint32_t sgn = b >> 31;
                 oi[pos] = (uint32_t)idx | (sgn << 31);
@@ -579,38 +620,78 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
 }  // namespace
 
 
-cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uint64_t cand_total, cudaStream_t stream) {
-  ProfileScope prof(stream, PT_CAND_SELECT_COMPACT);
-  static PerDeviceInt resident_of;                         // co-resident CTAs per SM, per device (0: not asked yet)
+namespace {
+
+// Co-resident CTAs of the kernel per SM on the current device, asked once per device (with the kernel's shared-memory
+// attribute set on the way); *dev receives the device.
+template <bool DENSE_IN>
+cudaError_t resident_ctas(int* resident_out, int* dev_out) {
+  static PerDeviceInt resident_of;                         // (0: not asked yet)
   int dev = -1;
   const size_t smem = sizeof(Shared);
   int resident = resident_of.get(&dev);
   if (dev < 0) return cudaErrorInvalidDevice;              // (the shared-memory attribute below is per device)
   if (resident == 0) {
-    cudaError_t e = cudaFuncSetAttribute(select_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(select_compact_kernel<DENSE_IN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int r = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, select_compact_kernel, kThreads, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, select_compact_kernel<DENSE_IN>, kThreads, smem);
     if (e != cudaSuccess) return e;
     if (r <= 0) return cudaErrorLaunchFailure;
     resident = r;
     resident_of.set(dev, r);
   }
+  *resident_out = resident;
+  *dev_out = dev;
+  return cudaSuccess;
+}
+
+template <bool DENSE_IN>
+cudaError_t launch_impl(const DevTables& T, uint64_t units, uint32_t dsel, uint32_t dchunks, uint32_t tag, cudaStream_t stream) {
+  ProfileScope prof(stream, tag);
+  const size_t smem = sizeof(Shared);
+  int resident = 0, dev = -1;
+  cudaError_t er = resident_ctas<DENSE_IN>(&resident, &dev);
+  if (er != cudaSuccess) return er;
   const uint32_t per_sm = resident < kCtasPerSm ? (uint32_t)resident : (uint32_t)kCtasPerSm;
   uint32_t grid = (uint32_t)sm_count() * per_sm;
-  // no more CTAs than units of work - counting the dense tiles this launch may have to take over
-  uint64_t units = (cand_total + kSub - 1) / kSub;
-  if (units < tiles[L_DSEL]) units = tiles[L_DSEL];
   if (units < 1) units = 1;
-  if (grid > units) grid = (uint32_t)units;
+  if (grid > units) grid = (uint32_t)units;                // no more CTAs than units of work
   if (grid > kSelectCompactMaxGrid) grid = kSelectCompactMaxGrid;
+  if (DENSE_IN && (units + grid - 1) / grid > kStage / kSub) return cudaErrorInvalidConfiguration;   // a share must fit the stage
   DevTables Tc = T;
-  uint32_t dsel = tiles[L_DSEL], dchunks = tiles[L_DCOMP];
   void* args[] = {(void*)&Tc, (void*)&dsel, (void*)&dchunks};
-  cudaError_t e = cudaLaunchCooperativeKernel((const void*)select_compact_kernel, dim3(grid), dim3(kThreads), args, smem, stream);
+  cudaError_t e = cudaLaunchCooperativeKernel((const void*)select_compact_kernel<DENSE_IN>, dim3(grid), dim3(kThreads), args,
+                                              smem, stream);
   if (e != cudaSuccess) return e;
   note_launches(1);
   return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uint64_t cand_total, cudaStream_t stream) {
+  // units of work: the lists' capacity - or the dense tiles this launch may have to take over, if there are more
+  uint64_t units = (cand_total + kSub - 1) / kSub;
+  if (units < tiles[L_DSEL]) units = tiles[L_DSEL];
+  return launch_impl<false>(T, units, tiles[L_DSEL], tiles[L_DCOMP], PT_CAND_SELECT_COMPACT, stream);
+}
+
+// Short vectors: residual add, exact selection and compaction over the dense range itself, in one launch.
+// dense_units: the scopes' lengths in units of 1024 elements, summed.
+cudaError_t launch_dense_fused(const DevTables& T, uint64_t dense_units, cudaStream_t stream) {
+  return launch_impl<true>(T, dense_units, 0u, 0u, PT_DENSE_FUSED, stream);
+}
+
+// How many units launch_dense_fused can take on the current device: every CTA's share must fit its shared-memory
+// stage.  0 if the kernel cannot run here.
+uint64_t dense_fused_capacity() {
+  int resident = 0, dev = -1;
+  if (resident_ctas<true>(&resident, &dev) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+  const uint64_t per_sm = resident < kCtasPerSm ? (uint64_t)resident : (uint64_t)kCtasPerSm;
+  uint64_t grid = (uint64_t)sm_count() * per_sm;
+  if (grid > kSelectCompactMaxGrid) grid = kSelectCompactMaxGrid;
+  return grid * (kStage / kSub);
 }
 
 }  // namespace gd

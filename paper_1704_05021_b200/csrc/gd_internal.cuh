@@ -236,6 +236,8 @@ cudaError_t launch_feedback(const DevTables& T, cudaStream_t stream);
 cudaError_t launch_pack_sampled(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uint64_t cand_total, cudaStream_t stream);
 cudaError_t launch_dense_bound(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
+cudaError_t launch_dense_fused(const DevTables& T, uint64_t dense_units, cudaStream_t stream);
+uint64_t dense_fused_capacity();   // how many 1024-element units launch_dense_fused takes on the current device (0: none)
 cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream);
 int sm_count();   // multiprocessors of the current device (148 if it cannot be asked)
 // A small per-device cache of one int (0 = not known yet), for values that belong to the device a call runs on:
@@ -259,7 +261,7 @@ void note_launches(uint32_t count);
 enum ProfileTag : uint32_t { PT_SETUP = 0, PT_PACK_SAMPLED = 9, PT_MEANS = 10, PT_SAMPLE_SELECT = 1, PT_ADD_EMIT = 2, PT_DENSE_SELECT = 3, PT_DENSE_COMPACT = 4,
                              PT_CAND_SELECT = 5, PT_CAND_COMPACT = 6, PT_FINALIZE = 7, PT_APPLY = 8, PT_FEEDBACK = 11,
                              PT_CAND_SELECT_COMPACT = 12, PT_SETUP_PREDICT = 13,
-                             PT_DENSE_HIST = 14, PT_DENSE_FIND = 15 };
+                             PT_DENSE_HIST = 14, PT_DENSE_FIND = 15, PT_DENSE_FUSED = 16 };
 void profile_mark(cudaStream_t stream, bool begin, uint32_t tag);
 struct ProfileScope {   // records an event pair around the launches made during its lifetime
   cudaStream_t stream;

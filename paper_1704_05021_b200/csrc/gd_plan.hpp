@@ -25,7 +25,9 @@ constexpr uint64_t kSampleAllMax = 8192;         // scopes up to this length are
 constexpr uint64_t kClusterMaxStride = 1024;      // strata up to this many elements wide are sampled in groups of 8
 constexpr uint64_t kAutoDenseMax = 3ull << 18;   // vectors up to this length skip the prediction (measured, step time
                                                  // with L2 flushed: dense 56 us against 58 us predicted at 2^19 elements,
-                                                 // 65 against 59 at 2^20, 83 against 63 at 2^21)
+                                                 // 65 against 59 at 2^20, 83 against 63 at 2^21) - and so do all that the
+                                                 // one-launch kernel for short vectors can hold (38 / 40 / 46 / 54 us against
+                                                 // 56 / 58 / 60 / 65 us predicted at 2^18 .. 2^21 elements)
 
 inline uint64_t kept_count(uint64_t n, uint32_t drop_ppm) {
   return n - (n * (uint64_t)drop_ppm) / 1000000ull;   // n <= 2^32, drop_ppm <= 1e6: no overflow
@@ -98,6 +100,8 @@ struct Plan {
   bool predict = true;
   bool local_predict = false;   // the prediction shares a launch with the start of the call (gd_predict.cu)
   bool dense_bound = false;     // no sample: the lower bounds come from a histogram pass over the dense vector (gd_dense.cu)
+  bool dense_fused = false;     // no sample, short vector: add, selection and compaction in one launch (gd_candidates.cu)
+  uint64_t dense_units = 0;     // the scopes' lengths in units of 1024 elements, summed
   uint32_t emit_chunk_tiles = 1, dense_sel_tile = kDenseSelTileMax, dense_chunk_tiles = kDenseChunkTilesMax;
   uint32_t samp_tile = kTile;
   // workspace layout (byte offsets)
@@ -123,7 +127,7 @@ inline int check_offsets(const uint64_t* off, uint32_t count, uint64_t* n_out) {
 
 // layer_cols == NULL: one (mu+, mu-) pair per layer.
 inline int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_t* layer_cols, uint32_t n_shards, int scope_mode,
-              uint32_t drop_ppm, uint32_t flags, Plan* P) {
+              uint32_t drop_ppm, uint32_t flags, Plan* P, uint64_t fused_units = 0) {
   uint64_t n = 0;
   int rc = check_offsets(layer_off, n_layers, &n);
   if (rc != GD_OK) return rc;
@@ -131,16 +135,24 @@ inline int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_
   if (scope_mode != GD_SCOPE_GLOBAL && scope_mode != GD_SCOPE_PER_LAYER) return GD_ERR_INVALID_ARG;
   if (n > (1ull << 32)) return GD_ERR_TOO_LARGE;
   const bool sampled = (flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
+  const uint32_t ns_planned = scope_mode == GD_SCOPE_GLOBAL ? 1u : n_layers;
+  // fused_units: how many units of 1024 elements the one-launch kernel for short vectors holds on this device (0: not
+  // available).  A scope's last unit may be partial.
+  uint64_t units = 0;
+  if (scope_mode == GD_SCOPE_GLOBAL) units = (n + 1023) / 1024;
+  else for (uint32_t l = 0; l < n_layers; ++l) units += (layer_off[l + 1] - layer_off[l] + 1023) / 1024;
+  P->dense_units = units;
+  const bool fused_fits = ns_planned <= kSmemScopes && units <= fused_units;
   // Short vectors are selected densely right away: below about 2^20 elements the three dense passes
   // run out of L2 and cost less than sampling, predicting and selecting among candidates.
-  const bool predict = !(flags & GD_FLAG_NO_PREDICTION) && (sampled || n > kAutoDenseMax);
+  const bool predict = !(flags & GD_FLAG_NO_PREDICTION) && (sampled || (flags & GD_FLAG_PREDICT_ALWAYS) || (!fused_fits && n > kAutoDenseMax));
   P->predict = predict;
+  P->dense_fused = !predict && fused_fits;
   // Without a sample, long vectors still go through the candidate lists: one histogram pass over the dense vector
   // gives every scope an exact lower bound of its threshold (gd_dense.cu).  Short vectors, whose passes run out
   // of L2, and calls with more scopes than the kernels over the lists keep in shared memory take the plain dense
   // selection and compaction.
-  const uint32_t ns_planned = scope_mode == GD_SCOPE_GLOBAL ? 1u : n_layers;
-  P->dense_bound = !predict && !sampled && n > kAutoDenseMax && ns_planned <= kSmemScopes;
+  P->dense_bound = !predict && !P->dense_fused && n > kAutoDenseMax && ns_planned <= kSmemScopes;
   P->pair_off.assign((size_t)n_layers + 1, 0);
   P->layer_cols.assign(n_layers, 1);
   for (uint32_t l = 0; l < n_layers; ++l) {

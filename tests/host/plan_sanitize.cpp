@@ -22,12 +22,12 @@ using namespace gd;
 static uint64_t kept(uint64_t n, uint32_t ppm) { return n - n * ppm / 1000000ull; }
 
 static int check(const std::vector<uint64_t>& sizes, uint32_t n_shards, int scope_mode, uint32_t ppm, uint32_t flags,
-                 const uint32_t* cols) {
+                 const uint32_t* cols, uint64_t fused_units = 0) {
   std::vector<uint64_t> off(sizes.size() + 1, 0);
   for (size_t i = 0; i < sizes.size(); ++i) off[i + 1] = off[i] + sizes[i];
   const uint64_t n = off.back();
   Plan P;
-  const int rc = make_plan(off.data(), (uint32_t)sizes.size(), cols, n_shards, scope_mode, ppm, flags, &P);
+  const int rc = make_plan(off.data(), (uint32_t)sizes.size(), cols, n_shards, scope_mode, ppm, flags, &P, fused_units);
   if (n > (1ull << 32)) { REQUIRE(rc == GD_ERR_TOO_LARGE); return 0; }
   REQUIRE(rc == GD_OK);
   const uint32_t ns = scope_mode == GD_SCOPE_GLOBAL ? 1u : (uint32_t)sizes.size();
@@ -79,7 +79,15 @@ static int check(const std::vector<uint64_t>& sizes, uint32_t n_shards, int scop
     for (uint32_t s = 0; s < ns; ++s) REQUIRE(P.scopes[s].samp_m <= kLocalSampleMax);
     REQUIRE(P.samp_tile == 256 || P.samp_tile == 512 || P.samp_tile == 1024);
   }
-  if (P.dense_bound) REQUIRE(!P.predict && ns <= kSmemScopes);
+  if (P.dense_bound) REQUIRE(!P.predict && !P.dense_fused && ns <= kSmemScopes);
+  uint64_t units = 0;
+  for (uint32_t s = 0; s < ns; ++s) units += (P.scopes[s].hi - P.scopes[s].lo + 1023) / 1024;
+  REQUIRE(P.dense_units == units);
+  if (P.dense_fused) REQUIRE(!P.predict && ns <= kSmemScopes && units <= fused_units);
+  if (flags & GD_FLAG_PREDICT_ALWAYS) REQUIRE(P.predict && !P.dense_fused && !P.dense_bound);
+  if (flags & GD_FLAG_NO_PREDICTION) REQUIRE(!P.predict);
+  if (fused_units >= units && ns <= kSmemScopes && !(flags & (GD_FLAG_SAMPLED_THRESHOLD | GD_FLAG_PREDICT_ALWAYS)))
+    REQUIRE(P.dense_fused);
   return 1;
 }
 
@@ -105,6 +113,12 @@ int main() {
       for (uint32_t ppm : {0u, 300000u, 900000u, 990000u, 999000u, 999999u, 1000000u})
         for (uint32_t flags : {0u, (uint32_t)GD_FLAG_NO_PREDICTION, (uint32_t)GD_FLAG_SAMPLED_THRESHOLD, (uint32_t)GD_FLAG_NO_EARLY_ZERO})
           for (uint32_t shards : {1u, 4u, 33u}) plans += check(sizes, shards, scope, ppm, flags, nullptr);
+  // with the one-launch kernel for short vectors on offer (a small and a large device), and prediction forced
+  for (const auto& sizes : layouts)
+    for (int scope : {GD_SCOPE_GLOBAL, GD_SCOPE_PER_LAYER})
+      for (uint32_t flags : {0u, (uint32_t)GD_FLAG_NO_PREDICTION, (uint32_t)GD_FLAG_SAMPLED_THRESHOLD, (uint32_t)GD_FLAG_PREDICT_ALWAYS})
+        for (uint64_t fused_units : {(uint64_t)1, (uint64_t)296, (uint64_t)2368, ~(uint64_t)0})
+          plans += check(sizes, 3, scope, 990000u, flags, nullptr, fused_units);
   // hundreds of layers of random sizes (the tables no longer fit a kernel argument), with and without columns
   std::mt19937_64 rng(7);
   for (int rep = 0; rep < 40; ++rep) {

@@ -93,10 +93,12 @@ def _one_step(sess, g, views):
     assert sess.status() == B.GD_OK
 
 
-@pytest.mark.parametrize("path", ["predicted", "dense"])
+@pytest.mark.parametrize("path", ["predicted", "dense", "dense_short_vector"])
 def test_profile_pairs_and_launch_count(cuda_device, path):
     """Every kernel of a step is one launch and, with the hooks on, one tagged event pair, in launch order."""
     w = _layout(B.GD_VALUES_FP32)
+    if path == "dense_short_vector":                             # what one launch of the dense kernel holds
+        w = W.small_layered(4, [700_000, 13, 300_003, 4096], 990_000, B.GD_SCOPE_PER_LAYER, B.GD_VALUES_FP32, 3)
     flags = B.GD_FLAG_NO_PREDICTION if path == "dense" else 0
     sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, flags, cuda_device)
     params = torch.zeros(w.n, device=cuda_device)
@@ -126,7 +128,7 @@ def test_profile_pairs_and_launch_count(cuda_device, path):
         B.gd_profile_enable(1)                                   # the fused full pass only
         _one_step(sess, g, views)
         pairs = B.gd_profile_collect(with_tags=True)
-        assert [t for t, _ in pairs] == ["add_emit"]
+        assert [t for t, _ in pairs] == ["dense_fused" if path == "dense_short_vector" else "add_emit"]
         # the fused pass streams 12 bytes per element: its duration must be consistent with the device
         assert pairs[0][1] > 12.0 * w.n / 20e12 * 1e3            # not faster than 20 TB/s
     finally:

@@ -97,9 +97,12 @@ def run_steps(w, device, steps, flags=0, method="sort", grads=None, alpha=1.0, w
 
 
 # ---------------------------------------------------------------- workload 1: 2^20 flat, 5 steps
-@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
+@pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION, B.GD_FLAG_PREDICT_ALWAYS,
+                                   B.GD_FLAG_PREDICT_ALWAYS | B.GD_FLAG_PLAIN_RADIX])
 def test_config1_five_steps(cuda_device, flags):
-    run_steps(W.workload(1), cuda_device, 5, flags=flags, expect_dense=bool(flags & B.GD_FLAG_NO_PREDICTION))
+    """Short enough for the one-launch dense kernel, which is the default here; with GD_FLAG_PREDICT_ALWAYS through the
+    sample, the fused pass and the lists."""
+    run_steps(W.workload(1), cuda_device, 5, flags=flags, expect_dense=not flags & B.GD_FLAG_PREDICT_ALWAYS)
 
 
 @pytest.mark.parametrize("flags", [0, B.GD_FLAG_NO_PREDICTION])
@@ -1134,7 +1137,7 @@ def test_random_layouts_and_modes(cuda_device, seed):
     ppm = int(rng.choice([0, 300_000, 900_000, 984_000, 990_000, 999_000, 999_999, 1_000_000]))
     scope_mode = int(rng.integers(0, 2))
     value_mode = int(rng.choice([B.GD_VALUES_FP32, B.GD_VALUES_TWO_MEANS, B.GD_VALUES_THRESHOLD, B.GD_VALUES_COLUMN_MEANS]))
-    flags = int(rng.choice([0, 0, B.GD_FLAG_NO_PREDICTION]))
+    flags = int(rng.choice([0, B.GD_FLAG_PREDICT_ALWAYS, B.GD_FLAG_NO_PREDICTION]))
     shards = int(rng.integers(1, 7))
     cols = None
     if value_mode == B.GD_VALUES_COLUMN_MEANS:
@@ -1156,8 +1159,8 @@ def test_random_layouts_and_modes(cuda_device, seed):
             g = rng.choice(np.array([0.0, 0.25, -0.25, 0.5, 1.0, -2.0]), w.n)           # few distinct values
         grads.append(torch.from_numpy(g.astype(np.float32)))
     alpha = float(rng.choice([1.0, 0.5, -1.25]))
-    if flags == 0 and rng.random() < 0.3:
-        flags = B.GD_FLAG_NO_EARLY_ZERO
+    if not flags & B.GD_FLAG_NO_PREDICTION and rng.random() < 0.3:
+        flags |= B.GD_FLAG_NO_EARLY_ZERO
     if value_mode == B.GD_VALUES_THRESHOLD and rng.random() < 0.5:
         flags |= B.GD_FLAG_QUANT_ERROR_FEEDBACK      # the +-tau table is exact, so the fed-back residual is too
     run_steps(w, cuda_device, 3, flags=flags, grads=grads, layer_cols=cols, alpha=alpha)
@@ -1181,6 +1184,8 @@ def test_random_models_of_few_large_tensors(cuda_device, seed):
         flags |= B.GD_FLAG_QUANT_ERROR_FEEDBACK
     if seed % 2 == 1 and not flags & B.GD_FLAG_NO_PREDICTION:
         flags |= B.GD_FLAG_PLAIN_RADIX                # the selection's three plain radix passes instead of its short cut
+    if not flags & B.GD_FLAG_NO_PREDICTION:
+        flags |= B.GD_FLAG_PREDICT_ALWAYS             # (the models short enough for the one-launch dense kernel too)
     cols = None
     if value_mode == B.GD_VALUES_COLUMN_MEANS:
         cols = []
