@@ -169,6 +169,9 @@ inline int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_
   const uint64_t dense_tiles = (n + kTile - 1) / kTile;
   uint32_t chunk_tiles = 8;
   while (chunk_tiles > 1 && dense_tiles < (uint64_t)chunk_tiles * 888u) chunk_tiles >>= 1;
+#ifdef GD_FORCE_CHUNK
+  chunk_tiles = GD_FORCE_CHUNK;
+#endif
   P->emit_chunk_tiles = chunk_tiles;
   const uint64_t CH = (uint64_t)chunk_tiles * kTile;
   // The dense kernels (used when a prediction fails) take large tiles on long vectors, where the
