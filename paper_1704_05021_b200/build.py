@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(PKG_DIR, "libgd.so")
-SOURCES = ["gd_emit.cu", "gd_select.cu", "gd_compact.cu", "gd_candidates.cu", "gd_predict.cu", "gd_dense.cu", "gd_apply.cu", "gd_api.cu"]
+SOURCES = ["gd_emit.cu", "gd_emit_pipe.cu", "gd_select.cu", "gd_compact.cu", "gd_candidates.cu", "gd_predict.cu", "gd_dense.cu", "gd_apply.cu", "gd_api.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",

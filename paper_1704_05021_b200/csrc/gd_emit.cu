@@ -296,6 +296,14 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
 cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
   if (!tiles[L_EMIT]) return cudaSuccess;
   ProfileScope prof(stream, PT_ADD_EMIT);
+#ifndef GD_NO_EMIT_PIPE
+  if (add_emit_pipe_takes(T)) {
+    cudaError_t e = launch_add_emit_pipe(T, tiles, stream);
+    if (e != cudaSuccess) return e;
+    note_launches(1);
+    return cudaSuccess;
+  }
+#endif
   switch (T.emit_chunk_tiles) {
     case 1: add_emit_kernel<1><<<tiles[L_EMIT], kEmitThreads, 0, stream>>>(T); break;
     case 2: add_emit_kernel<2><<<tiles[L_EMIT], kEmitThreads, 0, stream>>>(T); break;

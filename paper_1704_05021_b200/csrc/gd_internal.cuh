@@ -236,6 +236,8 @@ cudaError_t launch_feedback(const DevTables& T, cudaStream_t stream);
 cudaError_t launch_pack_sampled(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uint64_t cand_total, cudaStream_t stream);
 cudaError_t launch_dense_bound(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
+bool add_emit_pipe_takes(const DevTables& T);        // the pipelined fused pass (gd_emit_pipe.cu) can take the call
+cudaError_t launch_add_emit_pipe(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_dense_fused(const DevTables& T, uint64_t dense_units, cudaStream_t stream);
 uint64_t dense_fused_capacity();   // how many 1024-element units launch_dense_fused takes on the current device (0: none)
 cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream);

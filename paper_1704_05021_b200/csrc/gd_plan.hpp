@@ -163,12 +163,15 @@ inline int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_
     P->pair_off[l + 1] = P->pair_off[l] + cols;
   }
   P->n_pairs = P->pair_off[n_layers];
-  // The fused pass gives each CTA a chunk of 1, 2, 4 or 8 tiles: as large as still leaves a wave and a
-  // half of CTAs (4 per SM on 148 SMs) for the whole vector.  (Measured on 2^21 .. 2^26 elements: four
-  // waves, the first rule, cost 20-30 % more time at 2^23 .. 2^25; one wave loses to the tail.)
+  // The fused pass works in chunks of 1, 2, 4 or 8 tiles.  One CTA per chunk (more than 32 scopes, gd_emit.cu): as
+  // large as still leaves a wave and a half of CTAs (4 per SM on 148 SMs) for the whole vector.  (Measured on
+  // 2^21 .. 2^26 elements: four waves, the first rule, cost 20-30 % more time at 2^23 .. 2^25; one wave loses to the
+  // tail.)  The persistent pipeline (gd_emit_pipe.cu) hides a chunk's start-up and look-back, so its chunks are
+  // smaller - the last ones end closer together - but not so small that the look-back, two chunks deep, falls behind.
   const uint64_t dense_tiles = (n + kTile - 1) / kTile;
-  uint32_t chunk_tiles = 8;
-  while (chunk_tiles > 1 && dense_tiles < (uint64_t)chunk_tiles * 888u) chunk_tiles >>= 1;
+  uint32_t chunk_tiles = ns_planned <= kSmemScopes ? 4 : 8;
+  const uint64_t per_size = ns_planned <= kSmemScopes ? 296u : 888u;
+  while (chunk_tiles > 1 && dense_tiles < (uint64_t)chunk_tiles * per_size) chunk_tiles >>= 1;
 #ifdef GD_FORCE_CHUNK
   chunk_tiles = GD_FORCE_CHUNK;
 #endif

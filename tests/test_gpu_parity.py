@@ -1120,6 +1120,24 @@ def test_quantisation_error_feedback_needs_a_one_bit_mode(cuda_device):
         sess.compress(torch.zeros(w.n, device=cuda_device))
 
 
+@pytest.mark.parametrize("which", ["grad", "residual"])
+def test_vectors_must_be_aligned_to_16_bytes(cuda_device, which):
+    """The kernels read and write 128 bits at a time (and the fused pass copies whole tiles in bulk): a gradient or
+    residual that starts off a 16-byte boundary is refused, with nothing launched."""
+    w = W.small_layered(2, [300_000, 17], 990_000, B.GD_SCOPE_PER_LAYER, B.GD_VALUES_FP32, 1)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
+    buf = torch.zeros(w.n + 8, dtype=torch.float32, device=cuda_device)
+    g = torch.zeros(w.n, dtype=torch.float32, device=cuda_device)
+    if which == "grad":
+        g = buf[1:1 + w.n]
+    else:
+        sess.residual = buf[1:1 + w.n]                       # before the first call: the argument block is built then
+    before = B.gd_launch_count()
+    with pytest.raises(B.GdError):
+        sess.compress(g)
+    assert B.gd_launch_count() == before
+
+
 # ---------------------------------------------------------------- randomised layouts
 @pytest.mark.parametrize("seed", range(12))
 def test_random_layouts_and_modes(cuda_device, seed):
