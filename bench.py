@@ -539,7 +539,7 @@ def run_cuda(args):
     fused_avg_ms = sum(fused_ms) / len(fused_ms) if fused_ms else None
     cand_per_call = stats["n_candidates"]
     fused_bytes = 12.0 * w.n + 8.0 * cand_per_call         # read g, read r, write r; candidates written
-    roofline = {"bound": "hbm", "kernel": "add_emit_kernel", "achieved": None, "peak": peak, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": "add_emit_pipe_kernel", "achieved": None, "peak": peak, "unit": "GB/s",
                 "frac": None, "traffic": None, "peak_kind": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch": fused_bytes, "launches_timed": len(fused_ms)}
     if fused_avg_ms:

@@ -81,6 +81,7 @@ struct PipeSmem {
   ChunkMeta cmeta[kBufs];
   uint64_t excl[kBufs];                              // candidates of the scope before the chunk
   uint32_t total[kBufs];                             // candidates of the chunk
+  uint32_t tau_lo[kSmemScopes], zmin[kSmemScopes];   // per scope: candidates are keys >= tau_lo, cleared early keys >= zmin
   int abort;
   SmemTables tab;
 };
@@ -386,6 +387,25 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
   const uint32_t* tile0;
   if (tid == 0) GD_PSTAMP(0);
   load_tables(T, L_EMIT, &sm.tab, &scopes, &tile0);           // (at most kSmemScopes scopes: the launcher checks)
+  if (warp == (uint32_t)kScanWarp && lane < T.n_scopes) {
+    // Every scope's thresholds, fetched once, along with the tables.  Zeros are never candidates: when the
+    // prediction is 0 the list holds the non-zero entries, and if there are fewer than k of them the threshold is 0
+    // and the zeros that are kept are found by the dense compaction.  Entries with key >= zmin (above tau_hi, the
+    // sample's estimate of the threshold itself) are almost surely kept: their residual slot gets +0 in the streaming
+    // store.  Each is a candidate, so its value is in the list, from which the compaction puts it back should it not
+    // be kept after all.  In sampled-threshold mode tau_lo is the threshold itself and every candidate is kept.
+    const bool sampled = (T.flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
+    const uint32_t s = lane;
+    uint32_t tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || T.scopes[s].k == 0) ? 0xFFFFFFFFu : T.state[s].tau_lo;
+    if (tau_lo == 0u && !sampled) tau_lo = 1u;
+    uint32_t zmin = 0xFFFFFFFFu;
+    if (tau_lo != 0xFFFFFFFFu) {
+      if (sampled) { if (!(T.flags & GD_FLAG_NO_EARLY_ZERO)) zmin = tau_lo; }
+      else if (early_zero_enabled(T)) zmin = T.state[s].tau_hi + 1u;
+    }
+    sm.tau_lo[s] = tau_lo;
+    sm.zmin[s] = zmin;
+  }
   if (tid == 0) {
     for (int st = 0; st < kStages; ++st) {
       mbar_init(&sm.full[st], 1u);                            // the producer's arrive (+ the bytes of its two copies)
@@ -410,34 +430,19 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
   if (warp == (uint32_t)kProducerWarp) {
     // ------------------------------------------------------------ producer
     if (lane != 0) return;
-    const bool sampled = (T.flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;   // tau_lo is the threshold itself: keep key >= tau_lo
     int stage = 0;
     uint32_t parity = 1;                   // (a fresh mbarrier reads as "the phase of parity 1 has completed")
     uint32_t armed = 0, armed_parity = 0;  // stages used, and the parity of the latest phase of each one's full barrier
-    uint32_t cached_s = 0xFFFFFFFFu, tau_lo = 0xFFFFFFFFu, zmin = 0xFFFFFFFFu;
     bool ok = true;
-    uint32_t t_next = atomicAdd(&T.ctl->ticket[L_EMIT], 1u);
+    // the CTAs' first chunks are theirs by number; the ticket counter hands out the rest
+    uint32_t t_next = blockIdx.x;
     while (ok) {
       const uint32_t t = t_next;
       if (t >= total_chunks) break;
-      t_next = atomicAdd(&T.ctl->ticket[L_EMIT], 1u);         // (in flight while this chunk's copies are issued)
+      t_next = gridDim.x + atomicAdd(&T.ctl->ticket[L_EMIT], 1u);   // (in flight while this chunk's copies are issued)
       const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
       const ScopeDesc& d = scopes[s];
-      if (s != cached_s) {
-        // Zeros are never candidates: when the prediction is 0 the list holds the non-zero entries, and if there
-        // are fewer than k of them the threshold is 0 and the zeros that are kept are found by the dense compaction.
-        tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || d.k == 0) ? 0xFFFFFFFFu : T.state[s].tau_lo;
-        if (tau_lo == 0u && !sampled) tau_lo = 1u;
-        // Entries with key >= zmin (above tau_hi, the sample's estimate of the threshold itself) are almost surely
-        // kept: their residual slot gets +0 in the streaming store.  Each is a candidate, so its value is in the
-        // list, from which the compaction puts it back should it not be kept after all.
-        zmin = 0xFFFFFFFFu;
-        if (tau_lo != 0xFFFFFFFFu) {
-          if (sampled) { if (!(T.flags & GD_FLAG_NO_EARLY_ZERO)) zmin = tau_lo; }
-          else if (early_zero_enabled(T)) zmin = T.state[s].tau_hi + 1u;
-        }
-        cached_s = s;
-      }
+      const uint32_t tau_lo = sm.tau_lo[s], zmin = sm.zmin[s];
       const uint64_t lo = d.lo, hi = d.hi;
       const uint64_t cbase = (lo / CH + (t - tile0[s])) * CH;
       // the chunk's tiles that overlap the scope are consecutive
