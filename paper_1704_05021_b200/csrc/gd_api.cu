@@ -22,6 +22,8 @@ namespace {
 
 __global__ void __launch_bounds__(kThreads) setup_kernel(const __grid_constant__ SetupBlob blob, uint4* tables_dst,
                                                          uint32_t tables_vec, uint4* zero_dst, uint64_t zero_vec) {
+  pdl_trigger();
+  pdl_wait();      // (may have been brought onto the GPU early: see launch_dependent)
   const uint64_t stride = (uint64_t)gridDim.x * kThreads;
   const uint64_t g = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
   for (uint64_t i = g; i < zero_vec; i += stride) zero_dst[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -160,8 +162,9 @@ cudaError_t launch_setup(void* tables_dst, const void* tables_src, size_t tables
   SetupBlob blob;
   const size_t first = tables_bytes <= kSetupBlobBytes ? tables_bytes : (src_is_pinned ? 0 : kSetupBlobBytes);
   std::memcpy(blob.bytes, tables_src, first);
-  setup_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(blob, (uint4*)tables_dst, (uint32_t)(first / 16), (uint4*)zero_dst,
-                                                         zero_vec);
+  const cudaError_t le = launch_dependent(setup_kernel, dim3((unsigned)blocks), dim3(kThreads), 0, stream, blob, (uint4*)tables_dst,
+                                          (uint32_t)(first / 16), (uint4*)zero_dst, zero_vec);
+  if (le != cudaSuccess) return le;
   GD_LAUNCH_CHECK();
   if (first == tables_bytes) return cudaSuccess;
   if (src_is_pinned) return cudaMemcpyAsync(tables_dst, tables_src, tables_bytes, cudaMemcpyHostToDevice, stream);

@@ -52,6 +52,8 @@ __global__ void __launch_bounds__(kThreads) apply_kernel(const __grid_constant__
   const uint64_t* layer_off = INLINE ? I.layer_off : A.layer_off;
   const uint64_t* pair_off = INLINE ? I.pair_off : A.pair_off;
   const uint32_t* layer_cols = INLINE ? I.layer_cols : A.layer_cols;
+  pdl_trigger();   // (the start of the next call may be brought onto the GPU behind this kernel)
+  pdl_wait();      // nothing of the kernels before this one - the push, parameters another push has just updated - is read above
   const uint64_t begin = A.cnt_off[0], end = A.cnt_off[A.n_shards];
   const uint64_t lo_all = shard_off[0], hi_all = shard_off[A.n_shards];
   // Each thread takes kBatch entries at a time, a grid-stride apart, and has all their loads in flight before the
@@ -272,11 +274,9 @@ int gd_decompress_apply(const gd_apply_args* a, void* stream_v) {
       A.cnt_off = p.shard_cnt_off;
       A.means = p.means;
       ProfileScope prof(stream, PT_APPLY);
-      if (use_inline)
-        apply_kernel<true><<<grid, kThreads, 0, stream>>>(A, I);
-      else
-        apply_kernel<false><<<grid, kThreads, 0, stream>>>(A, I);
-      if (cudaPeekAtLastError() != cudaSuccess) return GD_ERR_CUDA;
+      const cudaError_t le = use_inline ? launch_dependent(apply_kernel<true>, dim3(grid), dim3(kThreads), 0, stream, A, I)
+                                        : launch_dependent(apply_kernel<false>, dim3(grid), dim3(kThreads), 0, stream, A, I);
+      if (le != cudaSuccess || cudaPeekAtLastError() != cudaSuccess) return GD_ERR_CUDA;
       note_launches(1);
     }
     return GD_OK;

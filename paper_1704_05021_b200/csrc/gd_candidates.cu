@@ -113,6 +113,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
   const uint32_t ltm = lanemask_lt();
 
   GD_STAMP(0);
+  pdl_trigger();   // (the apply of the push, enqueued behind this kernel, may be brought onto the GPU from now on)
   if (T.ctl->status != GD_OK) return;               // set only by an earlier kernel of this call: uniform over the grid
   if (!DENSE_IN && dense_sel_tiles != 0u && T.ctl->dense_needed != 0u) {
     if (!dense_takeover(T, dense_sel_tiles, dense_chunks, smem_raw)) return;

@@ -105,6 +105,7 @@ __global__ void __launch_bounds__(kThreads) dense_find_kernel(const __grid_const
   __shared__ unsigned long long s_part[kWarps];
   __shared__ int s_valid;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  pdl_trigger();   // (the fused pass is enqueued behind the second walk)
   if (FULL && T.ctl->hist_redo == 0u) return;
   const uint32_t s = blockIdx.x;
   const ScopeDesc& d = T.scopes[s];

@@ -385,6 +385,21 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const ScopeDesc* scopes;
   const uint32_t* tile0;
+  if (tid == 0) {
+    for (int st = 0; st < kStages; ++st) {
+      mbar_init(&sm.full[st], 1u);                            // the producer's arrive (+ the bytes of its two copies)
+      mbar_init(&sm.empty[st], (uint32_t)kConsumerWarps);
+    }
+    for (int b = 0; b < kBufs; ++b) {
+      mbar_init(&sm.chunk_done[b], (uint32_t)kConsumerWarps);
+      mbar_init(&sm.counted[b], 1u);
+      mbar_init(&sm.prefix_ready[b], 1u);
+    }
+    sm.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  pdl_wait();   // nothing the kernels before this one wrote - tables, thresholds, the residual - is read above this line
   if (tid == 0) GD_PSTAMP(0);
   load_tables(T, L_EMIT, &sm.tab, &scopes, &tile0);           // (at most kSmemScopes scopes: the launcher checks)
   if (warp == (uint32_t)kScanWarp && lane < T.n_scopes) {
@@ -405,20 +420,6 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
     }
     sm.tau_lo[s] = tau_lo;
     sm.zmin[s] = zmin;
-  }
-  if (tid == 0) {
-    for (int st = 0; st < kStages; ++st) {
-      mbar_init(&sm.full[st], 1u);                            // the producer's arrive (+ the bytes of its two copies)
-      mbar_init(&sm.empty[st], (uint32_t)kConsumerWarps);
-    }
-    for (int b = 0; b < kBufs; ++b) {
-      mbar_init(&sm.chunk_done[b], (uint32_t)kConsumerWarps);
-      mbar_init(&sm.counted[b], 1u);
-      mbar_init(&sm.prefix_ready[b], 1u);
-    }
-    sm.abort = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
   const volatile int* abort = &sm.abort;
@@ -683,8 +684,8 @@ cudaError_t launch_add_emit_pipe(const DevTables& T, const uint32_t* tiles, cuda
   }
   uint32_t grid = (uint32_t)sm_count();
   if (grid > tiles[L_EMIT]) grid = tiles[L_EMIT];
-  add_emit_pipe_kernel<<<grid, kPipeThreads, smem, stream>>>(T, tiles[L_EMIT]);
-  return cudaGetLastError();
+  const cudaError_t e = launch_dependent(add_emit_pipe_kernel, dim3(grid), dim3(kPipeThreads), smem, stream, T, tiles[L_EMIT]);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace gd

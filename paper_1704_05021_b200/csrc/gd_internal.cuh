@@ -3,6 +3,7 @@
 #pragma once
 
 #include <atomic>
+#include <utility>
 
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -62,6 +63,31 @@ struct DevTables {       // passed by value to every kernel
   uint32_t* out_tau;
   float* out_means;
 };
+
+// ---------------------------------------------------------------- programmatic dependent launches
+// A kernel launched with launch_dependent() may be brought onto the GPU while the kernel before it in the stream is
+// still running - from the moment all CTAs of that kernel have called pdl_trigger() (or ended) - so that its launch
+// latency is spent then and not after.  It must call pdl_wait() before it reads or writes anything the earlier
+// kernels of the stream touch: that returns when the kernel before it has completed and its writes are visible.
+// Where the kernel before it does not trigger, or is no kernel at all, the launch is an ordinary one.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // ---------------------------------------------------------------- device helpers
 __device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31u; }

@@ -75,6 +75,8 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
   __shared__ int s_is_last;
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   const ScopeDesc* scopes = reinterpret_cast<const ScopeDesc*>(blob.bytes + scopes_off);
+  pdl_trigger();   // the fused pass, enqueued behind this kernel, may be brought onto the GPU from now on
+  pdl_wait();      // (this kernel itself may have been: nothing is read or written before the stream's earlier kernels are done)
 
   if (blockIdx.x >= gather_ctas) {
     // ---- the start of the call: clear the control region (the scope states are cleared by the CTAs that fill them
@@ -229,9 +231,10 @@ cudaError_t launch_setup_predict(const DevTables& T, uint32_t gather_ctas, uint3
   if (zero_ctas < 1) zero_ctas = 1;
   const uint64_t state_beg = state_off / 16;
   const uint64_t state_end = (state_off + sizeof(ScopeState) * (size_t)T.n_scopes + 15) / 16;
-  setup_predict_kernel<<<(unsigned)(gather_ctas + zero_ctas), kPredictThreads, 0, stream>>>(
-      T, blob, gather_ctas, gather_tile, call, flags, (uint4*)tables_dst, (uint32_t)(tables_bytes / 16), (uint4*)zero_dst, zero_vec, state_beg,
-      state_end, (uint32_t)scopes_off, (uint32_t)tile0_off);
+  const cudaError_t le = launch_dependent(setup_predict_kernel, dim3((unsigned)(gather_ctas + zero_ctas)), dim3(kPredictThreads), 0, stream,
+                                          T, blob, gather_ctas, gather_tile, call, flags, (uint4*)tables_dst, (uint32_t)(tables_bytes / 16),
+                                          (uint4*)zero_dst, zero_vec, state_beg, state_end, (uint32_t)scopes_off, (uint32_t)tile0_off);
+  if (le != cudaSuccess) return le;
   GD_LAUNCH_CHECK();
   return cudaSuccess;
 }

@@ -23,6 +23,7 @@ template <int VIEW, bool MANY>
 __global__ void __launch_bounds__(kThreads, (MANY && VIEW != V_DENSE) ? 2 : 4) select_kernel(const __grid_constant__ DevTables T, uint32_t total_tiles,
                                                                                              uint32_t dense_tiles) {
   __shared__ SelectSmem<VIEW, MANY> S;
+  pdl_trigger();   // (the fused pass, enqueued behind the selection on the sample, may be brought onto the GPU from now on)
   if (VIEW == V_CAND) {
     // (the dense selection borrows this selection's shared memory, which is large enough: asserted below)
     if (dense_tiles != 0u && T.ctl->dense_needed != 0u)
