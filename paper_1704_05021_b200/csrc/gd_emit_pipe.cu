@@ -435,12 +435,13 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
     uint32_t parity = 1;                   // (a fresh mbarrier reads as "the phase of parity 1 has completed")
     uint32_t armed = 0, armed_parity = 0;  // stages used, and the parity of the latest phase of each one's full barrier
     bool ok = true;
-    // the CTAs' first chunks are theirs by number; the ticket counter hands out the rest
-    uint32_t t_next = blockIdx.x;
+    // Chunks are handed out by a ticket counter, the first ones too: a chunk that another CTA's look-back waits for
+    // is then always held by a CTA that is running, however many of the grid's CTAs are resident at once.
+    uint32_t t_next = atomicAdd(&T.ctl->ticket[L_EMIT], 1u);
     while (ok) {
       const uint32_t t = t_next;
       if (t >= total_chunks) break;
-      t_next = gridDim.x + atomicAdd(&T.ctl->ticket[L_EMIT], 1u);   // (in flight while this chunk's copies are issued)
+      t_next = atomicAdd(&T.ctl->ticket[L_EMIT], 1u);         // (in flight while this chunk's copies are issued)
       const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
       const ScopeDesc& d = scopes[s];
       const uint32_t tau_lo = sm.tau_lo[s], zmin = sm.zmin[s];

@@ -456,7 +456,8 @@ def test_many_layers_on_the_predicted_path(cuda_device, scope_mode, value_mode):
 
 
 # ---------------------------------------------------------------- guard words around every buffer
-@pytest.mark.parametrize("case", ["predicted_fp32", "predicted_two_means", "dense_fp32", "sampled", "many_scopes"])
+@pytest.mark.parametrize("case", ["predicted_fp32", "predicted_two_means", "dense_fp32", "dense_one_launch", "sampled",
+                                  "many_scopes"])
 def test_nothing_is_written_outside_the_buffers(cuda_device, case):
     """Every buffer the library writes (residual, outputs, workspace, parameters) sits between guard words; the guards
     must be intact after compress + apply and the outputs must equal the oracle's.  Buffers have exactly the sizes the
@@ -464,9 +465,11 @@ def test_nothing_is_written_outside_the_buffers(cuda_device, case):
     rng = np.random.default_rng(5150)
     G = 1024                                                       # guard elements on either side
     value_mode, flags, scope = B.GD_VALUES_FP32, 0, B.GD_SCOPE_PER_LAYER
-    sizes = [1_300_000, 9, 4097, 1_000_003]
-    if case == "predicted_two_means":
-        value_mode = B.GD_VALUES_TWO_MEANS
+    sizes = [1_300_000, 9, 4097, 1_000_003]                        # short enough for the one-launch dense kernel ...
+    if case == "predicted_fp32":
+        flags = B.GD_FLAG_PREDICT_ALWAYS                            # ... so the predicted path is asked for
+    elif case == "predicted_two_means":
+        value_mode, flags = B.GD_VALUES_TWO_MEANS, B.GD_FLAG_PREDICT_ALWAYS
     elif case == "dense_fp32":
         sizes = [200_001, 9, 4097]
     elif case == "sampled":
@@ -507,6 +510,11 @@ def test_nothing_is_written_outside_the_buffers(cuda_device, case):
                           mean.view(-1, 2), ws, flags=flags)
     B.gd_compress(call)
     assert B.gd_status(ws) == B.GD_OK
+    st = B.gd_get_stats(ws)
+    if case.startswith("predicted"):
+        assert st["n_scopes_predicted"] >= 2 and st["n_scopes_dense"] == 0, st
+    elif case.startswith("dense"):
+        assert st["n_scopes_dense"] == len(sizes) and st["n_candidates"] == 0, st   # the one-launch kernel: no lists
     views = [par[w.shard_off[j]:w.shard_off[j + 1]] for j in range(w.n_shards)]
     push = {"idx": idx, "val": None if value_mode != B.GD_VALUES_FP32 else val, "shard_cnt_off": off,
             "means": mean.view(-1, 2) if value_mode != B.GD_VALUES_FP32 else None}
@@ -665,8 +673,8 @@ def test_delta_pull_matches_oracle_and_client_copy(cuda_device, flags, layout):
     rng = np.random.default_rng(23)
     # short vectors are selected densely; the long ones take the predicted path (fused subtraction, candidates,
     # slots cleared in the stream), the last one with more scopes than the kernels keep in shared memory
-    sizes = {"short": [70_000, 9, 4096, 130_003], "long_global": [1_500_000, 9, 4096, 900_003],
-             "long_per_layer": [1_500_000, 9, 4096, 900_003],
+    sizes = {"short": [70_000, 9, 4096, 130_003], "long_global": [2_500_000, 9, 4096, 900_003],
+             "long_per_layer": [2_500_000, 9, 4096, 900_003],
              "long_many": [1_200_000] + [int(x) for x in rng.integers(1, 6000, size=50)] + [1_000_000]}[layout]
     scope = B.GD_SCOPE_GLOBAL if layout in ("short", "long_global") else B.GD_SCOPE_PER_LAYER
     w = W.small_layered(len(sizes), sizes, 980_000, scope, B.GD_VALUES_FP32, 2)
@@ -682,6 +690,8 @@ def test_delta_pull_matches_oracle_and_client_copy(cuda_device, flags, layout):
         exp = orc.compress_delta(p_host, last_host, w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode)
         sess.compress_delta(p_dev, last_dev)
         compare_step(sess, exp, f"pull {step} flags {flags}")
+        if flags == 0:
+            assert (sess.stats()["n_scopes_predicted"] >= 1) == (layout != "short"), sess.stats()
         assert np.array_equal(_np_u32(last_dev), exp["last_pulled"].view(np.uint32)), f"pull {step}: last pulled copy"
         assert torch.equal(p_dev.cpu(), torch.from_numpy(p_host)), "parameters were modified"
         sess.apply(client_views, 1.0)
