@@ -1240,6 +1240,47 @@ def test_random_models_of_few_large_tensors(cuda_device, seed):
     run_steps(w, cuda_device, 2, flags=flags, grads=grads, layer_cols=cols, alpha=float(rng.choice([1.0, 0.5])))
 
 
+@pytest.mark.parametrize("case", ["boundaries_at_every_offset", "dense_rows", "tiny_between_large", "full_lists"])
+def test_pipelined_pass_edges(cuda_device, case):
+    """What the pipelined fused pass treats specially, each on a layout too long for the one-launch dense kernel:
+    scope boundaries at every offset modulo 4 inside a tile (tiles cut by a boundary are read element by element, the
+    rest in bulk), a vector whose length is no multiple of 4, runs in which most entries are candidates (a warp's
+    stash overflows and it reads its part of the chunk back), scopes shorter than a tile between long ones (chunks of a
+    single cut tile), and candidate lists that fill up (a scope of ties: the early clearing is undone, the scope is
+    selected densely).  Three steps each, residual carried, everything compared with the oracle."""
+    rng = np.random.default_rng({"boundaries_at_every_offset": 1, "dense_rows": 2, "tiny_between_large": 3,
+                                 "full_lists": 4}[case])
+    if case == "boundaries_at_every_offset":
+        sizes = [1_000_001, 500_002, 700_003, 4096 * 60 + 1, 300_007, 1_234_567 + 2]
+    elif case == "dense_rows":
+        sizes = [2_000_000, 1_500_000]
+    elif case == "tiny_between_large":
+        sizes = [1_200_000, 3, 0, 4095, 1, 1_300_000, 17, 4097, 900_000]
+    else:
+        sizes = [1_500_000, 1_000_000, 800_000]
+    w = W.small_layered(len(sizes), sizes, 990_000, B.GD_SCOPE_PER_LAYER, B.GD_VALUES_FP32, 3)
+    assert w.n > 2368 * 1024                                     # (more than the one-launch dense kernel holds)
+    grads = []
+    for step in range(3):
+        g = rng.laplace(0, 1e-3, w.n).astype(np.float32)
+        if case == "dense_rows":
+            g[:] = 0.0                                            # row-sparse: 2 % of the rows of 500 are non-zero
+            rows = rng.choice(w.n // 500, w.n // 500 // 50, replace=False)
+            for r_ in rows[:2000]:
+                g[r_ * 500:(r_ + 1) * 500] = rng.standard_normal(500).astype(np.float32) * 1e-3
+            g[100_000:160_000] = rng.standard_normal(60_000).astype(np.float32)      # and one long run far above the rest
+        elif case == "full_lists":
+            lo, hi = w.layer_off[1], w.layer_off[2]
+            g[lo:hi] = 0.25                                       # every entry of the second scope ties
+        grads.append(torch.from_numpy(g))
+    sess = run_steps(w, cuda_device, 3, grads=grads)
+    st = sess.stats()
+    if case == "full_lists":
+        assert st["n_scopes_dense"] == 1 and st["n_scopes_predicted"] == 2, st
+    else:
+        assert st["n_scopes_dense"] == 0, st
+
+
 @pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
 def test_threshold_far_above_the_prediction(cuda_device, scope_mode):
     """Magnitudes spread evenly over 120 binades: the prediction's safety margin (a multiple of the expected rank for
