@@ -352,13 +352,15 @@ int gd_profile_collect(float* ms_out, uint32_t* tags_out, uint32_t capacity, uin
 
 /*
  * Self-test of the bounded device-side waits (no counterpart in the paper).  Every wait in the
- * library's kernels - on a predecessor tile of a scan, on a grid barrier - gives up after a fixed
- * number of polls, marks its tile aborted so that nothing waits on it, and records
- * GD_ERR_DEVICE_TIMEOUT in the workspace.  This call enqueues a one-warp kernel that waits, for at
- * most spin_limit polls, on a tile nothing will ever publish, and then lets a second tile meet the
- * aborted one.  Afterwards gd_status(workspace) is GD_ERR_DEVICE_TIMEOUT and gd_get_stats reports
- * n_scopes = 1 if the first wait gave up (as it must) and n_scopes_predicted = 1 if the second tile
- * aborted without waiting.  The context stays usable.  workspace: device, 256-byte aligned, >= 512 bytes.
+ * library's kernels - on a predecessor tile of a scan, on a grid barrier, on the mbarrier of a
+ * pipeline stage - gives up after a fixed number of polls or a fixed time, marks its tile aborted so
+ * that nothing waits on it, and records GD_ERR_DEVICE_TIMEOUT in the workspace.  This call enqueues a
+ * one-warp kernel that waits, for at most spin_limit polls, on a tile nothing will ever publish, and
+ * then lets a second tile meet the aborted one; and a second one-warp kernel that waits, for at most
+ * 100 ns x spin_limit, on an mbarrier at which nothing arrives.  Afterwards gd_status(workspace) is
+ * GD_ERR_DEVICE_TIMEOUT and gd_get_stats reports n_scopes = 1 if the first wait gave up (as it must),
+ * n_scopes_predicted = 1 if the second tile aborted without waiting, and n_kept = 1 if the wait on
+ * the mbarrier gave up.  The context stays usable.  workspace: device, 256-byte aligned, >= 512 bytes.
  */
 int gd_selftest_bounded_wait(void* workspace, size_t workspace_bytes, uint32_t spin_limit, void* stream);
 

@@ -532,6 +532,8 @@ int gd_selftest_bounded_wait(void* workspace, size_t workspace_bytes, uint32_t s
   if (!workspace || ((uintptr_t)workspace & (kAlign - 1)) || workspace_bytes < 512) return GD_ERR_WORKSPACE;
   if (spin_limit == 0 || spin_limit > kLookbackSpinLimit) return GD_ERR_INVALID_ARG;
   if (launch_bounded_wait_selftest(workspace, spin_limit, (cudaStream_t)stream) != cudaSuccess) return GD_ERR_CUDA;
+  // the waits on mbarriers (the pipelined fused pass) are bounded by time: 100 ns per poll of the other limit
+  if (launch_mbar_wait_selftest(workspace, 100ull * spin_limit, (cudaStream_t)stream) != cudaSuccess) return GD_ERR_CUDA;
   return GD_OK;
 }
 

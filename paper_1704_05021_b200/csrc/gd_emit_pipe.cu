@@ -114,7 +114,8 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
 
 // Waits until the phase of parity `parity` of b has completed.  Gives up (false) when the CTA's abort flag is up or
 // after kWaitBudgetNs.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, const volatile int* abort) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, const volatile int* abort,
+                                          uint64_t budget_ns = kWaitBudgetNs) {
   uint32_t spins = 0;
   uint64_t t0 = 0;
   while (!mbar_try_wait(b, parity)) {
@@ -122,7 +123,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, const vo
     if (spins == 32u) t0 = global_timer_ns();
     if (spins > 32u && (spins & 31u) == 0u) {
       if (*abort) return false;
-      if (global_timer_ns() - t0 > kWaitBudgetNs) return false;
+      if (global_timer_ns() - t0 > budget_ns) return false;
     }
   }
   return true;
@@ -664,7 +665,31 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
   if (warp == 0) GD_PSTAMP(3);
 }
 
+// Self-test of the bounded mbarrier wait: one warp waits, for at most budget_ns, on an mbarrier at which nothing
+// arrives, records the timeout the way the pipeline does and notes that the wait gave up in the statistics' n_kept.
+__global__ void __launch_bounds__(32) mbar_wait_selftest_kernel(Ctl* ctl, uint64_t budget_ns) {
+  __shared__ alignas(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1u);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  const bool ok = mbar_wait(&bar, 0u, &abort_flag, budget_ns);
+  if (threadIdx.x == 0) {
+    if (!ok) atomicCAS(&ctl->status, (int)GD_OK, (int)GD_ERR_DEVICE_TIMEOUT);
+    ctl->n_kept = ok ? 0u : 1u;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_mbar_wait_selftest(void* workspace, uint64_t budget_ns, cudaStream_t stream) {
+  mbar_wait_selftest_kernel<<<1, 32, 0, stream>>>((Ctl*)workspace, budget_ns);
+  GD_LAUNCH_CHECK();
+  return cudaSuccess;
+}
 
 // Whether the pipelined kernel takes this call: tables that fit shared memory, 16-byte aligned vectors.
 bool add_emit_pipe_takes(const DevTables& T) {

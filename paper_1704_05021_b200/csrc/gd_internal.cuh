@@ -267,6 +267,7 @@ cudaError_t launch_add_emit_pipe(const DevTables& T, const uint32_t* tiles, cuda
 cudaError_t launch_dense_fused(const DevTables& T, uint64_t dense_units, cudaStream_t stream);
 uint64_t dense_fused_capacity();   // how many 1024-element units launch_dense_fused takes on the current device (0: none)
 cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream);
+cudaError_t launch_mbar_wait_selftest(void* workspace, uint64_t budget_ns, cudaStream_t stream);   // after the former: the workspace is prepared
 int sm_count();   // multiprocessors of the current device (148 if it cannot be asked)
 // A small per-device cache of one int (0 = not known yet), for values that belong to the device a call runs on:
 // multiprocessor counts, how many CTAs of a kernel fit on one of them.  Devices beyond kMaxDevices are not cached.

@@ -280,14 +280,18 @@ def test_config3_threshold_quantisation(cuda_device):
 
 
 def test_bounded_wait_gives_up_and_context_survives(cuda_device):
-    """A wait on a tile that nothing publishes runs out of polls, reports a timeout, and the next call works."""
+    """A wait on a tile that nothing publishes runs out of polls, one on an mbarrier at which nothing arrives runs out
+    of time; both report a timeout, and the next calls (short and long vectors) work."""
     ws = torch.zeros(4096, dtype=torch.uint8, device=cuda_device)
     B.gd_selftest_bounded_wait(ws, spin_limit=2000)
     st = B.gd_get_stats(ws)
     assert st["status"] == B.GD_ERR_DEVICE_TIMEOUT
     assert st["n_scopes"] == 1            # the first wait gave up
     assert st["n_scopes_predicted"] == 1  # the tile behind it aborted instead of waiting
+    assert st["n_kept"] == 1              # the wait on an mbarrier at which nothing arrives gave up too
     run_steps(W.workload(1), cuda_device, 1)
+    w = W.small_layered(2, [2_000_000, 900_001], 990_000, B.GD_SCOPE_PER_LAYER, B.GD_VALUES_FP32, 2)
+    run_steps(w, cuda_device, 1, grads=[torch.randn(w.n, generator=torch.Generator().manual_seed(3)) * 1e-3])
 
 
 def test_config2_no_prediction(cuda_device):
