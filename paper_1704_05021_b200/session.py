@@ -5,6 +5,7 @@ gd_decompress_apply need, and issues the calls.  No arithmetic happens here.
 """
 from __future__ import annotations
 
+import json
 from typing import List, Optional, Sequence
 
 import torch
@@ -109,3 +110,14 @@ class GradDropSession:
 
     def stats(self) -> dict:
         return B.gd_get_stats(self.workspace)
+
+    def log_step(self, fh, step: int, **extra) -> dict:
+        """Appends one JSON line about the last compress call to the open text file `fh` and returns it: the step
+        number, the call's status and counters (gd_get_stats), the survivors per shard and the scopes' threshold keys.
+        Waits for the stream (the figures are read from the device), so it is for logs, not for the timed path."""
+        off = self.out_shard_cnt_off.cpu().tolist()
+        rec = {"step": int(step), **self.stats(),
+               "kept_per_shard": [int(off[j + 1] - off[j]) for j in range(self.n_shards)],
+               "tau_keys": [int(x) & 0xFFFFFFFF for x in self.out_tau.cpu().tolist()], **extra}
+        fh.write(json.dumps(rec) + "\n")
+        return rec

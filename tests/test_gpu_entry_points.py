@@ -166,3 +166,20 @@ def test_apply_with_two_alphas_in_one_session(cuda_device):
         bound += b
     assert np.all(np.abs(got - ref) <= REL_TOL * bound + 1e-45)
     assert np.count_nonzero(got) == np.count_nonzero(ref)
+
+
+def test_per_step_metrics_log(cuda_device, tmp_path):
+    """One JSON line per step: status, counters, survivors per shard (they add up to k), threshold keys."""
+    import json
+    w = _layout(B.GD_VALUES_FP32)
+    sess = GradDropSession(w.layer_off, w.shard_off, w.drop_ppm, w.scope_mode, w.value_mode, 0, cuda_device)
+    path = tmp_path / "steps.jsonl"
+    with open(path, "w") as fh:
+        for step in range(3):
+            sess.compress(torch.randn(w.n, device=cuda_device) * 1e-3)
+            sess.log_step(fh, step, note="test")
+    recs = [json.loads(line) for line in open(path)]
+    assert [r["step"] for r in recs] == [0, 1, 2]
+    for r in recs:
+        assert r["status"] == B.GD_OK and r["n_kept"] == sess.k_total and sum(r["kept_per_shard"]) == sess.k_total
+        assert r["n_scopes"] == len(w.layer_off) - 1 and len(r["tau_keys"]) == r["n_scopes"] and r["note"] == "test"
