@@ -86,49 +86,6 @@ struct PipeSmem {
   SmemTables tab;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
-  asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"(smem_u32(b)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* b, uint32_t bytes) {
-  asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(smem_u32(b)), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* b, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok)
-               : "r"(smem_u32(b)), "r"(parity)
-               : "memory");
-  return ok != 0u;
-}
-// Global -> shared bulk copy of `bytes` (a multiple of 16; both addresses 16-byte aligned), counted on mbarrier b.
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* b) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(b))
-               : "memory");
-}
-
-// Waits until the phase of parity `parity` of b has completed.  Gives up (false) when the CTA's abort flag is up or
-// after kWaitBudgetNs.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, const volatile int* abort,
-                                          uint64_t budget_ns = kWaitBudgetNs) {
-  uint32_t spins = 0;
-  uint64_t t0 = 0;
-  while (!mbar_try_wait(b, parity)) {
-    ++spins;
-    if (spins == 32u) t0 = global_timer_ns();
-    if (spins > 32u && (spins & 31u) == 0u) {
-      if (*abort) return false;
-      if (global_timer_ns() - t0 > budget_ns) return false;
-    }
-  }
-  return true;
-}
-
 #ifdef GD_PIPE_STAMPS
 // debug: earliest and latest time over the CTAs at which point `i` was reached (slots behind the control block)
 #define GD_PSTAMP(i)                                                                                              \
