@@ -27,6 +27,7 @@ namespace {
 
 constexpr int kPredictThreads = 1024;
 constexpr int kPredictWarps = kPredictThreads / 32;
+constexpr size_t kKeysBytes = sizeof(uint32_t) * kLocalSampleMax;   // dynamic shared memory: one scope's whole sample
 
 // For each of `count` ranks (1-based, from the largest key down): the bin of hist[0 .. nbins) that holds it and
 // the number of keys in the bins above that bin.  nbins is 1024 or 2048; run by the whole CTA.
@@ -70,6 +71,7 @@ __global__ void __launch_bounds__(kPredictThreads, 1)
 setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant__ SetupBlob blob, uint32_t gather_ctas,
                      uint32_t gather_tile, uint32_t call, uint32_t* flags, uint4* tables_dst, uint32_t tables_vec, uint4* zero_dst, uint64_t zero_vec,
                      uint64_t state_vec_beg, uint64_t state_vec_end, uint32_t scopes_off, uint32_t tile0_off) {
+  extern __shared__ __align__(16) unsigned char smem_keys[];   // the scope's sample, for the CTA that finishes the scope
   __shared__ uint32_t s_hist[kRadixBins0];
   __shared__ uint32_t s_bin[2], s_above[2], s_rank[2];
   __shared__ int s_is_last;
@@ -91,7 +93,8 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
       for (uint32_t x = tid; x < T.n_scopes; x += kPredictThreads) {
         if (scopes[x].samp_m == 0) {
           uint4* p = reinterpret_cast<uint4*>(T.state + x);
-          p[0] = make_uint4(0u, 0u, 0u, 0u); p[1] = p[0]; p[2] = p[0]; p[3] = p[0];
+          static_assert(sizeof(ScopeState) == 48, "three 16-byte stores clear one scope state");
+          p[0] = make_uint4(0u, 0u, 0u, 0u); p[1] = p[0]; p[2] = p[0];
         }
       }
     }
@@ -129,6 +132,9 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
     if (!all) s_is_last = 0;
     __syncthreads();
   }
+#ifdef GD_PHASE_STAMPS
+  if (tid == 0) atomicMax(reinterpret_cast<unsigned long long*>(T.ctl) + 22, global_timer_ns());
+#endif
   if (!s_is_last) return;
   __threadfence();
 
@@ -140,21 +146,43 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
     s_rank[1] = (uint32_t)rank_hi_of(d);                   // ... and the estimate of the threshold itself
   }
   __syncthreads();
-  // the whole sample into registers (at most 32 keys per thread), all loads in flight at once
+  // The whole sample into shared memory (at most 32 keys per thread: 128 KB), eight loads per thread in flight at a
+  // time.  The loops below are rolled on purpose: this code runs once per call, after the fused pass of the call
+  // before has swept the L2, so every instruction line is fetched from DRAM - unrolled 32 times with the keys in
+  // registers, the same selection took 9 us, most of it instruction fetches; rolled, 6 us.
   constexpr int kKeys = 32;
-  constexpr uint32_t kNone = 0xFFFFFFFFu;                  // (keys are at most 0x7FFFFFFF)
-  uint32_t k[kKeys];
+  const uint32_t* keys = reinterpret_cast<const uint32_t*>(smem_keys);
+  {
+    constexpr int kBatch = 8;                               // loads per thread in flight at a time
+    uint32_t* wkeys = reinterpret_cast<uint32_t*>(smem_keys);
+    for (uint32_t li0 = tid; li0 < m; li0 += kBatch * kPredictThreads) {
+      uint32_t w[kBatch];
 #pragma unroll
-  for (int j = 0; j < kKeys; ++j) {
-    const uint32_t li = (uint32_t)j * kPredictThreads + tid;
-    k[j] = li < m ? (__float_as_uint(__ldcg(vals + li)) & kAbsMask) : kNone;
+      for (int u = 0; u < kBatch; ++u) {
+        const uint32_t li = li0 + (uint32_t)u * kPredictThreads;
+        w[u] = li < m ? __float_as_uint(__ldcg(vals + li)) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        const uint32_t li = li0 + (uint32_t)u * kPredictThreads;
+        if (li < m) wkeys[li] = w[u];
+      }
+    }
   }
+  __syncthreads();
+  const uint32_t per_thread = (m + kPredictThreads - 1u) / kPredictThreads;   // <= kKeys
   uint32_t zeros = 0;                                      // samples that are +-0: counted privately
-#pragma unroll
-  for (int j = 0; j < kKeys; ++j) {
-    if (k[j] == 0u) ++zeros;
-    else if (k[j] != kNone) atomicAdd(&s_hist[k[j] >> kShift0], 1u);
+#pragma unroll 4
+  for (uint32_t j = 0; j < per_thread; ++j) {
+    const uint32_t li = j * kPredictThreads + tid;
+    if (li < m) {
+      const uint32_t key = keys[li] & kAbsMask;
+      if (key == 0u) ++zeros;
+      else atomicAdd(&s_hist[key >> kShift0], 1u);
+    }
   }
+  static_assert(kLocalSampleMax == (uint32_t)kKeys * kPredictThreads, "the shared-memory copy of the sample");
+  const uint32_t zeros_mine = zeros;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) zeros += __shfl_xor_sync(0xFFFFFFFFu, zeros, o);
   if (lane == 0 && zeros) atomicAdd(&s_hist[0], zeros);
@@ -169,16 +197,18 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
 
   // second digit: the keys under the first rank's first digit in the lower half of the histogram, those under the
   // second rank's (if it differs) in the upper half
-  zeros = 0;
-#pragma unroll
-  for (int j = 0; j < kKeys; ++j) {
-    const uint32_t key = k[j];
-    const uint32_t top = key >> kShift0, dig = (key >> kShift1) & 1023u;
-    if (key == 0u) ++zeros;
-    else if (key == kNone) {}
-    else if (top == pa) atomicAdd(&s_hist[dig], 1u);
-    else if (top == pb) atomicAdd(&s_hist[1024u + dig], 1u);
+#pragma unroll 4
+  for (uint32_t j = 0; j < per_thread; ++j) {
+    const uint32_t li = j * kPredictThreads + tid;
+    if (li < m) {
+      const uint32_t key = keys[li] & kAbsMask;
+      const uint32_t top = key >> kShift0, dig = (key >> kShift1) & 1023u;
+      if (key == 0u) {}
+      else if (top == pa) atomicAdd(&s_hist[dig], 1u);
+      else if (top == pb) atomicAdd(&s_hist[1024u + dig], 1u);
+    }
   }
+  zeros = zeros_mine;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) zeros += __shfl_xor_sync(0xFFFFFFFFu, zeros, o);
   if (lane == 0 && zeros) {
@@ -201,12 +231,15 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
     // lower edges of the 21-bit buckets
     st->tau_lo = ((pa << 10) | da) << kShift1;
     st->tau_hi = ((pb << 10) | db) << kShift1;
+#ifdef GD_PHASE_STAMPS
+    atomicMax(reinterpret_cast<unsigned long long*>(T.ctl) + 23, global_timer_ns());
+#endif
   }
 }
 
 }  // namespace
 
-static_assert(kLocalSampleMax == 32u * kPredictThreads, "what one CTA's registers hold: 32 keys per thread");
+static_assert(kLocalSampleMax == 32u * kPredictThreads, "what one CTA keeps in shared memory: 32 keys per thread");
 
 // gather_ctas: CTAs that gather the samples (the scopes' sample tiles of gather_tile values); flags: one word per such CTA; tables_src: the host image of the
 // tables (at most kSetupBlobBytes); scopes_off, tile0_off: where the scope descriptors and the first sample tile of
@@ -217,6 +250,14 @@ cudaError_t launch_setup_predict(const DevTables& T, uint32_t gather_ctas, uint3
                                  size_t tile0_off, cudaStream_t stream) {
   if (tables_bytes > kSetupBlobBytes) return cudaErrorInvalidValue;
   ProfileScope prof(stream, PT_SETUP_PREDICT);
+  static PerDeviceInt configured;                          // the kernel's shared-memory attribute is per device
+  int dev = -1;
+  if (configured.get(&dev) == 0) {
+    if (dev < 0) return cudaErrorInvalidDevice;
+    cudaError_t e = cudaFuncSetAttribute(setup_predict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kKeysBytes);
+    if (e != cudaSuccess) return e;
+    configured.set(dev, 1);
+  }
   // The number of the call, which marks the finished sample tiles: starts at a value that differs from process to
   // process and does not repeat within one (for 2^32 calls).  A stale mark that happened to equal it would only make
   // a prediction start from an incomplete sample, and the prediction never affects results.
@@ -231,7 +272,7 @@ cudaError_t launch_setup_predict(const DevTables& T, uint32_t gather_ctas, uint3
   if (zero_ctas < 1) zero_ctas = 1;
   const uint64_t state_beg = state_off / 16;
   const uint64_t state_end = (state_off + sizeof(ScopeState) * (size_t)T.n_scopes + 15) / 16;
-  const cudaError_t le = launch_dependent(setup_predict_kernel, dim3((unsigned)(gather_ctas + zero_ctas)), dim3(kPredictThreads), 0, stream,
+  const cudaError_t le = launch_dependent(setup_predict_kernel, dim3((unsigned)(gather_ctas + zero_ctas)), dim3(kPredictThreads), kKeysBytes, stream,
                                           T, blob, gather_ctas, gather_tile, call, flags, (uint4*)tables_dst, (uint32_t)(tables_bytes / 16),
                                           (uint4*)zero_dst, zero_vec, state_beg, state_end, (uint32_t)scopes_off, (uint32_t)tile0_off);
   if (le != cudaSuccess) return le;

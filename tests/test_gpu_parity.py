@@ -1285,6 +1285,24 @@ def test_pipelined_pass_edges(cuda_device, case):
         assert st["n_scopes_dense"] == 0, st
 
 
+def test_empty_scopes_leave_their_neighbours_alone(cuda_device):
+    """Empty tensors between others: the start of a call clears the state of every scope without a sample, and must
+    clear exactly that (a store that reached 16 bytes into the next scope's state used to wipe that scope's
+    prediction whenever it landed late, which sent the scope down the dense path: right results, at a cost).
+    Thirty calls; every non-empty scope must stay on the predicted path in each, and the first two are compared with
+    the oracle."""
+    sizes = [1_500_000, 0, 4095, 0, 1_300_000, 0, 0, 17, 600_000]
+    w = W.small_layered(len(sizes), sizes, 990_000, B.GD_SCOPE_PER_LAYER, B.GD_VALUES_FP32, 2)
+    gen = torch.Generator().manual_seed(99)
+    grads = [torch.randn(w.n, generator=gen) * 1e-3 for _ in range(2)]
+    sess = run_steps(w, cuda_device, 2, grads=grads, with_apply=False)
+    g = grads[0].to(cuda_device)
+    for call in range(30):
+        sess.compress(g)
+        st = sess.stats()
+        assert st["status"] == B.GD_OK and st["n_scopes_dense"] == 0 and st["n_scopes_predicted"] == len(sizes), (call, st)
+
+
 @pytest.mark.parametrize("scope_mode", [B.GD_SCOPE_GLOBAL, B.GD_SCOPE_PER_LAYER])
 def test_threshold_far_above_the_prediction(cuda_device, scope_mode):
     """Magnitudes spread evenly over 120 binades: the prediction's safety margin (a multiple of the expected rank for
