@@ -292,7 +292,7 @@ STEP_KERNELS = {
     "predicted_large_sample": ["setup", "sample_select", "add_emit", "cand_select_compact"],
     "predicted_many_scopes": ["setup", "sample_select", "add_emit", "cand_select", "cand_compact"],
     "dense": ["setup", "dense_hist", "dense_find", "dense_hist", "dense_find", "add_emit", "cand_select_compact"],
-    "dense_short_vector": ["setup", "dense_fused"],
+    "dense_short_vector": ["dense_fused"],
     "dense_many_scopes": ["setup", "add_emit", "dense_select", "dense_compact"],
     "sampled": ["setup", "sample_select", "add_emit", "pack_sampled"],
 }

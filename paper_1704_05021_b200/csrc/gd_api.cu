@@ -382,7 +382,10 @@ int compress_impl(const gd_compress_args* a, void* stream_v, bool may_allocate) 
     // The start of the call (clearing the control region, writing the tables) shares a launch with the prediction
     // when every scope's sample is small enough for one CTA; otherwise it is a launch of its own.
     const bool local_predict = P.local_predict;
-    if (local_predict) {
+    // (short vectors: the one launch that does everything also starts the call, where the tables fit its argument)
+    const bool fused_starts = P.dense_fused && !sampled && P.tables_bytes <= kSetupBlobBytes && P.zero_bytes != 0;
+    if (fused_starts) {
+    } else if (local_predict) {
       if (launch_setup_predict(T, tiles[L_SAMP], P.samp_tile, (uint32_t*)(ws + P.off_flags), ws + P.off_tables, tables_image, P.tables_bytes, ws, P.zero_bytes, P.off_state,
                                P.t_scopes, P.t_tile0[L_SAMP], stream) != cudaSuccess)
         return GD_ERR_CUDA;
@@ -412,7 +415,9 @@ int compress_impl(const gd_compress_args* a, void* stream_v, bool may_allocate) 
       // short vectors: add, select and compact over the dense range in one cooperative launch where the vector
       // fits its CTAs' shared memory and the scopes its tables (the plan says); else the three separate kernels
       if (P.dense_fused) {
-        if (launch_dense_fused(T, P.dense_units, stream) != cudaSuccess) return GD_ERR_CUDA;
+        if (launch_dense_fused(T, P.dense_units, stream, ws + P.off_tables, fused_starts ? tables_image : nullptr, P.tables_bytes, ws,
+                               P.zero_bytes) != cudaSuccess)
+          return GD_ERR_CUDA;
       } else {
         if (launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
         if (launch_dense_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;

@@ -24,8 +24,12 @@
 // would be paid for in instruction fetches, not saved in issue slots.  Used when the call has at most kSmemScopes
 // scopes; models with more tensors than that run the two separate kernels.
 #include <atomic>
+#include <cstring>
+#include <mutex>
 
 #include "gd_compact_body.cuh"
+#include <cooperative_groups.h>
+
 #include "gd_select_body.cuh"
 
 namespace gd {
@@ -92,9 +96,23 @@ static_assert(sizeof(SelectSmem<V_DENSE, false>) <= sizeof(Shared) && sizeof(Com
 // need no prediction): the "list" of a scope is its dense range itself - the kernel forms v = grad + residual as it
 // loads its share, selects with the three plain radix passes, and writes the whole new residual (v where dropped,
 // +0 where kept) as it places the survivors: add, select and compact of Algorithm 1 in one launch.
+// What the kernel needs when it is also the start of the call (short vectors: no launch before it has cleared the
+// control region or written the tables): the host-built tables, as a kernel argument, and the two regions.
+struct CallStart {
+  SetupBlob blob;
+  uint4* tables_dst;
+  uint4* zero_dst;
+  uint64_t zero_vec;       // 16-byte words to clear (0: an earlier launch has started the call)
+  uint32_t tables_vec;     // 16-byte words of tables
+};
+struct NoCallStart {};
+template <bool DENSE_IN> struct StartOf { using type = NoCallStart; };
+template <> struct StartOf<true> { using type = CallStart; };
+
 template <bool DENSE_IN>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(const __grid_constant__ DevTables T,
-                                                                      uint32_t dense_sel_tiles, uint32_t dense_chunks) {
+                                                                      uint32_t dense_sel_tiles, uint32_t dense_chunks,
+                                                                      const __grid_constant__ typename StartOf<DENSE_IN>::type start) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sm = *reinterpret_cast<Shared*>(smem_raw);
   __shared__ ScopeDesc s_scope[kSmemScopes];
@@ -116,6 +134,18 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
 
   GD_STAMP(0);
   pdl_trigger();   // (the apply of the push, enqueued behind this kernel, may be brought onto the GPU from now on)
+  if constexpr (DENSE_IN) {
+    if (start.zero_vec != 0u) {
+      // the start of the call, by the whole grid: clear the control region, write the tables, and meet (the runtime's
+      // own grid barrier: the one in the control region is among the words being cleared)
+      const uint64_t stride = (uint64_t)gridDim.x * kThreads, g0 = (uint64_t)blockIdx.x * kThreads + tid;
+      for (uint64_t i = g0; i < start.zero_vec; i += stride) start.zero_dst[i] = make_uint4(0u, 0u, 0u, 0u);
+      const uint4* src = reinterpret_cast<const uint4*>(start.blob.bytes);
+      for (uint64_t i = g0; i < start.tables_vec; i += stride) start.tables_dst[i] = src[i];
+      __threadfence();
+      cooperative_groups::this_grid().sync();
+    }
+  }
   if (T.ctl->status != GD_OK) return;               // set only by an earlier kernel of this call: uniform over the grid
   if (!DENSE_IN && dense_sel_tiles != 0u && T.ctl->dense_needed != 0u) {
     if (!dense_takeover(T, dense_sel_tiles, dense_chunks, smem_raw)) return;
@@ -677,7 +707,8 @@ cudaError_t resident_ctas(int* resident_out, int* dev_out) {
 }
 
 template <bool DENSE_IN>
-cudaError_t launch_impl(const DevTables& T, uint64_t units, uint32_t dsel, uint32_t dchunks, uint32_t tag, cudaStream_t stream) {
+cudaError_t launch_impl(const DevTables& T, uint64_t units, uint32_t dsel, uint32_t dchunks, uint32_t tag, cudaStream_t stream,
+                        const typename StartOf<DENSE_IN>::type& start) {
   ProfileScope prof(stream, tag);
   const size_t smem = sizeof(Shared);
   int resident = 0, dev = -1;
@@ -690,7 +721,7 @@ cudaError_t launch_impl(const DevTables& T, uint64_t units, uint32_t dsel, uint3
   if (grid > kSelectCompactMaxGrid) grid = kSelectCompactMaxGrid;
   if (DENSE_IN && (units + grid - 1) / grid > kStage / kSub) return cudaErrorInvalidConfiguration;   // a share must fit the stage
   DevTables Tc = T;
-  void* args[] = {(void*)&Tc, (void*)&dsel, (void*)&dchunks};
+  void* args[] = {(void*)&Tc, (void*)&dsel, (void*)&dchunks, (void*)&start};
   cudaError_t e = cudaLaunchCooperativeKernel((const void*)select_compact_kernel<DENSE_IN>, dim3(grid), dim3(kThreads), args,
                                               smem, stream);
   if (e != cudaSuccess) return e;
@@ -704,13 +735,31 @@ cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uin
   // units of work: the lists' capacity - or the dense tiles this launch may have to take over, if there are more
   uint64_t units = (cand_total + kSub - 1) / kSub;
   if (units < tiles[L_DSEL]) units = tiles[L_DSEL];
-  return launch_impl<false>(T, units, tiles[L_DSEL], tiles[L_DCOMP], PT_CAND_SELECT_COMPACT, stream);
+  return launch_impl<false>(T, units, tiles[L_DSEL], tiles[L_DCOMP], PT_CAND_SELECT_COMPACT, stream, NoCallStart{});
 }
 
 // Short vectors: residual add, exact selection and compaction over the dense range itself, in one launch.
 // dense_units: the scopes' lengths in units of 1024 elements, summed.
-cudaError_t launch_dense_fused(const DevTables& T, uint64_t dense_units, cudaStream_t stream) {
-  return launch_impl<true>(T, dense_units, 0u, 0u, PT_DENSE_FUSED, stream);
+// tables_src != NULL: the launch is also the start of the call - it clears zero_bytes at zero_dst and writes the
+// tables_bytes (at most kSetupBlobBytes) of host-built tables to tables_dst before anything else.
+cudaError_t launch_dense_fused(const DevTables& T, uint64_t dense_units, cudaStream_t stream, void* tables_dst,
+                               const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes) {
+  static CallStart start;                                    // (large: kept off the stack; filled under the lock below)
+  static std::mutex start_mutex;
+  std::lock_guard<std::mutex> lock(start_mutex);
+  start.zero_vec = 0;
+  start.tables_vec = 0;
+  start.tables_dst = nullptr;
+  start.zero_dst = nullptr;
+  if (tables_src) {
+    if (tables_bytes > kSetupBlobBytes) return cudaErrorInvalidValue;
+    std::memcpy(start.blob.bytes, tables_src, tables_bytes);
+    start.tables_dst = (uint4*)tables_dst;
+    start.tables_vec = (uint32_t)(tables_bytes / 16);
+    start.zero_dst = (uint4*)zero_dst;
+    start.zero_vec = zero_bytes / 16;
+  }
+  return launch_impl<true>(T, dense_units, 0u, 0u, PT_DENSE_FUSED, stream, start);
 }
 
 // How many units launch_dense_fused can take on the current device: every CTA's share must fit its shared-memory

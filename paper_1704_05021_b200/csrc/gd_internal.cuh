@@ -311,7 +311,8 @@ cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uin
 cudaError_t launch_dense_bound(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 bool add_emit_pipe_takes(const DevTables& T);        // the pipelined fused pass (gd_emit_pipe.cu) can take the call
 cudaError_t launch_add_emit_pipe(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
-cudaError_t launch_dense_fused(const DevTables& T, uint64_t dense_units, cudaStream_t stream);
+cudaError_t launch_dense_fused(const DevTables& T, uint64_t dense_units, cudaStream_t stream, void* tables_dst,
+                               const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes);
 uint64_t dense_fused_capacity();   // how many 1024-element units launch_dense_fused takes on the current device (0: none)
 cudaError_t launch_bounded_wait_selftest(void* workspace, uint32_t spin_limit, cudaStream_t stream);
 cudaError_t launch_mbar_wait_selftest(void* workspace, uint64_t budget_ns, cudaStream_t stream);   // after the former: the workspace is prepared
