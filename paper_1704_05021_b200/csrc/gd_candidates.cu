@@ -146,17 +146,33 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       cooperative_groups::this_grid().sync();
     }
   }
-  if (T.ctl->status != GD_OK) return;               // set only by an earlier kernel of this call: uniform over the grid
-  if (!DENSE_IN && dense_sel_tiles != 0u && T.ctl->dense_needed != 0u) {
-    if (!dense_takeover(T, dense_sel_tiles, dense_chunks, smem_raw)) return;
+  // ---- tables, lengths, partition.  Everything the start reads - the call's status, the scope descriptors, what the
+  // earlier kernels left in the scopes' states - is asked for at once: one round trip to L2 instead of three.
+  static_assert(kSmemScopes * (sizeof(ScopeDesc) / 8) <= 2 * kThreads, "two descriptor words per thread");
+  const uint32_t words = T.n_scopes * (uint32_t)(sizeof(ScopeDesc) / 8);
+  const uint64_t* src = reinterpret_cast<const uint64_t*>(T.scopes);
+  const int call_status = T.ctl->status;             // set only by an earlier kernel of this call: uniform over the grid
+  const uint32_t dense_needed = (!DENSE_IN && dense_sel_tiles != 0u) ? T.ctl->dense_needed : 0u;
+  const uint64_t w0 = tid < words ? src[tid] : 0ull, w1 = tid + kThreads < words ? src[tid + kThreads] : 0ull;
+  uint64_t x_count = 0;
+  uint32_t x_tau_lo = 0, x_tau_hi = 0;
+  if (tid < T.n_scopes) {
+    const ScopeState* sx = T.state + tid;
+    x_count = sx->cand_count; x_tau_lo = sx->tau_lo; x_tau_hi = sx->tau_hi;
   }
-
-  // ---- tables, lengths, partition
+  if (call_status != GD_OK) return;
+  if (dense_needed != 0u) {
+    if (!dense_takeover(T, dense_sel_tiles, dense_chunks, smem_raw)) return;
+    if (tid < T.n_scopes) {                          // (the takeover has rewritten the states of the scopes it took)
+      const ScopeState* sx = T.state + tid;
+      x_count = __ldcg(reinterpret_cast<const unsigned long long*>(&sx->cand_count));
+      x_tau_lo = __ldcg(&sx->tau_lo); x_tau_hi = __ldcg(&sx->tau_hi);
+    }
+  }
   {
-    const uint32_t words = T.n_scopes * (uint32_t)(sizeof(ScopeDesc) / 8);
-    const uint64_t* src = reinterpret_cast<const uint64_t*>(T.scopes);
     uint64_t* dst = reinterpret_cast<uint64_t*>(s_scope);
-    for (uint32_t i = tid; i < words; i += kThreads) dst[i] = src[i];
+    if (tid < words) dst[tid] = w0;
+    if (tid + kThreads < words) dst[tid + kThreads] = w1;
     for (uint32_t i = tid; i < kSmemScopes; i += kThreads) s_level[i] = 0;
     if (tid == 0) {
       mbar_init(&s_stage_bar, 1u);
@@ -165,14 +181,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) select_compact_kernel(co
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
-    for (uint32_t x = tid; x < T.n_scopes; x += kThreads) {
-      const ScopeState* sx = T.state + x;
-      const uint64_t m = DENSE_IN ? s_scope[x].hi - s_scope[x].lo : (predicted_ok(T, s_scope[x], *sx) ? sx->cand_count : 0ull);
+    if (tid < T.n_scopes) {
+      const uint32_t x = tid;
+      const bool ok = !(T.flags & GD_FLAG_NO_PREDICTION) && x_count >= s_scope[x].k && x_count <= s_scope[x].cand_cap;   // predicted_ok()
+      const uint64_t m = DENSE_IN ? s_scope[x].hi - s_scope[x].lo : (ok ? x_count : 0ull);
       s_len[x] = m;
       // the window of fine bins is centred on the sample's estimate of the threshold, but starts no lower than
       // the smallest key a candidate can have
-      const uint32_t base = candidate_base_key(sx->tau_lo), half = (kWinBins / 2u) << kFineShift;
-      const uint32_t est = sx->tau_hi;
+      const uint32_t base = candidate_base_key(x_tau_lo), half = (kWinBins / 2u) << kFineShift;
+      const uint32_t est = x_tau_hi;
       s_wlo[x] = (est > half && est - half > base) ? est - half : base;
       s_vt0[x + 1] = (uint32_t)((m + kSub - 1) / kSub);
     }
