@@ -472,7 +472,9 @@ def run_cuda(args):
         ev_end[it].record()
     barrier()
     launches = B.gd_launch_count() - launches0
-    fused_ms = B.gd_profile_collect()
+    fused_pairs = B.gd_profile_collect(with_tags=True)       # ("add_emit", ms), or ("dense_fused", ms) on short vectors
+    fused_ms = [ms for _, ms in fused_pairs]
+    fused_tag = fused_pairs[0][0] if fused_pairs else "add_emit"
     B.gd_profile_enable(False)
     clocks = sampler.stop() if rank == 0 else None
     stats = sess.stats()
@@ -539,7 +541,11 @@ def run_cuda(args):
     fused_avg_ms = sum(fused_ms) / len(fused_ms) if fused_ms else None
     cand_per_call = stats["n_candidates"]
     fused_bytes = 12.0 * w.n + 8.0 * cand_per_call         # read g, read r, write r; candidates written
-    roofline = {"bound": "hbm", "kernel": "add_emit_pipe_kernel", "achieved": None, "peak": peak, "unit": "GB/s",
+    # (short vectors: one kernel does the whole call; the persistent pipeline otherwise, or - with more than 32
+    # scopes - its first version, one CTA per chunk)
+    kernel_name = ("select_compact_kernel<DENSE_IN>" if fused_tag == "dense_fused"
+                   else ("add_emit_pipe_kernel" if sess.n_scopes <= 32 else "add_emit_kernel"))
+    roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": None, "peak": peak, "unit": "GB/s",
                 "frac": None, "traffic": None, "peak_kind": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch": fused_bytes, "launches_timed": len(fused_ms)}
     if fused_avg_ms:
@@ -549,7 +555,7 @@ def run_cuda(args):
     # DRAM traffic of the fused pass: ncu's figure for a smaller launch of the same kernel on the same kind of input,
     # scaled by the elements of this launch (every element is read twice and written once, so it grows with n)
     traffic = dram_traffic_per_element(w)
-    if traffic and not args.no_prediction and not args.sampled:
+    if traffic and not args.no_prediction and not args.sampled and kernel_name == "add_emit_pipe_kernel":
         roofline["traffic"] = traffic["bytes_per_element"] * w.n
         roofline["traffic_source"] = (f"ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch at n = "
                                       f"{traffic['captured_n']} ({traffic['workload']}, captured {traffic['captured']}), "
