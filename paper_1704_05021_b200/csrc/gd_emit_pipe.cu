@@ -648,26 +648,38 @@ cudaError_t launch_mbar_wait_selftest(void* workspace, uint64_t budget_ns, cudaS
   return cudaSuccess;
 }
 
-// Whether the pipelined kernel takes this call: tables that fit shared memory, 16-byte aligned vectors.
+namespace {
+
+// 1 if the current device gives the kernel its shared memory (asked once per device, with the attribute set on the
+// way), -1 if it does not or cannot be asked.
+int pipe_configured() {
+  static PerDeviceInt configured;                          // 0: not asked yet
+  int dev = -1;
+  int c = configured.get(&dev);
+  if (c != 0) return c;
+  if (dev < 0) return -1;
+  const cudaError_t e = cudaFuncSetAttribute(add_emit_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
+  if (e != cudaSuccess) (void)cudaGetLastError();          // (a device with less shared memory: the first version of the pass runs)
+  c = e == cudaSuccess ? 1 : -1;
+  configured.set(dev, c);
+  return c;
+}
+
+}  // namespace
+
+// Whether the pipelined kernel takes this call: tables that fit shared memory, 16-byte aligned vectors, a device that
+// has the shared memory.
 bool add_emit_pipe_takes(const DevTables& T) {
   if (T.n_scopes > kSmemScopes || T.emit_chunk_tiles > (uint32_t)kMaxChunkTiles) return false;
   const uintptr_t a = (uintptr_t)T.grad | (uintptr_t)T.residual | (uintptr_t)T.delta_base;
-  return (a & 15u) == 0u;
+  return (a & 15u) == 0u && pipe_configured() > 0;
 }
 
 cudaError_t launch_add_emit_pipe(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
-  static PerDeviceInt configured;
-  int dev = -1;
-  const size_t smem = sizeof(PipeSmem);
-  if (configured.get(&dev) == 0) {
-    if (dev < 0) return cudaErrorInvalidDevice;
-    cudaError_t e = cudaFuncSetAttribute(add_emit_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured.set(dev, 1);
-  }
+  if (pipe_configured() <= 0) return cudaErrorInvalidDevice;
   uint32_t grid = (uint32_t)sm_count();
   if (grid > tiles[L_EMIT]) grid = tiles[L_EMIT];
-  const cudaError_t e = launch_dependent(add_emit_pipe_kernel, dim3(grid), dim3(kPipeThreads), smem, stream, T, tiles[L_EMIT]);
+  const cudaError_t e = launch_dependent(add_emit_pipe_kernel, dim3(grid), dim3(kPipeThreads), sizeof(PipeSmem), stream, T, tiles[L_EMIT]);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
