@@ -382,13 +382,31 @@ int compress_impl(const gd_compress_args* a, void* stream_v, bool may_allocate) 
     // The start of the call (clearing the control region, writing the tables) shares a launch with the prediction
     // when every scope's sample is small enough for one CTA; otherwise it is a launch of its own.
     const bool local_predict = P.local_predict;
+    EmitEarly early;
+    const EmitEarly* early_ptr = nullptr;
     // (short vectors: the one launch that does everything also starts the call, where the tables fit its argument)
     const bool fused_starts = P.dense_fused && !sampled && P.tables_bytes <= kSetupBlobBytes && P.zero_bytes != 0;
     if (fused_starts) {
     } else if (local_predict) {
+      uint32_t call = 0, clearing_ctas = 0;
       if (launch_setup_predict(T, tiles[L_SAMP], P.samp_tile, (uint32_t*)(ws + P.off_flags), ws + P.off_tables, tables_image, P.tables_bytes, ws, P.zero_bytes, P.off_state,
-                               P.t_scopes, P.t_tile0[L_SAMP], stream) != cudaSuccess)
+                               P.t_scopes, P.t_tile0[L_SAMP], stream, &call, &clearing_ctas) != cudaSuccess)
         return GD_ERR_CUDA;
+      // the fused pass may start while that launch is still selecting: it gets the tables itself and waits only for
+      // the marks of what it is about to use (at most 32 scopes)
+      if (P.n_scopes <= kSmemScopes) {
+        early.tables_src = tables_image;
+        early.tables_bytes = P.tables_bytes;
+        early.scopes_off = P.t_scopes;
+        early.tile0_emit_off = P.t_tile0[L_EMIT];
+        early.ready = (const uint32_t*)(ws + P.off_flags) + tiles[L_SAMP];
+        early.cleared = early.ready + kSmemScopes;
+        early.call = call;
+        early.clearing_ctas = clearing_ctas;
+#ifndef GD_NO_EARLY
+        early_ptr = &early;
+#endif
+      }
     } else if (launch_setup(ws + P.off_tables, tables_image, P.tables_bytes, ws, P.zero_bytes, stream, image_is_pinned) != cudaSuccess) {
       return GD_ERR_CUDA;
     }
@@ -400,7 +418,7 @@ int compress_impl(const gd_compress_args* a, void* stream_v, bool may_allocate) 
     }
     const bool predict = P.predict;
     if (predict && !local_predict && launch_sample_select(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
-    if (predict && launch_add_emit(T, tiles, stream) != cudaSuccess) return GD_ERR_CUDA;
+    if (predict && launch_add_emit(T, tiles, stream, early_ptr) != cudaSuccess) return GD_ERR_CUDA;
     // Without a prediction: the selection and compaction over the dense range.  With one: the two kernels over
     // the candidate lists, which first do the dense work of the scopes whose prediction failed (usually none).
     // The compaction that runs last also finishes the call (thresholds, shard offsets, means).

@@ -293,12 +293,12 @@ __global__ void __launch_bounds__(kEmitThreads, 1024 / kEmitThreads) add_emit_ke
 
 }  // namespace
 
-cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
+cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStream_t stream, const EmitEarly* early) {
   if (!tiles[L_EMIT]) return cudaSuccess;
   ProfileScope prof(stream, PT_ADD_EMIT);
 #ifndef GD_NO_EMIT_PIPE
   if (add_emit_pipe_takes(T)) {
-    cudaError_t e = launch_add_emit_pipe(T, tiles, stream);
+    cudaError_t e = launch_add_emit_pipe(T, tiles, stream, early);
     if (e != cudaSuccess) return e;
     note_launches(1);
     return cudaSuccess;

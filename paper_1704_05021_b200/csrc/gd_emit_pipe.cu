@@ -22,6 +22,9 @@
 //
 // Every wait - on an mbarrier, in the look-back - is bounded; one that runs out records GD_ERR_DEVICE_TIMEOUT, raises
 // the CTA's abort flag (all other waits look at it) and the CTA leaves after its copies in flight have landed.
+#include <cstring>
+#include <mutex>
+
 #include "gd_scan.cuh"
 
 namespace gd {
@@ -70,6 +73,13 @@ struct ChunkFacts {      // what a consumer warp remembers of a chunk until it p
   uint32_t fill;         // candidates of this warp in the chunk (warp-uniform)
 };
 
+struct PipeStart {       // kernel argument: what lets the pass start before the launch before it has ended (enabled != 0)
+  SetupBlob blob;        // the call's tables
+  const uint32_t* ready; // per scope: the call's number once the scope's prediction is final
+  const uint32_t* cleared;   // per clearing CTA of the launch before: the call's number once its part is cleared
+  uint32_t call, clearing_ctas, scopes_off, tile0_off, enabled;
+};
+
 struct PipeSmem {
   alignas(128) float g[kStages][kTile];
   alignas(128) float r[kStages][kTile];
@@ -81,7 +91,6 @@ struct PipeSmem {
   ChunkMeta cmeta[kBufs];
   uint64_t excl[kBufs];                              // candidates of the scope before the chunk
   uint32_t total[kBufs];                             // candidates of the chunk
-  uint32_t tau_lo[kSmemScopes], zmin[kSmemScopes];   // per scope: candidates are keys >= tau_lo, cleared early keys >= zmin
   int abort;
   SmemTables tab;
 };
@@ -103,6 +112,25 @@ struct PipeSmem {
 __device__ __forceinline__ void give_up(PipeSmem& sm, Ctl* ctl) {
   atomicCAS(&ctl->status, (int)GD_OK, (int)GD_ERR_DEVICE_TIMEOUT);
   *(volatile int*)&sm.abort = 1;
+}
+
+// A scope's thresholds for the pass.  Zeros are never candidates: when the prediction is 0 the list holds the non-zero
+// entries, and if there are fewer than k of them the threshold is 0 and the zeros that are kept are found by the dense
+// compaction.  Entries with key >= zmin (above tau_hi, the sample's estimate of the threshold itself) are almost surely
+// kept: their residual slot gets +0 in the streaming store.  Each is a candidate, so its value is in the list, from
+// which the compaction puts it back should it not be kept after all.  In sampled-threshold mode tau_lo is the
+// threshold itself and every candidate is kept.  (Read from L2: the launch that wrote them may still be running.)
+__device__ __forceinline__ void scope_thresholds(const DevTables& T, uint32_t s, uint64_t k, uint32_t* tau_lo_out, uint32_t* zmin_out) {
+  const bool sampled = (T.flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
+  uint32_t tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || k == 0) ? 0xFFFFFFFFu : __ldcg(&T.state[s].tau_lo);
+  if (tau_lo == 0u && !sampled) tau_lo = 1u;
+  uint32_t zmin = 0xFFFFFFFFu;
+  if (tau_lo != 0xFFFFFFFFu) {
+    if (sampled) { if (!(T.flags & GD_FLAG_NO_EARLY_ZERO)) zmin = tau_lo; }
+    else if (early_zero_enabled(T)) zmin = __ldcg(&T.state[s].tau_hi) + 1u;
+  }
+  *tau_lo_out = tau_lo;
+  *zmin_out = zmin;
 }
 
 // A consumer warp's part of one tile: v = g + r (or g - base), the store of v, candidates into the stash.
@@ -337,7 +365,8 @@ __device__ __forceinline__ void place_chunk(const DevTables& T, PipeSmem& sm, in
   }
 }
 
-__global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __grid_constant__ DevTables T, uint32_t total_chunks) {
+__global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __grid_constant__ DevTables T, uint32_t total_chunks,
+                                                                        const __grid_constant__ PipeStart start) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   PipeSmem& sm = *reinterpret_cast<PipeSmem*>(smem_raw);
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
@@ -357,28 +386,24 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  pdl_wait();   // nothing the kernels before this one wrote - tables, thresholds, the residual - is read above this line
-  if (tid == 0) GD_PSTAMP(0);
-  load_tables(T, L_EMIT, &sm.tab, &scopes, &tile0);           // (at most kSmemScopes scopes: the launcher checks)
-  if (warp == (uint32_t)kScanWarp && lane < T.n_scopes) {
-    // Every scope's thresholds, fetched once, along with the tables.  Zeros are never candidates: when the
-    // prediction is 0 the list holds the non-zero entries, and if there are fewer than k of them the threshold is 0
-    // and the zeros that are kept are found by the dense compaction.  Entries with key >= zmin (above tau_hi, the
-    // sample's estimate of the threshold itself) are almost surely kept: their residual slot gets +0 in the streaming
-    // store.  Each is a candidate, so its value is in the list, from which the compaction puts it back should it not
-    // be kept after all.  In sampled-threshold mode tau_lo is the threshold itself and every candidate is kept.
-    const bool sampled = (T.flags & GD_FLAG_SAMPLED_THRESHOLD) != 0;
-    const uint32_t s = lane;
-    uint32_t tau_lo = ((T.flags & GD_FLAG_NO_PREDICTION) || T.scopes[s].k == 0) ? 0xFFFFFFFFu : T.state[s].tau_lo;
-    if (tau_lo == 0u && !sampled) tau_lo = 1u;
-    uint32_t zmin = 0xFFFFFFFFu;
-    if (tau_lo != 0xFFFFFFFFu) {
-      if (sampled) { if (!(T.flags & GD_FLAG_NO_EARLY_ZERO)) zmin = tau_lo; }
-      else if (early_zero_enabled(T)) zmin = T.state[s].tau_hi + 1u;
-    }
-    sm.tau_lo[s] = tau_lo;
-    sm.zmin[s] = zmin;
+  if (start.enabled) {
+    // The tables come with the launch, and nothing else of the launch before this one (the start of the call and the
+    // prediction) is touched before that launch has marked it done: the cleared control region before the first
+    // ticket is taken, a scope's prediction before its first chunk is handed out.  So this grid need not wait for
+    // that one to end - only for the CTA that finishes the prediction of the scope it is about to stream.
+    const uint32_t words = T.n_scopes * (uint32_t)(sizeof(ScopeDesc) / 8);
+    const uint64_t* src = reinterpret_cast<const uint64_t*>(start.blob.bytes + start.scopes_off);
+    uint64_t* dst = reinterpret_cast<uint64_t*>(sm.tab.scopes);
+    for (uint32_t i = tid; i < words; i += kPipeThreads) dst[i] = src[i];
+    const uint32_t* t0 = reinterpret_cast<const uint32_t*>(start.blob.bytes + start.tile0_off);
+    for (uint32_t i = tid; i <= T.n_scopes; i += kPipeThreads) sm.tab.tile0[i] = t0[i];
+    scopes = sm.tab.scopes;
+    tile0 = sm.tab.tile0;
+  } else {
+    pdl_wait();   // nothing the kernels before this one wrote - tables, thresholds, the residual - is read above this line
+    load_tables(T, L_EMIT, &sm.tab, &scopes, &tile0);         // (at most kSmemScopes scopes: the launcher checks)
   }
+  if (tid == 0) GD_PSTAMP(0);
   __syncthreads();
   const volatile int* abort = &sm.abort;
   const bool delta = T.delta_base != nullptr;                 // v = g - base instead of g + r
@@ -388,7 +413,27 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
 
   if (warp == (uint32_t)kProducerWarp) {
     // ------------------------------------------------------------ producer
+    if (start.enabled) {
+      // the control region (ticket counter, look-back descriptors, status) must have been cleared: all lanes look
+      uint32_t spins = 0;
+      uint64_t t0w = 0;
+      for (;;) {
+        bool all = true;
+        for (uint32_t z = lane; z < start.clearing_ctas; z += 32) all = all && ld_acquire_u32(start.cleared + z) == start.call;
+        if (__all_sync(0xFFFFFFFFu, all)) break;
+        ++spins;
+        if (spins == 8u) t0w = global_timer_ns();
+        if (spins > 8u) {
+          __nanosleep(100);
+          if (__any_sync(0xFFFFFFFFu, global_timer_ns() - t0w > kWaitBudgetNs)) {
+            if (lane == 0) give_up(sm, T.ctl);
+            return;
+          }
+        }
+      }
+    }
     if (lane != 0) return;
+    uint32_t cached_s = 0xFFFFFFFFu, tau_lo = 0xFFFFFFFFu, zmin = 0xFFFFFFFFu;
     int stage = 0;
     uint32_t parity = 1;                   // (a fresh mbarrier reads as "the phase of parity 1 has completed")
     uint32_t armed = 0, armed_parity = 0;  // stages used, and the parity of the latest phase of each one's full barrier
@@ -402,7 +447,23 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
       t_next = atomicAdd(&T.ctl->ticket[L_EMIT], 1u);         // (in flight while this chunk's copies are issued)
       const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
       const ScopeDesc& d = scopes[s];
-      const uint32_t tau_lo = sm.tau_lo[s], zmin = sm.zmin[s];
+      if (s != cached_s) {
+        if (start.enabled) {                               // the scope's prediction must be final
+          uint32_t spins = 0;
+          uint64_t t0w = 0;
+          while (ld_acquire_u32(start.ready + s) != start.call) {
+            ++spins;
+            if (spins == 8u) t0w = global_timer_ns();
+            if (spins > 8u) {
+              __nanosleep(100);
+              if (*abort || global_timer_ns() - t0w > kWaitBudgetNs) { ok = false; break; }
+            }
+          }
+          if (!ok) break;
+        }
+        scope_thresholds(T, s, d.k, &tau_lo, &zmin);
+        cached_s = s;
+      }
       const uint64_t lo = d.lo, hi = d.hi;
       const uint64_t cbase = (lo / CH + (t - tile0[s])) * CH;
       // the chunk's tiles that overlap the scope are consecutive
@@ -675,11 +736,25 @@ bool add_emit_pipe_takes(const DevTables& T) {
   return (a & 15u) == 0u && pipe_configured() > 0;
 }
 
-cudaError_t launch_add_emit_pipe(const DevTables& T, const uint32_t* tiles, cudaStream_t stream) {
+cudaError_t launch_add_emit_pipe(const DevTables& T, const uint32_t* tiles, cudaStream_t stream, const EmitEarly* early) {
   if (pipe_configured() <= 0) return cudaErrorInvalidDevice;
   uint32_t grid = (uint32_t)sm_count();
   if (grid > tiles[L_EMIT]) grid = tiles[L_EMIT];
-  const cudaError_t e = launch_dependent(add_emit_pipe_kernel, dim3(grid), dim3(kPipeThreads), sizeof(PipeSmem), stream, T, tiles[L_EMIT]);
+  static PipeStart start;                                    // (large: kept off the stack; filled under the lock below)
+  static std::mutex start_mutex;
+  std::lock_guard<std::mutex> lock(start_mutex);
+  start.enabled = 0;
+  if (early && early->tables_bytes <= kSetupBlobBytes && early->clearing_ctas <= kStartMarks && T.n_scopes <= kSmemScopes) {
+    std::memcpy(start.blob.bytes, early->tables_src, early->tables_bytes);
+    start.ready = early->ready;
+    start.cleared = early->cleared;
+    start.call = early->call;
+    start.clearing_ctas = early->clearing_ctas;
+    start.scopes_off = (uint32_t)early->scopes_off;
+    start.tile0_off = (uint32_t)early->tile0_emit_off;
+    start.enabled = 1;
+  }
+  const cudaError_t e = launch_dependent(add_emit_pipe_kernel, dim3(grid), dim3(kPipeThreads), sizeof(PipeSmem), stream, T, tiles[L_EMIT], start);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 

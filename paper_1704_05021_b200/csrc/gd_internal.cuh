@@ -102,6 +102,11 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 // True when a wait that began at t0 (global_timer_ns) and has polled `spins` times should give up.
 __device__ __forceinline__ bool wait_expired(uint32_t spins, uint32_t spin_limit, uint64_t t0, uint64_t budget_ns) {
   return spins > spin_limit && (budget_ns == 0 || global_timer_ns() - t0 > budget_ns);
@@ -291,15 +296,25 @@ struct SetupBlob {
   unsigned char bytes[kSetupBlobBytes];
 };
 
+// What lets the pipelined fused pass start before the setup-and-predict launch has ended: the tables in its own
+// argument, and where that launch marks (with the call's number) the scopes whose predictions are final and the CTAs
+// that have cleared their part of the control region.
+struct EmitEarly {
+  const void* tables_src;        // host image of the tables (at most kSetupBlobBytes)
+  size_t tables_bytes, scopes_off, tile0_emit_off;
+  const uint32_t* ready;         // [kSmemScopes]
+  const uint32_t* cleared;       // [clearing_ctas]
+  uint32_t call, clearing_ctas;
+};
 // Host-side launchers of the kernel groups (one per .cu file); `tiles` is indexed by Launch.
 cudaError_t upload_by_launches(void* dst, const void* src, size_t bytes, cudaStream_t stream);
 cudaError_t launch_setup(void* tables_dst, const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes,
                          cudaStream_t stream, bool src_is_pinned);
 cudaError_t launch_setup_predict(const DevTables& T, uint32_t gather_ctas, uint32_t gather_tile, uint32_t* flags, void* tables_dst, const void* tables_src,
                                  size_t tables_bytes, void* zero_dst, size_t zero_bytes, size_t state_off, size_t scopes_off,
-                                 size_t tile0_off, cudaStream_t stream);
+                                 size_t tile0_off, cudaStream_t stream, uint32_t* call_out, uint32_t* clearing_ctas_out);
 cudaError_t launch_sample_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
-cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
+cudaError_t launch_add_emit(const DevTables& T, const uint32_t* tiles, cudaStream_t stream, const EmitEarly* early = nullptr);
 cudaError_t launch_candidate_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_dense_select(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 cudaError_t launch_compact(const DevTables& T, const uint32_t* tiles, bool dense, bool finalize, cudaStream_t stream);
@@ -310,7 +325,7 @@ cudaError_t launch_pack_sampled(const DevTables& T, const uint32_t* tiles, cudaS
 cudaError_t launch_select_compact(const DevTables& T, const uint32_t* tiles, uint64_t cand_total, cudaStream_t stream);
 cudaError_t launch_dense_bound(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
 bool add_emit_pipe_takes(const DevTables& T);        // the pipelined fused pass (gd_emit_pipe.cu) can take the call
-cudaError_t launch_add_emit_pipe(const DevTables& T, const uint32_t* tiles, cudaStream_t stream);
+cudaError_t launch_add_emit_pipe(const DevTables& T, const uint32_t* tiles, cudaStream_t stream, const EmitEarly* early);
 cudaError_t launch_dense_fused(const DevTables& T, uint64_t dense_units, cudaStream_t stream, void* tables_dst,
                                const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes);
 uint64_t dense_fused_capacity();   // how many 1024-element units launch_dense_fused takes on the current device (0: none)

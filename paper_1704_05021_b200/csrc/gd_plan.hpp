@@ -307,7 +307,8 @@ inline int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_
       if (tt <= 2u * 148u || P->samp_tile == 1024u) break;
     }
   }
-  P->off_flags = off;        off = align_up(off + sizeof(uint32_t) * (size_t)P->tiles[L_SAMP]);   // not cleared
+  // (marks of the sample tiles, then one per scope - its prediction is written - and one per CTA that clears: not cleared)
+  P->off_flags = off;        off = align_up(off + sizeof(uint32_t) * ((size_t)P->tiles[L_SAMP] + kSmemScopes + kStartMarks));
   P->off_agg = off;          off = align_up(off + 32 * (size_t)kSelectCompactMaxGrid);   // per-CTA records, not cleared
   P->off_samp = off;         off = align_up(off + sizeof(float) * P->samp_total);
   P->off_cand_idx = off;     off = align_up(off + sizeof(uint32_t) * P->cand_total);

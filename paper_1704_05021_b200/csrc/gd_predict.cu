@@ -89,15 +89,25 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
       if (i < state_vec_beg || i >= state_vec_end) zero_dst[i] = make_uint4(0u, 0u, 0u, 0u);
     const uint4* src = reinterpret_cast<const uint4*>(blob.bytes);
     for (uint64_t i = z * kPredictThreads + tid; i < tables_vec; i += stride) tables_dst[i] = src[i];
+    // Marks for the fused pass, which may be running already (it is a programmatic dependent of this launch and, with
+    // its tables in its own argument, does not wait for this grid to end): one per scope whose prediction is final -
+    // here the scopes without a sample - and one per CTA that has done its part of the clearing.
+    uint32_t* ready = flags + gather_ctas;
+    uint32_t* cleared = ready + kSmemScopes;
     if (z == 0) {
       for (uint32_t x = tid; x < T.n_scopes; x += kPredictThreads) {
         if (scopes[x].samp_m == 0) {
           uint4* p = reinterpret_cast<uint4*>(T.state + x);
           static_assert(sizeof(ScopeState) == 48, "three 16-byte stores clear one scope state");
           p[0] = make_uint4(0u, 0u, 0u, 0u); p[1] = p[0]; p[2] = p[0];
+          __threadfence();
+          if (x < kSmemScopes) __stcg(ready + x, call);
         }
       }
     }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0 && z < kStartMarks) __stcg(cleared + z, call);
     return;
   }
 
@@ -231,6 +241,8 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
     // lower edges of the 21-bit buckets
     st->tau_lo = ((pa << 10) | da) << kShift1;
     st->tau_hi = ((pb << 10) | db) << kShift1;
+    __threadfence();
+    if (s < kSmemScopes) __stcg(flags + gather_ctas + s, call);   // the scope's prediction is final (see the clearing CTAs)
 #ifdef GD_PHASE_STAMPS
     atomicMax(reinterpret_cast<unsigned long long*>(T.ctl) + 23, global_timer_ns());
 #endif
@@ -247,7 +259,7 @@ static_assert(kLocalSampleMax == 32u * kPredictThreads, "what one CTA keeps in s
 cudaError_t launch_setup_predict(const DevTables& T, uint32_t gather_ctas, uint32_t gather_tile, uint32_t* flags,
                                  void* tables_dst,
                                  const void* tables_src, size_t tables_bytes, void* zero_dst, size_t zero_bytes, size_t state_off, size_t scopes_off,
-                                 size_t tile0_off, cudaStream_t stream) {
+                                 size_t tile0_off, cudaStream_t stream, uint32_t* call_out, uint32_t* clearing_ctas_out) {
   if (tables_bytes > kSetupBlobBytes) return cudaErrorInvalidValue;
   ProfileScope prof(stream, PT_SETUP_PREDICT);
   static PerDeviceInt configured;                          // the kernel's shared-memory attribute is per device
@@ -267,7 +279,8 @@ cudaError_t launch_setup_predict(const DevTables& T, uint32_t gather_ctas, uint3
   std::memcpy(blob.bytes, tables_src, tables_bytes);
   const uint64_t zero_vec = zero_bytes / 16;              // both regions are 256-byte aligned and padded
   uint64_t zero_ctas = (zero_vec + kPredictThreads * 4 - 1) / (kPredictThreads * 4);
-  const uint64_t cap = (uint64_t)sm_count();
+  uint64_t cap = (uint64_t)sm_count();
+  if (cap > kStartMarks) cap = kStartMarks;
   if (zero_ctas > cap) zero_ctas = cap;
   if (zero_ctas < 1) zero_ctas = 1;
   const uint64_t state_beg = state_off / 16;
@@ -277,6 +290,8 @@ cudaError_t launch_setup_predict(const DevTables& T, uint32_t gather_ctas, uint3
                                           (uint4*)zero_dst, zero_vec, state_beg, state_end, (uint32_t)scopes_off, (uint32_t)tile0_off);
   if (le != cudaSuccess) return le;
   GD_LAUNCH_CHECK();
+  *call_out = call;
+  *clearing_ctas_out = (uint32_t)zero_ctas;
   return cudaSuccess;
 }
 

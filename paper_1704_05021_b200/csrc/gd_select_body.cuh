@@ -15,11 +15,6 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
   return x;
 }
 
-__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
-  uint32_t v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
 
 // All CTAs of a cooperative launch meet here.  `phase` counts the barriers this CTA has passed.
 // Returns false (after recording GD_ERR_DEVICE_TIMEOUT) if the others did not arrive in time.
