@@ -1285,6 +1285,24 @@ def test_pipelined_pass_edges(cuda_device, case):
         assert st["n_scopes_dense"] == 0, st
 
 
+@pytest.mark.parametrize("n_layers", [25, 26, 32])
+def test_as_many_scopes_as_the_shared_tables_hold(cuda_device, n_layers):
+    """25 tensors: the most for which the start of the call, the prediction and the tables still travel in one launch's
+    argument (the fused pass then starts under that launch and waits for each scope's mark); 26: the first for which
+    they do not; 32: the most the kernels keep in shared memory (the tables are written by a launch of their own).  Empty, tiny and long tensors mixed, two
+    means per tensor, three steps."""
+    rng = np.random.default_rng(2400 + n_layers)
+    sizes = [int(x) for x in rng.integers(1, 20_000, size=n_layers)]
+    sizes[0], sizes[3], sizes[7], sizes[n_layers - 1] = 900_000, 0, 1_400_001, 700_003
+    sizes[5] = 1
+    w = W.small_layered(n_layers, sizes, 990_000, B.GD_SCOPE_PER_LAYER, B.GD_VALUES_TWO_MEANS, 4)
+    assert w.n > 2368 * 1024
+    grads = [torch.from_numpy(rng.laplace(0, 1e-3, w.n).astype(np.float32)) for _ in range(3)]
+    sess = run_steps(w, cuda_device, 3, grads=grads)
+    st = sess.stats()
+    assert st["n_scopes_dense"] == 0 and st["n_scopes_predicted"] == n_layers, st
+
+
 def test_empty_scopes_leave_their_neighbours_alone(cuda_device):
     """Empty tensors between others: the start of a call clears the state of every scope without a sample, and must
     clear exactly that (a store that reached 16 bytes into the next scope's state used to wipe that scope's
