@@ -86,7 +86,16 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+  static std::atomic<int> refused{0};                        // a driver that does not take the attribute: ordinary launches
+  if (!refused.load(std::memory_order_relaxed)) {
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, args...);
+    if (e != cudaErrorNotSupported && e != cudaErrorInvalidValue) return e;
+    (void)cudaGetLastError();
+    refused.store(1, std::memory_order_relaxed);
+  }
+  cfg.attrs = nullptr;
+  cfg.numAttrs = 0;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 // ---------------------------------------------------------------- device helpers
