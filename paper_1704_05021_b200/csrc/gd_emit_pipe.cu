@@ -7,7 +7,7 @@
 //                   mbarrier per stage), across chunk boundaries, whatever the other warps are doing;
 //   16 consumer     wait for a tile, form v = g + r from shared memory, store v over r (128-bit stores), and put the
 //   warps           rare entries with |v| >= tau_lo, in index order, into a per-warp stash; a chunk's candidates are
-//                   copied to their final, index-ordered positions in the scope's list one chunk LATER, when the
+//                   copied to their final, index-ordered positions in the scope's list two chunks LATER, when the
 //                   prefix of the chunk is long known;
 //   count warp      per finished chunk: its total is published at once, its (tile, warp) counts become offsets;
 //   scan warp       per finished chunk: one decoupled look-back over the earlier chunks of the scope - off the
@@ -20,7 +20,11 @@
 // last of them to end together.  Tiles cut by a scope's boundary or by the end of the vector are read with plain
 // loads from global memory (bulk copies need 16-byte alignment and whole tiles are what they are good at).
 //
-// Every wait - on an mbarrier, in the look-back - is bounded; one that runs out records GD_ERR_DEVICE_TIMEOUT, raises
+// Behind the launch that starts a call and predicts the thresholds, the pass is a programmatic dependent that does
+// not wait for that grid's end: it carries the tables in its own argument and looks at marks - the control region is
+// cleared, a scope's prediction is final - before it uses what they stand for (PipeStart).
+//
+// Every wait - on an mbarrier, on a mark, in the look-back - is bounded; one that runs out records GD_ERR_DEVICE_TIMEOUT, raises
 // the CTA's abort flag (all other waits look at it) and the CTA leaves after its copies in flight have landed.
 #include <cstring>
 #include <mutex>
