@@ -88,7 +88,8 @@ struct Ctl {             // zeroed at the start of every call
 };
 
 constexpr uint32_t kSmemScopes = 32;          // most scopes whose tables the kernels keep in shared memory
-constexpr size_t kSetupBlobBytes = 3584;      // the small host-built tables of a call travel as a kernel argument of this size at most
+constexpr size_t kSetupBlobBytes = 6144;      // the small host-built tables of a call travel as a kernel argument of this size at most
+                                              // (the tables of 32 scopes are 4.6 KB; kernel arguments beyond 4 KB need CUDA 12.1)
 constexpr uint32_t kSelectCompactMaxGrid = 4096;   // most CTAs of the kernel that selects and compacts in one launch
 constexpr uint32_t kStartMarks = 128;                 // most CTAs that clear the control region in the setup-and-predict launch
 constexpr uint32_t kLocalSampleMax = 32768;        // most samples of one scope that the setup-and-predict launch handles

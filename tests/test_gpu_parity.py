@@ -1287,9 +1287,9 @@ def test_pipelined_pass_edges(cuda_device, case):
 
 @pytest.mark.parametrize("n_layers", [25, 26, 32])
 def test_as_many_scopes_as_the_shared_tables_hold(cuda_device, n_layers):
-    """25 tensors: the most for which the start of the call, the prediction and the tables still travel in one launch's
-    argument (the fused pass then starts under that launch and waits for each scope's mark); 26: the first for which
-    they do not; 32: the most the kernels keep in shared memory (the tables are written by a launch of their own).  Empty, tiny and long tensors mixed, two
+    """Up to 32 tensors - as many scopes as the kernels keep in shared memory - the start of the call, the prediction
+    and the tables travel in one launch's argument (4.6 KB of tables at 32), and the fused pass starts under that
+    launch and waits for each scope's mark.  Empty, tiny and long tensors mixed, two
     means per tensor, three steps."""
     rng = np.random.default_rng(2400 + n_layers)
     sizes = [int(x) for x in rng.integers(1, 20_000, size=n_layers)]
@@ -1301,6 +1301,9 @@ def test_as_many_scopes_as_the_shared_tables_hold(cuda_device, n_layers):
     sess = run_steps(w, cuda_device, 3, grads=grads)
     st = sess.stats()
     assert st["n_scopes_dense"] == 0 and st["n_scopes_predicted"] == n_layers, st
+    before = B.gd_launch_count()
+    sess.compress(grads[0].to(cuda_device))
+    assert B.gd_launch_count() - before == 3          # setup + prediction, fused pass, selection + compaction
 
 
 def test_empty_scopes_leave_their_neighbours_alone(cuda_device):
