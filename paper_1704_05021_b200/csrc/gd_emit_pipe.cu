@@ -22,7 +22,8 @@
 //
 // Behind the launch that starts a call and predicts the thresholds, the pass is a programmatic dependent that does
 // not wait for that grid's end: it carries the tables in its own argument and looks at marks - the control region is
-// cleared, a scope's prediction is final - before it uses what they stand for (PipeStart).
+// cleared, a scope's prediction is final - before it uses what they stand for (PipeStart).  The copies of a scope's
+// first chunk are issued before the scope's mark is up; only the consumers' view of them waits for it.
 //
 // Every wait - on an mbarrier, on a mark, in the look-back - is bounded; one that runs out records GD_ERR_DEVICE_TIMEOUT, raises
 // the CTA's abort flag (all other waits look at it) and the CTA leaves after its copies in flight have landed.
@@ -393,7 +394,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
   if (start.enabled) {
     // The tables come with the launch, and nothing else of the launch before this one (the start of the call and the
     // prediction) is touched before that launch has marked it done: the cleared control region before the first
-    // ticket is taken, a scope's prediction before its first chunk is handed out.  So this grid need not wait for
+    // ticket is taken, a scope's prediction before a tile of it is handed to the consumers.  So this grid need not wait for
     // that one to end - only for the CTA that finishes the prediction of the scope it is about to stream.
     const uint32_t words = T.n_scopes * (uint32_t)(sizeof(ScopeDesc) / 8);
     const uint64_t* src = reinterpret_cast<const uint64_t*>(start.blob.bytes + start.scopes_off);
@@ -451,31 +452,62 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
       t_next = atomicAdd(&T.ctl->ticket[L_EMIT], 1u);         // (in flight while this chunk's copies are issued)
       const uint32_t s = scope_of_tile(tile0, T.n_scopes, t);
       const ScopeDesc& d = scopes[s];
-      if (s != cached_s) {
-        if (start.enabled) {                               // the scope's prediction must be final
-          uint32_t spins = 0;
-          uint64_t t0w = 0;
-          while (ld_acquire_u32(start.ready + s) != start.call) {
-            ++spins;
-            if (spins == 8u) t0w = global_timer_ns();
-            if (spins > 8u) {
-              __nanosleep(100);
-              if (*abort || global_timer_ns() - t0w > kWaitBudgetNs) { ok = false; break; }
-            }
-          }
-          if (!ok) break;
-        }
-        scope_thresholds(T, s, d.k, &tau_lo, &zmin);
-        cached_s = s;
-      }
       const uint64_t lo = d.lo, hi = d.hi;
       const uint64_t cbase = (lo / CH + (t - tile0[s])) * CH;
       // the chunk's tiles that overlap the scope are consecutive
       uint32_t i_first = 0, i_last = C - 1u;
       while (i_first < C && cbase + (uint64_t)(i_first + 1u) * kTile <= lo) ++i_first;
       while (i_last > i_first && cbase + (uint64_t)i_last * kTile >= hi) --i_last;
+      uint32_t issued = 0;                 // tiles of this chunk whose copies are under way already
+      if (s != cached_s) {
+        if (start.enabled && ld_acquire_u32(start.ready + s) != start.call) {
+          // The scope's prediction must be final before a consumer sees a tile of it - the copies need not wait:
+          // they are issued now (their bytes announced on the stage's barrier, the producer's arrive held back), so
+          // that the chunk has landed by the time the thresholds exist.
+#ifndef GD_NO_EARLY_LOADS
+          if (i_last - i_first < (uint32_t)kStages)
+#else
+          if (false)
+#endif
+          {
+            int st = stage;
+            uint32_t par = parity;
+            for (uint32_t i = i_first; i <= i_last; ++i) {
+              if (!mbar_wait(&sm.empty[st], par, abort)) { ok = false; break; }
+              const uint64_t base = cbase + (uint64_t)i * kTile;
+              if (base >= lo && base + kTile <= hi) {
+                mbar_expect_tx(&sm.full[st], 2u * kTileBytes);
+                bulk_load(sm.g[st], T.grad + base, kTileBytes, &sm.full[st]);
+                bulk_load(sm.r[st], second + base, kTileBytes, &sm.full[st]);
+              }
+              ++issued;
+              if (++st == kStages) { st = 0; par ^= 1u; }
+            }
+          }
+          uint32_t spins = 0;
+          uint64_t t0w = 0;
+          while (ok && ld_acquire_u32(start.ready + s) != start.call) {
+            ++spins;
+            if (spins == 8u) t0w = global_timer_ns();
+            if (spins > 8u) {
+              __nanosleep(100);
+              if (*abort || global_timer_ns() - t0w > kWaitBudgetNs) ok = false;
+            }
+          }
+        }
+        if (ok) {
+          scope_thresholds(T, s, d.k, &tau_lo, &zmin);
+          cached_s = s;
+        } else {
+          tau_lo = 0xFFFFFFFFu; zmin = 0xFFFFFFFFu;             // (giving up: the tiles under way are handed on empty-handed)
+        }
+      }
       for (uint32_t i = i_first; i <= i_last; ++i) {
-        if (!mbar_wait(&sm.empty[stage], parity, abort)) { ok = false; break; }
+        const bool under_way = i - i_first < issued;
+        if (!under_way) {
+          if (!ok) break;
+          if (!mbar_wait(&sm.empty[stage], parity, abort)) { ok = false; break; }
+        }
         const uint64_t base = cbase + (uint64_t)i * kTile;
         const bool cut = !(base >= lo && base + kTile <= hi);
         TileMeta m;
@@ -484,7 +516,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) add_emit_pipe_kernel(const __
         m.i = i - i_first;
         m.tau_lo = tau_lo; m.zmin = zmin;
         sm.meta[stage] = m;
-        if (cut) {
+        if (cut || under_way) {
           mbar_arrive(&sm.full[stage]);
         } else {
           mbar_arrive_expect_tx(&sm.full[stage], 2u * kTileBytes);

@@ -1244,6 +1244,43 @@ def test_random_models_of_few_large_tensors(cuda_device, seed):
     run_steps(w, cuda_device, 2, flags=flags, grads=grads, layer_cols=cols, alpha=float(rng.choice([1.0, 0.5])))
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_random_models_of_ten_to_48_tensors(cuda_device, seed):
+    """Ten to 48 tensors from empty to 1.2 M elements (on both sides of the 32 scopes whose tables fit shared memory and
+    the kernel argument, and of the length the one-launch dense kernel holds), random drop ratio, scope, value mode,
+    shard count, flags and value distribution; three steps with the residual carried, everything compared with the
+    oracle."""
+    rng = np.random.default_rng(770000 + seed)
+    n_layers = int(rng.integers(10, 49))
+    sizes = []
+    for _ in range(n_layers):
+        kind = rng.integers(0, 6)
+        sizes.append(int([0, rng.integers(1, 40), rng.integers(40, 5000), rng.integers(5000, 70_000),
+                          rng.integers(70_000, 400_000), rng.integers(400_000, 1_200_000)][kind]))
+    if sum(sizes) == 0:
+        sizes[0] = 99_999
+    ppm = int(rng.choice([300_000, 900_000, 984_000, 990_000, 990_000, 999_000, 999_900, 1_000_000]))
+    scope_mode = int(rng.integers(0, 2))
+    value_mode = int(rng.choice([0, 0, 1, 2]))
+    flags = int(rng.choice([0, 0, B.GD_FLAG_PREDICT_ALWAYS, B.GD_FLAG_PREDICT_ALWAYS, B.GD_FLAG_NO_PREDICTION]))
+    if not flags & B.GD_FLAG_NO_PREDICTION and rng.random() < 0.3:
+        flags |= B.GD_FLAG_NO_EARLY_ZERO
+    w = W.small_layered(n_layers, sizes, ppm, scope_mode, value_mode, int(rng.integers(1, 9)))
+    dist = int(rng.integers(0, 4))
+    grads = []
+    for _ in range(3):
+        if dist == 0:
+            g = rng.laplace(0, 1e-3, w.n)
+        elif dist == 1:
+            g = rng.standard_normal(w.n) * 10.0 ** rng.integers(-6, 1, w.n)
+        elif dist == 2:
+            g = np.where(rng.random(w.n) < 0.02, rng.standard_normal(w.n), 0.0)
+        else:
+            g = rng.choice(np.array([0.0, 0.25, -0.25, 0.5, 1.0, -2.0]), w.n)
+        grads.append(torch.from_numpy(g.astype(np.float32)))
+    run_steps(w, cuda_device, 3, flags=flags, grads=grads, alpha=float(rng.choice([1.0, 0.5])))
+
+
 @pytest.mark.parametrize("case", ["boundaries_at_every_offset", "dense_rows", "tiny_between_large", "full_lists"])
 def test_pipelined_pass_edges(cuda_device, case):
     """What the pipelined fused pass treats specially, each on a layout too long for the one-launch dense kernel:
