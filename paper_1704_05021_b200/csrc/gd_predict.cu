@@ -162,6 +162,7 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
   // registers, the same selection took 9 us, most of it instruction fetches; rolled, 6 us.
   constexpr int kKeys = 32;
   const uint32_t* keys = reinterpret_cast<const uint32_t*>(smem_keys);
+  uint32_t zeros = 0;                                      // samples that are +-0: counted privately
   {
     constexpr int kBatch = 8;                               // loads per thread in flight at a time
     uint32_t* wkeys = reinterpret_cast<uint32_t*>(smem_keys);
@@ -175,22 +176,17 @@ setup_predict_kernel(const __grid_constant__ DevTables T, const __grid_constant_
 #pragma unroll
       for (int u = 0; u < kBatch; ++u) {
         const uint32_t li = li0 + (uint32_t)u * kPredictThreads;
-        if (li < m) wkeys[li] = w[u];
+        if (li < m) {
+          wkeys[li] = w[u];
+          // first digit: counted as the keys arrive
+          const uint32_t key = w[u] & kAbsMask;
+          if (key == 0u) ++zeros;
+          else atomicAdd(&s_hist[key >> kShift0], 1u);
+        }
       }
     }
   }
-  __syncthreads();
   const uint32_t per_thread = (m + kPredictThreads - 1u) / kPredictThreads;   // <= kKeys
-  uint32_t zeros = 0;                                      // samples that are +-0: counted privately
-#pragma unroll 4
-  for (uint32_t j = 0; j < per_thread; ++j) {
-    const uint32_t li = j * kPredictThreads + tid;
-    if (li < m) {
-      const uint32_t key = keys[li] & kAbsMask;
-      if (key == 0u) ++zeros;
-      else atomicAdd(&s_hist[key >> kShift0], 1u);
-    }
-  }
   static_assert(kLocalSampleMax == (uint32_t)kKeys * kPredictThreads, "the shared-memory copy of the sample");
   const uint32_t zeros_mine = zeros;
 #pragma unroll
