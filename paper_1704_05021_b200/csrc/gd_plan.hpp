@@ -20,7 +20,13 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // factors of 0.12, 0.25 and 0.5 were timed on layered models of 12 to 387 tensors), so:
 // hits = kHitsFactor * k^(2/3) within [kHitsMin, kHitsMax], and never more than kSampleMax samples or a
 // sixteenth of the scope.
-constexpr double kHitsFactor = 0.25, kHitsMin = 32.0, kHitsMax = 256.0, kSampleMax = 262144.0;
+// While the lists are short - the call keeps at most kShortListsK entries in all - the sample is on the critical path (the
+// fused pass waits for the prediction) and a longer list costs next to nothing: the cap is 128 there (step time at
+// R = 99 %, 256 / 128 / 64 hits: 2^22 elements 65 / 62 / 60 us, 2^24 94 / 91 / 89 us, 2^25 136 / 133 / 132 us, the MNIST-shaped
+// model 104 / 103 / 104 us; from 2^26 elements on 256 is as good or better, and on the NMT-shaped model 128 costs 16 us:
+// its lists then outgrow the shared-memory stage of the kernel that selects among them).
+constexpr double kHitsFactor = 0.25, kHitsMin = 32.0, kHitsMax = 256.0, kHitsMaxShortLists = 128.0, kSampleMax = 262144.0;
+constexpr uint64_t kShortListsK = 1ull << 19;
 constexpr uint64_t kSampleAllMax = 8192;         // scopes up to this length are sampled completely
 constexpr uint64_t kClusterMaxStride = 1024;      // strata up to this many elements wide are sampled in groups of 8
 constexpr uint64_t kAutoDenseMax = 3ull << 18;   // vectors up to this length skip the prediction (measured, step time
@@ -39,12 +45,13 @@ inline uint64_t kept_count(uint64_t n, uint32_t drop_ppm) {
 // above the prediction is at least k with a margin of six standard deviations plus 12.5 %.  Small
 // scopes are sampled completely, which makes the prediction the exact threshold.  None of this
 // affects results: a scope whose prediction fails is selected densely.
-inline void plan_prediction(uint64_t ns, uint64_t k, uint64_t* m, uint64_t* rank, uint64_t* cap, uint32_t* cluster) {
+inline void plan_prediction(uint64_t ns, uint64_t k, double hits_max, uint64_t* m, uint64_t* rank, uint64_t* cap,
+                            uint32_t* cluster) {
   *cluster = 1;
   if (k == 0 || ns == 0) { *m = 0; *rank = 0; *cap = 0; return; }
   double hits = kHitsFactor * std::cbrt((double)k * (double)k);
   if (hits < kHitsMin) hits = kHitsMin;
-  if (hits > kHitsMax) hits = kHitsMax;
+  if (hits > hits_max) hits = hits_max;
   double target = hits * (double)ns / (double)k;
   if (target > kSampleMax) target = kSampleMax;
   if (target > (double)ns / 16.0) target = (double)ns / 16.0;
@@ -194,6 +201,7 @@ inline int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_
   P->samp_off.assign(ns_count + 1, 0);
   uint64_t tiles[L_COUNT] = {0, 0, 0, 0, 0};
   uint64_t out_base = 0, cand_base = 0, samp_base = 0;
+  const double hits_max = kept_count(n, drop_ppm) <= kShortListsK ? kHitsMaxShortLists : kHitsMax;
   for (uint32_t s = 0; s < ns_count; ++s) {
     ScopeDesc& d = P->scopes[s];
     d.lo = scope_mode == GD_SCOPE_GLOBAL ? 0 : layer_off[s];
@@ -210,7 +218,7 @@ inline int make_plan(const uint64_t* layer_off, uint32_t n_layers, const uint32_
       rank = kept_count(m, drop_ppm);
       cap = sampled_cap(ns, d.k);
     } else if (predict) {
-      plan_prediction(ns, d.k, &m, &rank, &cap, &cluster);
+      plan_prediction(ns, d.k, hits_max, &m, &rank, &cap, &cluster);
     } else if (P->dense_bound) {
       // the candidates are the keys above the bin of the k-th largest key (fewer than k) and that bin itself
       const uint64_t c = 3 * d.k + 4096;
