@@ -53,6 +53,13 @@ inline void plan_prediction(uint64_t ns, uint64_t k, double hits_max, uint64_t* 
   if (hits < kHitsMin) hits = kHitsMin;
   if (hits > hits_max) hits = hits_max;
   double target = hits * (double)ns / (double)k;
+#ifndef GD_NO_LOCAL_CLAMP
+  // Short lists (hits_max below kHitsMax): a sample that one CTA can hold is predicted from in the launch that starts
+  // the call (kLocalSampleMax values; gd_predict.cu) instead of two launches more - worth a wider margin, as long as
+  // the expected hits stay at or above kHitsMin.
+  if (hits_max < kHitsMax && target > (double)kLocalSampleMax && (double)kLocalSampleMax * (double)k >= kHitsMin * (double)ns)
+    target = (double)kLocalSampleMax;
+#endif
   if (target > kSampleMax) target = kSampleMax;
   if (target > (double)ns / 16.0) target = (double)ns / 16.0;
   uint64_t mt = (uint64_t)target;
