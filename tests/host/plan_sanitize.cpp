@@ -133,6 +133,35 @@ int main() {
       for (uint32_t flags : {0u, (uint32_t)GD_FLAG_NO_PREDICTION, (uint32_t)GD_FLAG_SAMPLED_THRESHOLD})
         plans += check(sizes, 1 + (uint32_t)(rng() % 40), scope, 990000u, flags, rep % 2 ? cols.data() : nullptr);
   }
+  // how large a sample is: short lists (at most 2^19 entries kept by the call) stay within what the launch that starts
+  // the call selects from, down to 32 expected samples above the threshold; long lists and thinner samples do not
+  {
+    auto plan_of = [](const std::vector<uint64_t>& sizes, int scope, uint32_t ppm, Plan* P) {
+      std::vector<uint64_t> off(sizes.size() + 1, 0);
+      for (size_t i = 0; i < sizes.size(); ++i) off[i + 1] = off[i] + sizes[i];
+      REQUIRE(make_plan(off.data(), (uint32_t)sizes.size(), nullptr, 4, scope, ppm, 0, P) == GD_OK);
+    };
+    Plan P;
+    const std::vector<uint64_t> nmt = {42500000, 42500000, 42500000, 85000, 1500000, 1000000, 1500000, 1000000, 1500000, 1000000, 1500000, 1000000};
+    for (uint32_t ppm : {990000u, 999000u}) {
+      plan_of({1ull << 24}, GD_SCOPE_GLOBAL, ppm, &P);
+      REQUIRE(P.predict && P.local_predict);
+      plan_of(nmt, GD_SCOPE_PER_LAYER, ppm, &P);
+      REQUIRE(P.predict && P.local_predict);
+      for (const ScopeDesc& d : P.scopes)                  // at least 32 expected hits, unless a sixteenth of the scope is sampled
+        if (d.samp_m + 8 < (d.hi - d.lo) / 16) REQUIRE((double)d.k * (double)d.samp_m >= 31.0 * (double)(d.hi - d.lo));
+    }
+    plan_of({1ull << 28}, GD_SCOPE_GLOBAL, 999000u, &P);   // 268 435 kept: still short
+    REQUIRE(P.local_predict && P.scopes[0].samp_m == kLocalSampleMax);
+    plan_of({1ull << 30}, GD_SCOPE_GLOBAL, 999000u, &P);   // 1 073 742 kept: the sample keeps its 256 expected hits
+    REQUIRE(P.predict && !P.local_predict && P.scopes[0].samp_m > kLocalSampleMax);
+    plan_of({1ull << 24}, GD_SCOPE_GLOBAL, 999500u, &P);   // 32 hits would need more than one CTA holds
+    REQUIRE(P.predict && !P.local_predict);
+    plan_of({1ull << 30}, GD_SCOPE_GLOBAL, 990000u, &P);   // long lists at R = 99 %: 256 hits are 25 600 samples
+    REQUIRE(P.local_predict && P.scopes[0].samp_m >= 25000 && P.scopes[0].samp_m <= 26000);
+    plan_of({1ull << 24}, GD_SCOPE_GLOBAL, 990000u, &P);   // short lists at R = 99 %: 128 hits
+    REQUIRE(P.local_predict && P.scopes[0].samp_m >= 12500 && P.scopes[0].samp_m <= 13000);
+  }
   // arguments that must be refused
   {
     Plan P;
