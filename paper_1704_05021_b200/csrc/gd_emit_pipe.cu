@@ -270,22 +270,36 @@ __device__ __forceinline__ void place_chunk(const DevTables& T, PipeSmem& sm, in
   StashEntry* stash = sm.stash[buf][warp];
   const uint32_t ltm = lanemask_lt();
   if (fill <= kPipeStash) {
-    uint32_t a = 0;                          // first stash entry of tile i
-    for (uint32_t i = 0; i < cm.ntiles; ++i) {
-      const uint32_t c = sm.cnt[buf][i * kConsumerWarps + warp];
-      const uint64_t dst = excl + sm.off[buf][i * kConsumerWarps + warp];
-      for (uint32_t e = lane; e < c; e += 32) {
-        const uint64_t pos = dst + e;
-        if (pos < cap) {
-          cidx[pos] = stash[a + e].idx;
-          cval[pos] = stash[a + e].val;
-        } else if ((__float_as_uint(stash[a + e].val) & kAbsMask) >= zmin) {
-          // the list is full (the scope will be selected densely): the slot must hold v again
-          T.residual[stash[a + e].idx] = stash[a + e].val;
-          T.state[cm.s].early_bad = 1u;
-        }
+    // One loop over the warp's stash (a few entries per tile: a loop per tile would run with most lanes idle and four
+    // times the shared-memory round trips).  Entry e belongs to the last tile whose run starts at or before it.
+    uint32_t first[kMaxChunkTiles], shift[kMaxChunkTiles];   // first stash entry of tile i; (offset in the chunk) - first
+    {
+      uint32_t a = 0;
+#pragma unroll
+      for (int i = 0; i < kMaxChunkTiles; ++i) {
+        const bool live = (uint32_t)i < cm.ntiles;
+        const uint32_t c = live ? sm.cnt[buf][i * kConsumerWarps + warp] : 0u;
+        const uint32_t o = live ? sm.off[buf][i * kConsumerWarps + warp] : 0u;
+        first[i] = a;
+        shift[i] = o - a;
+        a += c;
       }
-      a += c;
+    }
+    for (uint32_t e = lane; e < fill; e += 32) {
+      uint32_t sh = shift[0];
+#pragma unroll
+      for (int i = 1; i < kMaxChunkTiles; ++i)
+        if (e >= first[i]) sh = shift[i];
+      const uint64_t pos = excl + (uint32_t)(e + sh);
+      const StashEntry se = stash[e];
+      if (pos < cap) {
+        cidx[pos] = se.idx;
+        cval[pos] = se.val;
+      } else if ((__float_as_uint(se.val) & kAbsMask) >= zmin) {
+        // the list is full (the scope will be selected densely): the slot must hold v again
+        T.residual[se.idx] = se.val;
+        T.state[cm.s].early_bad = 1u;
+      }
     }
     return;
   }
